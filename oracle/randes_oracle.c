@@ -1,0 +1,412 @@
+/*
+ * RanDeS CPU oracle -- TEST INFRASTRUCTURE, not a product path.
+ *
+ * A plain, slow, element-by-element implementation of delta superposition and
+ * retrieval under seed-defined random orthogonal transforms, written from the
+ * paper's equations.  It exists so that the CUDA library can be compared with
+ * something that can be checked against the paper by eye.  Only tests, the
+ * smoke check and the benchmark's CPU-baseline leg may call it; it shares no
+ * code with the CUDA library and neither includes the other.
+ *
+ * Notation (paper symbol in brackets):
+ *   W_0  base model            [Theta_0]
+ *   W_i  fine-tuned model i    [Theta_i]
+ *   d_i  = W_i - W_0           [Delta_i, Section 3]
+ *   T_i  orthogonal transform  [O_i, Section 4]
+ *   M    = sum_i T_i(d_i)      [the superposed delta, Section 4 / Eq. in 4.4]
+ *   sigma_i^g  permutation of the members of group g for task i [Section 4.3]
+ *   s_i(l,c)   +-1 diagonal entry for task i, slot l, column c   [Section 4.4]
+ *
+ * Readings of points the paper leaves open (all are stated again in the
+ * design notes of this repository):
+ *   - T_i = D_i o P_i: the layers of a delta are shuffled first, the sign flip
+ *     is indexed by the position ("slot") the layer lands on in M.
+ *   - Shuffle is the gather the paper prints: slot k receives member sigma(k).
+ *   - lambda is applied at retrieval; M is kept in fp32 whatever the storage
+ *     type of the weights.
+ *   - "Column" is the second (contiguous) index of a row-major [rows, cols]
+ *     array; a 1-D parameter is [1, cols].
+ *   - Random numbers: Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11),
+ *     key = the task's 64-bit seed, counter = (index, layer-or-group, domain
+ *     tag, task id).
+ *   - Arithmetic: fp32; the subtraction W_i - W_0 and each accumulation are
+ *     separately rounded; retrieval is one fused multiply-add; bf16 is
+ *     round-to-nearest-even.
+ *
+ * Every function below is pinned by the CPU test-suite to something other
+ * than itself (known-answer vectors, dense signed-permutation matrices in
+ * double precision, closed forms, invariants).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define RO_F32 0
+#define RO_BF16 1
+#define RO_SHUFFLE 1u
+#define RO_FLIP 2u
+
+#define RO_TAG_PERM 0x5045524Du /* "PERM" */
+#define RO_TAG_SIGN 0x5349474Eu /* "SIGN" */
+
+/* ------------------------------------------------------------------------ */
+/* Philox4x32-10, from the published definition (SC'11, Section 3.3 / Table  */
+/* of multipliers): ten rounds of two 32x32->64 multiplies, the key bumped   */
+/* by the Weyl constants between rounds.                                     */
+/* ------------------------------------------------------------------------ */
+void ro_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    const uint32_t MUL0 = 0xD2511F53u, MUL1 = 0xCD9E8D57u;
+    const uint32_t WEYL0 = 0x9E3779B9u, WEYL1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) {
+            k0 += WEYL0;
+            k1 += WEYL1;
+        }
+        uint64_t p0 = (uint64_t)MUL0 * (uint64_t)c0;
+        uint64_t p1 = (uint64_t)MUL1 * (uint64_t)c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+static void seed_key(uint64_t seed, uint32_t key[2])
+{
+    key[0] = (uint32_t)(seed & 0xFFFFFFFFu);
+    key[1] = (uint32_t)(seed >> 32);
+}
+
+/* ------------------------------------------------------------------------ */
+/* Section 4.3: sigma ~ S_G, one per (task, group).  Fisher-Yates from the   */
+/* top, random words taken from consecutive Philox blocks in output order,   */
+/* reduced to [0, k] by multiply-shift.                                      */
+/* sigma[k] = index (within the group) of the member that lands on slot k.   */
+/* ------------------------------------------------------------------------ */
+void ro_permutation(uint64_t seed, uint32_t task_id, uint32_t group_index,
+                    uint32_t G, uint32_t *sigma)
+{
+    uint32_t key[2], ctr[4], blk[4];
+    uint32_t n_block = 0, used = 4;
+    seed_key(seed, key);
+    for (uint32_t k = 0; k < G; ++k) sigma[k] = k;
+    for (uint32_t k = G; k-- > 1;) {
+        if (used == 4) {
+            ctr[0] = n_block++; ctr[1] = group_index; ctr[2] = RO_TAG_PERM; ctr[3] = task_id;
+            ro_philox4x32_10(ctr, key, blk);
+            used = 0;
+        }
+        uint32_t r = blk[used++];
+        uint32_t j = (uint32_t)(((uint64_t)r * (uint64_t)(k + 1)) >> 32);
+        uint32_t t = sigma[k]; sigma[k] = sigma[j]; sigma[j] = t;
+    }
+}
+
+/* ------------------------------------------------------------------------ */
+/* Section 4.4: diagonal entry of D for (task, slot, column): +1 or -1 with  */
+/* equal probability.  One Philox block holds the bits of 128 columns.       */
+/* ------------------------------------------------------------------------ */
+int ro_sign(uint64_t seed, uint32_t task_id, uint32_t slot, uint32_t col)
+{
+    uint32_t key[2], ctr[4], blk[4];
+    seed_key(seed, key);
+    ctr[0] = col >> 7; ctr[1] = slot; ctr[2] = RO_TAG_SIGN; ctr[3] = task_id;
+    ro_philox4x32_10(ctr, key, blk);
+    uint32_t bit = (blk[(col >> 5) & 3u] >> (col & 31u)) & 1u;
+    return bit ? -1 : +1;
+}
+
+void ro_sign_row(uint64_t seed, uint32_t task_id, uint32_t slot, uint32_t cols, int8_t *out)
+{
+    for (uint32_t c = 0; c < cols; ++c) out[c] = (int8_t)ro_sign(seed, task_id, slot, c);
+}
+
+/* ------------------------------------------------------------------------ */
+/* Per-task layer tables over the whole model.                               */
+/*   src_of_slot[l] = layer whose delta lands on slot l   (sigma)            */
+/*   slot_of_pos[p] = slot that holds layer p's delta     (sigma^-1)         */
+/* Group members are the layers carrying that group id, in layer order.      */
+/* Returns 0, or -1 if a group id is out of range / allocation fails.        */
+/* ------------------------------------------------------------------------ */
+int ro_task_tables(uint32_t n_layers, const uint32_t *group, uint32_t n_groups,
+                   const uint32_t *gflags, uint64_t seed, uint32_t task_id,
+                   uint32_t *src_of_slot, uint32_t *slot_of_pos)
+{
+    uint32_t *members = (uint32_t *)malloc(sizeof(uint32_t) * (n_layers + 1));
+    uint32_t *sigma = (uint32_t *)malloc(sizeof(uint32_t) * (n_layers + 1));
+    if (!members || !sigma) { free(members); free(sigma); return -1; }
+    for (uint32_t l = 0; l < n_layers; ++l) {
+        if (group[l] >= n_groups) { free(members); free(sigma); return -1; }
+        src_of_slot[l] = l;
+        slot_of_pos[l] = l;
+    }
+    for (uint32_t g = 0; g < n_groups; ++g) {
+        uint32_t G = 0;
+        for (uint32_t l = 0; l < n_layers; ++l)
+            if (group[l] == g) members[G++] = l;
+        if (G < 2 || !(gflags[g] & RO_SHUFFLE)) continue;
+        ro_permutation(seed, task_id, g, G, sigma);
+        for (uint32_t k = 0; k < G; ++k) {
+            src_of_slot[members[k]] = members[sigma[k]];
+            slot_of_pos[members[sigma[k]]] = members[k];
+        }
+    }
+    free(members);
+    free(sigma);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------ */
+/* bf16 <-> fp32                                                             */
+/* ------------------------------------------------------------------------ */
+static float bf16_to_f32(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+uint16_t ro_f32_to_bf16(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu) != 0u)
+        return (uint16_t)((u >> 16) | 0x0040u); /* NaN stays NaN */
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7FFFu + lsb; /* round to nearest, ties to even; carries into Inf */
+    return (uint16_t)(u >> 16);
+}
+
+static float load_elem(const void *p, int dtype, size_t i)
+{
+    if (dtype == RO_BF16) return bf16_to_f32(((const uint16_t *)p)[i]);
+    return ((const float *)p)[i];
+}
+
+/* ------------------------------------------------------------------------ */
+/* x = T_i(d_i) restricted to one slot l: the shuffled, sign-flipped delta.  */
+/* x[r,c] = s_i(l,c) * ( W_i[src][r,c] - W_0[src][r,c] ),  src = sigma_i(l). */
+/* base == NULL: `task` already holds the delta (PEFT / LoRA, Section 5.8).  */
+/* ------------------------------------------------------------------------ */
+static float transformed_delta(const void *w_task, const void *w_base, int dtype,
+                               size_t idx, int sign)
+{
+    float d;
+    if (w_base) {
+        d = load_elem(w_task, dtype, idx) - load_elem(w_base, dtype, idx); /* one rounding */
+    } else {
+        d = load_elem(w_task, dtype, idx);
+    }
+    return sign < 0 ? -d : d;
+}
+
+typedef struct {
+    uint32_t n_layers;
+    const uint32_t *rows, *cols, *group;
+    uint32_t n_groups;
+    const uint32_t *gflags;
+} ro_spec_t;
+
+static int spec_check(const ro_spec_t *s)
+{
+    /* all members of a group must have one shape (Section 4.3: same type) */
+    for (uint32_t a = 0; a < s->n_layers; ++a) {
+        if (s->group[a] >= s->n_groups) return -1;
+        for (uint32_t b = a + 1; b < s->n_layers; ++b)
+            if (s->group[a] == s->group[b] &&
+                (s->rows[a] != s->rows[b] || s->cols[a] != s->cols[b]))
+                return -2;
+    }
+    return 0;
+}
+
+/*
+ * M[l] (+)= sign_op * T_i(d_i)[l] for one task.  Used by compress (looping
+ * over tasks in the given order, starting from +0), add (sign_op=+1) and
+ * remove (sign_op=-1).  slot_mask (may be NULL) limits the work to chosen
+ * slots so that large cases can be spot-checked.
+ */
+static int accumulate_one(const ro_spec_t *s, int dtype, int sign_op,
+                          uint32_t task_id, uint64_t seed,
+                          const void *const *base, const void *const *task,
+                          float *const *M, const uint8_t *slot_mask)
+{
+    uint32_t L = s->n_layers;
+    uint32_t *src_of_slot = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
+    uint32_t *slot_of_pos = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
+    if (!src_of_slot || !slot_of_pos) { free(src_of_slot); free(slot_of_pos); return -1; }
+    if (ro_task_tables(L, s->group, s->n_groups, s->gflags, seed, task_id,
+                       src_of_slot, slot_of_pos)) {
+        free(src_of_slot); free(slot_of_pos); return -1;
+    }
+    for (uint32_t l = 0; l < L; ++l) {
+        if (slot_mask && !slot_mask[l]) continue;
+        uint32_t rows = s->rows[l], cols = s->cols[l];
+        uint32_t src = src_of_slot[l];
+        int flip = (s->gflags[s->group[l]] & RO_FLIP) != 0;
+        int8_t *sg = (int8_t *)malloc(cols ? cols : 1);
+        if (!sg) { free(src_of_slot); free(slot_of_pos); return -1; }
+        if (flip) ro_sign_row(seed, task_id, l, cols, sg);
+        else memset(sg, 1, cols);
+        const void *wt = task[src];
+        const void *wb = base ? base[src] : NULL;
+        float *m = M[l];
+#pragma omp parallel for schedule(static)
+        for (int64_t r = 0; r < (int64_t)rows; ++r) {
+            for (uint32_t c = 0; c < cols; ++c) {
+                size_t idx = (size_t)r * cols + c;
+                float x = transformed_delta(wt, wb, dtype, idx, sg[c]);
+                m[idx] = sign_op < 0 ? m[idx] - x : m[idx] + x; /* one rounding */
+            }
+        }
+        free(sg);
+    }
+    free(src_of_slot);
+    free(slot_of_pos);
+    return 0;
+}
+
+static ro_spec_t make_spec(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+                           const uint32_t *group, uint32_t n_groups, const uint32_t *gflags)
+{
+    ro_spec_t s;
+    s.n_layers = n_layers; s.rows = rows; s.cols = cols; s.group = group;
+    s.n_groups = n_groups; s.gflags = gflags;
+    return s;
+}
+
+/*
+ * compress (Section 4, first display; Section 4.4 first display):
+ *   M = sum_{i in given order} T_i(W_i - W_0), every slot started from +0.0f.
+ * tasks is a flattened [n_tasks][n_layers] array of host pointers.
+ */
+int ro_compress(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+                const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
+                int dtype, uint32_t n_tasks, const uint32_t *task_ids, const uint64_t *seeds,
+                const void *const *base, const void *const *tasks,
+                float *const *M, const uint8_t *slot_mask)
+{
+    ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
+    int rc = spec_check(&s);
+    if (rc) return rc;
+    for (uint32_t l = 0; l < n_layers; ++l) {
+        if (slot_mask && !slot_mask[l]) continue;
+        size_t n = (size_t)rows[l] * cols[l];
+        for (size_t e = 0; e < n; ++e) M[l][e] = 0.0f;
+    }
+    for (uint32_t i = 0; i < n_tasks; ++i) {
+        rc = accumulate_one(&s, dtype, +1, task_ids[i], seeds[i], base,
+                            tasks + (size_t)i * n_layers, M, slot_mask);
+        if (rc) return rc;
+    }
+    return 0;
+}
+
+/* Model hot swapping (Section 5.7): M <- M + T_j(d_j)  /  M <- M - T_j(d_j). */
+int ro_add_model(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+                 const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
+                 int dtype, uint32_t task_id, uint64_t seed,
+                 const void *const *base, const void *const *task,
+                 float *const *M, const uint8_t *slot_mask)
+{
+    ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
+    int rc = spec_check(&s);
+    if (rc) return rc;
+    return accumulate_one(&s, dtype, +1, task_id, seed, base, task, M, slot_mask);
+}
+
+int ro_remove_model(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+                    const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
+                    int dtype, uint32_t task_id, uint64_t seed,
+                    const void *const *base, const void *const *task,
+                    float *const *M, const uint8_t *slot_mask)
+{
+    ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
+    int rc = spec_check(&s);
+    if (rc) return rc;
+    return accumulate_one(&s, dtype, -1, task_id, seed, base, task, M, slot_mask);
+}
+
+/*
+ * retrieve (Section 4, second display; Section 4.4 second display):
+ *   What_t = W_0 + lambda * T_t^-1(M).
+ * T_t^-1 = P_t^-1 o D_t: undo the flip in M's frame (D is its own inverse),
+ * then send slot l back to the layer it came from.  For layer position p:
+ *   l = sigma_t^-1(p);  out[p][r,c] = fma(lambda, s_t(l,c) * M[l][r,c], W_0[p][r,c]).
+ * out is fp32 or bf16 (round to nearest even).  pos_mask (may be NULL) limits
+ * the work to chosen layer positions.
+ */
+int ro_retrieve(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+                const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
+                int dtype, int out_dtype, uint32_t task_id, uint64_t seed, float lambda,
+                const void *const *base, const float *const *M,
+                void *const *out, const uint8_t *pos_mask)
+{
+    ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
+    int rc = spec_check(&s);
+    if (rc) return rc;
+    uint32_t L = n_layers;
+    uint32_t *src_of_slot = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
+    uint32_t *slot_of_pos = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
+    if (!src_of_slot || !slot_of_pos) { free(src_of_slot); free(slot_of_pos); return -1; }
+    if (ro_task_tables(L, group, n_groups, gflags, seed, task_id, src_of_slot, slot_of_pos)) {
+        free(src_of_slot); free(slot_of_pos); return -1;
+    }
+    for (uint32_t p = 0; p < L; ++p) {
+        if (pos_mask && !pos_mask[p]) continue;
+        uint32_t nr = rows[p], nc = cols[p];
+        uint32_t l = slot_of_pos[p];
+        int flip = (gflags[group[p]] & RO_FLIP) != 0;
+        int8_t *sg = (int8_t *)malloc(nc ? nc : 1);
+        if (!sg) { free(src_of_slot); free(slot_of_pos); return -1; }
+        if (flip) ro_sign_row(seed, task_id, l, nc, sg);
+        else memset(sg, 1, nc);
+        const float *m = M[l];
+        const void *wb = base[p];
+        void *o = out[p];
+#pragma omp parallel for schedule(static)
+        for (int64_t r = 0; r < (int64_t)nr; ++r) {
+            for (uint32_t c = 0; c < nc; ++c) {
+                size_t idx = (size_t)r * nc + c;
+                float mv = m[idx];
+                float signed_m = sg[c] < 0 ? -mv : mv;
+                float y = fmaf(lambda, signed_m, load_elem(wb, dtype, idx));
+                if (out_dtype == RO_BF16) ((uint16_t *)o)[idx] = ro_f32_to_bf16(y);
+                else ((float *)o)[idx] = y;
+            }
+        }
+        free(sg);
+    }
+    free(src_of_slot);
+    free(slot_of_pos);
+    return 0;
+}
+
+int ro_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void ro_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}

@@ -1,0 +1,195 @@
+/*
+ * randes.h -- C ABI of the B200 RanDeS library.
+ *
+ * RanDeS (Randomized Delta Superposition) stores T models fine-tuned from one
+ * base W_0 as W_0 plus ONE superposed delta
+ *
+ *        M = sum_i T_i (W_i - W_0)                       (Section 4, first display)
+ *
+ * where every T_i is a random orthogonal transform fixed by a seed, and brings
+ * one model back on demand as
+ *
+ *        What_t = W_0 + lambda * T_t^-1 (M)              (Section 4, second display)
+ *
+ * T_i is a shuffle of same-shape layers (Section 4.3), a per-column +-1 sign
+ * flip (Section 4.4), or both.  Models are added to and removed from M without
+ * recomputation (Section 5.7).
+ *
+ * General conventions
+ * -------------------
+ * - A model is a list of n_layers row-major tensors [rows, cols]; a 1-D
+ *   parameter is [1, cols].  "Column" = the second, contiguous index.
+ * - Layers with the same `group` id must have the same shape; a group is the
+ *   set of "layers of the same type" that may be shuffled among each other.
+ *   Group members are ordered by layer index.
+ * - Pointer arrays (`base`, `tasks`, `out`) are HOST arrays of DEVICE
+ *   pointers, one per layer, in layer order.  The library copies them; the
+ *   caller may free or reuse the arrays as soon as the call returns.
+ * - All tensor data, M and the workspace are DEVICE memory owned by the
+ *   caller.  The library allocates no device memory and frees nothing it is
+ *   handed.  Weight tensors must be aligned to their element size; 16-byte
+ *   aligned tensors with cols % 4 == 0 take the vectorised path.
+ * - M is one fp32 arena of randes_superposition_bytes() bytes, 256-byte
+ *   aligned; slot l starts at byte randes_layer_offset(plan, l).  M is fp32
+ *   whatever the storage type of the weights.
+ * - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   Calls enqueue work and return; results are ordered on `stream`.  All calls
+ *   on one plan must be issued on one stream or otherwise ordered by the
+ *   caller: they share the plan's device workspace.
+ * - Every entry point returns 0 (RANDES_OK) or a negative randes_status_t;
+ *   randes_last_error() then describes the failure.  Arguments are validated
+ *   before anything is launched; nothing crosses the ABI as an exception.
+ * - Results are deterministic: every output element is written by exactly one
+ *   thread, tasks are summed in plan order, each fp32 operation is rounded
+ *   once (W_i - W_0, then the accumulation; retrieval is one fused
+ *   multiply-add), bf16 conversion is round-to-nearest-even.
+ * - Not thread-safe per plan; distinct plans may be used from distinct threads.
+ */
+#ifndef RANDES_H
+#define RANDES_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct randes_plan_s randes_plan_t; /* opaque, host memory, library-owned */
+
+typedef enum { RANDES_F32 = 0, RANDES_BF16 = 1 } randes_dtype_t;
+
+/* per-group transform flags */
+enum { RANDES_SHUFFLE = 1, RANDES_FLIP = 2 };
+
+typedef struct { uint32_t rows, cols, group; } randes_layer_t;
+typedef struct { uint32_t flags; } randes_group_t;
+
+typedef enum {
+    RANDES_OK = 0,
+    RANDES_INVALID_ARGUMENT = -1,
+    RANDES_SHAPE_MISMATCH = -2,   /* members of one group differ in shape */
+    RANDES_UNKNOWN_TASK = -3,
+    RANDES_DUPLICATE_TASK = -4,
+    RANDES_WORKSPACE_TOO_SMALL = -5,
+    RANDES_UNSUPPORTED_DTYPE = -6,
+    RANDES_MISALIGNED = -7,       /* pointer not aligned to its element size */
+    RANDES_CAPACITY = -8,         /* plan already holds max_tasks tasks */
+    RANDES_CUDA_ERROR = -9,
+    RANDES_OUT_OF_MEMORY = -10    /* host allocation failed */
+} randes_status_t;
+
+/*
+ * Bytes of device workspace a plan over these layers needs for up to max_tasks
+ * registered tasks.  Returns 0 on invalid arguments.  Host-only.
+ */
+size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_layers,
+                                   uint32_t max_tasks);
+
+/*
+ * Build a plan (Sections 4.2-4.4; seeds as in the appendix on the default
+ * experimental setup: one seed per model drives both its shuffle and its sign
+ * matrices).
+ *
+ *   layers[n_layers], groups[n_groups]  host arrays, copied.
+ *   storage_dtype   element type of every W_0 / W_i tensor.
+ *   task_ids/seeds[n_tasks]  the initially registered models, in the order in
+ *                   which compress sums them.  Ids must be distinct.
+ *   max_tasks       capacity of the registry (>= n_tasks, >= 1).
+ *   dev_workspace   device memory, 256-byte aligned, at least
+ *                   randes_plan_workspace_bytes() bytes; used by the plan until
+ *                   randes_plan_destroy.  The layer, tile and permutation
+ *                   tables are copied into it on `stream`.
+ *   out_plan        receives the plan; free with randes_plan_destroy.
+ *
+ * For every registered task and every group with RANDES_SHUFFLE and >= 2
+ * members a permutation sigma is drawn from the task's seed (Fisher-Yates on a
+ * Philox4x32-10 stream); slot k of the shuffled delta holds member sigma(k).
+ * Errors: INVALID_ARGUMENT, SHAPE_MISMATCH, DUPLICATE_TASK,
+ * WORKSPACE_TOO_SMALL, UNSUPPORTED_DTYPE, MISALIGNED, CUDA_ERROR.
+ */
+int randes_plan(const randes_layer_t* layers, uint32_t n_layers,
+                const randes_group_t* groups, uint32_t n_groups,
+                randes_dtype_t storage_dtype,
+                const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
+                uint32_t max_tasks,
+                void* dev_workspace, size_t dev_workspace_bytes, void* stream,
+                randes_plan_t** out_plan);
+
+void randes_plan_destroy(randes_plan_t* plan); /* NULL is allowed; frees host memory only */
+
+/* Size of the fp32 arena M: sum of 4*rows*cols, each slot padded to 256 bytes.
+ * Independent of the number of tasks (Section 4.1: a seed per added model). */
+size_t randes_superposition_bytes(const randes_plan_t* plan);
+
+/* Byte offset of slot `layer` inside M; (size_t)-1 if out of range. */
+size_t randes_layer_offset(const randes_plan_t* plan, uint32_t layer);
+
+uint32_t randes_num_layers(const randes_plan_t* plan);
+uint32_t randes_num_tasks(const randes_plan_t* plan);
+
+/* Copies the registered ids / seeds, in summation order, into host arrays of
+ * randes_num_tasks() entries (either may be NULL). */
+int randes_task_list(const randes_plan_t* plan, uint32_t* task_ids, uint64_t* seeds);
+
+/*
+ * Host copies of one task's layer tables (n_layers entries each, either may be
+ * NULL):  src_of_slot[l] = layer whose delta lands on slot l (sigma);
+ * slot_of_pos[p] = slot holding layer p's delta (sigma^-1).   (Section 4.3)
+ * Errors: UNKNOWN_TASK.
+ */
+int randes_task_tables(const randes_plan_t* plan, uint32_t task_id,
+                       uint32_t* src_of_slot, uint32_t* slot_of_pos);
+
+/*
+ * compress (Section 4, first display; Section 4.4, first display):
+ *   M[l][r,c] = sum over registered tasks i, in plan order, of
+ *               s_i(l,c) * ( W_i[sigma_i(l)][r,c] - W_0[sigma_i(l)][r,c] )
+ * starting from +0.  M is overwritten.
+ *   base[n_layers]             W_0, or NULL: `tasks` then hold the deltas
+ *                              themselves (adapter deltas, Section 5.8).
+ *   tasks[n_tasks * n_layers]  tasks[i*n_layers + l] = layer l of the i-th
+ *                              registered task.
+ * One kernel launch.  Errors: INVALID_ARGUMENT, MISALIGNED, CUDA_ERROR.
+ */
+int randes_compress(randes_plan_t* plan, const void* const* base, const void* const* tasks,
+                    void* M, void* stream);
+
+/*
+ * Model hot swapping (Section 5.7).
+ *   add:     registers (task_id, seed) at the end of the summation order and
+ *            performs  M <- M + T_j(W_j - W_0)  in place.
+ *   remove:  performs  M <- M - T_j(W_j - W_0)  in place and drops the task.
+ *            The library keeps no deltas: the caller passes the same weights
+ *            that were added.  Exact up to one fp32 rounding per element.
+ * base may be NULL (task holds the delta).  One kernel launch each.
+ * Errors: DUPLICATE_TASK, CAPACITY (add); UNKNOWN_TASK (remove);
+ * INVALID_ARGUMENT, MISALIGNED, CUDA_ERROR.
+ */
+int randes_add_model(randes_plan_t* plan, uint32_t task_id, uint64_t seed,
+                     const void* const* base, const void* const* task, void* M, void* stream);
+int randes_remove_model(randes_plan_t* plan, uint32_t task_id,
+                        const void* const* base, const void* const* task, void* M, void* stream);
+
+/*
+ * retrieve (Section 4, second display; Section 4.4, second display):
+ *   out[p][r,c] = fma(lambda, s_t(l,c) * M[l][r,c], W_0[p][r,c]),  l = sigma_t^-1(p)
+ * written as out_dtype (fp32, or bf16 rounded to nearest even).
+ *   base[n_layers], out[n_layers]; out must not alias base or M.
+ * One kernel launch.  Errors: UNKNOWN_TASK, UNSUPPORTED_DTYPE,
+ * INVALID_ARGUMENT, MISALIGNED, CUDA_ERROR.
+ */
+int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda,
+                    randes_dtype_t out_dtype, const void* const* base, const void* M,
+                    void* const* out, void* stream);
+
+/* Number of kernels this library has launched in this process (all plans). */
+uint64_t randes_launch_count(void);
+
+/* Description of the calling thread's most recent failure; never NULL. */
+const char* randes_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RANDES_H */

@@ -133,6 +133,9 @@ def _spec_args(spec):
 def _ptr_array(arrs: Sequence[np.ndarray]):
     pa = (ctypes.c_void_p * max(len(arrs), 1))()
     for i, a in enumerate(arrs):
+        if a is None:   # a layer the masked computation never touches
+            pa[i] = None
+            continue
         assert a.flags["C_CONTIGUOUS"]
         pa[i] = a.ctypes.data
     return pa
@@ -151,6 +154,8 @@ def _check_layers(spec, layers, dtype):
     want = np.uint16 if dtype == BF16 else np.float32
     assert len(layers) == len(rows)
     for l, a in enumerate(layers):
+        if a is None:
+            continue
         assert a.dtype == want, (l, a.dtype, want)
         assert a.size == int(rows[l]) * int(cols[l]), (l, a.shape)
 
@@ -171,8 +176,11 @@ def task_tables(spec, seed: int, task_id: int) -> Tuple[np.ndarray, np.ndarray]:
     return src[:L], pos[:L]
 
 
-def new_superposition(spec) -> List[np.ndarray]:
-    return [np.zeros((int(r), int(c)), dtype=np.float32) for r, c in zip(spec[0], spec[1])]
+def new_superposition(spec, slots=None) -> List[np.ndarray]:
+    """One zeroed fp32 array per slot; with ``slots`` given, only those are allocated."""
+    keep = None if slots is None else set(int(x) for x in slots)
+    return [np.zeros((int(r), int(c)), dtype=np.float32) if keep is None or l in keep else None
+            for l, (r, c) in enumerate(zip(spec[0], spec[1]))]
 
 
 def compress(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
@@ -191,7 +199,7 @@ def compress(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
         _check_layers(spec, t, dtype)
         flat.extend(t)
     if M is None:
-        M = new_superposition(spec)
+        M = new_superposition(spec, slots)
     ids = _u32(task_ids)
     sd = np.ascontiguousarray(np.asarray(seeds, dtype=np.uint64))
     mptr, mkeep = _mask(slots, L)
@@ -240,7 +248,9 @@ def retrieve(spec, dtype: int, out_dtype: int, task_id: int, seed: int, lam: flo
     _check_layers(spec, base, dtype)
     _check_layers(spec, M, F32)
     odt = np.uint16 if out_dtype == BF16 else np.float32
-    out = [np.zeros((int(r), int(c)), dtype=odt) for r, c in zip(spec[0], spec[1])]
+    wanted = None if positions is None else set(int(x) for x in positions)
+    out = [np.zeros((int(r), int(c)), dtype=odt) if wanted is None or l in wanted else None
+           for l, (r, c) in enumerate(zip(spec[0], spec[1]))]
     mptr, mkeep = _mask(positions, L)
     rc = lib.ro_retrieve(*sargs, ctypes.c_int(dtype), ctypes.c_int(out_dtype),
                          ctypes.c_uint32(task_id), ctypes.c_uint64(seed), ctypes.c_float(lam),

@@ -1,0 +1,594 @@
+// Host side of the RanDeS library: the C ABI, the plan (layer table, unit list,
+// per-task permutation tables drawn from seeds), argument validation and the
+// staging of pointer tables into the caller's device workspace.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/randes.h"
+#include "randes_internal.h"
+
+using namespace randes;
+
+namespace {
+
+thread_local std::string g_error;
+std::atomic<uint64_t> g_launches{0};
+
+int fail(int code, const char* fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_error = buf;
+    return code;
+}
+
+int fail_cuda(cudaError_t e, const char* what)
+{
+    return fail(RANDES_CUDA_ERROR, "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
+}
+
+// ---- random streams ----------------------------------------------------------------------
+// Philox4x32-10 as published (SC'11): a 4-word counter is mixed by ten rounds;
+// round = two 32x32->64 products whose halves are crossed with the other two
+// counter words and the key; the key advances by a Weyl sequence per round.
+struct Philox {
+    uint32_t key[2];
+    explicit Philox(uint64_t seed) { key[0] = static_cast<uint32_t>(seed); key[1] = static_cast<uint32_t>(seed >> 32); }
+    void block(uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t out[4]) const
+    {
+        uint32_t x[4] = {a, b, c, d};
+        uint32_t k[2] = {key[0], key[1]};
+        for (int round = 0; round < 10; ++round) {
+            const uint64_t left = 0xD2511F53ull * x[0];
+            const uint64_t right = 0xCD9E8D57ull * x[2];
+            const uint32_t y[4] = {static_cast<uint32_t>(right >> 32) ^ x[1] ^ k[0], static_cast<uint32_t>(right),
+                                   static_cast<uint32_t>(left >> 32) ^ x[3] ^ k[1], static_cast<uint32_t>(left)};
+            std::memcpy(x, y, sizeof x);
+            k[0] += 0x9E3779B9u;
+            k[1] += 0xBB67AE85u;
+        }
+        std::memcpy(out, x, sizeof x);
+    }
+};
+
+// sigma ~ S_G for (task, group): Fisher-Yates from the last position down; the
+// r-th random word of the (group, task) stream picks j in [0, k] as (word*(k+1)) >> 32.
+void draw_sigma(uint64_t seed, uint32_t task_id, uint32_t group, uint32_t G, std::vector<uint32_t>& sigma)
+{
+    sigma.resize(G);
+    for (uint32_t k = 0; k < G; ++k) sigma[k] = k;
+    const Philox rng(seed);
+    uint32_t words[4];
+    uint32_t drawn = 0;
+    for (uint32_t k = G; k > 1; --k) {
+        if ((drawn & 3u) == 0) rng.block(drawn >> 2, group, kTagPerm, task_id, words);
+        const uint32_t word = words[drawn & 3u];
+        ++drawn;
+        const uint32_t j = static_cast<uint32_t>((static_cast<uint64_t>(word) * k) >> 32);
+        std::swap(sigma[k - 1], sigma[j]);
+    }
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct TaskEntry {
+    uint32_t id;
+    uint64_t seed;
+    std::vector<uint32_t> src_of_slot;   // sigma over the whole layer list
+    std::vector<uint32_t> slot_of_pos;   // sigma^-1
+};
+
+struct WorkspaceLayout {
+    size_t layers, units, tasks, src_of_slot, slot_of_pos, base_ptrs, out_ptrs, task_ptrs, total;
+};
+
+WorkspaceLayout layout_workspace(size_t n_layers, size_t n_units, size_t max_tasks)
+{
+    WorkspaceLayout w;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    w.layers = take(n_layers * sizeof(DevLayer));
+    w.units = take(n_units * sizeof(DevUnit));
+    w.tasks = take(max_tasks * sizeof(DevTask));
+    w.src_of_slot = take(max_tasks * n_layers * sizeof(uint32_t));
+    w.slot_of_pos = take(max_tasks * n_layers * sizeof(uint32_t));
+    w.base_ptrs = take(n_layers * sizeof(void*));
+    w.out_ptrs = take(n_layers * sizeof(void*));
+    w.task_ptrs = take(max_tasks * n_layers * sizeof(void*));
+    w.total = off;
+    return w;
+}
+
+// Units in group order; inside a group, all members at one (row block, column
+// chunk) are adjacent, so that tiles of W_0 which several slots read (under a
+// shuffle) are touched close together in time and stay in L2.
+void build_units(const randes_layer_t* layers, uint32_t n_layers, std::vector<DevUnit>& units)
+{
+    units.clear();
+    std::vector<char> done(n_layers, 0);
+    std::vector<uint32_t> members;
+    for (uint32_t first = 0; first < n_layers; ++first) {
+        if (done[first]) continue;
+        members.clear();
+        for (uint32_t l = first; l < n_layers; ++l)
+            if (!done[l] && layers[l].group == layers[first].group) { members.push_back(l); done[l] = 1; }
+        const uint32_t rows = layers[first].rows, cols = layers[first].cols;
+        if (rows == 0 || cols == 0) continue;
+        const uint32_t nb = (cols + kColsPerWarp - 1) / kColsPerWarp;
+        uint32_t nbc = 1;
+        while (nbc < static_cast<uint32_t>(kWarpsPerCta) && nb % (nbc * 2) == 0) nbc *= 2;
+        const uint32_t rows_per_unit = kRowsPerWarp * (kWarpsPerCta / nbc);
+        for (uint32_t r0 = 0; r0 < rows; r0 += rows_per_unit)
+            for (uint32_t cb0 = 0; cb0 < nb; cb0 += nbc)
+                for (uint32_t l : members) {
+                    DevUnit u;
+                    u.layer = l;
+                    u.row0 = r0;
+                    u.nrows = std::min(rows_per_unit, rows - r0);
+                    u.cb0 = static_cast<uint16_t>(cb0);
+                    u.nbc = static_cast<uint16_t>(nbc);
+                    units.push_back(u);
+                }
+    }
+}
+
+int check_layers(const randes_layer_t* layers, uint32_t n_layers)
+{
+    if (!layers || n_layers == 0) return fail(RANDES_INVALID_ARGUMENT, "layers is NULL or empty");
+    for (uint32_t l = 0; l < n_layers; ++l)
+        if (layers[l].cols > 65535u * kColsPerWarp)
+            return fail(RANDES_INVALID_ARGUMENT, "layer %u: cols %u exceeds the supported %u", l, layers[l].cols,
+                        65535u * kColsPerWarp);
+    return RANDES_OK;
+}
+
+}  // namespace
+
+struct randes_plan_s {
+    uint32_t n_layers = 0, n_groups = 0, max_tasks = 0;
+    int storage = RANDES_F32;
+    std::vector<randes_layer_t> layers;
+    std::vector<uint32_t> gflags;
+    std::vector<std::vector<uint32_t>> members;   // per group, in layer order
+    std::vector<DevLayer> dev_layers;
+    std::vector<DevUnit> units;
+    std::vector<size_t> m_off_bytes;
+    size_t m_bytes = 0;
+    std::vector<TaskEntry> tasks;                 // summation order
+    // device side
+    char* ws = nullptr;
+    WorkspaceLayout lay{};
+    int sm_count = 0;
+    int grid_acc = 0;
+    int grid_ret[2] = {0, 0};
+    // host mirrors of what the device pointer tables currently hold
+    std::vector<const void*> h_base, h_out, h_tasks;
+    std::vector<DevTask> h_dev_tasks;
+    bool base_valid = false, out_valid = false;
+    size_t tasks_valid = 0;
+
+    template <typename T> T* dev(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+namespace {
+
+void make_task_tables(const randes_plan_t& p, TaskEntry& t)
+{
+    t.src_of_slot.resize(p.n_layers);
+    t.slot_of_pos.resize(p.n_layers);
+    for (uint32_t l = 0; l < p.n_layers; ++l) t.src_of_slot[l] = t.slot_of_pos[l] = l;
+    std::vector<uint32_t> sigma;
+    for (uint32_t g = 0; g < p.n_groups; ++g) {
+        const std::vector<uint32_t>& mem = p.members[g];
+        if (mem.size() < 2 || !(p.gflags[g] & RANDES_SHUFFLE)) continue;
+        draw_sigma(t.seed, t.id, g, static_cast<uint32_t>(mem.size()), sigma);
+        for (size_t k = 0; k < mem.size(); ++k) {
+            t.src_of_slot[mem[k]] = mem[sigma[k]];     // slot k receives member sigma(k)
+            t.slot_of_pos[mem[sigma[k]]] = mem[k];
+        }
+    }
+}
+
+int find_task(const randes_plan_t& p, uint32_t id)
+{
+    for (size_t i = 0; i < p.tasks.size(); ++i)
+        if (p.tasks[i].id == id) return static_cast<int>(i);
+    return -1;
+}
+
+// copy task rows [first, end) (descriptors + both tables) to the device
+int upload_task_rows(randes_plan_t& p, size_t first, cudaStream_t s)
+{
+    const size_t L = p.n_layers;
+    p.h_dev_tasks.resize(p.max_tasks);
+    for (size_t i = first; i < p.tasks.size(); ++i) {
+        const TaskEntry& t = p.tasks[i];
+        DevTask d;
+        d.id = t.id;
+        d.key0 = static_cast<uint32_t>(t.seed);
+        d.key1 = static_cast<uint32_t>(t.seed >> 32);
+        d.pad = 0;
+        p.h_dev_tasks[i] = d;
+        cudaError_t e = cudaMemcpyAsync(p.dev<uint32_t>(p.lay.src_of_slot) + i * L, t.src_of_slot.data(),
+                                        L * sizeof(uint32_t), cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(p.dev<uint32_t>(p.lay.slot_of_pos) + i * L, t.slot_of_pos.data(), L * sizeof(uint32_t),
+                                cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return fail_cuda(e, "copy of task tables");
+    }
+    if (first < p.tasks.size()) {
+        cudaError_t e = cudaMemcpyAsync(p.dev<DevTask>(p.lay.tasks) + first, p.h_dev_tasks.data() + first,
+                                        (p.tasks.size() - first) * sizeof(DevTask), cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return fail_cuda(e, "copy of task descriptors");
+    }
+    return RANDES_OK;
+}
+
+int check_ptrs(const randes_plan_t& p, const void* const* ptrs, const char* what, size_t elem, bool allow_null_array)
+{
+    if (!ptrs) return allow_null_array ? RANDES_OK : fail(RANDES_INVALID_ARGUMENT, "%s is NULL", what);
+    for (uint32_t l = 0; l < p.n_layers; ++l) {
+        const bool empty = p.layers[l].rows == 0 || p.layers[l].cols == 0;
+        if (!ptrs[l] && !empty) return fail(RANDES_INVALID_ARGUMENT, "%s[%u] is NULL", what, l);
+        if (reinterpret_cast<uintptr_t>(ptrs[l]) % elem)
+            return fail(RANDES_MISALIGNED, "%s[%u] = %p is not aligned to %zu bytes", what, l, ptrs[l], elem);
+    }
+    return RANDES_OK;
+}
+
+// bring a device pointer table up to date; skips the copy when nothing changed
+int stage_ptrs(randes_plan_t& p, std::vector<const void*>& mirror, bool& valid, size_t dev_off, const void* const* ptrs,
+               cudaStream_t s)
+{
+    const size_t L = p.n_layers;
+    if (valid && std::memcmp(mirror.data(), ptrs, L * sizeof(void*)) == 0) return RANDES_OK;
+    mirror.assign(ptrs, ptrs + L);
+    valid = true;
+    cudaError_t e = cudaMemcpyAsync(p.ws + dev_off, mirror.data(), L * sizeof(void*), cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) { valid = false; return fail_cuda(e, "copy of pointer table"); }
+    return RANDES_OK;
+}
+
+int stage_task_ptrs(randes_plan_t& p, const void* const* ptrs, size_t n_tasks, cudaStream_t s)
+{
+    const size_t n = n_tasks * p.n_layers;
+    if (p.tasks_valid == n && std::memcmp(p.h_tasks.data(), ptrs, n * sizeof(void*)) == 0) return RANDES_OK;
+    if (p.h_tasks.size() < n) p.h_tasks.resize(static_cast<size_t>(p.max_tasks) * p.n_layers);
+    std::memcpy(p.h_tasks.data(), ptrs, n * sizeof(void*));
+    p.tasks_valid = n;
+    cudaError_t e = cudaMemcpyAsync(p.ws + p.lay.task_ptrs, p.h_tasks.data(), n * sizeof(void*), cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) { p.tasks_valid = 0; return fail_cuda(e, "copy of task pointer table"); }
+    return RANDES_OK;
+}
+
+size_t elem_size(int dtype) { return dtype == RANDES_BF16 ? 2 : 4; }
+
+int check_m(const void* M)
+{
+    if (!M) return fail(RANDES_INVALID_ARGUMENT, "M is NULL");
+    if (reinterpret_cast<uintptr_t>(M) % 256) return fail(RANDES_MISALIGNED, "M = %p is not 256-byte aligned", M);
+    return RANDES_OK;
+}
+
+int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_from_m, bool negate,
+                   const void* const* base, const void* const* task_ptrs, void* M, cudaStream_t s)
+{
+    int rc;
+    if (base && (rc = stage_ptrs(p, p.h_base, p.base_valid, p.lay.base_ptrs, base, s))) return rc;
+    if ((rc = stage_task_ptrs(p, task_ptrs, n_rows, s))) return rc;
+    AccumulateArgs a;
+    a.layers = p.dev<DevLayer>(p.lay.layers);
+    a.units = p.dev<DevUnit>(p.lay.units);
+    a.n_units = static_cast<uint32_t>(p.units.size());
+    a.n_layers = p.n_layers;
+    a.src_of_slot = p.dev<uint32_t>(p.lay.src_of_slot) + first_row * p.n_layers;
+    a.tasks = p.dev<DevTask>(p.lay.tasks) + first_row;
+    a.n_tasks = static_cast<uint32_t>(n_rows);
+    a.init_from_m = init_from_m;
+    a.negate = negate;
+    a.has_base = base != nullptr;
+    a.base = p.dev<const void*>(p.lay.base_ptrs);
+    a.task_ptrs = p.dev<const void*>(p.lay.task_ptrs);
+    a.M = static_cast<float*>(M);
+    if (a.n_units == 0) return RANDES_OK;
+    const int grid = std::min<int>(p.grid_acc, static_cast<int>(a.n_units));
+    const int e = launch_accumulate(p.storage, a, grid, s);
+    if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the accumulate kernel");
+    ++g_launches;
+    return RANDES_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* randes_last_error(void) { return g_error.c_str(); }
+
+uint64_t randes_launch_count(void) { return g_launches.load(); }
+
+size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_layers, uint32_t max_tasks)
+{
+    if (check_layers(layers, n_layers) || max_tasks == 0) return 0;
+    std::vector<DevUnit> units;
+    build_units(layers, n_layers, units);
+    return layout_workspace(n_layers, units.size(), max_tasks).total;
+}
+
+int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_group_t* groups, uint32_t n_groups,
+                randes_dtype_t storage_dtype, const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
+                uint32_t max_tasks, void* dev_workspace, size_t dev_workspace_bytes, void* stream,
+                randes_plan_t** out_plan)
+{
+    if (!out_plan) return fail(RANDES_INVALID_ARGUMENT, "out_plan is NULL");
+    *out_plan = nullptr;
+    int rc = check_layers(layers, n_layers);
+    if (rc) return rc;
+    if (!groups || n_groups == 0) return fail(RANDES_INVALID_ARGUMENT, "groups is NULL or empty");
+    if (storage_dtype != RANDES_F32 && storage_dtype != RANDES_BF16)
+        return fail(RANDES_UNSUPPORTED_DTYPE, "storage dtype %d is not supported", static_cast<int>(storage_dtype));
+    if (max_tasks == 0 || n_tasks > max_tasks)
+        return fail(RANDES_INVALID_ARGUMENT, "max_tasks = %u must be >= max(1, n_tasks = %u)", max_tasks, n_tasks);
+    if (n_tasks && (!task_ids || !seeds)) return fail(RANDES_INVALID_ARGUMENT, "task_ids / seeds is NULL");
+    for (uint32_t g = 0; g < n_groups; ++g)
+        if (groups[g].flags & ~static_cast<uint32_t>(RANDES_SHUFFLE | RANDES_FLIP))
+            return fail(RANDES_INVALID_ARGUMENT, "group %u: unknown flag bits 0x%x", g, groups[g].flags);
+    for (uint32_t i = 0; i < n_tasks; ++i)
+        for (uint32_t j = 0; j < i; ++j)
+            if (task_ids[i] == task_ids[j]) return fail(RANDES_DUPLICATE_TASK, "task id %u appears twice", task_ids[i]);
+
+    randes_plan_t* p = new (std::nothrow) randes_plan_t;
+    if (!p) return fail(RANDES_OUT_OF_MEMORY, "host allocation failed");
+    try {
+        p->n_layers = n_layers;
+        p->n_groups = n_groups;
+        p->max_tasks = max_tasks;
+        p->storage = storage_dtype;
+        p->layers.assign(layers, layers + n_layers);
+        p->gflags.resize(n_groups);
+        for (uint32_t g = 0; g < n_groups; ++g) p->gflags[g] = groups[g].flags;
+        p->members.assign(n_groups, {});
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            if (layers[l].group >= n_groups) {
+                delete p;
+                return fail(RANDES_INVALID_ARGUMENT, "layer %u: group %u out of range (n_groups = %u)", l, layers[l].group,
+                            n_groups);
+            }
+            const std::vector<uint32_t>& mem = p->members[layers[l].group];
+            if (!mem.empty() && (layers[mem[0]].rows != layers[l].rows || layers[mem[0]].cols != layers[l].cols)) {
+                delete p;
+                return fail(RANDES_SHAPE_MISMATCH, "group %u: layer %u is %ux%u but layer %u is %ux%u", layers[l].group, l,
+                            layers[l].rows, layers[l].cols, mem[0], layers[mem[0]].rows, layers[mem[0]].cols);
+            }
+            p->members[layers[l].group].push_back(l);
+        }
+        p->dev_layers.resize(n_layers);
+        p->m_off_bytes.resize(n_layers);
+        size_t off = 0;
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            const uint32_t g = layers[l].group;
+            const std::vector<uint32_t>& mem = p->members[g];
+            DevLayer d;
+            d.m_off = off / sizeof(float);
+            d.rows = layers[l].rows;
+            d.cols = layers[l].cols;
+            d.flags = (p->gflags[g] & RANDES_FLIP ? kFlagFlip : 0u) |
+                      ((p->gflags[g] & RANDES_SHUFFLE) && mem.size() >= 2 ? kFlagShuffle : 0u);
+            d.group = g;
+            d.member = static_cast<uint32_t>(std::find(mem.begin(), mem.end(), l) - mem.begin());
+            d.group_size = static_cast<uint32_t>(mem.size());
+            p->dev_layers[l] = d;
+            p->m_off_bytes[l] = off;
+            off = align_up(off + static_cast<size_t>(layers[l].rows) * layers[l].cols * sizeof(float), 256);
+        }
+        p->m_bytes = off;
+        build_units(layers, n_layers, p->units);
+        p->tasks.resize(n_tasks);
+        for (uint32_t i = 0; i < n_tasks; ++i) {
+            p->tasks[i].id = task_ids[i];
+            p->tasks[i].seed = seeds[i];
+            make_task_tables(*p, p->tasks[i]);
+        }
+        p->lay = layout_workspace(n_layers, p->units.size(), max_tasks);
+    } catch (const std::bad_alloc&) {
+        delete p;
+        return fail(RANDES_OUT_OF_MEMORY, "host allocation failed");
+    }
+
+    if (dev_workspace) {
+        // A plan without a workspace is host-only: tables and sizes can be
+        // queried, the compute entry points refuse to run.
+        if (reinterpret_cast<uintptr_t>(dev_workspace) % 256) {
+            delete p;
+            return fail(RANDES_MISALIGNED, "dev_workspace = %p is not 256-byte aligned", dev_workspace);
+        }
+        if (dev_workspace_bytes < p->lay.total) {
+            const size_t need = p->lay.total;
+            delete p;
+            return fail(RANDES_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, plan needs %zu", dev_workspace_bytes, need);
+        }
+        p->ws = static_cast<char*>(dev_workspace);
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) { delete p; return fail_cuda(e, "device query"); }
+        const int occ_acc = accumulate_ctas_per_sm(p->storage);
+        const int occ_r0 = retrieve_ctas_per_sm(p->storage, RANDES_F32);
+        const int occ_r1 = retrieve_ctas_per_sm(p->storage, RANDES_BF16);
+        if (occ_acc <= 0 || occ_r0 <= 0 || occ_r1 <= 0) {
+            delete p;
+            return fail(RANDES_CUDA_ERROR, "kernels are not loadable on this device (built for sm_100a)");
+        }
+        p->grid_acc = p->sm_count * occ_acc;
+        p->grid_ret[0] = p->sm_count * occ_r0;
+        p->grid_ret[1] = p->sm_count * occ_r1;
+        e = cudaMemcpyAsync(p->ws + p->lay.layers, p->dev_layers.data(), n_layers * sizeof(DevLayer),
+                            cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess && !p->units.empty())
+            e = cudaMemcpyAsync(p->ws + p->lay.units, p->units.data(), p->units.size() * sizeof(DevUnit),
+                                cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) { delete p; return fail_cuda(e, "copy of plan tables"); }
+        if ((rc = upload_task_rows(*p, 0, s))) { delete p; return rc; }
+    }
+    *out_plan = p;
+    return RANDES_OK;
+}
+
+void randes_plan_destroy(randes_plan_t* plan) { delete plan; }
+
+size_t randes_superposition_bytes(const randes_plan_t* plan) { return plan ? plan->m_bytes : 0; }
+
+size_t randes_layer_offset(const randes_plan_t* plan, uint32_t layer)
+{
+    if (!plan || layer >= plan->n_layers) return static_cast<size_t>(-1);
+    return plan->m_off_bytes[layer];
+}
+
+uint32_t randes_num_layers(const randes_plan_t* plan) { return plan ? plan->n_layers : 0; }
+uint32_t randes_num_tasks(const randes_plan_t* plan) { return plan ? static_cast<uint32_t>(plan->tasks.size()) : 0; }
+
+int randes_task_list(const randes_plan_t* plan, uint32_t* task_ids, uint64_t* seeds)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    for (size_t i = 0; i < plan->tasks.size(); ++i) {
+        if (task_ids) task_ids[i] = plan->tasks[i].id;
+        if (seeds) seeds[i] = plan->tasks[i].seed;
+    }
+    return RANDES_OK;
+}
+
+int randes_task_tables(const randes_plan_t* plan, uint32_t task_id, uint32_t* src_of_slot, uint32_t* slot_of_pos)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    const int i = find_task(*plan, task_id);
+    if (i < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_id);
+    const TaskEntry& t = plan->tasks[i];
+    if (src_of_slot) std::memcpy(src_of_slot, t.src_of_slot.data(), plan->n_layers * sizeof(uint32_t));
+    if (slot_of_pos) std::memcpy(slot_of_pos, t.slot_of_pos.data(), plan->n_layers * sizeof(uint32_t));
+    return RANDES_OK;
+}
+
+int randes_compress(randes_plan_t* plan, const void* const* base, const void* const* tasks, void* M, void* stream)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
+    int rc;
+    if ((rc = check_m(M))) return rc;
+    if (plan->tasks.empty()) return fail(RANDES_INVALID_ARGUMENT, "no task is registered");
+    if (!tasks) return fail(RANDES_INVALID_ARGUMENT, "tasks is NULL");
+    const size_t es = elem_size(plan->storage);
+    if ((rc = check_ptrs(*plan, base, "base", es, true))) return rc;
+    for (size_t i = 0; i < plan->tasks.size(); ++i)
+        if ((rc = check_ptrs(*plan, tasks + i * plan->n_layers, "tasks", es, false))) return rc;
+    return run_accumulate(*plan, 0, plan->tasks.size(), false, false, base, tasks, M, static_cast<cudaStream_t>(stream));
+}
+
+int randes_add_model(randes_plan_t* plan, uint32_t task_id, uint64_t seed, const void* const* base,
+                     const void* const* task, void* M, void* stream)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
+    int rc;
+    if ((rc = check_m(M))) return rc;
+    if (find_task(*plan, task_id) >= 0) return fail(RANDES_DUPLICATE_TASK, "task id %u is already registered", task_id);
+    if (plan->tasks.size() >= plan->max_tasks)
+        return fail(RANDES_CAPACITY, "plan already holds max_tasks = %u tasks", plan->max_tasks);
+    const size_t es = elem_size(plan->storage);
+    if ((rc = check_ptrs(*plan, base, "base", es, true))) return rc;
+    if ((rc = check_ptrs(*plan, task, "task", es, false))) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    TaskEntry t;
+    t.id = task_id;
+    t.seed = seed;
+    try {
+        make_task_tables(*plan, t);
+        plan->tasks.push_back(std::move(t));
+    } catch (const std::bad_alloc&) {
+        return fail(RANDES_OUT_OF_MEMORY, "host allocation failed");
+    }
+    const size_t row = plan->tasks.size() - 1;
+    if ((rc = upload_task_rows(*plan, row, s)) ||
+        (rc = run_accumulate(*plan, row, 1, true, false, base, task, M, s))) {
+        plan->tasks.pop_back();
+        return rc;
+    }
+    return RANDES_OK;
+}
+
+int randes_remove_model(randes_plan_t* plan, uint32_t task_id, const void* const* base, const void* const* task,
+                        void* M, void* stream)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
+    int rc;
+    if ((rc = check_m(M))) return rc;
+    const int row = find_task(*plan, task_id);
+    if (row < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_id);
+    const size_t es = elem_size(plan->storage);
+    if ((rc = check_ptrs(*plan, base, "base", es, true))) return rc;
+    if ((rc = check_ptrs(*plan, task, "task", es, false))) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((rc = run_accumulate(*plan, row, 1, true, true, base, task, M, s))) return rc;
+    // close the gap in the registry; later rows move up one place on the device too
+    plan->tasks.erase(plan->tasks.begin() + row);
+    return upload_task_rows(*plan, row, s);
+}
+
+int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
+                    const void* const* base, const void* M, void* const* out, void* stream)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
+    if (out_dtype != RANDES_F32 && out_dtype != RANDES_BF16)
+        return fail(RANDES_UNSUPPORTED_DTYPE, "output dtype %d is not supported", static_cast<int>(out_dtype));
+    int rc;
+    if ((rc = check_m(M))) return rc;
+    const int row = find_task(*plan, task_id);
+    if (row < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_id);
+    if ((rc = check_ptrs(*plan, base, "base", elem_size(plan->storage), false))) return rc;
+    if ((rc = check_ptrs(*plan, const_cast<const void* const*>(out), "out", elem_size(out_dtype), false))) return rc;
+    const char* m_lo = static_cast<const char*>(M);
+    const char* m_hi = m_lo + plan->m_bytes;
+    for (uint32_t l = 0; l < plan->n_layers; ++l) {
+        const char* o = static_cast<const char*>(out[l]);
+        if (out[l] && (out[l] == base[l] || (o >= m_lo && o < m_hi)))
+            return fail(RANDES_INVALID_ARGUMENT, "out[%u] aliases base or M", l);
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((rc = stage_ptrs(*plan, plan->h_base, plan->base_valid, plan->lay.base_ptrs, base, s))) return rc;
+    if ((rc = stage_ptrs(*plan, plan->h_out, plan->out_valid, plan->lay.out_ptrs, const_cast<const void* const*>(out), s)))
+        return rc;
+    RetrieveArgs a;
+    a.layers = plan->dev<DevLayer>(plan->lay.layers);
+    a.units = plan->dev<DevUnit>(plan->lay.units);
+    a.n_units = static_cast<uint32_t>(plan->units.size());
+    a.n_layers = plan->n_layers;
+    a.slot_of_pos = plan->dev<uint32_t>(plan->lay.slot_of_pos) + static_cast<size_t>(row) * plan->n_layers;
+    a.base = plan->dev<const void*>(plan->lay.base_ptrs);
+    a.out = plan->dev<void*>(plan->lay.out_ptrs);
+    a.M = static_cast<const float*>(M);
+    a.task.id = plan->tasks[row].id;
+    a.task.key0 = static_cast<uint32_t>(plan->tasks[row].seed);
+    a.task.key1 = static_cast<uint32_t>(plan->tasks[row].seed >> 32);
+    a.task.pad = 0;
+    a.lambda = lambda;
+    if (a.n_units == 0) return RANDES_OK;
+    const int grid = std::min<int>(plan->grid_ret[out_dtype], static_cast<int>(a.n_units));
+    const int e = launch_retrieve(plan->storage, out_dtype, a, grid, s);
+    if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the retrieve kernel");
+    ++g_launches;
+    return RANDES_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,86 @@
+// Structures shared by the host side (plan, C ABI) and the kernels of the
+// RanDeS library.  Not part of the public interface.
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+
+namespace randes {
+
+constexpr uint32_t kFlagShuffle = 1u;   // layer may move inside its group for some task
+constexpr uint32_t kFlagFlip = 2u;      // per-column sign flip on this slot
+
+constexpr int kWarpsPerCta = 8;
+constexpr int kThreadsPerCta = kWarpsPerCta * 32;
+constexpr int kColsPerWarp = 128;       // one Philox block of sign bits; 4 columns per lane
+constexpr int kRowsPerWarp = 16;        // rows one warp walks per unit
+constexpr int kTaskChunk = 32;          // tasks whose pointers / sign blocks a warp holds at once
+constexpr uint32_t kTagSign = 0x5349474Eu;  // counter word 2 of the sign stream ("SIGN")
+constexpr uint32_t kTagPerm = 0x5045524Du;  // counter word 2 of the permutation stream ("PERM")
+
+// One layer of the model == one slot of M (same index space).
+struct DevLayer {
+    unsigned long long m_off;  // first element of this slot in the fp32 arena M
+    uint32_t rows, cols;
+    uint32_t flags;            // kFlagShuffle | kFlagFlip, already resolved (shuffle only if group size >= 2)
+    uint32_t group;
+    uint32_t member;           // index of this layer inside its group
+    uint32_t group_size;
+};
+static_assert(sizeof(DevLayer) == 32, "DevLayer layout");
+
+// One unit of work for a CTA: `nrows` rows x `nbc` column blocks of 128 columns
+// of one layer.  Warp w owns column block cb0 + (w % nbc) and the rows
+// row0 + (w / nbc), stepping by kWarpsPerCta / nbc.
+struct DevUnit {
+    uint32_t layer;
+    uint32_t row0;
+    uint32_t nrows;
+    uint16_t cb0;
+    uint16_t nbc;              // 1, 2, 4 or 8
+};
+static_assert(sizeof(DevUnit) == 16, "DevUnit layout");
+
+struct DevTask {
+    uint32_t id;
+    uint32_t key0, key1;       // low / high half of the 64-bit seed
+    uint32_t pad;
+};
+
+struct RetrieveArgs {
+    const DevLayer* layers;
+    const DevUnit* units;
+    uint32_t n_units;
+    uint32_t n_layers;
+    const uint32_t* slot_of_pos;   // this task's sigma^-1, n_layers entries
+    const void* const* base;       // device array of n_layers device pointers
+    void* const* out;
+    const float* M;
+    DevTask task;
+    float lambda;
+};
+
+struct AccumulateArgs {
+    const DevLayer* layers;
+    const DevUnit* units;
+    uint32_t n_units;
+    uint32_t n_layers;
+    const uint32_t* src_of_slot;   // rows of sigma, one per task to sum, n_layers entries each
+    const DevTask* tasks;          // matching task descriptors
+    uint32_t n_tasks;
+    uint32_t init_from_m;          // 0: start from +0 (compress); 1: start from M (add / remove)
+    uint32_t negate;               // 1: subtract (remove)
+    uint32_t has_base;             // 0: task tensors already hold deltas
+    const void* const* base;       // device array [n_layers]
+    const void* const* task_ptrs;  // device array [n_tasks][n_layers]
+    float* M;
+};
+
+// Launchers (randes_kernels.cu).  Return a cudaError_t as int.
+int launch_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, int grid, void* stream);
+int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void* stream);
+// Resident CTAs per SM of each kernel (for sizing persistent grids).
+int retrieve_ctas_per_sm(int storage_dtype, int out_dtype);
+int accumulate_ctas_per_sm(int storage_dtype);
+
+}  // namespace randes

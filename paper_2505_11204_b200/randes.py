@@ -1,0 +1,327 @@
+"""Thin binding over the CUDA C-ABI library (``include/randes.h``).
+
+Argument marshalling only: every step of the path runs in the library's
+kernels.  PyTorch supplies device memory and the stream.  There is no CPU
+fallback: if the compiled library is missing, loading raises.
+
+Two levels:
+
+* module functions ``randes_plan``, ``randes_compress``, ``randes_add_model``,
+  ``randes_remove_model``, ``randes_retrieve`` ... with the C names, taking
+  ctypes pointer arrays / raw addresses;
+* ``Plan``: the same calls on lists of torch CUDA tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+F32 = 0
+BF16 = 1
+SHUFFLE = 1
+FLIP = 2
+
+OK = 0
+INVALID_ARGUMENT = -1
+SHAPE_MISMATCH = -2
+UNKNOWN_TASK = -3
+DUPLICATE_TASK = -4
+WORKSPACE_TOO_SMALL = -5
+UNSUPPORTED_DTYPE = -6
+MISALIGNED = -7
+CAPACITY = -8
+CUDA_ERROR = -9
+OUT_OF_MEMORY = -10
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librandes.so")
+_lib = None
+
+
+class RandesError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__("randes error %d: %s" % (code, message))
+        self.code = code
+
+
+class Layer(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_uint32), ("cols", ctypes.c_uint32), ("group", ctypes.c_uint32)]
+
+
+class Group(ctypes.Structure):
+    _fields_ = [("flags", ctypes.c_uint32)]
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "%s is missing: build it with `python -m paper_2505_11204_b200.build` "
+                "(there is no CPU fallback)" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, u32, u64, sz = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_size_t
+        L.randes_plan_workspace_bytes.argtypes = [vp, u32, u32]
+        L.randes_plan_workspace_bytes.restype = sz
+        L.randes_plan.argtypes = [vp, u32, vp, u32, ctypes.c_int, vp, vp, u32, u32, vp, sz, vp,
+                                  ctypes.POINTER(vp)]
+        L.randes_plan.restype = ctypes.c_int
+        L.randes_plan_destroy.argtypes = [vp]
+        L.randes_plan_destroy.restype = None
+        L.randes_superposition_bytes.argtypes = [vp]
+        L.randes_superposition_bytes.restype = sz
+        L.randes_layer_offset.argtypes = [vp, u32]
+        L.randes_layer_offset.restype = sz
+        L.randes_num_layers.argtypes = [vp]
+        L.randes_num_layers.restype = u32
+        L.randes_num_tasks.argtypes = [vp]
+        L.randes_num_tasks.restype = u32
+        L.randes_task_list.argtypes = [vp, vp, vp]
+        L.randes_task_list.restype = ctypes.c_int
+        L.randes_task_tables.argtypes = [vp, u32, vp, vp]
+        L.randes_task_tables.restype = ctypes.c_int
+        L.randes_compress.argtypes = [vp, vp, vp, vp, vp]
+        L.randes_compress.restype = ctypes.c_int
+        L.randes_add_model.argtypes = [vp, u32, u64, vp, vp, vp, vp]
+        L.randes_add_model.restype = ctypes.c_int
+        L.randes_remove_model.argtypes = [vp, u32, vp, vp, vp, vp]
+        L.randes_remove_model.restype = ctypes.c_int
+        L.randes_retrieve.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
+        L.randes_retrieve.restype = ctypes.c_int
+        L.randes_launch_count.argtypes = []
+        L.randes_launch_count.restype = u64
+        L.randes_last_error.argtypes = []
+        L.randes_last_error.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+EXPORTS = [
+    "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_superposition_bytes",
+    "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
+    "randes_task_tables", "randes_compress", "randes_add_model", "randes_remove_model",
+    "randes_retrieve", "randes_launch_count", "randes_last_error",
+]
+
+
+def randes_last_error() -> str:
+    return lib().randes_last_error().decode()
+
+
+def _check(rc: int) -> None:
+    if rc != OK:
+        raise RandesError(rc, randes_last_error())
+
+
+def _addr(x) -> Optional[int]:
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, ctypes.Array):
+        return ctypes.addressof(x)
+    return int(x.data_ptr())  # torch tensor
+
+
+# ---- C-named entry points (raw addresses / ctypes arrays) ----------------------------------
+def randes_plan_workspace_bytes(layers, n_layers: int, max_tasks: int) -> int:
+    return int(lib().randes_plan_workspace_bytes(_addr(layers), n_layers, max_tasks))
+
+
+def randes_plan(layers, n_layers, groups, n_groups, storage_dtype, task_ids, seeds, n_tasks, max_tasks,
+                dev_workspace, dev_workspace_bytes, stream) -> int:
+    """Returns the plan handle (an address); raises RandesError on failure."""
+    out = ctypes.c_void_p()
+    _check(lib().randes_plan(_addr(layers), n_layers, _addr(groups), n_groups, storage_dtype,
+                             _addr(task_ids), _addr(seeds), n_tasks, max_tasks, _addr(dev_workspace),
+                             dev_workspace_bytes, stream, ctypes.byref(out)))
+    return out.value
+
+
+def randes_plan_destroy(plan) -> None:
+    lib().randes_plan_destroy(plan)
+
+
+def randes_superposition_bytes(plan) -> int:
+    return int(lib().randes_superposition_bytes(plan))
+
+
+def randes_layer_offset(plan, layer: int) -> int:
+    return int(lib().randes_layer_offset(plan, layer))
+
+
+def randes_num_layers(plan) -> int:
+    return int(lib().randes_num_layers(plan))
+
+
+def randes_num_tasks(plan) -> int:
+    return int(lib().randes_num_tasks(plan))
+
+
+def randes_compress(plan, base, tasks, M, stream) -> None:
+    _check(lib().randes_compress(plan, _addr(base), _addr(tasks), _addr(M), stream))
+
+
+def randes_add_model(plan, task_id, seed, base, task, M, stream) -> None:
+    _check(lib().randes_add_model(plan, task_id, seed, _addr(base), _addr(task), _addr(M), stream))
+
+
+def randes_remove_model(plan, task_id, base, task, M, stream) -> None:
+    _check(lib().randes_remove_model(plan, task_id, _addr(base), _addr(task), _addr(M), stream))
+
+
+def randes_retrieve(plan, task_id, lam, out_dtype, base, M, out, stream) -> None:
+    _check(lib().randes_retrieve(plan, task_id, lam, out_dtype, _addr(base), _addr(M), _addr(out), stream))
+
+
+def randes_launch_count() -> int:
+    return int(lib().randes_launch_count())
+
+
+def ptr_array(tensors: Sequence) -> ctypes.Array:
+    """Host array of device addresses, one per tensor (nested lists are flattened)."""
+    flat = []
+    for t in tensors:
+        if isinstance(t, (list, tuple)):
+            flat.extend(t)
+        else:
+            flat.append(t)
+    arr = (ctypes.c_void_p * max(len(flat), 1))()
+    for i, t in enumerate(flat):
+        arr[i] = None if t is None else (t if isinstance(t, int) else int(t.data_ptr()))
+    return arr
+
+
+def _as_ptrs(x):
+    if x is None or isinstance(x, ctypes.Array):
+        return x
+    return ptr_array(x)
+
+
+# ---- convenience object over torch tensors --------------------------------------------------
+class Plan:
+    """A plan plus the device workspace it lives in.
+
+    ``rows, cols, group`` describe the layers, ``gflags`` the groups (see
+    ``include/randes.h``).  Tensors passed to the methods are torch CUDA tensors
+    of the storage dtype (float32 or bfloat16), one per layer.
+    """
+
+    def __init__(self, rows, cols, group, gflags, storage: int = F32, task_ids=(), seeds=(),
+                 max_tasks: Optional[int] = None, device="cuda", host_only: bool = False):
+        n_layers, n_groups = len(rows), len(gflags)
+        self._layers = (Layer * max(n_layers, 1))()
+        for l in range(n_layers):
+            self._layers[l] = Layer(int(rows[l]), int(cols[l]), int(group[l]))
+        self._groups = (Group * max(n_groups, 1))()
+        for g in range(n_groups):
+            self._groups[g] = Group(int(gflags[g]))
+        n_tasks = len(task_ids)
+        if max_tasks is None:
+            max_tasks = max(1, n_tasks + 8)
+        ids = (ctypes.c_uint32 * max(n_tasks, 1))(*[int(t) for t in task_ids])
+        sds = (ctypes.c_uint64 * max(n_tasks, 1))(*[int(s) for s in seeds])
+        self.n_layers = n_layers
+        self.rows, self.cols = [int(r) for r in rows], [int(c) for c in cols]
+        self.storage = storage
+        self.handle = None
+        self.workspace = None
+        self.device = device
+        ws_ptr, ws_bytes, stream = None, 0, None
+        if not host_only:
+            import torch
+
+            ws_bytes = randes_plan_workspace_bytes(self._layers, n_layers, max_tasks)
+            if ws_bytes == 0:
+                raise RandesError(INVALID_ARGUMENT, randes_last_error())
+            self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+            ws_ptr = self.workspace.data_ptr()
+            stream = self._stream()
+        self.handle = randes_plan(self._layers, n_layers, self._groups, n_groups, storage, ids, sds, n_tasks,
+                                  max_tasks, ws_ptr, ws_bytes, stream)
+        self.m_bytes = randes_superposition_bytes(self.handle)
+        self.offsets = [randes_layer_offset(self.handle, l) for l in range(n_layers)]
+
+    @classmethod
+    def from_workload(cls, w, **kw) -> "Plan":
+        kw.setdefault("task_ids", w.task_ids)
+        kw.setdefault("seeds", w.seeds)
+        return cls(w.rows, w.cols, w.group, w.gflags, storage=w.storage, **kw)
+
+    def _stream(self):
+        import torch
+
+        return torch.cuda.current_stream(self.device).cuda_stream
+
+    def close(self) -> None:
+        if self.handle is not None:
+            randes_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- queries
+    @property
+    def n_tasks(self) -> int:
+        return randes_num_tasks(self.handle)
+
+    def task_list(self):
+        n = self.n_tasks
+        ids = (ctypes.c_uint32 * max(n, 1))()
+        sds = (ctypes.c_uint64 * max(n, 1))()
+        _check(lib().randes_task_list(self.handle, ctypes.addressof(ids), ctypes.addressof(sds)))
+        return [int(x) for x in ids[:n]], [int(x) for x in sds[:n]]
+
+    def task_tables(self, task_id: int):
+        src = (ctypes.c_uint32 * max(self.n_layers, 1))()
+        pos = (ctypes.c_uint32 * max(self.n_layers, 1))()
+        _check(lib().randes_task_tables(self.handle, task_id, ctypes.addressof(src), ctypes.addressof(pos)))
+        return [int(x) for x in src[:self.n_layers]], [int(x) for x in pos[:self.n_layers]]
+
+    # -- device buffers
+    def new_superposition(self):
+        import torch
+
+        return torch.empty(self.m_bytes // 4, dtype=torch.float32, device=self.device)
+
+    def slot(self, M, layer: int):
+        """View of slot ``layer`` of the arena M as a [rows, cols] tensor."""
+        o = self.offsets[layer] // 4
+        n = self.rows[layer] * self.cols[layer]
+        return M[o:o + n].view(self.rows[layer], self.cols[layer])
+
+    def new_output(self, out_dtype: int = F32):
+        import torch
+
+        dt = torch.bfloat16 if out_dtype == BF16 else torch.float32
+        return [torch.empty(r, c, dtype=dt, device=self.device) for r, c in zip(self.rows, self.cols)]
+
+    # -- the path
+    def compress(self, base, tasks, M=None):
+        if M is None:
+            M = self.new_superposition()
+        randes_compress(self.handle, _as_ptrs(base), _as_ptrs(tasks), M, self._stream())
+        return M
+
+    def add_model(self, task_id: int, seed: int, base, task, M):
+        randes_add_model(self.handle, task_id, seed, _as_ptrs(base), _as_ptrs(task), M, self._stream())
+        return M
+
+    def remove_model(self, task_id: int, base, task, M):
+        randes_remove_model(self.handle, task_id, _as_ptrs(base), _as_ptrs(task), M, self._stream())
+        return M
+
+    def retrieve(self, task_id: int, lam: float, base, M, out=None, out_dtype: int = F32):
+        out_list = None
+        if out is None:
+            out = out_list = self.new_output(out_dtype)
+        elif not isinstance(out, ctypes.Array):
+            out_list = out
+        randes_retrieve(self.handle, task_id, lam, out_dtype, _as_ptrs(base), M, _as_ptrs(out), self._stream())
+        return out_list

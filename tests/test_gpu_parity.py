@@ -1,0 +1,301 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle.
+
+Bars: permutation tables, sign bits and the fp32 superposition M are bit-exact;
+fp32 outputs of retrieve are bit-exact (one fused multiply-add on both sides;
+the accepted bound would be 1e-6 * max|W|); bf16 outputs are bit-exact (accepted
+bound: 1 bf16 ulp).  All inputs are seeded and synthetic.
+"""
+import numpy as np
+import pytest
+
+from oracle import randes_oracle as ro
+from paper_2505_11204_b200 import build, randes, workloads as wl
+
+from gpu_util import (assert_bits_equal, check_model, check_superposition, from_dev, model_to_dev, poison,
+                      to_dev)
+
+pytestmark = pytest.mark.gpu
+S, F = randes.SHUFFLE, randes.FLIP
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build_library()
+
+
+def make_workload(shapes, flags=S | F, storage=wl.F32, n_tasks=3, seed0=42, data_seed=7, interleave=True):
+    """shapes: list of (rows, cols, group_size).  Layers of different groups are
+    interleaved so that group-local and global indices differ."""
+    names, rows, cols, group = [], [], [], []
+    maxg = max(s[2] for s in shapes)
+    order = [(k, g) for k in range(maxg) for g in range(len(shapes)) if k < shapes[g][2]] if interleave else \
+            [(k, g) for g in range(len(shapes)) for k in range(shapes[g][2])]
+    for k, g in order:
+        names.append("g%d.%d" % (g, k)); rows.append(shapes[g][0]); cols.append(shapes[g][1]); group.append(g)
+    gflags = [flags if isinstance(flags, int) else flags[g] for g in range(len(shapes))]
+    return wl.Workload(name="case", layer_names=names, rows=rows, cols=cols, group=group, gflags=gflags,
+                       storage=storage, n_tasks=n_tasks, task_ids=list(range(n_tasks)),
+                       seeds=[seed0 + i for i in range(n_tasks)], scale=1e-3, lam=0.3, data_seed=data_seed)
+
+
+def run_full_cycle(w, out_dtypes=(wl.F32, wl.BF16), lam=None, extra_task=True):
+    """compress -> retrieve all -> add -> retrieve -> remove -> retrieve, each
+    step compared with the oracle replaying the same calls."""
+    import torch
+
+    lam = w.lam if lam is None else lam
+    ids, seeds = list(w.task_ids), list(w.seeds)
+    all_ids = ids + ([max(ids) + 5] if extra_task else [])
+    base, tasks = wl.model_set(w, all_ids)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, max_tasks=len(all_ids) + 1)
+    K = len(ids)
+
+    M_dev = poison(plan.new_superposition())
+    plan.compress(d_base, d_tasks[:K], M_dev)
+    M_ref = ro.compress(w.spec, w.storage, ids, seeds, base, tasks[:K])
+    check_superposition(plan, M_dev, M_ref, "compress")
+    # padding between slots is never written
+    raw = M_dev.view(torch.int32)
+    for l in range(w.n_layers):
+        end = plan.offsets[l] // 4 + w.rows[l] * w.cols[l]
+        nxt = plan.offsets[l + 1] // 4 if l + 1 < w.n_layers else plan.m_bytes // 4
+        assert bool((raw[end:nxt] == -1).all()), "padding after slot %d was written" % l
+
+    def retrieve_all(tag):
+        cur_ids, cur_seeds = plan.task_list()
+        for od in out_dtypes:
+            for t, s in zip(cur_ids, cur_seeds):
+                out = [poison(o) for o in plan.new_output(od)]
+                plan.retrieve(t, lam, d_base, M_dev, out=out, out_dtype=od)
+                ref = ro.retrieve(w.spec, w.storage, od, t, s, lam, base, M_ref)
+                check_model(out, ref, "%s retrieve task %d dtype %d" % (tag, t, od))
+
+    retrieve_all("after compress")
+    if extra_task:
+        new_id, new_seed = all_ids[-1], 100
+        plan.add_model(new_id, new_seed, d_base, d_tasks[K], M_dev)
+        ro.add_model(w.spec, w.storage, new_id, new_seed, base, tasks[K], M_ref)
+        check_superposition(plan, M_dev, M_ref, "add")
+        assert plan.task_list() == (ids + [new_id], seeds + [new_seed])
+        retrieve_all("after add")
+        gone = ids[len(ids) // 2]
+        j = ids.index(gone)
+        plan.remove_model(gone, d_base, d_tasks[j], M_dev)
+        ro.remove_model(w.spec, w.storage, gone, seeds[j], base, tasks[j], M_ref)
+        check_superposition(plan, M_dev, M_ref, "remove")
+        assert gone not in plan.task_list()[0]
+        retrieve_all("after remove")
+    torch.cuda.synchronize()
+    plan.close()
+
+
+# --------------------------------------------------------------------------- small cases
+def test_toy_config_all_steps():
+    run_full_cycle(wl.toy())
+
+
+RAGGED = [(1, 1, 3), (5, 3, 3), (37, 12, 2), (3, 127, 3), (2, 129, 4), (7, 130, 2), (19, 260, 3),
+          (1, 4100, 2), (33, 768, 3), (50, 640, 1), (130, 256, 2), (1, 4096, 5), (17, 384, 2)]
+
+
+@pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
+def test_ragged_shapes_span_tiles_and_tails(storage):
+    run_full_cycle(make_workload(RAGGED, storage=storage, n_tasks=3))
+
+
+@pytest.mark.parametrize("flags", [0, S, F])
+def test_single_transform_modes(flags):
+    run_full_cycle(make_workload(RAGGED[3:10], flags=flags, n_tasks=2), out_dtypes=(wl.F32,))
+
+
+def test_mixed_group_flags():
+    shapes = [(9, 132, 3), (1, 132, 3), (4, 256, 1), (6, 20, 4)]
+    run_full_cycle(make_workload(shapes, flags=[S | F, S, F, 0], n_tasks=4), out_dtypes=(wl.F32,))
+
+
+def test_more_tasks_than_one_chunk():
+    # 40 tasks: the kernel holds 32 task descriptors at a time
+    run_full_cycle(make_workload([(5, 260, 3), (1, 33, 2), (24, 128, 2)], n_tasks=40), out_dtypes=(wl.F32,),
+                   extra_task=True)
+
+
+def test_single_task_round_trip_and_lambda_one():
+    w = make_workload(RAGGED[2:9], n_tasks=1)
+    base, tasks = wl.model_set(w)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w)
+    M = plan.compress(d_base, d_tasks)
+    out = plan.retrieve(0, 1.0, d_base, M)
+    for b, t, o in zip(base, tasks[0], out):
+        want = (b + (t - b).astype(np.float32)).astype(np.float32)
+        assert_bits_equal(from_dev(o), want, "K=1 round trip")
+    plan.close()
+
+
+def test_delta_input_without_base():
+    # adapter deltas given directly (Section 5.8): base = NULL
+    w = make_workload([(16, 768, 3), (768, 16, 2), (1, 100, 2)], n_tasks=3)
+    deltas = [[wl.lora_delta_layer(w, l, t) for l in range(w.n_layers)] for t in w.task_ids]
+    d_deltas = [model_to_dev(d) for d in deltas]
+    plan = randes.Plan.from_workload(w)
+    M = plan.compress(None, d_deltas)
+    M_ref = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, None, deltas)
+    check_superposition(plan, M, M_ref, "delta compress")
+    extra = [wl.lora_delta_layer(w, l, 9) for l in range(w.n_layers)]
+    plan.add_model(9, 77, None, model_to_dev(extra), M)
+    ro.add_model(w.spec, w.storage, 9, 77, None, extra, M_ref)
+    check_superposition(plan, M, M_ref, "delta add")
+    plan.remove_model(1, None, d_deltas[1], M)
+    ro.remove_model(w.spec, w.storage, 1, w.seeds[1], None, deltas[1], M_ref)
+    check_superposition(plan, M, M_ref, "delta remove")
+    plan.close()
+
+
+def test_sign_bits_and_permutation_seen_through_the_kernels():
+    # delta == 1 everywhere except a per-layer tag: M exposes s_i(l, c) and sigma_i(l) directly
+    w = make_workload([(3, 300, 5)], n_tasks=1)
+    ones = [np.full((r, c), float(l + 1), dtype=np.float32) for l, (r, c) in enumerate(zip(w.rows, w.cols))]
+    plan = randes.Plan.from_workload(w)
+    M = plan.compress(None, [model_to_dev(ones)])
+    src, _ = ro.task_tables(w.spec, w.seeds[0], 0)
+    for l in range(w.n_layers):
+        want = np.tile(ro.sign_row(w.seeds[0], 0, l, w.cols[l]).astype(np.float32) * float(src[l] + 1), (w.rows[l], 1))
+        assert_bits_equal(from_dev(plan.slot(M, l)), want, "sign/perm slot %d" % l)
+    plan.close()
+
+
+def test_unaligned_tensors_take_the_scalar_path():
+    import torch
+
+    for storage in (wl.F32, wl.BF16):
+        w = make_workload([(6, 132, 3), (3, 260, 2)], storage=storage, n_tasks=2)
+        base, tasks = wl.model_set(w)
+
+        def shifted(a, k):  # same values, start address off by k elements
+            t = to_dev(a)
+            buf = torch.empty(a.size + 8, dtype=t.dtype, device="cuda")
+            v = buf[k:k + a.size].view(a.shape)
+            v.copy_(t)
+            return v
+
+        d_base = [shifted(a, 1 + (l % 3)) for l, a in enumerate(base)]
+        d_tasks = [[shifted(a, 1 + ((l + i) % 2)) for l, a in enumerate(t)] for i, t in enumerate(tasks)]
+        plan = randes.Plan.from_workload(w)
+        M = plan.compress(d_base, d_tasks)
+        M_ref = ro.compress(w.spec, storage, w.task_ids, w.seeds, base, tasks)
+        check_superposition(plan, M, M_ref, "unaligned compress")
+        for od in (wl.F32, wl.BF16):
+            dt = torch.bfloat16 if od == wl.BF16 else torch.float32
+            bufs = [torch.empty(r * c + 8, dtype=dt, device="cuda") for r, c in zip(w.rows, w.cols)]
+            out = [b[1:1 + r * c].view(r, c) for b, r, c in zip(bufs, w.rows, w.cols)]
+            plan.retrieve(1, 0.3, d_base, M, out=out, out_dtype=od)
+            ref = ro.retrieve(w.spec, storage, od, 1, w.seeds[1], 0.3, base, M_ref)
+            check_model(out, ref, "unaligned retrieve")
+        plan.close()
+
+
+def test_gpu_argument_validation():
+    import torch
+
+    w = make_workload([(4, 128, 2)], n_tasks=1)
+    base, tasks = wl.model_set(w)
+    d_base, d_task = model_to_dev(base), model_to_dev(tasks[0])
+    plan = randes.Plan.from_workload(w, max_tasks=2)
+    M = plan.compress(d_base, [d_task])
+
+    def expect(code, fn):
+        with pytest.raises(randes.RandesError) as e:
+            fn()
+        assert e.value.code == code, str(e.value)
+
+    before = randes.randes_launch_count()
+    expect(randes.UNKNOWN_TASK, lambda: plan.retrieve(5, 1.0, d_base, M))
+    expect(randes.UNSUPPORTED_DTYPE, lambda: plan.retrieve(0, 1.0, d_base, M, out=plan.new_output(), out_dtype=3))
+    expect(randes.INVALID_ARGUMENT, lambda: plan.retrieve(0, 1.0, d_base, M, out=d_base))          # aliases base
+    expect(randes.INVALID_ARGUMENT, lambda: plan.retrieve(0, 1.0, d_base, M, out=[plan.slot(M, 0), plan.slot(M, 1)]))
+    expect(randes.MISALIGNED, lambda: plan.compress(d_base, [d_task], M[1:]))
+    expect(randes.INVALID_ARGUMENT, lambda: randes.randes_compress(plan.handle, randes.ptr_array(d_base),
+                                                                   randes.ptr_array(d_task), None, None))
+    expect(randes.DUPLICATE_TASK, lambda: plan.add_model(0, 9, d_base, d_task, M))
+    expect(randes.UNKNOWN_TASK, lambda: plan.remove_model(4, d_base, d_task, M))
+    odd = torch.empty(4 * 128 * 4 + 2, dtype=torch.uint8, device="cuda")[1:1 + 4 * 128 * 4]
+    expect(randes.MISALIGNED, lambda: plan.compress([odd, d_base[1]], [d_task], M))
+    plan.add_model(1, 9, d_base, d_task, M)
+    expect(randes.CAPACITY, lambda: plan.add_model(2, 9, d_base, d_task, M))
+    assert randes.randes_launch_count() == before + 1      # only the valid add launched
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(randes.RandesError) as e:
+        randes.randes_plan(plan._layers, 2, plan._groups, 1, 0, None, None, 0, 1, small, 256, None)
+    assert e.value.code == randes.WORKSPACE_TOO_SMALL
+    plan.close()
+
+
+# --------------------------------------------------------------------------- the paper-shaped configs, full size
+def test_vit_b32_shaped_full():
+    w = wl.vit_b32()
+    run_full_cycle(w, out_dtypes=(wl.F32,), extra_task=False)
+
+
+def test_gpt2_shaped_bf16_hot_swap_full():
+    # K = 7 in bf16 storage; then remove task 3 and add task 7 (seed 100), retrieving every task after each change
+    import torch
+
+    w = wl.gpt2_small()
+    ids, seeds = list(w.task_ids), list(w.seeds)
+    base, tasks = wl.model_set(w, ids + [7])
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, max_tasks=9)
+    M = plan.compress(d_base, d_tasks[:7])
+    M_ref = ro.compress(w.spec, w.storage, ids, seeds, base, tasks[:7])
+    check_superposition(plan, M, M_ref, "compress")
+
+    def sweep(tag):
+        cur_ids, cur_seeds = plan.task_list()
+        out = plan.new_output(wl.BF16)
+        for t, s in zip(cur_ids, cur_seeds):
+            plan.retrieve(t, w.lam, d_base, M, out=out, out_dtype=wl.BF16)
+            ref = ro.retrieve(w.spec, w.storage, wl.BF16, t, s, w.lam, base, M_ref)
+            check_model(out, ref, "%s task %d" % (tag, t))
+
+    sweep("initial")
+    plan.remove_model(3, d_base, d_tasks[3], M)
+    ro.remove_model(w.spec, w.storage, 3, seeds[3], base, tasks[3], M_ref)
+    check_superposition(plan, M, M_ref, "remove 3")
+    sweep("after remove")
+    plan.add_model(7, 100, d_base, d_tasks[7], M)
+    ro.add_model(w.spec, w.storage, 7, 100, base, tasks[7], M_ref)
+    check_superposition(plan, M, M_ref, "add 7")
+    sweep("after add")
+    torch.cuda.synchronize()
+    plan.close()
+
+
+def test_flan_t5_shaped_full_and_lora_variant():
+    w = wl.flan_t5_base()
+    base, tasks = wl.model_set(w)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w)
+    M = plan.compress(d_base, d_tasks)
+    M_ref = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, base, tasks)
+    check_superposition(plan, M, M_ref, "compress")
+    for t in (0, 5):
+        out = plan.retrieve(t, w.lam, d_base, M)
+        ref = ro.retrieve(w.spec, w.storage, wl.F32, t, w.seeds[t], w.lam, base, M_ref)
+        check_model(out, ref, "retrieve %d" % t)
+    plan.close()
+    del d_tasks, tasks, M
+    # rank-16 adapters on q and v of every attention module, materialised, plan over those 72 matrices only
+    targets = wl.flan_t5_lora_targets(w)
+    assert len(targets) == 72
+    wlora = wl.subset(w, targets, "flan_t5_base_lora")
+    deltas = [[wl.lora_delta_layer(wlora, l, t) for l in range(wlora.n_layers)] for t in wlora.task_ids]
+    lbase = [base[l] for l in targets]
+    plan = randes.Plan.from_workload(wlora)
+    M = plan.compress(None, [model_to_dev(d) for d in deltas])
+    M_ref = ro.compress(wlora.spec, wlora.storage, wlora.task_ids, wlora.seeds, None, deltas)
+    check_superposition(plan, M, M_ref, "lora compress")
+    out = plan.retrieve(2, w.lam, model_to_dev(lbase), M)
+    ref = ro.retrieve(wlora.spec, wlora.storage, wl.F32, 2, wlora.seeds[2], w.lam, lbase, M_ref)
+    check_model(out, ref, "lora retrieve")
+    plan.close()

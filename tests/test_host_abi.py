@@ -1,0 +1,132 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports what
+the header declares, validates arguments, and draws the same permutations as
+the oracle (two independent implementations of the seed -> sigma rule)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import randes_oracle as ro
+from paper_2505_11204_b200 import build, randes, workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "randes.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(randes_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert len(names) >= 15
+    L = ctypes.CDLL(randes.LIB_PATH)
+    for n in names:
+        assert hasattr(L, n), n
+    assert sorted(randes.EXPORTS) == names
+
+
+def test_host_only_plan_tables_match_oracle():
+    for w in (wl.toy(), wl.vit_b32(), wl.gpt2_small(), wl.flan_t5_base(), wl.vit_l14()):
+        ids = list(range(w.n_tasks)) + [1000]
+        seeds = w.seeds + [2**63 + 12345]
+        p = randes.Plan(w.rows, w.cols, w.group, w.gflags, storage=w.storage, task_ids=ids, seeds=seeds,
+                        host_only=True)
+        for t, s in zip(ids, seeds):
+            src, pos = p.task_tables(t)
+            osrc, opos = ro.task_tables(w.spec, s, t)
+            assert src == osrc.tolist() and pos == opos.tolist()
+        assert p.task_list() == (ids, seeds)
+        p.close()
+
+
+def test_sigma_agrees_for_many_seeds_and_group_sizes():
+    rng = np.random.default_rng(5)
+    for _ in range(300):
+        G = int(rng.integers(1, 40))
+        seed = int(rng.integers(0, 2**63))
+        tid = int(rng.integers(0, 2**32))
+        n_pad = int(rng.integers(0, 3))   # singleton groups before the one under test shift its index
+        rows = [1] * n_pad + [2] * G
+        cols = [3 + i for i in range(n_pad)] + [8] * G
+        group = list(range(n_pad)) + [n_pad] * G
+        gflags = [randes.FLIP] * n_pad + [randes.SHUFFLE]
+        p = randes.Plan(rows, cols, group, gflags, task_ids=[tid], seeds=[seed], host_only=True)
+        src, pos = p.task_tables(tid)
+        sigma = ro.permutation(seed, tid, n_pad, G)
+        assert src[n_pad:] == [n_pad + int(s) for s in sigma]
+        assert all(pos[src[l]] == l for l in range(len(rows)))
+        p.close()
+
+
+def test_superposition_layout_is_one_fp32_copy_independent_of_task_count():
+    w = wl.vit_b32()
+    p1 = randes.Plan.from_workload(w.with_tasks(1), host_only=True)
+    p8 = randes.Plan.from_workload(w, host_only=True)
+    assert p1.m_bytes == p8.m_bytes
+    assert p1.offsets == p8.offsets
+    assert all(o % 256 == 0 for o in p8.offsets)
+    raw = 4 * w.n_params
+    assert raw <= p8.m_bytes <= raw + 256 * w.n_layers
+    for l in range(w.n_layers - 1):
+        assert p8.offsets[l + 1] - p8.offsets[l] >= 4 * w.rows[l] * w.cols[l]
+    assert randes.randes_layer_offset(p8.handle, w.n_layers) == 2**64 - 1
+    # memory figures of the paper's first results table: 0.564 -> 0.89 (GiB) is one fp32 copy of the encoder
+    assert abs(0.564 + raw / 2**30 - 0.89) < 0.005
+
+
+def test_workspace_size_grows_with_capacity_and_rejects_bad_input():
+    w = wl.toy()
+    p = randes.Plan.from_workload(w, host_only=True)
+    a = randes.randes_plan_workspace_bytes(p._layers, w.n_layers, 4)
+    b = randes.randes_plan_workspace_bytes(p._layers, w.n_layers, 64)
+    assert 0 < a < b
+    assert randes.randes_plan_workspace_bytes(p._layers, w.n_layers, 0) == 0
+    assert randes.randes_plan_workspace_bytes(None, 3, 4) == 0
+
+
+def _expect(code, fn):
+    with pytest.raises(randes.RandesError) as e:
+        fn()
+    assert e.value.code == code, (e.value.code, str(e.value))
+    assert randes.randes_last_error()
+
+
+def test_plan_argument_validation():
+    S, F = randes.SHUFFLE, randes.FLIP
+    mk = lambda **kw: randes.Plan(kw.get("rows", [2, 2]), kw.get("cols", [4, 4]), kw.get("group", [0, 0]),
+                                  kw.get("gflags", [S | F]), storage=kw.get("storage", randes.F32),
+                                  task_ids=kw.get("ids", [0]), seeds=kw.get("seeds", [1]),
+                                  max_tasks=kw.get("max_tasks", 4), host_only=True)
+    mk().close()
+    _expect(randes.SHAPE_MISMATCH, lambda: mk(cols=[4, 5]))
+    _expect(randes.DUPLICATE_TASK, lambda: mk(ids=[3, 3], seeds=[1, 2]))
+    _expect(randes.INVALID_ARGUMENT, lambda: mk(group=[0, 1]))          # group id out of range
+    _expect(randes.INVALID_ARGUMENT, lambda: mk(gflags=[8]))            # unknown flag bit
+    _expect(randes.INVALID_ARGUMENT, lambda: mk(max_tasks=0, ids=[], seeds=[]))
+    _expect(randes.INVALID_ARGUMENT, lambda: mk(ids=[0, 1, 2], seeds=[0, 1, 2], max_tasks=2))
+    _expect(randes.UNSUPPORTED_DTYPE, lambda: mk(storage=7))
+    p = mk()
+    _expect(randes.UNKNOWN_TASK, lambda: p.task_tables(99))
+    # a host-only plan cannot compute
+    arr = (ctypes.c_void_p * 2)(256, 512)
+    _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_compress(p.handle, arr, arr, 256, None))
+    _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_retrieve(p.handle, 0, 1.0, randes.F32, arr, 256, arr, None))
+    _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_add_model(p.handle, 5, 5, arr, arr, 256, None))
+    _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_remove_model(p.handle, 0, arr, arr, 256, None))
+    p.close()
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(randes, "_lib", None)
+    monkeypatch.setattr(randes, "LIB_PATH", str(tmp_path / "absent.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        randes.lib()

@@ -113,8 +113,9 @@ WorkspaceLayout layout_workspace(size_t n_layers, size_t n_units, size_t max_tas
 // Units in group order; inside a group, all members at one (row block, column
 // chunk) are adjacent, so that tiles of W_0 which several slots read (under a
 // shuffle) are touched close together in time and stay in L2.
-void build_units(const randes_layer_t* layers, uint32_t n_layers, std::vector<DevUnit>& units)
+void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, std::vector<DevUnit>& units)
 {
+    const uint32_t wcols = cols_per_warp(storage);
     units.clear();
     std::vector<char> done(n_layers, 0);
     std::vector<uint32_t> members;
@@ -125,7 +126,7 @@ void build_units(const randes_layer_t* layers, uint32_t n_layers, std::vector<De
             if (!done[l] && layers[l].group == layers[first].group) { members.push_back(l); done[l] = 1; }
         const uint32_t rows = layers[first].rows, cols = layers[first].cols;
         if (rows == 0 || cols == 0) continue;
-        const uint32_t nb = (cols + kColsPerWarp - 1) / kColsPerWarp;
+        const uint32_t nb = (cols + wcols - 1) / wcols;
         uint32_t nbc = 1;
         while (nbc < static_cast<uint32_t>(kWarpsPerCta) && nb % (nbc * 2) == 0) nbc *= 2;
         const uint32_t rows_per_unit = kRowsPerWarp * (kWarpsPerCta / nbc);
@@ -147,9 +148,9 @@ int check_layers(const randes_layer_t* layers, uint32_t n_layers)
 {
     if (!layers || n_layers == 0) return fail(RANDES_INVALID_ARGUMENT, "layers is NULL or empty");
     for (uint32_t l = 0; l < n_layers; ++l)
-        if (layers[l].cols > 65535u * kColsPerWarp)
+        if (layers[l].cols > 65535u * 128u)
             return fail(RANDES_INVALID_ARGUMENT, "layer %u: cols %u exceeds the supported %u", l, layers[l].cols,
-                        65535u * kColsPerWarp);
+                        65535u * 128u);
     return RANDES_OK;
 }
 
@@ -170,7 +171,7 @@ struct randes_plan_s {
     char* ws = nullptr;
     WorkspaceLayout lay{};
     int sm_count = 0;
-    int grid_acc = 0;
+    int grid_acc[2] = {0, 0};   // [0] compress, [1] one task (add / remove)
     int grid_ret[2] = {0, 0};
     // host mirrors of what the device pointer tables currently hold
     std::vector<const void*> h_base, h_out, h_tasks;
@@ -302,7 +303,7 @@ int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_
     a.task_ptrs = p.dev<const void*>(p.lay.task_ptrs);
     a.M = static_cast<float*>(M);
     if (a.n_units == 0) return RANDES_OK;
-    const int grid = std::min<int>(p.grid_acc, static_cast<int>(a.n_units));
+    const int grid = std::min<int>(p.grid_acc[n_rows == 1], static_cast<int>(a.n_units));
     const int e = launch_accumulate(p.storage, a, grid, s);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the accumulate kernel");
     ++g_launches;
@@ -320,9 +321,13 @@ uint64_t randes_launch_count(void) { return g_launches.load(); }
 size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_layers, uint32_t max_tasks)
 {
     if (check_layers(layers, n_layers) || max_tasks == 0) return 0;
+    // the unit list depends on the storage type, which is not known here: take the larger
     std::vector<DevUnit> units;
-    build_units(layers, n_layers, units);
-    return layout_workspace(n_layers, units.size(), max_tasks).total;
+    build_units(layers, n_layers, RANDES_F32, units);
+    size_t n_units = units.size();
+    build_units(layers, n_layers, RANDES_BF16, units);
+    n_units = std::max(n_units, units.size());
+    return layout_workspace(n_layers, n_units, max_tasks).total;
 }
 
 int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_group_t* groups, uint32_t n_groups,
@@ -392,7 +397,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
             off = align_up(off + static_cast<size_t>(layers[l].rows) * layers[l].cols * sizeof(float), 256);
         }
         p->m_bytes = off;
-        build_units(layers, n_layers, p->units);
+        build_units(layers, n_layers, p->storage, p->units);
         p->tasks.resize(n_tasks);
         for (uint32_t i = 0; i < n_tasks; ++i) {
             p->tasks[i].id = task_ids[i];
@@ -423,14 +428,16 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         cudaError_t e = cudaGetDevice(&dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) { delete p; return fail_cuda(e, "device query"); }
-        const int occ_acc = accumulate_ctas_per_sm(p->storage);
+        const int occ_acc = accumulate_ctas_per_sm(p->storage, false);
+        const int occ_acc1 = accumulate_ctas_per_sm(p->storage, true);
         const int occ_r0 = retrieve_ctas_per_sm(p->storage, RANDES_F32);
         const int occ_r1 = retrieve_ctas_per_sm(p->storage, RANDES_BF16);
-        if (occ_acc <= 0 || occ_r0 <= 0 || occ_r1 <= 0) {
+        if (occ_acc <= 0 || occ_acc1 <= 0 || occ_r0 <= 0 || occ_r1 <= 0) {
             delete p;
             return fail(RANDES_CUDA_ERROR, "kernels are not loadable on this device (built for sm_100a)");
         }
-        p->grid_acc = p->sm_count * occ_acc;
+        p->grid_acc[0] = p->sm_count * occ_acc;
+        p->grid_acc[1] = p->sm_count * occ_acc1;
         p->grid_ret[0] = p->sm_count * occ_r0;
         p->grid_ret[1] = p->sm_count * occ_r1;
         e = cudaMemcpyAsync(p->ws + p->lay.layers, p->dev_layers.data(), n_layers * sizeof(DevLayer),

@@ -12,11 +12,16 @@ constexpr uint32_t kFlagFlip = 2u;      // per-column sign flip on this slot
 
 constexpr int kWarpsPerCta = 8;
 constexpr int kThreadsPerCta = kWarpsPerCta * 32;
-constexpr int kColsPerWarp = 128;       // one Philox block of sign bits; 4 columns per lane
 constexpr int kRowsPerWarp = 16;        // rows one warp walks per unit
 constexpr int kTaskChunk = 32;          // tasks whose pointers / sign blocks a warp holds at once
 constexpr uint32_t kTagSign = 0x5349474Eu;  // counter word 2 of the sign stream ("SIGN")
 constexpr uint32_t kTagPerm = 0x5045524Du;  // counter word 2 of the permutation stream ("PERM")
+
+// A lane always moves 16 bytes of a weight tensor: 4 fp32 or 8 bf16 columns.  A
+// warp therefore spans 128 (fp32) or 256 (bf16) columns = 1 or 2 Philox blocks
+// of sign bits.
+constexpr int cols_per_lane(int storage_dtype) { return storage_dtype == 1 ? 8 : 4; }
+constexpr int cols_per_warp(int storage_dtype) { return 32 * cols_per_lane(storage_dtype); }
 
 // One layer of the model == one slot of M (same index space).
 struct DevLayer {
@@ -29,8 +34,8 @@ struct DevLayer {
 };
 static_assert(sizeof(DevLayer) == 32, "DevLayer layout");
 
-// One unit of work for a CTA: `nrows` rows x `nbc` column blocks of 128 columns
-// of one layer.  Warp w owns column block cb0 + (w % nbc) and the rows
+// One unit of work for a CTA: `nrows` rows x `nbc` warp-wide column blocks of
+// one layer.  Warp w owns column block cb0 + (w % nbc) and the rows
 // row0 + (w / nbc), stepping by kWarpsPerCta / nbc.
 struct DevUnit {
     uint32_t layer;
@@ -79,8 +84,10 @@ struct AccumulateArgs {
 // Launchers (randes_kernels.cu).  Return a cudaError_t as int.
 int launch_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, int grid, void* stream);
 int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void* stream);
-// Resident CTAs per SM of each kernel (for sizing persistent grids).
+// Resident CTAs per SM of each kernel (for sizing persistent grids); 0 if the
+// kernels cannot run on the current device.  Also opts the kernels into the
+// dynamic shared memory they need: call once per device before launching.
 int retrieve_ctas_per_sm(int storage_dtype, int out_dtype);
-int accumulate_ctas_per_sm(int storage_dtype);
+int accumulate_ctas_per_sm(int storage_dtype, bool single_task);
 
 }  // namespace randes

@@ -1,16 +1,22 @@
 // sm_100a kernels of the RanDeS hot path: retrieve, and accumulate
-// (compress / add_model / remove_model).  HBM-bound streaming kernels:
-// 128-bit loads, fp32 arithmetic with one rounding per operation, sign bits
-// generated in registers from Philox4x32-10 and never stored to memory, the
-// per-task layer permutation resolved per unit of work from small index tables.
+// (compress / add_model / remove_model).  HBM-bound streaming kernels: every
+// lane moves 16 bytes of a weight tensor per request, arithmetic is fp32 with
+// one rounding per operation, sign bits are generated in registers from
+// Philox4x32-10 and never stored to global memory, the per-task layer
+// permutation is resolved per unit of work from small index tables.
 //
 // Work decomposition.  A CTA (8 warps) walks a list of units; a unit is a block
-// of rows x up to 8 column blocks of 128 columns of one layer.  A warp owns one
-// column block (lane = 4 adjacent columns, so one Philox block of 128 bits is
-// exactly the warp's sign bits) and walks down the rows: the sign bits are
+// of rows x up to 8 warp-wide column blocks of one layer.  A warp owns one
+// column block (32 lanes x 16 bytes: 128 fp32 or 256 bf16 columns, i.e. one or
+// two Philox blocks of sign bits) and walks down the rows: the sign bits are
 // computed once per unit and reused for every row.  Every output element is
-// written by exactly one thread, tasks are summed in a fixed order: results are
-// bit-reproducible.
+// written by exactly one thread and tasks are summed in a fixed order, so
+// results are bit-reproducible.
+//
+// The accumulate kernel keeps its weight streams in flight with cp.async into a
+// per-thread ring in shared memory (each lane reads back only what it copied,
+// so no barrier is needed): the number of bytes in flight is set by shared
+// memory, not by registers.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -22,8 +28,8 @@ namespace {
 typedef __nv_bfloat16 bf16;
 
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): counter (c0..c3), key (k0,k1).
-__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4])
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                               uint32_t k1)
 {
 #pragma unroll
     for (int round = 0; round < 10; ++round) {
@@ -36,83 +42,113 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
         k0 += 0x9E3779B9u;
         k1 += 0xBB67AE85u;
     }
-    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
-}
-
-// The four sign bits of this lane's columns (bit j = column 4*lane + j of the
-// warp's 128-column block) out of the block's four words.
-__device__ __forceinline__ uint32_t lane_nibble(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, int lane)
-{
-    const int q = lane >> 3;
-    const uint32_t w = q == 0 ? w0 : (q == 1 ? w1 : (q == 2 ? w2 : w3));
-    return (w >> ((lane & 7) * 4)) & 0xFu;
+    return make_uint4(c0, c1, c2, c3);
 }
 
 __device__ __forceinline__ float flip(float x, uint32_t mask) { return __uint_as_float(__float_as_uint(x) ^ mask); }
 
-// ---- element access: fp32 and bf16 storage, 4 columns per lane -------------------------
-template <typename T> struct Io;
+// ---- storage types: a lane's 16 bytes hold CPL columns -------------------------------------
+template <typename T> struct Store;
 
-template <> struct Io<float> {
-    static constexpr uintptr_t kVecAlign = 16;
-    static __device__ __forceinline__ float4 load4_stream(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
-    static __device__ __forceinline__ float4 load4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+template <> struct Store<float> {
+    static constexpr int CPL = 4;
+    static __device__ __forceinline__ void widen(const uint4& raw, float (&v)[4])
+    {
+        v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
+        v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
+    }
     static __device__ __forceinline__ float load1(const float* p) { return __ldg(p); }
-    static __device__ __forceinline__ void store4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
-    static __device__ __forceinline__ void store1(float* p, float v) { *p = v; }
 };
 
-template <> struct Io<bf16> {
-    static constexpr uintptr_t kVecAlign = 8;
-    static __device__ __forceinline__ float4 widen(uint2 raw)
+template <> struct Store<bf16> {
+    static constexpr int CPL = 8;
+    static __device__ __forceinline__ void widen(const uint4& raw, float (&v)[8])
     {
-        float4 f;
-        f.x = __uint_as_float(raw.x << 16);
-        f.y = __uint_as_float(raw.x & 0xFFFF0000u);
-        f.z = __uint_as_float(raw.y << 16);
-        f.w = __uint_as_float(raw.y & 0xFFFF0000u);
-        return f;
+        v[0] = __uint_as_float(raw.x << 16); v[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+        v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+        v[4] = __uint_as_float(raw.z << 16); v[5] = __uint_as_float(raw.z & 0xFFFF0000u);
+        v[6] = __uint_as_float(raw.w << 16); v[7] = __uint_as_float(raw.w & 0xFFFF0000u);
     }
-    static __device__ __forceinline__ float4 load4_stream(const bf16* p) { return widen(__ldcs(reinterpret_cast<const uint2*>(p))); }
-    static __device__ __forceinline__ float4 load4(const bf16* p) { return widen(__ldg(reinterpret_cast<const uint2*>(p))); }
     static __device__ __forceinline__ float load1(const bf16* p)
     {
         return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
     }
-    static __device__ __forceinline__ void store4(bf16* p, float4 v)
-    {
-        // round to nearest even, two values per conversion
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
-        const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
-        uint2 raw;
-        raw.x = *reinterpret_cast<const uint32_t*>(&lo);
-        raw.y = *reinterpret_cast<const uint32_t*>(&hi);
-        __stcs(reinterpret_cast<uint2*>(p), raw);
-    }
-    static __device__ __forceinline__ void store1(bf16* p, float v) { *p = __float2bfloat16_rn(v); }
 };
 
-template <typename T>
-__device__ __forceinline__ bool vec_aligned(const void* p)
+// ---- output types: CPL consecutive values ---------------------------------------------------
+template <typename T> struct Out;
+
+template <> struct Out<float> {
+    template <int CPL> static __device__ __forceinline__ void store(float* p, const float (&y)[CPL])
+    {
+#pragma unroll
+        for (int j = 0; j < CPL / 4; ++j)
+            __stcs(reinterpret_cast<float4*>(p) + j, make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]));
+    }
+    static __device__ __forceinline__ void store1(float* p, float v) { *p = v; }
+    template <int CPL> static __device__ __forceinline__ bool aligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+};
+
+template <> struct Out<bf16> {
+    // round to nearest even, two values per conversion
+    static __device__ __forceinline__ uint32_t pack(float lo, float hi)
+    {
+        const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t*>(&v);
+    }
+    template <int CPL> static __device__ __forceinline__ void store(bf16* p, const float (&y)[CPL])
+    {
+        if (CPL == 4) {
+            __stcs(reinterpret_cast<uint2*>(p), make_uint2(pack(y[0], y[1]), pack(y[2], y[3])));
+        } else {
+            __stcs(reinterpret_cast<uint4*>(p),
+                   make_uint4(pack(y[0], y[1]), pack(y[2], y[3]), pack(y[4 % CPL], y[5 % CPL]), pack(y[6 % CPL], y[7 % CPL])));
+        }
+    }
+    static __device__ __forceinline__ void store1(bf16* p, float v) { *p = __float2bfloat16_rn(v); }
+    template <int CPL> static __device__ __forceinline__ bool aligned(const void* p)
+    {
+        return (reinterpret_cast<uintptr_t>(p) & (2 * CPL - 1)) == 0;
+    }
+};
+
+__device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// The sign bits of this lane's CPL columns (bit e = column c + e), out of the
+// Philox block that covers them.
+template <int CPL> __device__ __forceinline__ uint32_t lane_bits(const uint4& blk, int lane)
 {
-    return (reinterpret_cast<uintptr_t>(p) & (Io<T>::kVecAlign - 1)) == 0;
+    if (CPL == 4) {
+        const int q = lane >> 3;
+        const uint32_t w = q == 0 ? blk.x : (q == 1 ? blk.y : (q == 2 ? blk.z : blk.w));
+        return (w >> ((lane & 7) * 4)) & 0xFu;
+    }
+    const int q = (lane & 15) >> 2;
+    const uint32_t w = q == 0 ? blk.x : (q == 1 ? blk.y : (q == 2 ? blk.z : blk.w));
+    return (w >> ((lane & 3) * 8)) & 0xFFu;
+}
+
+// Which 128-column Philox block holds this lane's columns.
+template <int CPL> __device__ __forceinline__ uint32_t lane_block(uint32_t cb, int lane)
+{
+    return CPL == 4 ? cb : cb * 2 + (lane >> 4);
 }
 
 // geometry of this warp inside a unit
 struct WarpTile {
-    uint32_t cb;      // column block (128 columns) of the layer
-    uint32_t c;       // first of this lane's 4 columns
+    uint32_t cb;      // warp-wide column block of the layer
+    uint32_t c;       // first of this lane's CPL columns
     uint32_t r0;      // first row of this warp
     uint32_t r_end;   // one past the last row of the unit
     uint32_t rstep;   // row stride between this warp's rows
 };
 
-__device__ __forceinline__ WarpTile warp_tile(const DevUnit& un, int warp, int lane)
+template <int CPL> __device__ __forceinline__ WarpTile warp_tile(const DevUnit& un, int warp, int lane)
 {
     WarpTile t;
     const uint32_t nbc = un.nbc;
     t.cb = un.cb0 + (warp & (nbc - 1));
-    t.c = t.cb * kColsPerWarp + lane * 4;
+    t.c = (t.cb * 32 + lane) * CPL;
     t.rstep = kWarpsPerCta / nbc;
     t.r0 = un.row0 + warp / nbc;
     t.r_end = un.row0 + un.nrows;
@@ -126,26 +162,30 @@ __device__ __forceinline__ WarpTile warp_tile(const DevUnit& un, int warp, int l
 // =========================================================================================
 template <typename ST, typename OT, bool VEC>
 __device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, const float* __restrict__ mp,
-                                              const ST* __restrict__ wp, OT* __restrict__ op, const float (&lam)[4])
+                                              const ST* __restrict__ wp, OT* __restrict__ op,
+                                              const float (&lam)[Store<ST>::CPL])
 {
-    constexpr int U = 4;
+    constexpr int CPL = Store<ST>::CPL;
+    constexpr int U = CPL == 4 ? 4 : 2;
     for (uint32_t r = t.r0; r < t.r_end; r += t.rstep * U) {
-        float4 m[U], w[U];
+        float4 m[U][CPL / 4];
+        uint4 w[U];
+        float ms[U][CPL], wsc[U][CPL];
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             const uint32_t rr = r + j * t.rstep;
             if (rr < t.r_end) {
                 const size_t off = static_cast<size_t>(rr) * cols + t.c;
                 if (VEC) {
-                    m[j] = __ldcs(reinterpret_cast<const float4*>(mp + off));
-                    w[j] = Io<ST>::load4_stream(wp + off);
-                } else {
-                    float mm[4] = {0.f, 0.f, 0.f, 0.f}, ww[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (t.c + e < cols) { mm[e] = mp[off + e]; ww[e] = Io<ST>::load1(wp + off + e); }
-                    m[j] = make_float4(mm[0], mm[1], mm[2], mm[3]);
-                    w[j] = make_float4(ww[0], ww[1], ww[2], ww[3]);
+                    for (int h = 0; h < CPL / 4; ++h) m[j][h] = __ldcs(reinterpret_cast<const float4*>(mp + off) + h);
+                    w[j] = __ldcs(reinterpret_cast<const uint4*>(wp + off));
+                } else {
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) {
+                        ms[j][e] = 0.f; wsc[j][e] = 0.f;
+                        if (t.c + e < cols) { ms[j][e] = mp[off + e]; wsc[j][e] = Store<ST>::load1(wp + off + e); }
+                    }
                 }
             }
         }
@@ -154,18 +194,25 @@ __device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, 
             const uint32_t rr = r + j * t.rstep;
             if (rr < t.r_end) {
                 const size_t off = static_cast<size_t>(rr) * cols + t.c;
-                float4 y;
-                y.x = __fmaf_rn(lam[0], m[j].x, w[j].x);
-                y.y = __fmaf_rn(lam[1], m[j].y, w[j].y);
-                y.z = __fmaf_rn(lam[2], m[j].z, w[j].z);
-                y.w = __fmaf_rn(lam[3], m[j].w, w[j].w);
+                float mv[CPL], wv[CPL], y[CPL];
                 if (VEC) {
-                    Io<OT>::store4(op + off, y);
-                } else {
-                    const float yy[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        if (t.c + e < cols) Io<OT>::store1(op + off + e, yy[e]);
+                    for (int h = 0; h < CPL / 4; ++h) {
+                        mv[4 * h] = m[j][h].x; mv[4 * h + 1] = m[j][h].y; mv[4 * h + 2] = m[j][h].z; mv[4 * h + 3] = m[j][h].w;
+                    }
+                    Store<ST>::widen(w[j], wv);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) { mv[e] = ms[j][e]; wv[e] = wsc[j][e]; }
+                }
+#pragma unroll
+                for (int e = 0; e < CPL; ++e) y[e] = __fmaf_rn(lam[e], mv[e], wv[e]);
+                if (VEC) {
+                    Out<OT>::template store<CPL>(op + off, y);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e)
+                        if (t.c + e < cols) Out<OT>::store1(op + off + e, y[e]);
                 }
             }
         }
@@ -175,6 +222,7 @@ __device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, 
 template <typename ST, typename OT>
 __global__ void __launch_bounds__(kThreadsPerCta) retrieve_kernel(const RetrieveArgs a)
 {
+    constexpr int CPL = Store<ST>::CPL;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
@@ -182,23 +230,22 @@ __global__ void __launch_bounds__(kThreadsPerCta) retrieve_kernel(const Retrieve
         const DevLayer lp = a.layers[p];
         const uint32_t slot = (lp.flags & kFlagShuffle) ? a.slot_of_pos[p] : p;   // sigma^-1
         const unsigned long long m_off = slot == p ? lp.m_off : a.layers[slot].m_off;
-        const WarpTile t = warp_tile(un, warp, lane);
+        const WarpTile t = warp_tile<CPL>(un, warp, lane);
         if (t.c >= lp.cols || t.r0 >= t.r_end) continue;
 
-        uint32_t nib = 0;
+        uint32_t bits = 0;
         if (lp.flags & kFlagFlip) {
-            uint32_t blk[4];
-            philox4x32_10(t.cb, slot, kTagSign, a.task.id, a.task.key0, a.task.key1, blk);
-            nib = lane_nibble(blk[0], blk[1], blk[2], blk[3], lane);
+            const uint4 blk = philox4x32_10(lane_block<CPL>(t.cb, lane), slot, kTagSign, a.task.id, a.task.key0, a.task.key1);
+            bits = lane_bits<CPL>(blk, lane);
         }
-        float lam[4];
+        float lam[CPL];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) lam[e] = flip(a.lambda, ((nib >> e) & 1u) << 31);
+        for (int e = 0; e < CPL; ++e) lam[e] = flip(a.lambda, ((bits >> e) & 1u) << 31);
 
         const ST* wp = static_cast<const ST*>(a.base[p]);
         OT* op = static_cast<OT*>(a.out[p]);
         const float* mp = a.M + m_off;
-        const bool vec = (lp.cols & 3u) == 0 && vec_aligned<ST>(wp) && vec_aligned<OT>(op);
+        const bool vec = lp.cols % CPL == 0 && aligned16(wp) && Out<OT>::template aligned<CPL>(op);
         if (vec) retrieve_rows<ST, OT, true>(t, lp.cols, mp, wp, op, lam);
         else retrieve_rows<ST, OT, false>(t, lp.cols, mp, wp, op, lam);
     }
@@ -211,115 +258,239 @@ __global__ void __launch_bounds__(kThreadsPerCta) retrieve_kernel(const Retrieve
 // A warp keeps the resolved source pointers and the Philox sign blocks of up to
 // kTaskChunk tasks in its private shared-memory scratch: lane i prepares task i.
 // =========================================================================================
-struct WarpScratch {
+template <int CPL> struct WarpScratch {
     const void* pw[kTaskChunk];
     const void* pb[kTaskChunk];
-    uint4 sign[kTaskChunk];
+    uint4 sign[kTaskChunk][CPL / 4];
 };
 
-template <typename ST, bool VEC>
-__device__ __forceinline__ float4 load_tile(const ST* p, size_t off, uint32_t c, uint32_t cols, bool stream)
+// How W_0 enters the difference W_i - W_0.
+constexpr int kNoBase = 0;        // the task tensors already hold deltas
+constexpr int kSharedBase = 1;    // no shuffle: every task subtracts the same W_0 tile, fetched once per row
+constexpr int kPerTaskBase = 2;   // shuffle: task i subtracts W_0[sigma_i(l)]; tiles repeat across slots and hit in L2
+
+constexpr int kInitZero = 0;      // start from +0
+constexpr int kInitAsync = 1;     // start from M written by an earlier launch: staged like the weights
+constexpr int kInitPlain = 2;     // start from M written earlier by this thread: plain load
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 {
-    if (VEC) return stream ? Io<ST>::load4_stream(p + off) : Io<ST>::load4(p + off);
-    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    const uint32_t s = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Position in the flattened (row, batch-of-tasks) sequence a warp walks.
+struct Cursor {
+    uint32_t row, b;
+    __device__ __forceinline__ void advance(uint32_t nbat) { if (++b == nbat) { b = 0; ++row; } }
+};
+
+// Shared-memory ring of one thread: NSTAGE stages x SLOTS 16-byte slots, slot-major
+// across the CTA's threads (consecutive lanes are contiguous: conflict-free).
+//   slots [0, NB)            W_i tiles of the batch
+//   slot  NB                 W_0 tile of the row (kSharedBase), filled with the row's first batch
+//   slots NB+1 .. NB+CPL/4   M tile of the row (kInitAsync), filled with the row's first batch
+template <int CPL, int NB> struct Ring {
+    static constexpr int SLOTS = NB + 1 + CPL / 4;
+    uint4* base;   // this thread's slot 0 of stage 0
+    __device__ __forceinline__ uint4* slot(int stage, int s) const { return base + (stage * SLOTS + s) * kThreadsPerCta; }
+};
+
+template <typename ST, int BASE, int NB, int NSTAGE>
+__device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_t cols, const WarpScratch<Store<ST>::CPL>& ws,
+                                                      int lane, uint32_t nt, int init_mode, uint32_t negate_bits,
+                                                      float* __restrict__ mp, uint4* ring_base)
+{
+    constexpr int CPL = Store<ST>::CPL;
+    const Ring<CPL, NB> ring{ring_base};
+    const uint32_t nrows = (t.r_end - t.r0 + t.rstep - 1) / t.rstep;
+    const uint32_t nbat = (nt + NB - 1) / NB;
+    const uint32_t N = nrows * nbat;
+    const int sblk = CPL == 8 ? (lane >> 4) : 0;
+
+    auto offset_of = [&](uint32_t row) { return static_cast<size_t>(t.r0 + row * t.rstep) * cols + t.c; };
+
+    auto issue = [&](const Cursor& cu, int stage) {
+        const size_t off = offset_of(cu.row);
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
-        if (c + e < cols) v[e] = Io<ST>::load1(p + off + e);
-    return make_float4(v[0], v[1], v[2], v[3]);
+        for (int k = 0; k < NB; ++k) {
+            const uint32_t i = cu.b * NB + k;
+            if (i < nt) cp_async16(ring.slot(stage, k), static_cast<const ST*>(ws.pw[i]) + off);
+        }
+        if (cu.b == 0) {
+            if (BASE == kSharedBase) cp_async16(ring.slot(stage, NB), static_cast<const ST*>(ws.pb[0]) + off);
+            if (init_mode == kInitAsync) {
+#pragma unroll
+                for (int h = 0; h < CPL / 4; ++h) cp_async16(ring.slot(stage, NB + 1 + h), mp + off + 4 * h);
+            }
+        }
+    };
+
+    // W_0 tiles under a shuffle come from L2 (each is shared by several slots): they
+    // are fetched into registers one batch ahead instead of occupying the ring.
+    uint4 w0_next[NB];
+    auto prefetch_base = [&](const Cursor& cu) {
+        if (BASE != kPerTaskBase) return;
+        const size_t off = offset_of(cu.row);
+#pragma unroll
+        for (int k = 0; k < NB; ++k) {
+            const uint32_t i = cu.b * NB + k;
+            if (i < nt) w0_next[k] = __ldg(reinterpret_cast<const uint4*>(static_cast<const ST*>(ws.pb[i]) + off));
+        }
+    };
+
+    Cursor ci{0, 0}, cc{0, 0}, cp{0, 0};
+    uint32_t issued = 0;
+#pragma unroll
+    for (int s = 0; s < NSTAGE - 1; ++s) {
+        if (issued < N) { issue(ci, s); ci.advance(nbat); ++issued; }
+        cp_async_commit();
+    }
+    prefetch_base(cp);
+    cp.advance(nbat);
+
+    float acc[CPL], w0row[CPL];
+    int stage_c = 0, stage_i = NSTAGE - 1;
+    for (uint32_t it = 0; it < N; ++it) {
+        if (issued < N) { issue(ci, stage_i); ci.advance(nbat); ++issued; }
+        cp_async_commit();
+        stage_i = stage_i + 1 == NSTAGE ? 0 : stage_i + 1;
+
+        uint4 w0_cur[NB];
+        if (BASE == kPerTaskBase) {
+#pragma unroll
+            for (int k = 0; k < NB; ++k) w0_cur[k] = w0_next[k];
+            if (it + 1 < N) { prefetch_base(cp); cp.advance(nbat); }
+        }
+        cp_async_wait<NSTAGE - 1>();   // everything but the newest NSTAGE-1 groups has landed: stage_c is ready
+
+        const size_t off = offset_of(cc.row);
+        if (cc.b == 0) {
+#pragma unroll
+            for (int e = 0; e < CPL; ++e) { acc[e] = 0.f; w0row[e] = 0.f; }
+            if (init_mode == kInitAsync) {
+#pragma unroll
+                for (int h = 0; h < CPL / 4; ++h) {
+                    const uint4 raw = *ring.slot(stage_c, NB + 1 + h);
+                    acc[4 * h] = __uint_as_float(raw.x); acc[4 * h + 1] = __uint_as_float(raw.y);
+                    acc[4 * h + 2] = __uint_as_float(raw.z); acc[4 * h + 3] = __uint_as_float(raw.w);
+                }
+            } else if (init_mode == kInitPlain) {
+#pragma unroll
+                for (int h = 0; h < CPL / 4; ++h) {
+                    const float4 v = *reinterpret_cast<const float4*>(mp + off + 4 * h);
+                    acc[4 * h] = v.x; acc[4 * h + 1] = v.y; acc[4 * h + 2] = v.z; acc[4 * h + 3] = v.w;
+                }
+            }
+            if (BASE == kSharedBase) Store<ST>::widen(*ring.slot(stage_c, NB), w0row);
+        }
+#pragma unroll
+        for (int k = 0; k < NB; ++k) {
+            const uint32_t i = cc.b * NB + k;
+            if (i < nt) {
+                float d[CPL];
+                Store<ST>::widen(*ring.slot(stage_c, k), d);
+                if (BASE == kPerTaskBase) {
+                    float s[CPL];
+                    Store<ST>::widen(w0_cur[k], s);
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) d[e] = __fsub_rn(d[e], s[e]);
+                } else if (BASE == kSharedBase) {
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) d[e] = __fsub_rn(d[e], w0row[e]);
+                }
+                const uint32_t bits = lane_bits<CPL>(ws.sign[i][sblk], lane) ^ negate_bits;
+#pragma unroll
+                for (int e = 0; e < CPL; ++e) acc[e] = __fadd_rn(acc[e], flip(d[e], ((bits >> e) & 1u) << 31));
+            }
+        }
+        if (cc.b + 1 == nbat) {
+#pragma unroll
+            for (int h = 0; h < CPL / 4; ++h)
+                *reinterpret_cast<float4*>(mp + off + 4 * h) = make_float4(acc[4 * h], acc[4 * h + 1], acc[4 * h + 2], acc[4 * h + 3]);
+        }
+        cc.advance(nbat);
+        stage_c = stage_c + 1 == NSTAGE ? 0 : stage_c + 1;
+    }
+    cp_async_wait<0>();
 }
 
-template <typename ST, bool VEC>
-__device__ __forceinline__ void accumulate_rows(const WarpTile& t, uint32_t cols, const WarpScratch& ws, int lane,
-                                                uint32_t nt, bool init, bool has_base, bool per_task_base,
-                                                uint32_t negate_nib, float* __restrict__ mp)
+// Element-at-a-time path for layers whose width is not a multiple of the lane
+// width or whose tensors are not 16-byte aligned.  Kept out of line: it is rare
+// and must not set the register budget of the vector path.
+template <typename ST>
+__device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, const WarpScratch<Store<ST>::CPL>* wsp, int lane,
+                                                    uint32_t nt, int init_mode, uint32_t negate_bits, float* mp, int base_mode)
 {
-    constexpr int U = 2;
-    const int q = lane >> 3, sh = (lane & 7) * 4;
-    for (uint32_t r = t.r0; r < t.r_end; r += t.rstep * U) {
-        float4 acc[U], w0[U];
-        size_t off[U];
-        bool on[U];
-#pragma unroll
-        for (int j = 0; j < U; ++j) {
-            const uint32_t rr = r + j * t.rstep;
-            on[j] = rr < t.r_end;
-            off[j] = static_cast<size_t>(rr) * cols + t.c;
-            acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            w0[j] = acc[j];
-            if (on[j]) {
-                if (init) {
-                    if (VEC) {
-                        acc[j] = *reinterpret_cast<const float4*>(mp + off[j]);
-                    } else {
-                        float v[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            if (t.c + e < cols) v[e] = mp[off[j] + e];
-                        acc[j] = make_float4(v[0], v[1], v[2], v[3]);
-                    }
-                }
-                // without a shuffle every task subtracts the same W_0 tile: fetch it once
-                if (has_base && !per_task_base)
-                    w0[j] = load_tile<ST, VEC>(static_cast<const ST*>(ws.pb[0]), off[j], t.c, cols, true);
+    constexpr int CPL = Store<ST>::CPL;
+    const WarpScratch<CPL>& ws = *wsp;
+    const int sblk = CPL == 8 ? (lane >> 4) : 0;
+    for (uint32_t r = t.r0; r < t.r_end; r += t.rstep) {
+        const size_t off = static_cast<size_t>(r) * cols + t.c;
+        for (int e = 0; e < CPL; ++e) {
+            if (t.c + e >= cols) break;
+            float acc = init_mode == kInitZero ? 0.f : mp[off + e];
+            for (uint32_t i = 0; i < nt; ++i) {
+                float d = Store<ST>::load1(static_cast<const ST*>(ws.pw[i]) + off + e);
+                if (base_mode != kNoBase) d = __fsub_rn(d, Store<ST>::load1(static_cast<const ST*>(ws.pb[i]) + off + e));
+                const uint32_t bits = lane_bits<CPL>(ws.sign[i][sblk], lane) ^ negate_bits;
+                acc = __fadd_rn(acc, flip(d, ((bits >> e) & 1u) << 31));
             }
-        }
-#pragma unroll 4
-        for (uint32_t i = 0; i < nt; ++i) {
-            const ST* pw = static_cast<const ST*>(ws.pw[i]);
-            const ST* pb = static_cast<const ST*>(ws.pb[i]);
-            const uint4 sw = ws.sign[i];
-            const uint32_t word = q == 0 ? sw.x : (q == 1 ? sw.y : (q == 2 ? sw.z : sw.w));
-            const uint32_t nib = ((word >> sh) & 0xFu) ^ negate_nib;
-            const uint32_t m0 = (nib & 1u) << 31, m1 = (nib & 2u) << 30, m2 = (nib & 4u) << 29, m3 = (nib & 8u) << 28;
-#pragma unroll
-            for (int j = 0; j < U; ++j) {
-                if (!on[j]) continue;
-                float4 d = load_tile<ST, VEC>(pw, off[j], t.c, cols, true);
-                if (has_base) {
-                    const float4 b = per_task_base ? load_tile<ST, VEC>(pb, off[j], t.c, cols, false) : w0[j];
-                    d.x = __fsub_rn(d.x, b.x);
-                    d.y = __fsub_rn(d.y, b.y);
-                    d.z = __fsub_rn(d.z, b.z);
-                    d.w = __fsub_rn(d.w, b.w);
-                }
-                acc[j].x = __fadd_rn(acc[j].x, flip(d.x, m0));
-                acc[j].y = __fadd_rn(acc[j].y, flip(d.y, m1));
-                acc[j].z = __fadd_rn(acc[j].z, flip(d.z, m2));
-                acc[j].w = __fadd_rn(acc[j].w, flip(d.w, m3));
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < U; ++j) {
-            if (!on[j]) continue;
-            if (VEC) {
-                *reinterpret_cast<float4*>(mp + off[j]) = acc[j];
-            } else {
-                const float v[4] = {acc[j].x, acc[j].y, acc[j].z, acc[j].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (t.c + e < cols) mp[off[j] + e] = v[e];
-            }
+            mp[off + e] = acc;
         }
     }
 }
 
-template <typename ST>
-__global__ void __launch_bounds__(kThreadsPerCta) accumulate_kernel(const AccumulateArgs a)
+#ifndef RANDES_COMPRESS_NB
+#define RANDES_COMPRESS_NB 4
+#endif
+#ifndef RANDES_COMPRESS_NSTAGE_F32
+#define RANDES_COMPRESS_NSTAGE_F32 4
+#endif
+#ifndef RANDES_COMPRESS_NSTAGE_BF16
+#define RANDES_COMPRESS_NSTAGE_BF16 3
+#endif
+#ifndef RANDES_SINGLE_NSTAGE_F32
+#define RANDES_SINGLE_NSTAGE_F32 8
+#endif
+#ifndef RANDES_SINGLE_NSTAGE_BF16
+#define RANDES_SINGLE_NSTAGE_BF16 6
+#endif
+
+template <typename ST, bool SINGLE> struct AccConfig {
+    static constexpr int CPL = Store<ST>::CPL;
+    static constexpr int NB = SINGLE ? 1 : RANDES_COMPRESS_NB;
+    static constexpr int NSTAGE = SINGLE ? (CPL == 4 ? RANDES_SINGLE_NSTAGE_F32 : RANDES_SINGLE_NSTAGE_BF16)
+                                         : (CPL == 4 ? RANDES_COMPRESS_NSTAGE_F32 : RANDES_COMPRESS_NSTAGE_BF16);
+    static constexpr size_t kRingBytes = static_cast<size_t>(NSTAGE) * Ring<CPL, NB>::SLOTS * kThreadsPerCta * sizeof(uint4);
+    static constexpr size_t kSmemBytes = kRingBytes + kWarpsPerCta * sizeof(WarpScratch<CPL>);
+};
+
+// SINGLE: one task per launch (add / remove): a deep ring of rows.  Otherwise
+// (compress): NB tasks per stage.
+template <typename ST, bool SINGLE>
+__global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const AccumulateArgs a)
 {
-    __shared__ WarpScratch scratch[kWarpsPerCta];
+    typedef AccConfig<ST, SINGLE> Cfg;
+    constexpr int CPL = Cfg::CPL;
+    extern __shared__ __align__(16) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    WarpScratch& ws = scratch[warp];
+    uint4* ring_base = reinterpret_cast<uint4*>(smem) + threadIdx.x;
+    WarpScratch<CPL>& ws = reinterpret_cast<WarpScratch<CPL>*>(smem + Cfg::kRingBytes)[warp];
     const uint32_t L = a.n_layers;
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
         const uint32_t slot = un.layer;
         const DevLayer ls = a.layers[slot];
-        const WarpTile t = warp_tile(un, warp, lane);
-        if (t.r0 >= t.r_end || t.cb * kColsPerWarp >= ls.cols) continue;   // warp-uniform: nothing for this warp
+        const WarpTile t = warp_tile<CPL>(un, warp, lane);
+        if (t.r0 >= t.r_end || t.cb * 32 * CPL >= ls.cols) continue;   // warp-uniform: nothing for this warp
         const bool lane_on = t.c < ls.cols;
         const bool shuffled = (ls.flags & kFlagShuffle) != 0;
         const bool flipped = (ls.flags & kFlagFlip) != 0;
         float* mp = a.M + ls.m_off;
+        const int base_mode = !a.has_base ? kNoBase : ((shuffled && !SINGLE) ? kPerTaskBase : kSharedBase);
 
         for (uint32_t chunk0 = 0; chunk0 < a.n_tasks; chunk0 += kTaskChunk) {
             const uint32_t nt = min(static_cast<uint32_t>(kTaskChunk), a.n_tasks - chunk0);
@@ -332,33 +503,40 @@ __global__ void __launch_bounds__(kThreadsPerCta) accumulate_kernel(const Accumu
                 const void* pb = a.has_base ? a.base[src] : nullptr;
                 ws.pw[lane] = pw;
                 ws.pb[lane] = pb;
-                ok = vec_aligned<ST>(pw) && vec_aligned<ST>(pb);
-                uint32_t blk[4] = {0u, 0u, 0u, 0u};
-                if (flipped) {
-                    const DevTask tk = a.tasks[ti];
-                    philox4x32_10(t.cb, slot, kTagSign, tk.id, tk.key0, tk.key1, blk);
-                }
-                ws.sign[lane] = make_uint4(blk[0], blk[1], blk[2], blk[3]);
+                ok = aligned16(pw) && aligned16(pb);
+                const DevTask tk = a.tasks[ti];
+#pragma unroll
+                for (int h = 0; h < CPL / 4; ++h)
+                    ws.sign[lane][h] = flipped ? philox4x32_10(t.cb * (CPL / 4) + h, slot, kTagSign, tk.id, tk.key0, tk.key1)
+                                               : make_uint4(0u, 0u, 0u, 0u);
             }
-            const bool vec = (ls.cols & 3u) == 0 && __all_sync(0xFFFFFFFFu, ok);
+            const bool vec = ls.cols % CPL == 0 && __all_sync(0xFFFFFFFFu, ok);
             __syncwarp();
             if (lane_on) {
-                const bool init = a.init_from_m != 0 || chunk0 > 0;
-                const uint32_t neg = a.negate ? 0xFu : 0u;
-                if (vec)
-                    accumulate_rows<ST, true>(t, ls.cols, ws, lane, nt, init, a.has_base != 0, shuffled, neg, mp);
+                const int init_mode = chunk0 > 0 ? kInitPlain : (a.init_from_m ? kInitAsync : kInitZero);
+                const uint32_t neg = a.negate ? (CPL == 4 ? 0xFu : 0xFFu) : 0u;
+                if (!vec)
+                    accumulate_rows_scalar<ST>(t, ls.cols, &ws, lane, nt, init_mode, neg, mp, base_mode);
+                else if (base_mode == kNoBase)
+                    accumulate_rows_async<ST, kNoBase, Cfg::NB, Cfg::NSTAGE>(t, ls.cols, ws, lane, nt, init_mode, neg, mp, ring_base);
+                else if (base_mode == kSharedBase)
+                    accumulate_rows_async<ST, kSharedBase, Cfg::NB, Cfg::NSTAGE>(t, ls.cols, ws, lane, nt, init_mode, neg, mp, ring_base);
                 else
-                    accumulate_rows<ST, false>(t, ls.cols, ws, lane, nt, init, a.has_base != 0, shuffled, neg, mp);
+                    accumulate_rows_async<ST, kPerTaskBase, Cfg::NB, Cfg::NSTAGE>(t, ls.cols, ws, lane, nt, init_mode, neg, mp, ring_base);
             }
         }
     }
 }
 
-template <typename K>
-int ctas_per_sm(K kernel)
+template <typename K> int ctas_per_sm(K kernel, size_t smem)
 {
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreadsPerCta, 0) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreadsPerCta, smem) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }
@@ -380,22 +558,32 @@ int launch_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, int
 int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void* stream)
 {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (storage_dtype == 0) accumulate_kernel<float><<<grid, kThreadsPerCta, 0, s>>>(a);
-    else accumulate_kernel<bf16><<<grid, kThreadsPerCta, 0, s>>>(a);
+    const bool single = a.n_tasks == 1;
+    if (storage_dtype == 0) {
+        if (single) accumulate_kernel<float, true><<<grid, kThreadsPerCta, AccConfig<float, true>::kSmemBytes, s>>>(a);
+        else accumulate_kernel<float, false><<<grid, kThreadsPerCta, AccConfig<float, false>::kSmemBytes, s>>>(a);
+    } else {
+        if (single) accumulate_kernel<bf16, true><<<grid, kThreadsPerCta, AccConfig<bf16, true>::kSmemBytes, s>>>(a);
+        else accumulate_kernel<bf16, false><<<grid, kThreadsPerCta, AccConfig<bf16, false>::kSmemBytes, s>>>(a);
+    }
     return static_cast<int>(cudaGetLastError());
 }
 
 int retrieve_ctas_per_sm(int storage_dtype, int out_dtype)
 {
-    if (storage_dtype == 0 && out_dtype == 0) return ctas_per_sm(retrieve_kernel<float, float>);
-    if (storage_dtype == 0 && out_dtype == 1) return ctas_per_sm(retrieve_kernel<float, bf16>);
-    if (storage_dtype == 1 && out_dtype == 0) return ctas_per_sm(retrieve_kernel<bf16, float>);
-    return ctas_per_sm(retrieve_kernel<bf16, bf16>);
+    if (storage_dtype == 0 && out_dtype == 0) return ctas_per_sm(retrieve_kernel<float, float>, 0);
+    if (storage_dtype == 0 && out_dtype == 1) return ctas_per_sm(retrieve_kernel<float, bf16>, 0);
+    if (storage_dtype == 1 && out_dtype == 0) return ctas_per_sm(retrieve_kernel<bf16, float>, 0);
+    return ctas_per_sm(retrieve_kernel<bf16, bf16>, 0);
 }
 
-int accumulate_ctas_per_sm(int storage_dtype)
+int accumulate_ctas_per_sm(int storage_dtype, bool single)
 {
-    return storage_dtype == 0 ? ctas_per_sm(accumulate_kernel<float>) : ctas_per_sm(accumulate_kernel<bf16>);
+    if (storage_dtype == 0)
+        return single ? ctas_per_sm(accumulate_kernel<float, true>, AccConfig<float, true>::kSmemBytes)
+                      : ctas_per_sm(accumulate_kernel<float, false>, AccConfig<float, false>::kSmemBytes);
+    return single ? ctas_per_sm(accumulate_kernel<bf16, true>, AccConfig<bf16, true>::kSmemBytes)
+                  : ctas_per_sm(accumulate_kernel<bf16, false>, AccConfig<bf16, false>::kSmemBytes);
 }
 
 }  // namespace randes

@@ -255,14 +255,14 @@ __global__ void __launch_bounds__(kThreadsPerCta) retrieve_kernel(const Retrieve
 // accumulate:  M[l] (=|+=|-=) sum_i s_i(l, c) * ( W_i[sigma_i(l)] - W_0[sigma_i(l)] )
 // compress (Section 4, first display): all registered tasks, from +0, in plan order.
 // add / remove (Section 5.7): one task, starting from M, sign negated for remove.
-// A warp keeps the resolved source pointers and the Philox sign blocks of up to
-// kTaskChunk tasks in its private shared-memory scratch: lane i prepares task i.
+//
+// Per unit a warp first resolves, for up to MAXT tasks, the source pointers
+// (lane i looks up sigma_i(l) for task i) and the sign bits (lane i runs Philox
+// for task i; every lane then gathers its own columns' bits of NB tasks into one
+// word per batch).  The row loop is then a software pipeline over (row, batch of
+// NB tasks): W_i tiles travel through a per-thread cp.async ring in shared
+// memory, several stages ahead of their use.
 // =========================================================================================
-template <int CPL> struct WarpScratch {
-    const void* pw[kTaskChunk];
-    const void* pb[kTaskChunk];
-    uint4 sign[kTaskChunk][CPL / 4];
-};
 
 // How W_0 enters the difference W_i - W_0.
 constexpr int kNoBase = 0;        // the task tensors already hold deltas
@@ -273,125 +273,135 @@ constexpr int kInitZero = 0;      // start from +0
 constexpr int kInitAsync = 1;     // start from M written by an earlier launch: staged like the weights
 constexpr int kInitPlain = 2;     // start from M written earlier by this thread: plain load
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
+constexpr uint32_t kSlotBytes = kThreadsPerCta * 16;   // one 16-byte slot of every thread of the CTA
+
+template <int NB, int MAXT> struct WarpScratch {
+    const void* pw[MAXT];
+    const void* pb[MAXT];
+    uint32_t bits[(MAXT + NB - 1) / NB][32];   // [batch][lane]: bit k*CPL + e = sign of column e for task k of the batch
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src)
 {
-    const uint32_t s = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem_src) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint4 lds128(uint32_t saddr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t saddr, const uint4& v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 
-// Position in the flattened (row, batch-of-tasks) sequence a warp walks.
-struct Cursor {
-    uint32_t row, b;
-    __device__ __forceinline__ void advance(uint32_t nbat) { if (++b == nbat) { b = 0; ++row; } }
-};
-
-// Shared-memory ring of one thread: NSTAGE stages x SLOTS 16-byte slots, slot-major
-// across the CTA's threads (consecutive lanes are contiguous: conflict-free).
+// Ring of one thread: NSTAGE stages x SLOTS 16-byte slots, slot-major across the
+// CTA's threads (consecutive lanes are contiguous: conflict-free).  Per stage:
 //   slots [0, NB)            W_i tiles of the batch
 //   slot  NB                 W_0 tile of the row (kSharedBase), filled with the row's first batch
 //   slots NB+1 .. NB+CPL/4   M tile of the row (kInitAsync), filled with the row's first batch
-template <int CPL, int NB> struct Ring {
+template <int CPL, int NB> struct RingGeom {
     static constexpr int SLOTS = NB + 1 + CPL / 4;
-    uint4* base;   // this thread's slot 0 of stage 0
-    __device__ __forceinline__ uint4* slot(int stage, int s) const { return base + (stage * SLOTS + s) * kThreadsPerCta; }
+    static constexpr uint32_t kStageBytes = SLOTS * kSlotBytes;
 };
 
-template <typename ST, int BASE, int NB, int NSTAGE>
-__device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_t cols, const WarpScratch<Store<ST>::CPL>& ws,
-                                                      int lane, uint32_t nt, int init_mode, uint32_t negate_bits,
-                                                      float* __restrict__ mp, uint4* ring_base)
+template <typename ST, int BASE, int NB, int NSTAGE, int MAXT, bool FULL>
+__device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_t cols, const WarpScratch<NB, MAXT>& ws, int lane,
+                                                      uint32_t nt, int init_mode, float* __restrict__ mp, uint32_t ring)
 {
     constexpr int CPL = Store<ST>::CPL;
-    const Ring<CPL, NB> ring{ring_base};
+    typedef RingGeom<CPL, NB> G;
+    static_assert(NB * CPL <= 32, "a batch's sign bits must fit one word");
     const uint32_t nrows = (t.r_end - t.r0 + t.rstep - 1) / t.rstep;
     const uint32_t nbat = (nt + NB - 1) / NB;
     const uint32_t N = nrows * nbat;
-    const int sblk = CPL == 8 ? (lane >> 4) : 0;
+    const uint32_t row_stride = t.rstep * cols;          // elements between this warp's rows
+    const uint32_t off0 = t.r0 * cols + t.c;             // element offset of the first tile (layers hold < 2^32 elements)
 
-    auto offset_of = [&](uint32_t row) { return static_cast<size_t>(t.r0 + row * t.rstep) * cols + t.c; };
+    // three cursors over the same (row, batch) sequence: copies issued, W_0 prefetched, consumed
+    uint32_t off_i = off0, b_i = 0, off_p = off0, b_p = 0, off_c = off0, b_c = 0;
 
-    auto issue = [&](const Cursor& cu, int stage) {
-        const size_t off = offset_of(cu.row);
+    auto issue = [&](uint32_t stage) {
 #pragma unroll
         for (int k = 0; k < NB; ++k) {
-            const uint32_t i = cu.b * NB + k;
-            if (i < nt) cp_async16(ring.slot(stage, k), static_cast<const ST*>(ws.pw[i]) + off);
+            const uint32_t i = b_i * NB + k;
+            if (FULL || i < nt) cp_async16(stage + k * kSlotBytes, static_cast<const ST*>(ws.pw[i]) + off_i);
         }
-        if (cu.b == 0) {
-            if (BASE == kSharedBase) cp_async16(ring.slot(stage, NB), static_cast<const ST*>(ws.pb[0]) + off);
+        if (b_i == 0) {
+            if (BASE == kSharedBase) cp_async16(stage + NB * kSlotBytes, static_cast<const ST*>(ws.pb[0]) + off_i);
             if (init_mode == kInitAsync) {
 #pragma unroll
-                for (int h = 0; h < CPL / 4; ++h) cp_async16(ring.slot(stage, NB + 1 + h), mp + off + 4 * h);
+                for (int h = 0; h < CPL / 4; ++h) cp_async16(stage + (NB + 1 + h) * kSlotBytes, mp + off_i + 4 * h);
             }
         }
+        if (++b_i == nbat) { b_i = 0; off_i += row_stride; }
     };
 
     // W_0 tiles under a shuffle come from L2 (each is shared by several slots): they
     // are fetched into registers one batch ahead instead of occupying the ring.
     uint4 w0_next[NB];
-    auto prefetch_base = [&](const Cursor& cu) {
-        if (BASE != kPerTaskBase) return;
-        const size_t off = offset_of(cu.row);
+    auto prefetch_base = [&]() {
 #pragma unroll
         for (int k = 0; k < NB; ++k) {
-            const uint32_t i = cu.b * NB + k;
-            if (i < nt) w0_next[k] = __ldg(reinterpret_cast<const uint4*>(static_cast<const ST*>(ws.pb[i]) + off));
+            const uint32_t i = b_p * NB + k;
+            if (FULL || i < nt) w0_next[k] = __ldg(reinterpret_cast<const uint4*>(static_cast<const ST*>(ws.pb[i]) + off_p));
         }
+        if (++b_p == nbat) { b_p = 0; off_p += row_stride; }
     };
 
-    Cursor ci{0, 0}, cc{0, 0}, cp{0, 0};
     uint32_t issued = 0;
 #pragma unroll
     for (int s = 0; s < NSTAGE - 1; ++s) {
-        if (issued < N) { issue(ci, s); ci.advance(nbat); ++issued; }
+        if (issued < N) { issue(ring + s * G::kStageBytes); ++issued; }
         cp_async_commit();
     }
-    prefetch_base(cp);
-    cp.advance(nbat);
+    if (BASE == kPerTaskBase) prefetch_base();
 
     float acc[CPL], w0row[CPL];
-    int stage_c = 0, stage_i = NSTAGE - 1;
+    uint32_t stage_c = ring, stage_i = ring + (NSTAGE - 1) * G::kStageBytes;
+    const uint32_t ring_end = ring + NSTAGE * G::kStageBytes;
     for (uint32_t it = 0; it < N; ++it) {
-        if (issued < N) { issue(ci, stage_i); ci.advance(nbat); ++issued; }
+        if (issued < N) { issue(stage_i); ++issued; }
         cp_async_commit();
-        stage_i = stage_i + 1 == NSTAGE ? 0 : stage_i + 1;
+        stage_i += G::kStageBytes;
+        if (stage_i == ring_end) stage_i = ring;
 
         uint4 w0_cur[NB];
         if (BASE == kPerTaskBase) {
 #pragma unroll
             for (int k = 0; k < NB; ++k) w0_cur[k] = w0_next[k];
-            if (it + 1 < N) { prefetch_base(cp); cp.advance(nbat); }
+            if (it + 1 < N) prefetch_base();
         }
         cp_async_wait<NSTAGE - 1>();   // everything but the newest NSTAGE-1 groups has landed: stage_c is ready
 
-        const size_t off = offset_of(cc.row);
-        if (cc.b == 0) {
+        if (b_c == 0) {
 #pragma unroll
             for (int e = 0; e < CPL; ++e) { acc[e] = 0.f; w0row[e] = 0.f; }
             if (init_mode == kInitAsync) {
 #pragma unroll
                 for (int h = 0; h < CPL / 4; ++h) {
-                    const uint4 raw = *ring.slot(stage_c, NB + 1 + h);
+                    const uint4 raw = lds128(stage_c + (NB + 1 + h) * kSlotBytes);
                     acc[4 * h] = __uint_as_float(raw.x); acc[4 * h + 1] = __uint_as_float(raw.y);
                     acc[4 * h + 2] = __uint_as_float(raw.z); acc[4 * h + 3] = __uint_as_float(raw.w);
                 }
             } else if (init_mode == kInitPlain) {
 #pragma unroll
                 for (int h = 0; h < CPL / 4; ++h) {
-                    const float4 v = *reinterpret_cast<const float4*>(mp + off + 4 * h);
+                    const float4 v = *reinterpret_cast<const float4*>(mp + off_c + 4 * h);
                     acc[4 * h] = v.x; acc[4 * h + 1] = v.y; acc[4 * h + 2] = v.z; acc[4 * h + 3] = v.w;
                 }
             }
-            if (BASE == kSharedBase) Store<ST>::widen(*ring.slot(stage_c, NB), w0row);
+            if (BASE == kSharedBase) Store<ST>::widen(lds128(stage_c + NB * kSlotBytes), w0row);
         }
+        const uint32_t pack = ws.bits[b_c][lane];
 #pragma unroll
         for (int k = 0; k < NB; ++k) {
-            const uint32_t i = cc.b * NB + k;
-            if (i < nt) {
+            if (FULL || b_c * NB + k < nt) {
                 float d[CPL];
-                Store<ST>::widen(*ring.slot(stage_c, k), d);
+                Store<ST>::widen(lds128(stage_c + k * kSlotBytes), d);
                 if (BASE == kPerTaskBase) {
                     float s[CPL];
                     Store<ST>::widen(w0_cur[k], s);
@@ -401,18 +411,22 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
 #pragma unroll
                     for (int e = 0; e < CPL; ++e) d[e] = __fsub_rn(d[e], w0row[e]);
                 }
-                const uint32_t bits = lane_bits<CPL>(ws.sign[i][sblk], lane) ^ negate_bits;
 #pragma unroll
-                for (int e = 0; e < CPL; ++e) acc[e] = __fadd_rn(acc[e], flip(d[e], ((bits >> e) & 1u) << 31));
+                for (int e = 0; e < CPL; ++e)
+                    acc[e] = __fadd_rn(acc[e], flip(d[e], (pack << (31 - (k * CPL + e))) & 0x80000000u));
             }
         }
-        if (cc.b + 1 == nbat) {
+        if (b_c + 1 == nbat) {
 #pragma unroll
             for (int h = 0; h < CPL / 4; ++h)
-                *reinterpret_cast<float4*>(mp + off + 4 * h) = make_float4(acc[4 * h], acc[4 * h + 1], acc[4 * h + 2], acc[4 * h + 3]);
+                *reinterpret_cast<float4*>(mp + off_c + 4 * h) = make_float4(acc[4 * h], acc[4 * h + 1], acc[4 * h + 2], acc[4 * h + 3]);
+            b_c = 0;
+            off_c += row_stride;
+        } else {
+            ++b_c;
         }
-        cc.advance(nbat);
-        stage_c = stage_c + 1 == NSTAGE ? 0 : stage_c + 1;
+        stage_c += G::kStageBytes;
+        if (stage_c == ring_end) stage_c = ring;
     }
     cp_async_wait<0>();
 }
@@ -420,13 +434,12 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
 // Element-at-a-time path for layers whose width is not a multiple of the lane
 // width or whose tensors are not 16-byte aligned.  Kept out of line: it is rare
 // and must not set the register budget of the vector path.
-template <typename ST>
-__device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, const WarpScratch<Store<ST>::CPL>* wsp, int lane,
-                                                    uint32_t nt, int init_mode, uint32_t negate_bits, float* mp, int base_mode)
+template <typename ST, int NB, int MAXT>
+__device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, const WarpScratch<NB, MAXT>* wsp, int lane,
+                                                    uint32_t nt, int init_mode, float* mp, int base_mode)
 {
     constexpr int CPL = Store<ST>::CPL;
-    const WarpScratch<CPL>& ws = *wsp;
-    const int sblk = CPL == 8 ? (lane >> 4) : 0;
+    const WarpScratch<NB, MAXT>& ws = *wsp;
     for (uint32_t r = t.r0; r < t.r_end; r += t.rstep) {
         const size_t off = static_cast<size_t>(r) * cols + t.c;
         for (int e = 0; e < CPL; ++e) {
@@ -435,8 +448,8 @@ __device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, c
             for (uint32_t i = 0; i < nt; ++i) {
                 float d = Store<ST>::load1(static_cast<const ST*>(ws.pw[i]) + off + e);
                 if (base_mode != kNoBase) d = __fsub_rn(d, Store<ST>::load1(static_cast<const ST*>(ws.pb[i]) + off + e));
-                const uint32_t bits = lane_bits<CPL>(ws.sign[i][sblk], lane) ^ negate_bits;
-                acc = __fadd_rn(acc, flip(d, ((bits >> e) & 1u) << 31));
+                const uint32_t bit = (ws.bits[i / NB][lane] >> ((i % NB) * CPL + e)) & 1u;
+                acc = __fadd_rn(acc, flip(d, bit << 31));
             }
             mp[off + e] = acc;
         }
@@ -462,10 +475,12 @@ __device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, c
 template <typename ST, bool SINGLE> struct AccConfig {
     static constexpr int CPL = Store<ST>::CPL;
     static constexpr int NB = SINGLE ? 1 : RANDES_COMPRESS_NB;
+    static constexpr int MAXT = SINGLE ? 1 : kTaskChunk;
     static constexpr int NSTAGE = SINGLE ? (CPL == 4 ? RANDES_SINGLE_NSTAGE_F32 : RANDES_SINGLE_NSTAGE_BF16)
                                          : (CPL == 4 ? RANDES_COMPRESS_NSTAGE_F32 : RANDES_COMPRESS_NSTAGE_BF16);
-    static constexpr size_t kRingBytes = static_cast<size_t>(NSTAGE) * Ring<CPL, NB>::SLOTS * kThreadsPerCta * sizeof(uint4);
-    static constexpr size_t kSmemBytes = kRingBytes + kWarpsPerCta * sizeof(WarpScratch<CPL>);
+    typedef WarpScratch<NB, MAXT> Scratch;
+    static constexpr size_t kRingBytes = static_cast<size_t>(NSTAGE) * RingGeom<CPL, NB>::kStageBytes;
+    static constexpr size_t kSmemBytes = kRingBytes + kWarpsPerCta * sizeof(Scratch);
 };
 
 // SINGLE: one task per launch (add / remove): a deep ring of rows.  Otherwise
@@ -474,12 +489,15 @@ template <typename ST, bool SINGLE>
 __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const AccumulateArgs a)
 {
     typedef AccConfig<ST, SINGLE> Cfg;
-    constexpr int CPL = Cfg::CPL;
+    constexpr int CPL = Cfg::CPL, NB = Cfg::NB, MAXT = Cfg::MAXT, NS = Cfg::NSTAGE;
     extern __shared__ __align__(16) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint4* ring_base = reinterpret_cast<uint4*>(smem) + threadIdx.x;
-    WarpScratch<CPL>& ws = reinterpret_cast<WarpScratch<CPL>*>(smem + Cfg::kRingBytes)[warp];
+    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + threadIdx.x * 16;
+    // between units the ring is idle: its first slots double as the warp's table of Philox blocks
+    const uint32_t blocks = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * 512;
+    typename Cfg::Scratch& ws = reinterpret_cast<typename Cfg::Scratch*>(smem + Cfg::kRingBytes)[warp];
     const uint32_t L = a.n_layers;
+    const uint32_t negate_bits = a.negate ? 0xFFFFFFFFu : 0u;
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
         const uint32_t slot = un.layer;
@@ -492,8 +510,8 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const Acc
         float* mp = a.M + ls.m_off;
         const int base_mode = !a.has_base ? kNoBase : ((shuffled && !SINGLE) ? kPerTaskBase : kSharedBase);
 
-        for (uint32_t chunk0 = 0; chunk0 < a.n_tasks; chunk0 += kTaskChunk) {
-            const uint32_t nt = min(static_cast<uint32_t>(kTaskChunk), a.n_tasks - chunk0);
+        for (uint32_t chunk0 = 0; chunk0 < a.n_tasks; chunk0 += MAXT) {
+            const uint32_t nt = min(static_cast<uint32_t>(MAXT), a.n_tasks - chunk0);
             __syncwarp();   // the previous chunk's readers are done with the scratch
             bool ok = true;
             if (lane < nt) {
@@ -504,25 +522,46 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const Acc
                 ws.pw[lane] = pw;
                 ws.pb[lane] = pb;
                 ok = aligned16(pw) && aligned16(pb);
-                const DevTask tk = a.tasks[ti];
+                if (flipped) {
+                    const DevTask tk = a.tasks[ti];
 #pragma unroll
-                for (int h = 0; h < CPL / 4; ++h)
-                    ws.sign[lane][h] = flipped ? philox4x32_10(t.cb * (CPL / 4) + h, slot, kTagSign, tk.id, tk.key0, tk.key1)
-                                               : make_uint4(0u, 0u, 0u, 0u);
+                    for (int h = 0; h < CPL / 4; ++h)
+                        sts128(blocks + h * kSlotBytes + lane * 16,
+                               philox4x32_10(t.cb * (CPL / 4) + h, slot, kTagSign, tk.id, tk.key0, tk.key1));
+                }
             }
             const bool vec = ls.cols % CPL == 0 && __all_sync(0xFFFFFFFFu, ok);
             __syncwarp();
+            // every lane gathers the bits of its own columns, NB tasks to a word
+            const uint32_t nbat = (nt + NB - 1) / NB;
+            for (uint32_t b = 0; b < nbat; ++b) {
+                uint32_t pack = 0;
+                if (flipped) {
+#pragma unroll
+                    for (int k = 0; k < NB; ++k) {
+                        const uint32_t i = b * NB + k;
+                        if (i < nt)
+                            pack |= lane_bits<CPL>(lds128(blocks + (CPL == 8 ? (lane >> 4) : 0) * kSlotBytes + i * 16), lane) << (k * CPL);
+                    }
+                }
+                ws.bits[b][lane] = pack ^ negate_bits;
+            }
+            __syncwarp();   // the block table is free again before any lane's copies land in the ring
             if (lane_on) {
                 const int init_mode = chunk0 > 0 ? kInitPlain : (a.init_from_m ? kInitAsync : kInitZero);
-                const uint32_t neg = a.negate ? (CPL == 4 ? 0xFu : 0xFFu) : 0u;
+                const bool full = nt % NB == 0;
                 if (!vec)
-                    accumulate_rows_scalar<ST>(t, ls.cols, &ws, lane, nt, init_mode, neg, mp, base_mode);
-                else if (base_mode == kNoBase)
-                    accumulate_rows_async<ST, kNoBase, Cfg::NB, Cfg::NSTAGE>(t, ls.cols, ws, lane, nt, init_mode, neg, mp, ring_base);
-                else if (base_mode == kSharedBase)
-                    accumulate_rows_async<ST, kSharedBase, Cfg::NB, Cfg::NSTAGE>(t, ls.cols, ws, lane, nt, init_mode, neg, mp, ring_base);
-                else
-                    accumulate_rows_async<ST, kPerTaskBase, Cfg::NB, Cfg::NSTAGE>(t, ls.cols, ws, lane, nt, init_mode, neg, mp, ring_base);
+                    accumulate_rows_scalar<ST, NB, MAXT>(t, ls.cols, &ws, lane, nt, init_mode, mp, base_mode);
+                else if (base_mode == kNoBase) {
+                    if (full) accumulate_rows_async<ST, kNoBase, NB, NS, MAXT, true>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
+                    else accumulate_rows_async<ST, kNoBase, NB, NS, MAXT, false>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
+                } else if (base_mode == kSharedBase) {
+                    if (full) accumulate_rows_async<ST, kSharedBase, NB, NS, MAXT, true>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
+                    else accumulate_rows_async<ST, kSharedBase, NB, NS, MAXT, false>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
+                } else {
+                    if (full) accumulate_rows_async<ST, kPerTaskBase, NB, NS, MAXT, true>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
+                    else accumulate_rows_async<ST, kPerTaskBase, NB, NS, MAXT, false>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
+                }
             }
         }
     }

@@ -47,6 +47,35 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 
 __device__ __forceinline__ float flip(float x, uint32_t mask) { return __uint_as_float(__float_as_uint(x) ^ mask); }
 
+// Two fp32 values in one 64-bit register, for the packed add / sub / fma of sm_100.
+// Each half is rounded to nearest even exactly like the scalar instruction.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(uint32_t lo, uint32_t hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi)
+{
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
 // ---- storage types: a lane's 16 bytes hold CPL columns -------------------------------------
 template <typename T> struct Store;
 
@@ -56,6 +85,11 @@ template <> struct Store<float> {
     {
         v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
         v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
+    }
+    static __device__ __forceinline__ void widen2(const uint4& raw, f32x2 (&v)[2])
+    {
+        v[0] = pack2(raw.x, raw.y);
+        v[1] = pack2(raw.z, raw.w);
     }
     static __device__ __forceinline__ float load1(const float* p) { return __ldg(p); }
 };
@@ -68,6 +102,13 @@ template <> struct Store<bf16> {
         v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xFFFF0000u);
         v[4] = __uint_as_float(raw.z << 16); v[5] = __uint_as_float(raw.z & 0xFFFF0000u);
         v[6] = __uint_as_float(raw.w << 16); v[7] = __uint_as_float(raw.w & 0xFFFF0000u);
+    }
+    static __device__ __forceinline__ void widen2(const uint4& raw, f32x2 (&v)[4])
+    {
+        v[0] = pack2(raw.x << 16, raw.x & 0xFFFF0000u);
+        v[1] = pack2(raw.y << 16, raw.y & 0xFFFF0000u);
+        v[2] = pack2(raw.z << 16, raw.z & 0xFFFF0000u);
+        v[3] = pack2(raw.w << 16, raw.w & 0xFFFF0000u);
     }
     static __device__ __forceinline__ float load1(const bf16* p)
     {
@@ -259,9 +300,11 @@ __global__ void __launch_bounds__(kThreadsPerCta) retrieve_kernel(const Retrieve
 // Per unit a warp first resolves, for up to MAXT tasks, the source pointers
 // (lane i looks up sigma_i(l) for task i) and the sign bits (lane i runs Philox
 // for task i; every lane then gathers its own columns' bits of NB tasks into one
-// word per batch).  The row loop is then a software pipeline over (row, batch of
-// NB tasks): W_i tiles travel through a per-thread cp.async ring in shared
-// memory, several stages ahead of their use.
+// word per batch).  The row loop is then a software pipeline over (U rows, batch
+// of NB tasks): W_i tiles travel through a per-thread cp.async ring in shared
+// memory, several stages ahead of their use.  Arithmetic uses the packed fp32x2
+// instructions: d = W_i - W_0 (one rounding per half), acc = fma(d, +-1, acc)
+// (the product is exact, so this is acc + (+-d) with one rounding).
 // =========================================================================================
 
 // How W_0 enters the difference W_i - W_0.
@@ -269,22 +312,13 @@ constexpr int kNoBase = 0;        // the task tensors already hold deltas
 constexpr int kSharedBase = 1;    // no shuffle: every task subtracts the same W_0 tile, fetched once per row
 constexpr int kPerTaskBase = 2;   // shuffle: task i subtracts W_0[sigma_i(l)]; tiles repeat across slots and hit in L2
 
-constexpr int kInitZero = 0;      // start from +0
-constexpr int kInitAsync = 1;     // start from M written by an earlier launch: staged like the weights
-constexpr int kInitPlain = 2;     // start from M written earlier by this thread: plain load
-
 constexpr uint32_t kSlotBytes = kThreadsPerCta * 16;   // one 16-byte slot of every thread of the CTA
-
-template <int NB, int MAXT> struct WarpScratch {
-    const void* pw[MAXT];
-    const void* pb[MAXT];
-    uint32_t bits[(MAXT + NB - 1) / NB][32];   // [batch][lane]: bit k*CPL + e = sign of column e for task k of the batch
-};
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void* gmem) { asm volatile("prefetch.global.L2 [%0];" ::"l"(gmem)); }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ uint4 lds128(uint32_t saddr)
@@ -293,135 +327,212 @@ __device__ __forceinline__ uint4 lds128(uint32_t saddr)
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
     return v;
 }
+__device__ __forceinline__ const char* lds_ptr(uint32_t saddr)
+{
+    unsigned long long v;
+    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(saddr));
+    return reinterpret_cast<const char*>(v);
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t saddr)
+{
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(saddr));
+    return v;
+}
 __device__ __forceinline__ void sts128(uint32_t saddr, const uint4& v)
 {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+__device__ __forceinline__ void sts_u16(uint32_t saddr, uint32_t v)
+{
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(saddr), "h"(static_cast<unsigned short>(v)) : "memory");
+}
+__device__ __forceinline__ void sts_ptrs(uint32_t saddr, const void* a, const void* b)
+{
+    asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(saddr), "l"(a), "l"(b) : "memory");
+}
 
-// Ring of one thread: NSTAGE stages x SLOTS 16-byte slots, slot-major across the
-// CTA's threads (consecutive lanes are contiguous: conflict-free).  Per stage:
-//   slots [0, NB)            W_i tiles of the batch
-//   slot  NB                 W_0 tile of the row (kSharedBase), filled with the row's first batch
-//   slots NB+1 .. NB+CPL/4   M tile of the row (kInitAsync), filled with the row's first batch
-template <int CPL, int NB> struct RingGeom {
-    static constexpr int SLOTS = NB + 1 + CPL / 4;
-    static constexpr uint32_t kStageBytes = SLOTS * kSlotBytes;
+// Shared memory of the accumulate kernel, per CTA:
+//   ring     kRingSlots slots x (256 threads x 16 B), cut into stages whose layout
+//            depends on how W_0 comes in (StageGeom)
+//   per warp ptrs[MAXT] = {W_i layer, W_0 layer} resolved through sigma_i, 16 B each
+//            bits[MAXT/NB][32 lanes] 16-bit words: bit k*CPL + e = sign of column e for task k
+constexpr int kRingSlots = 24;    // 16-byte slots per thread: 96 KiB per CTA, two CTAs per SM
+
+template <typename ST, bool SINGLE> struct AccConfig {
+    static constexpr int CPL = Store<ST>::CPL;
+    static constexpr int U = SINGLE ? 1 : 2;          // rows per stage
+    static constexpr int NB = SINGLE ? 1 : 2;         // tasks per stage
+    static constexpr int MAXT = SINGLE ? 1 : kTaskChunk;
+    static constexpr bool kAsyncInit = SINGLE;        // add / remove start from M
+    static constexpr uint32_t kRingBytes = kRingSlots * kSlotBytes;
+    static constexpr int kBatches = (MAXT + NB - 1) / NB;
+    static constexpr uint32_t kPtrBytes = MAXT * 16;
+    static constexpr uint32_t kWarpBytes = kPtrBytes + kBatches * 64;
+    static constexpr size_t kSmemBytes = kRingBytes + kWarpsPerCta * kWarpBytes;
+    static_assert(NB * CPL <= 16, "a batch's sign bits must fit a 16-bit word");
 };
 
-template <typename ST, int BASE, int NB, int NSTAGE, int MAXT, bool FULL>
-__device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_t cols, const WarpScratch<NB, MAXT>& ws, int lane,
-                                                      uint32_t nt, int init_mode, float* __restrict__ mp, uint32_t ring)
+// Stage layout for one way of bringing W_0 in (slot-major across the CTA's threads):
+//   [0, U*NB)                 W_i tiles, slot u*NB + k = row u, task k of the batch
+//   kPerTaskBase: next U*NB   W_0[sigma_i(l)] tiles, same order (L2 hits, staged as deep as the W_i)
+//   kSharedBase:  next U      W_0 tile of row u, filled with the rows' first batch
+//   add / remove: next U*CPL/4  M tiles of the rows, filled likewise
+template <typename ST, bool SINGLE, int BASE> struct StageGeom {
+    typedef AccConfig<ST, SINGLE> C;
+    static constexpr int kW = 0;
+    static constexpr int kB = C::U * C::NB;
+    static constexpr int kM = kB + (BASE == kPerTaskBase ? C::U * C::NB : (BASE == kSharedBase ? C::U : 0));
+    static constexpr int SLOTS = kM + (C::kAsyncInit ? C::U * C::CPL / 4 : 0);
+    static constexpr int NSTAGE = (kRingSlots / SLOTS) > 8 ? 8 : (kRingSlots / SLOTS);
+    static constexpr uint32_t kStageBytes = SLOTS * kSlotBytes;
+    static_assert(NSTAGE >= 2, "ring too small");
+};
+
+template <typename ST, bool SINGLE, int BASE, bool FULL>
+__device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_t cols, uint32_t nt, bool init_plain, bool init_async,
+                                                      float* __restrict__ mp, uint32_t ring, uint32_t sptr, uint32_t sbits)
 {
-    constexpr int CPL = Store<ST>::CPL;
-    typedef RingGeom<CPL, NB> G;
-    static_assert(NB * CPL <= 32, "a batch's sign bits must fit one word");
+    typedef AccConfig<ST, SINGLE> C;
+    typedef StageGeom<ST, SINGLE, BASE> G;
+    constexpr int CPL = C::CPL, U = C::U, NB = C::NB, NSTAGE = G::NSTAGE;
+    constexpr uint32_t ES = sizeof(ST);
     const uint32_t nrows = (t.r_end - t.r0 + t.rstep - 1) / t.rstep;
     const uint32_t nbat = (nt + NB - 1) / NB;
-    const uint32_t N = nrows * nbat;
+    const uint32_t N = ((nrows + U - 1) / U) * nbat;
     const uint32_t row_stride = t.rstep * cols;          // elements between this warp's rows
     const uint32_t off0 = t.r0 * cols + t.c;             // element offset of the first tile (layers hold < 2^32 elements)
 
-    // three cursors over the same (row, batch) sequence: copies issued, W_0 prefetched, consumed
-    uint32_t off_i = off0, b_i = 0, off_p = off0, b_p = 0, off_c = off0, b_c = 0;
+    // two cursors over the same (row group, batch) sequence: copies issued, stages consumed
+    uint32_t off_i = off0, b_i = 0, left_i = nrows;
+    uint32_t off_c = off0, b_c = 0, left_c = nrows;
+    uint32_t issued = 0;
+    uint32_t stage_c = ring, stage_i = ring;
+    const uint32_t ring_end = ring + NSTAGE * G::kStageBytes;
 
-    auto issue = [&](uint32_t stage) {
+    auto issue = [&]() {
 #pragma unroll
         for (int k = 0; k < NB; ++k) {
             const uint32_t i = b_i * NB + k;
-            if (FULL || i < nt) cp_async16(stage + k * kSlotBytes, static_cast<const ST*>(ws.pw[i]) + off_i);
-        }
-        if (b_i == 0) {
-            if (BASE == kSharedBase) cp_async16(stage + NB * kSlotBytes, static_cast<const ST*>(ws.pb[0]) + off_i);
-            if (init_mode == kInitAsync) {
+            if (FULL || i < nt) {
+                const char* pw = lds_ptr(sptr + i * 16);
+                const char* pb = BASE == kPerTaskBase ? lds_ptr(sptr + i * 16 + 8) : nullptr;
 #pragma unroll
-                for (int h = 0; h < CPL / 4; ++h) cp_async16(stage + (NB + 1 + h) * kSlotBytes, mp + off_i + 4 * h);
+                for (int u = 0; u < U; ++u) {
+                    if (u == 0 || left_i > u) {
+                        const size_t byte_off = static_cast<size_t>(off_i + u * row_stride) * ES;
+                        cp_async16(stage_i + (G::kW + u * NB + k) * kSlotBytes, pw + byte_off);
+                        if (BASE == kPerTaskBase) cp_async16(stage_i + (G::kB + u * NB + k) * kSlotBytes, pb + byte_off);
+                    }
+                }
             }
         }
-        if (++b_i == nbat) { b_i = 0; off_i += row_stride; }
-    };
-
-    // W_0 tiles under a shuffle come from L2 (each is shared by several slots): they
-    // are fetched into registers one batch ahead instead of occupying the ring.
-    uint4 w0_next[NB];
-    auto prefetch_base = [&]() {
+        if (b_i == 0 && (BASE == kSharedBase || (C::kAsyncInit && init_async))) {
+            const char* pb0 = BASE == kSharedBase ? lds_ptr(sptr + 8) : nullptr;
 #pragma unroll
-        for (int k = 0; k < NB; ++k) {
-            const uint32_t i = b_p * NB + k;
-            if (FULL || i < nt) w0_next[k] = __ldg(reinterpret_cast<const uint4*>(static_cast<const ST*>(ws.pb[i]) + off_p));
+            for (int u = 0; u < U; ++u) {
+                if (u == 0 || left_i > u) {
+                    const uint32_t off = off_i + u * row_stride;
+                    if (BASE == kSharedBase) cp_async16(stage_i + (G::kB + u) * kSlotBytes, pb0 + static_cast<size_t>(off) * ES);
+                    if (C::kAsyncInit && init_async) {
+#pragma unroll
+                        for (int h = 0; h < CPL / 4; ++h)
+                            cp_async16(stage_i + (G::kM + u * (CPL / 4) + h) * kSlotBytes, mp + off + 4 * h);
+                    }
+                }
+            }
         }
-        if (++b_p == nbat) { b_p = 0; off_p += row_stride; }
-    };
-
-    uint32_t issued = 0;
-#pragma unroll
-    for (int s = 0; s < NSTAGE - 1; ++s) {
-        if (issued < N) { issue(ring + s * G::kStageBytes); ++issued; }
-        cp_async_commit();
-    }
-    if (BASE == kPerTaskBase) prefetch_base();
-
-    float acc[CPL], w0row[CPL];
-    uint32_t stage_c = ring, stage_i = ring + (NSTAGE - 1) * G::kStageBytes;
-    const uint32_t ring_end = ring + NSTAGE * G::kStageBytes;
-    for (uint32_t it = 0; it < N; ++it) {
-        if (issued < N) { issue(stage_i); ++issued; }
-        cp_async_commit();
+        if (++b_i == nbat) { b_i = 0; off_i += U * row_stride; left_i -= U; }
         stage_i += G::kStageBytes;
         if (stage_i == ring_end) stage_i = ring;
+        ++issued;
+    };
 
-        uint4 w0_cur[NB];
-        if (BASE == kPerTaskBase) {
 #pragma unroll
-            for (int k = 0; k < NB; ++k) w0_cur[k] = w0_next[k];
-            if (it + 1 < N) prefetch_base();
-        }
+    for (int s = 0; s < NSTAGE - 1; ++s) {
+        if (issued < N) issue();
+        cp_async_commit();
+    }
+
+    f32x2 acc[U][CPL / 2], w0row[U][CPL / 2];
+    const uint32_t one = 0x3F800000u;
+
+    for (uint32_t it = 0; it < N; ++it) {
+        if (issued < N) issue();
+        cp_async_commit();
         cp_async_wait<NSTAGE - 1>();   // everything but the newest NSTAGE-1 groups has landed: stage_c is ready
 
         if (b_c == 0) {
 #pragma unroll
-            for (int e = 0; e < CPL; ++e) { acc[e] = 0.f; w0row[e] = 0.f; }
-            if (init_mode == kInitAsync) {
+            for (int u = 0; u < U; ++u) {
 #pragma unroll
-                for (int h = 0; h < CPL / 4; ++h) {
-                    const uint4 raw = lds128(stage_c + (NB + 1 + h) * kSlotBytes);
-                    acc[4 * h] = __uint_as_float(raw.x); acc[4 * h + 1] = __uint_as_float(raw.y);
-                    acc[4 * h + 2] = __uint_as_float(raw.z); acc[4 * h + 3] = __uint_as_float(raw.w);
-                }
-            } else if (init_mode == kInitPlain) {
+                for (int e = 0; e < CPL / 2; ++e) { acc[u][e] = 0ull; w0row[u][e] = 0ull; }
+                if (u == 0 || left_c > u) {
+                    if (C::kAsyncInit && init_async) {
 #pragma unroll
-                for (int h = 0; h < CPL / 4; ++h) {
-                    const float4 v = *reinterpret_cast<const float4*>(mp + off_c + 4 * h);
-                    acc[4 * h] = v.x; acc[4 * h + 1] = v.y; acc[4 * h + 2] = v.z; acc[4 * h + 3] = v.w;
+                        for (int h = 0; h < CPL / 4; ++h) {
+                            const uint4 raw = lds128(stage_c + (G::kM + u * (CPL / 4) + h) * kSlotBytes);
+                            acc[u][2 * h] = pack2(raw.x, raw.y);
+                            acc[u][2 * h + 1] = pack2(raw.z, raw.w);
+                        }
+                    } else if (init_plain) {
+#pragma unroll
+                        for (int h = 0; h < CPL / 4; ++h) {
+                            const uint4 raw = *reinterpret_cast<const uint4*>(mp + off_c + u * row_stride + 4 * h);
+                            acc[u][2 * h] = pack2(raw.x, raw.y);
+                            acc[u][2 * h + 1] = pack2(raw.z, raw.w);
+                        }
+                    }
+                    if (BASE == kSharedBase) Store<ST>::widen2(lds128(stage_c + (G::kB + u) * kSlotBytes), w0row[u]);
                 }
             }
-            if (BASE == kSharedBase) Store<ST>::widen(lds128(stage_c + NB * kSlotBytes), w0row);
         }
-        const uint32_t pack = ws.bits[b_c][lane];
+        const uint32_t pack = lds_u16(sbits + b_c * 64);
 #pragma unroll
         for (int k = 0; k < NB; ++k) {
             if (FULL || b_c * NB + k < nt) {
-                float d[CPL];
-                Store<ST>::widen(lds128(stage_c + k * kSlotBytes), d);
-                if (BASE == kPerTaskBase) {
-                    float s[CPL];
-                    Store<ST>::widen(w0_cur[k], s);
+                // +-1.0f per column, shared by the U rows
+                f32x2 sg[CPL / 2];
 #pragma unroll
-                    for (int e = 0; e < CPL; ++e) d[e] = __fsub_rn(d[e], s[e]);
-                } else if (BASE == kSharedBase) {
+                for (int e = 0; e < CPL / 2; ++e)
+                    sg[e] = pack2(((pack << (31 - (k * CPL + 2 * e))) & 0x80000000u) | one,
+                                  ((pack << (31 - (k * CPL + 2 * e + 1))) & 0x80000000u) | one);
 #pragma unroll
-                    for (int e = 0; e < CPL; ++e) d[e] = __fsub_rn(d[e], w0row[e]);
+                for (int u = 0; u < U; ++u) {
+                    if (u == 0 || left_c > u) {
+                        f32x2 d[CPL / 2];
+                        Store<ST>::widen2(lds128(stage_c + (G::kW + u * NB + k) * kSlotBytes), d);
+                        if (BASE == kPerTaskBase) {
+                            f32x2 b[CPL / 2];
+                            Store<ST>::widen2(lds128(stage_c + (G::kB + u * NB + k) * kSlotBytes), b);
+#pragma unroll
+                            for (int e = 0; e < CPL / 2; ++e) d[e] = sub2(d[e], b[e]);
+                        } else if (BASE == kSharedBase) {
+#pragma unroll
+                            for (int e = 0; e < CPL / 2; ++e) d[e] = sub2(d[e], w0row[u][e]);
+                        }
+#pragma unroll
+                        for (int e = 0; e < CPL / 2; ++e) acc[u][e] = fma2(d[e], sg[e], acc[u][e]);
+                    }
                 }
-#pragma unroll
-                for (int e = 0; e < CPL; ++e)
-                    acc[e] = __fadd_rn(acc[e], flip(d[e], (pack << (31 - (k * CPL + e))) & 0x80000000u));
             }
         }
         if (b_c + 1 == nbat) {
 #pragma unroll
-            for (int h = 0; h < CPL / 4; ++h)
-                *reinterpret_cast<float4*>(mp + off_c + 4 * h) = make_float4(acc[4 * h], acc[4 * h + 1], acc[4 * h + 2], acc[4 * h + 3]);
+            for (int u = 0; u < U; ++u) {
+                if (u == 0 || left_c > u) {
+#pragma unroll
+                    for (int h = 0; h < CPL / 4; ++h) {
+                        float4 v;
+                        unpack2(acc[u][2 * h], v.x, v.y);
+                        unpack2(acc[u][2 * h + 1], v.z, v.w);
+                        *reinterpret_cast<float4*>(mp + off_c + u * row_stride + 4 * h) = v;
+                    }
+                }
+            }
             b_c = 0;
-            off_c += row_stride;
+            off_c += U * row_stride;
+            left_c -= U;
         } else {
             ++b_c;
         }
@@ -434,21 +545,20 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
 // Element-at-a-time path for layers whose width is not a multiple of the lane
 // width or whose tensors are not 16-byte aligned.  Kept out of line: it is rare
 // and must not set the register budget of the vector path.
-template <typename ST, int NB, int MAXT>
-__device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, const WarpScratch<NB, MAXT>* wsp, int lane,
-                                                    uint32_t nt, int init_mode, float* mp, int base_mode)
+template <typename ST, int NB>
+__device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, uint32_t nt, bool init, float* mp, int base_mode,
+                                                    uint32_t sptr, uint32_t sbits)
 {
     constexpr int CPL = Store<ST>::CPL;
-    const WarpScratch<NB, MAXT>& ws = *wsp;
     for (uint32_t r = t.r0; r < t.r_end; r += t.rstep) {
         const size_t off = static_cast<size_t>(r) * cols + t.c;
         for (int e = 0; e < CPL; ++e) {
             if (t.c + e >= cols) break;
-            float acc = init_mode == kInitZero ? 0.f : mp[off + e];
+            float acc = init ? mp[off + e] : 0.f;
             for (uint32_t i = 0; i < nt; ++i) {
-                float d = Store<ST>::load1(static_cast<const ST*>(ws.pw[i]) + off + e);
-                if (base_mode != kNoBase) d = __fsub_rn(d, Store<ST>::load1(static_cast<const ST*>(ws.pb[i]) + off + e));
-                const uint32_t bit = (ws.bits[i / NB][lane] >> ((i % NB) * CPL + e)) & 1u;
+                float d = Store<ST>::load1(reinterpret_cast<const ST*>(lds_ptr(sptr + i * 16)) + off + e);
+                if (base_mode != kNoBase) d = __fsub_rn(d, Store<ST>::load1(reinterpret_cast<const ST*>(lds_ptr(sptr + i * 16 + 8)) + off + e));
+                const uint32_t bit = (lds_u16(sbits + (i / NB) * 64) >> ((i % NB) * CPL + e)) & 1u;
                 acc = __fadd_rn(acc, flip(d, bit << 31));
             }
             mp[off + e] = acc;
@@ -456,48 +566,23 @@ __device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, c
     }
 }
 
-#ifndef RANDES_COMPRESS_NB
-#define RANDES_COMPRESS_NB 4
-#endif
-#ifndef RANDES_COMPRESS_NSTAGE_F32
-#define RANDES_COMPRESS_NSTAGE_F32 4
-#endif
-#ifndef RANDES_COMPRESS_NSTAGE_BF16
-#define RANDES_COMPRESS_NSTAGE_BF16 3
-#endif
-#ifndef RANDES_SINGLE_NSTAGE_F32
-#define RANDES_SINGLE_NSTAGE_F32 8
-#endif
-#ifndef RANDES_SINGLE_NSTAGE_BF16
-#define RANDES_SINGLE_NSTAGE_BF16 6
-#endif
-
-template <typename ST, bool SINGLE> struct AccConfig {
-    static constexpr int CPL = Store<ST>::CPL;
-    static constexpr int NB = SINGLE ? 1 : RANDES_COMPRESS_NB;
-    static constexpr int MAXT = SINGLE ? 1 : kTaskChunk;
-    static constexpr int NSTAGE = SINGLE ? (CPL == 4 ? RANDES_SINGLE_NSTAGE_F32 : RANDES_SINGLE_NSTAGE_BF16)
-                                         : (CPL == 4 ? RANDES_COMPRESS_NSTAGE_F32 : RANDES_COMPRESS_NSTAGE_BF16);
-    typedef WarpScratch<NB, MAXT> Scratch;
-    static constexpr size_t kRingBytes = static_cast<size_t>(NSTAGE) * RingGeom<CPL, NB>::kStageBytes;
-    static constexpr size_t kSmemBytes = kRingBytes + kWarpsPerCta * sizeof(Scratch);
-};
-
-// SINGLE: one task per launch (add / remove): a deep ring of rows.  Otherwise
-// (compress): NB tasks per stage.
+// SINGLE: one task per launch (add / remove): a deep ring of single rows, M staged
+// with the weights.  Otherwise (compress): 2 rows x 2 tasks per stage.
 template <typename ST, bool SINGLE>
 __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const AccumulateArgs a)
 {
-    typedef AccConfig<ST, SINGLE> Cfg;
-    constexpr int CPL = Cfg::CPL, NB = Cfg::NB, MAXT = Cfg::MAXT, NS = Cfg::NSTAGE;
+    typedef AccConfig<ST, SINGLE> C;
+    constexpr int CPL = C::CPL, NB = C::NB, MAXT = C::MAXT;
     extern __shared__ __align__(16) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + threadIdx.x * 16;
+    const uint32_t smem_s = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
+    const uint32_t ring = smem_s + threadIdx.x * 16;
     // between units the ring is idle: its first slots double as the warp's table of Philox blocks
-    const uint32_t blocks = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * 512;
-    typename Cfg::Scratch& ws = reinterpret_cast<typename Cfg::Scratch*>(smem + Cfg::kRingBytes)[warp];
+    const uint32_t blocks = smem_s + warp * 512;
+    const uint32_t sptr = smem_s + C::kRingBytes + warp * C::kWarpBytes;
+    const uint32_t sbits = sptr + C::kPtrBytes + lane * 2;
     const uint32_t L = a.n_layers;
-    const uint32_t negate_bits = a.negate ? 0xFFFFFFFFu : 0u;
+    const uint32_t negate_bits = a.negate ? 0xFFFFu : 0u;
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
         const uint32_t slot = un.layer;
@@ -519,8 +604,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const Acc
                 const uint32_t src = shuffled ? a.src_of_slot[static_cast<size_t>(ti) * L + slot] : slot;   // sigma_i(l)
                 const void* pw = a.task_ptrs[static_cast<size_t>(ti) * L + src];
                 const void* pb = a.has_base ? a.base[src] : nullptr;
-                ws.pw[lane] = pw;
-                ws.pb[lane] = pb;
+                sts_ptrs(sptr + lane * 16, pw, pb);
                 ok = aligned16(pw) && aligned16(pb);
                 if (flipped) {
                     const DevTask tk = a.tasks[ti];
@@ -544,23 +628,24 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const Acc
                             pack |= lane_bits<CPL>(lds128(blocks + (CPL == 8 ? (lane >> 4) : 0) * kSlotBytes + i * 16), lane) << (k * CPL);
                     }
                 }
-                ws.bits[b][lane] = pack ^ negate_bits;
+                sts_u16(sbits + b * 64, pack ^ negate_bits);
             }
             __syncwarp();   // the block table is free again before any lane's copies land in the ring
             if (lane_on) {
-                const int init_mode = chunk0 > 0 ? kInitPlain : (a.init_from_m ? kInitAsync : kInitZero);
+                const bool init_plain = chunk0 > 0 || (!SINGLE && a.init_from_m);
+                const bool init_async = SINGLE && chunk0 == 0 && a.init_from_m;
                 const bool full = nt % NB == 0;
                 if (!vec)
-                    accumulate_rows_scalar<ST, NB, MAXT>(t, ls.cols, &ws, lane, nt, init_mode, mp, base_mode);
+                    accumulate_rows_scalar<ST, NB>(t, ls.cols, nt, init_plain || a.init_from_m, mp, base_mode, sptr, sbits);
                 else if (base_mode == kNoBase) {
-                    if (full) accumulate_rows_async<ST, kNoBase, NB, NS, MAXT, true>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
-                    else accumulate_rows_async<ST, kNoBase, NB, NS, MAXT, false>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
+                    if (full) accumulate_rows_async<ST, SINGLE, kNoBase, true>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
+                    else accumulate_rows_async<ST, SINGLE, kNoBase, false>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
                 } else if (base_mode == kSharedBase) {
-                    if (full) accumulate_rows_async<ST, kSharedBase, NB, NS, MAXT, true>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
-                    else accumulate_rows_async<ST, kSharedBase, NB, NS, MAXT, false>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
+                    if (full) accumulate_rows_async<ST, SINGLE, kSharedBase, true>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
+                    else accumulate_rows_async<ST, SINGLE, kSharedBase, false>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
                 } else {
-                    if (full) accumulate_rows_async<ST, kPerTaskBase, NB, NS, MAXT, true>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
-                    else accumulate_rows_async<ST, kPerTaskBase, NB, NS, MAXT, false>(t, ls.cols, ws, lane, nt, init_mode, mp, ring);
+                    if (full) accumulate_rows_async<ST, SINGLE, kPerTaskBase, true>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
+                    else accumulate_rows_async<ST, SINGLE, kPerTaskBase, false>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
                 }
             }
         }

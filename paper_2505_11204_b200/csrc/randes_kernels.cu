@@ -361,7 +361,13 @@ constexpr int kRingSlots = 24;    // 16-byte slots per thread: 96 KiB per CTA, t
 
 template <typename ST, bool SINGLE> struct AccConfig {
     static constexpr int CPL = Store<ST>::CPL;
-    static constexpr int U = SINGLE ? 1 : 2;          // rows per stage
+#ifndef RANDES_SINGLE_U
+#define RANDES_SINGLE_U 1
+#endif
+#ifndef RANDES_COMPRESS_U_BF16
+#define RANDES_COMPRESS_U_BF16 1
+#endif
+    static constexpr int U = SINGLE ? RANDES_SINGLE_U : (CPL == 8 ? RANDES_COMPRESS_U_BF16 : 2);   // rows per stage
     static constexpr int NB = SINGLE ? 1 : 2;         // tasks per stage
     static constexpr int MAXT = SINGLE ? 1 : kTaskChunk;
     static constexpr bool kAsyncInit = SINGLE;        // add / remove start from M
@@ -383,7 +389,12 @@ template <typename ST, bool SINGLE, int BASE> struct StageGeom {
     static constexpr int kW = 0;
     static constexpr int kB = C::U * C::NB;
     static constexpr int kM = kB + (BASE == kPerTaskBase ? C::U * C::NB : (BASE == kSharedBase ? C::U : 0));
-    static constexpr int SLOTS = kM + (C::kAsyncInit ? C::U * C::CPL / 4 : 0);
+    // A lane's M tile is 16 B for fp32 storage and travels through the ring; for bf16 storage it
+    // is 32 B, which one 16-byte copy per lane can only fetch with a 32-byte stride between lanes
+    // (slow for cp.async): there M is prefetched into L2 and loaded into registers one step ahead.
+    static constexpr bool kInitViaRing = C::kAsyncInit && C::CPL == 4;
+    static constexpr bool kInitViaRegs = C::kAsyncInit && C::CPL == 8;
+    static constexpr int SLOTS = kM + (kInitViaRing ? C::U * C::CPL / 4 : 0);
     static constexpr int NSTAGE = (kRingSlots / SLOTS) > 8 ? 8 : (kRingSlots / SLOTS);
     static constexpr uint32_t kStageBytes = SLOTS * kSlotBytes;
     static_assert(NSTAGE >= 2, "ring too small");
@@ -434,11 +445,12 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
                 if (u == 0 || left_i > u) {
                     const uint32_t off = off_i + u * row_stride;
                     if (BASE == kSharedBase) cp_async16(stage_i + (G::kB + u) * kSlotBytes, pb0 + static_cast<size_t>(off) * ES);
-                    if (C::kAsyncInit && init_async) {
+                    if (G::kInitViaRing && init_async) {
 #pragma unroll
                         for (int h = 0; h < CPL / 4; ++h)
                             cp_async16(stage_i + (G::kM + u * (CPL / 4) + h) * kSlotBytes, mp + off + 4 * h);
                     }
+                    if (G::kInitViaRegs && init_async) prefetch_l2(mp + off);
                 }
             }
         }
@@ -457,6 +469,22 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
     f32x2 acc[U][CPL / 2], w0row[U][CPL / 2];
     const uint32_t one = 0x3F800000u;
 
+    // M tiles of the next row group, when they come through registers
+    uint4 m_next[U][CPL / 4];
+    uint32_t off_m = off0, left_m = nrows;
+    auto load_m_next = [&]() {
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (u == 0 || left_m > u) {
+#pragma unroll
+                for (int h = 0; h < CPL / 4; ++h)
+                    m_next[u][h] = *reinterpret_cast<const uint4*>(mp + off_m + u * row_stride + 4 * h);
+            }
+        off_m += U * row_stride;
+        left_m -= U;
+    };
+    if (G::kInitViaRegs && init_async && N > 0) load_m_next();
+
     for (uint32_t it = 0; it < N; ++it) {
         if (issued < N) issue();
         cp_async_commit();
@@ -468,12 +496,18 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
 #pragma unroll
                 for (int e = 0; e < CPL / 2; ++e) { acc[u][e] = 0ull; w0row[u][e] = 0ull; }
                 if (u == 0 || left_c > u) {
-                    if (C::kAsyncInit && init_async) {
+                    if (G::kInitViaRing && init_async) {
 #pragma unroll
                         for (int h = 0; h < CPL / 4; ++h) {
                             const uint4 raw = lds128(stage_c + (G::kM + u * (CPL / 4) + h) * kSlotBytes);
                             acc[u][2 * h] = pack2(raw.x, raw.y);
                             acc[u][2 * h + 1] = pack2(raw.z, raw.w);
+                        }
+                    } else if (G::kInitViaRegs && init_async) {
+#pragma unroll
+                        for (int h = 0; h < CPL / 4; ++h) {
+                            acc[u][2 * h] = pack2(m_next[u][h].x, m_next[u][h].y);
+                            acc[u][2 * h + 1] = pack2(m_next[u][h].z, m_next[u][h].w);
                         }
                     } else if (init_plain) {
 #pragma unroll
@@ -487,6 +521,7 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
                 }
             }
         }
+        if (G::kInitViaRegs && init_async && b_c == 0 && left_m > 0 && left_m <= nrows) load_m_next();
         const uint32_t pack = lds_u16(sbits + b_c * 64);
 #pragma unroll
         for (int k = 0; k < NB; ++k) {

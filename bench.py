@@ -1,0 +1,439 @@
+#!/usr/bin/env python
+"""Benchmark of the RanDeS hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload vit_l14] [--storage f32]
+    python bench.py --impl reference ...        # the CPU oracle on a bounded sample
+
+One step = one pass of the whole hot path over one synthetic weight set:
+compress all K task models into M, retrieve every task once, then stream-add
+`--swap` further models and remove them again.  The headline value is the
+algorithmic bytes of the step (what the method must move) divided by the
+device time of the step, summed over GPUs.  Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2505_11204_b200 import workloads as wl  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+WORKLOADS = {"toy": wl.toy, "vit_b32": wl.vit_b32, "gpt2_small": wl.gpt2_small, "flan_t5_base": wl.flan_t5_base,
+             "vit_l14": wl.vit_l14}
+
+
+def parse_args(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="vit_l14", choices=sorted(WORKLOADS))
+    ap.add_argument("--storage", default=None, choices=["f32", "bf16"])
+    ap.add_argument("--tasks", type=int, default=None, help="number of task models K (default: the workload's)")
+    ap.add_argument("--swap", type=int, default=5, help="models streamed in and out per step")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    return ap.parse_args(argv)
+
+
+def make_workload(args) -> wl.Workload:
+    w = WORKLOADS[args.workload]()
+    if args.storage is not None:
+        w = w.with_storage(wl.BF16 if args.storage == "bf16" else wl.F32)
+    if args.tasks is not None:
+        w = w.with_tasks(args.tasks)
+    return w
+
+
+def step_bytes(w: wl.Workload, n_swap: int, out_bytes: int = 4):
+    """Algorithmic bytes of each operation of one step (M is fp32)."""
+    s = 2 if w.storage == wl.BF16 else 4
+    P, K = w.n_params, w.n_tasks
+    b = {
+        "compress": (K * s + s + 4) * P,
+        "retrieve": (4 + s + out_bytes) * P,          # per call; K calls per step
+        "add": (8 + 2 * s) * P,                       # per call; n_swap calls per step
+        "remove": (8 + 2 * s) * P,
+    }
+    total = b["compress"] + K * b["retrieve"] + n_swap * (b["add"] + b["remove"])
+    return b, total
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def max_over_ranks(values, world, device=None):
+    """Element-wise maximum of a list of floats over all ranks (identity when world == 1)."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def aggregate_value(total_bytes_per_rank: float, ms_per_step_max: float, world: int) -> float:
+    """Whole-job GB/s: every rank moves total_bytes per step; time is the slowest rank's."""
+    return world * total_bytes_per_rank / (ms_per_step_max * 1e-3) / 1e9
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def config_dict(w, args, note=""):
+    return {"workload": "%s-shaped synthetic weights, K=%d tasks, %d layers, %.1f M params; step = compress + %d retrieves + %d adds + %d removes"
+                        % (w.name, w.n_tasks, w.n_layers, w.n_params / 1e6, w.n_tasks, args.swap, args.swap),
+            "storage": "bf16" if w.storage == wl.BF16 else "f32", "lambda": w.lam,
+            "l2": ("inputs exceed L2: every call streams at least %.2f GB" if (4 + 4) * w.n_params > 2 * 126e6 else
+                   "working set of %.3f GB fits in L2: latency-bound, not a roofline case")
+                  % ((4 + (2 if w.storage == wl.BF16 else 4)) * w.n_params / 1e9),
+            "note": note}
+
+
+# --------------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(w: wl.Workload):
+    """A bounded sample of the workload for the CPU oracle: the layers of the
+    first two blocks plus the unrepeated tensors, same K, same step structure."""
+    keep, sizes = [], w.group_sizes()
+    seen = [0] * len(sizes)
+    for l, g in enumerate(w.group):
+        if sizes[g] == 1 or seen[g] < 2:
+            keep.append(l)
+            seen[g] += 1
+    return wl.subset(w, keep, w.name + ":first-2-blocks")
+
+
+def run_oracle_step(ro, ws, base, tasks, extra, n_swap):
+    K = ws.n_tasks
+    M = ro.compress(ws.spec, ws.storage, ws.task_ids, ws.seeds, base, tasks)
+    for t, s in zip(ws.task_ids, ws.seeds):
+        ro.retrieve(ws.spec, ws.storage, wl.F32, t, s, ws.lam, base, M)
+    for j in range(n_swap):
+        ro.add_model(ws.spec, ws.storage, K + j, ws.seeds[0] + K + j, base, extra[j], M)
+    for j in range(n_swap):
+        ro.remove_model(ws.spec, ws.storage, K + j, ws.seeds[0] + K + j, base, extra[j], M)
+    return M
+
+
+def time_oracle(w: wl.Workload, n_swap: int, steps: int, warmup: int):
+    from oracle import randes_oracle as ro
+
+    ws = oracle_sample(w)
+    K = ws.n_tasks
+    ids = list(ws.task_ids) + [K + j for j in range(n_swap)]
+    base, models = wl.model_set(ws, ids, threads=os.cpu_count() or 1)
+    tasks, extra = models[:K], models[K:]
+    for _ in range(warmup):
+        run_oracle_step(ro, ws, base, tasks, extra, n_swap)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        run_oracle_step(ro, ws, base, tasks, extra, n_swap)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    _, total = step_bytes(ws, n_swap)
+    return {"value": total / dt / 1e9, "unit": "GB/s", "cores": ro.num_threads(), "kind": "oracle",
+            "sample": "%s: %d of %d layers, %.1f M of %.1f M params, K=%d, swap=%d, %.2f s per step"
+                      % (ws.name, ws.n_layers, w.n_layers, ws.n_params / 1e6, w.n_params / 1e6, K, n_swap, dt),
+            "ms_per_step": dt * 1e3}
+
+
+def run_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return 0
+    w = make_workload(args)
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    steps_run, warm_run = min(steps, 30), min(warmup, 3)   # bounded: about a second per step on the sample
+    r = time_oracle(w, args.swap, steps_run, warm_run)
+    line = {
+        "impl": "reference", "metric": "hot_path_algorithmic_bandwidth", "value": r["value"], "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "ms_per_step": r["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if w.storage == wl.F32 else "bf16 storage, f32 arithmetic", "data": "synthetic",
+        "config": config_dict(w, args, "CPU oracle on a bounded sample; timed %d step(s) after %d warm-up" % (steps_run, warm_run)),
+        "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------------- GPU legs
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2505_11204_b200 import build, randes
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if not os.path.exists(randes.LIB_PATH):
+        if rank == 0:
+            build.build_library()
+        if world > 1:
+            dist.barrier()
+    randes.lib()
+
+    w = make_workload(args)
+    K, n_swap = w.n_tasks, args.swap
+    ids = list(w.task_ids) + [K + j for j in range(n_swap)]
+    swap_seeds = [w.seeds[0] + K + j for j in range(n_swap)]
+    want_e2e = not args.no_e2e
+
+    # ---- inputs: generated on the host (seeded); pinned when the end-to-end leg needs them again
+    def host_tensor(a):
+        t = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+        return t.pin_memory() if want_e2e else t
+
+    base_np, models_np = wl.model_set(w, ids, threads=os.cpu_count() or 1)
+    h_base = [host_tensor(a) for a in base_np]
+    h_models = [[host_tensor(a) for a in m] for m in models_np]
+    del base_np, models_np
+    d_base = [t.to(dev, non_blocking=True) for t in h_base]
+    d_models = [[t.to(dev, non_blocking=True) for t in m] for m in h_models]
+    torch.cuda.synchronize()
+    if not want_e2e:
+        del h_base, h_models
+
+    plan = randes.Plan.from_workload(w, max_tasks=K + n_swap, device=dev)
+    M = plan.new_superposition()
+    out = plan.new_output(wl.F32)
+    p_base = randes.ptr_array(d_base)
+    p_tasks = randes.ptr_array(d_models[:K])
+    p_swap = [randes.ptr_array(m) for m in d_models[K:]]
+    p_out = randes.ptr_array(out)
+    stream = torch.cuda.current_stream(dev)
+    sh = stream.cuda_stream
+    names = ["compress", "retrieve", "add", "remove"]
+
+    def step(events=None):
+        def mark():
+            if events is not None:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record(stream)
+                events.append(e)
+        mark()
+        randes.randes_compress(plan.handle, p_base, p_tasks, M, sh)
+        mark()
+        for t in w.task_ids:
+            randes.randes_retrieve(plan.handle, t, w.lam, wl.F32, p_base, M, p_out, sh)
+        mark()
+        for j in range(n_swap):
+            randes.randes_add_model(plan.handle, K + j, swap_seeds[j], p_base, p_swap[j], M, sh)
+        mark()
+        for j in range(n_swap):
+            randes.randes_remove_model(plan.handle, K + j, p_base, p_swap[j], M, sh)
+        mark()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = randes.randes_launch_count()
+    evs = []
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_begin.record(stream)
+    for _ in range(args.steps):
+        step(evs)
+    t_end.record(stream)
+    barrier()
+    launches = randes.randes_launch_count() - launches0
+    total_ms = t_begin.elapsed_time(t_end)
+    clocks = sampler.stop() if rank == 0 else None
+
+    op_ms = {n: 0.0 for n in names}
+    for s_i in range(args.steps):
+        e = evs[s_i * 5:(s_i + 1) * 5]
+        for j, n in enumerate(names):
+            op_ms[n] += e[j].elapsed_time(e[j + 1])
+    red = max_over_ranks([total_ms] + [op_ms[n] for n in names], world, dev)
+    total_ms, op_ms = red[0], {n: red[1 + j] for j, n in enumerate(names)}
+
+    b, total_bytes = step_bytes(w, n_swap)
+    ms_per_step = total_ms / args.steps
+    value = aggregate_value(total_bytes, ms_per_step, world)
+    peak, peak_kind = measured_peak()
+    calls = {"compress": 1, "retrieve": K, "add": n_swap, "remove": n_swap}
+    ops = {}
+    for n in names:
+        c = calls[n] * args.steps
+        if c == 0:
+            continue
+        ms = op_ms[n] / c
+        gbs = b[n] / (ms * 1e-3) / 1e9
+        ops[n] = {"ms_per_call": ms, "GBps": gbs, "Gparams_per_s": w.n_params / (ms * 1e-3) / 1e9,
+                  "frac_of_%s_peak" % peak_kind: gbs / peak, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+                  "share_of_step": op_ms[n] / total_ms}
+    # dominant kernel by device time: retrieve_kernel vs accumulate_kernel (compress + add + remove)
+    acc_ms = op_ms["compress"] + op_ms.get("add", 0.0) + op_ms.get("remove", 0.0)
+    if op_ms["retrieve"] >= acc_ms:
+        dom, dom_bytes, dom_ms = "retrieve_kernel", b["retrieve"], ops["retrieve"]["ms_per_call"]
+    else:
+        dom = "accumulate_kernel (compress, add, remove launches)"
+        n_acc = (1 + 2 * n_swap) * args.steps
+        dom_bytes = (b["compress"] + n_swap * (b["add"] + b["remove"])) / (1 + 2 * n_swap)
+        dom_ms = acc_ms / n_acc
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak,
+                "peak_source": "%s copy bandwidth (MEASURED_PEAKS.json)" % peak_kind if peak_kind == "measured"
+                               else "fallback copy bandwidth",
+                "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "per_kernel": {k: {"achieved": ops[k]["GBps"], "frac": ops[k]["GBps"] / peak, "bytes_per_launch": b[k]}
+                               for k in ops}}
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    e2e = None
+    if want_e2e:
+        h_out = [torch.empty_like(o, device="cpu").pin_memory() for o in out]
+        h_M = torch.empty_like(M, device="cpu").pin_memory()
+
+        def e2e_step():
+            for dst, src in zip(d_base, h_base):
+                dst.copy_(src, non_blocking=True)
+            for dm, hm in zip(d_models, h_models):
+                for dst, src in zip(dm, hm):
+                    dst.copy_(src, non_blocking=True)
+            randes.randes_compress(plan.handle, p_base, p_tasks, M, sh)
+            for ti in w.task_ids:
+                randes.randes_retrieve(plan.handle, ti, w.lam, wl.F32, p_base, M, p_out, sh)
+                for dst, src in zip(h_out, out):
+                    dst.copy_(src, non_blocking=True)
+            for j in range(n_swap):
+                randes.randes_add_model(plan.handle, K + j, swap_seeds[j], p_base, p_swap[j], M, sh)
+            for j in range(n_swap):
+                randes.randes_remove_model(plan.handle, K + j, p_base, p_swap[j], M, sh)
+            h_M.copy_(M, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        z.record(stream)
+        barrier()
+        e2e_ms = max_over_ranks([a.elapsed_time(z)], world, dev)[0] / args.e2e_steps
+        s = 2 if w.storage == wl.BF16 else 4
+        e2e = {"value": aggregate_value(total_bytes, e2e_ms, world), "unit": "GB/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": (1 + K + n_swap) * w.n_params * s,
+               "d2h_bytes_per_step": (K + 1) * w.n_params * 4, "steps": args.e2e_steps}
+        del h_out, h_M, h_base, h_models
+
+    plan.close()
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        del d_models, d_base, M, out
+        torch.cuda.empty_cache()
+        cpu = time_oracle(w, n_swap, 5, 1)
+        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    if rank == 0:
+        line = {
+            "metric": "hot_path_algorithmic_bandwidth", "value": value, "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if w.storage == wl.F32 else "bf16 storage, f32 arithmetic", "data": "synthetic",
+            "config": config_dict(w, args, "every rank runs the whole workload on its own GPU; no collective on the data path"),
+            "Gparams_per_s": {n: ops[n]["Gparams_per_s"] for n in ops},
+            "ops": ops, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks,
+            "paper_context": "the paper times retrieval only: 658.19 ms per CLIP ViT-L/14 model and 292.70 ms per "
+                             "ViT-B/32 model on an Intel Xeon Gold 6448Y CPU (other hardware; context, not a target)",
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    args = parse_args()
+    return run_reference(args) if args.impl == "reference" else run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,87 @@
+"""The multi-rank path of the benchmark on CPU: two gloo ranks.
+
+The hot path shards by whole, independent problems (every rank runs the full
+workload on its own GPU; no collective touches the data), so what has to be
+right across ranks is only the timing reduction -- the slowest rank's time --
+and the whole-job aggregate built from it.
+"""
+import os
+import socket
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _rank_main(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import bench
+
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        # rank r pretends its step took (10 + 5 r) ms and its retrieves (2 + r) ms
+        red = bench.max_over_ranks([10.0 + 5.0 * rank, 2.0 + rank], world)
+        total_bytes = 1.5e9
+        value = bench.aggregate_value(total_bytes, red[0], world)
+        dist.barrier()
+        out[rank] = (red, value)
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_report_slowest_time_and_whole_job_throughput():
+    world = 2
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_rank_main, args=(world, _free_port(), out), nprocs=world, join=True)
+    assert len(out) == world
+    for rank in range(world):
+        red, value = out[rank]
+        assert red == [15.0, 3.0]                       # maximum over ranks, on every rank
+        assert value == pytest.approx(2 * 1.5e9 / 15e-3 / 1e9)   # both ranks' bytes over the slowest time
+
+
+def test_single_rank_is_identity():
+    import bench
+
+    assert bench.max_over_ranks([3.0, 4.0], 1) == [3.0, 4.0]
+    assert bench.aggregate_value(2e9, 1.0, 1) == pytest.approx(2000.0)
+
+
+def test_step_bytes_match_the_per_parameter_figures():
+    import bench
+    from paper_2505_11204_b200 import workloads as wl
+
+    w = wl.vit_l14()
+    b, total = bench.step_bytes(w, 5)
+    P = w.n_params
+    assert P == 303_966_208
+    assert b["compress"] == 88 * P and b["retrieve"] == 12 * P and b["add"] == 16 * P == b["remove"]
+    assert total == (88 + 20 * 12 + 10 * 16) * P
+    wb = w.with_storage(wl.BF16)
+    b, _ = bench.step_bytes(wb, 5, out_bytes=2)
+    assert b["compress"] == 46 * P and b["retrieve"] == 8 * P and b["add"] == 12 * P
+
+
+def test_workload_parameter_counts():
+    from paper_2505_11204_b200 import workloads as wl
+
+    want = {0: (1_575_936, 12, 2), 1: (87_849_216, 152, 20), 2: (124_439_808, 148, 16), 3: (247_577_856, 282, 29),
+            4: (303_966_208, 296, 20)}
+    for k, (P, L, G) in want.items():
+        w = wl.CONFIGS[k]()
+        assert (w.n_params, w.n_layers, len(w.gflags)) == (P, L, G), w.name
+    assert len(wl.flan_t5_lora_targets(wl.flan_t5_base())) == 72

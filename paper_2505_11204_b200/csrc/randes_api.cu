@@ -371,9 +371,10 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
             }
             const std::vector<uint32_t>& mem = p->members[layers[l].group];
             if (!mem.empty() && (layers[mem[0]].rows != layers[l].rows || layers[mem[0]].cols != layers[l].cols)) {
+                const uint32_t first = mem[0];   // `mem` dies with the plan
                 delete p;
                 return fail(RANDES_SHAPE_MISMATCH, "group %u: layer %u is %ux%u but layer %u is %ux%u", layers[l].group, l,
-                            layers[l].rows, layers[l].cols, mem[0], layers[mem[0]].rows, layers[mem[0]].cols);
+                            layers[l].rows, layers[l].cols, first, layers[first].rows, layers[first].cols);
             }
             p->members[layers[l].group].push_back(l);
         }

@@ -183,6 +183,39 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda,
                     randes_dtype_t out_dtype, const void* const* base, const void* M,
                     void* const* out, void* stream);
 
+/*
+ * retrieve for callers that cannot provide a device workspace.  (The paper has
+ * no counterpart: this entry point exists for deployment, not for the method.)
+ *
+ * Who needs it: code that is handed the weight tensors and a stream but does
+ * not own a device allocator -- a plug-in inside a serving process whose memory
+ * pool belongs to the host framework, or a request handler that swaps models in
+ * a latency-critical loop, where cudaMalloc / cudaFree would stall the device
+ * and are therefore forbidden.  Such a caller builds its plan with
+ * dev_workspace == NULL (host-only) and calls this instead of randes_retrieve.
+ *
+ * Same arguments, results and errors as randes_retrieve (bit-identical output);
+ * `plan` may be host-only.  The tables the kernel reads are copied, on
+ * `stream`, into a fixed array of RANDES_STATIC_SCRATCH_BYTES that lives inside
+ * the library on every GPU that loads it, for the life of the process.  The
+ * call allocates no device memory and frees none.
+ *   - Limit: 72 bytes per layer plus 16 bytes per tile of 16 rows x 1024 fp32
+ *     (2048 bf16) columns, rounded up, must fit the array (models up to roughly
+ *     a billion parameters); larger plans fail with RANDES_CAPACITY before
+ *     anything is launched.
+ *   - The first call on each device looks up the array's device address and
+ *     sizes the grid; make that first call outside any stream capture.
+ *   - All calls on one device share the array.  Calls on one stream are ordered
+ *     and safe; calls whose work may overlap on the GPU (different streams,
+ *     different plans or threads) race on the tables and must be serialised by
+ *     the caller.  Nothing in the array needs clearing between calls: each call
+ *     rewrites every entry it reads.
+ */
+#define RANDES_STATIC_SCRATCH_BYTES (1u << 20)
+int randes_retrieve_static(const randes_plan_t* plan, uint32_t task_id, float lambda,
+                           randes_dtype_t out_dtype, const void* const* base, const void* M,
+                           void* const* out, void* stream);
+
 /* Number of kernels this library has launched in this process (all plans). */
 uint64_t randes_launch_count(void);
 

@@ -599,4 +599,44 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_
     return RANDES_OK;
 }
 
+int randes_retrieve_static(const randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
+                           const void* const* base, const void* M, void* const* out, void* stream)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (out_dtype != RANDES_F32 && out_dtype != RANDES_BF16)
+        return fail(RANDES_UNSUPPORTED_DTYPE, "output dtype %d is not supported", static_cast<int>(out_dtype));
+    int rc;
+    if ((rc = check_m(M))) return rc;
+    const int row = find_task(*plan, task_id);
+    if (row < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_id);
+    if ((rc = check_ptrs(*plan, base, "base", elem_size(plan->storage), false))) return rc;
+    if ((rc = check_ptrs(*plan, const_cast<const void* const*>(out), "out", elem_size(out_dtype), false))) return rc;
+    const char* m_lo = static_cast<const char*>(M);
+    const char* m_hi = m_lo + plan->m_bytes;
+    for (uint32_t l = 0; l < plan->n_layers; ++l) {
+        const char* o = static_cast<const char*>(out[l]);
+        if (out[l] && (out[l] == base[l] || (o >= m_lo && o < m_hi)))
+            return fail(RANDES_INVALID_ARGUMENT, "out[%u] aliases base or M", l);
+    }
+    const size_t need = retrieve_static_bytes(plan->n_layers, static_cast<uint32_t>(plan->units.size()));
+    if (need > kStaticScratchBytes)
+        return fail(RANDES_CAPACITY,
+                    "this model needs %zu bytes of tables (%u layers, %zu tiles) but the built-in scratch holds %zu; "
+                    "use randes_retrieve with a workspace instead",
+                    need, plan->n_layers, plan->units.size(), static_cast<size_t>(kStaticScratchBytes));
+    const TaskEntry& t = plan->tasks[row];
+    DevTask dt;
+    dt.id = t.id;
+    dt.key0 = static_cast<uint32_t>(t.seed);
+    dt.key1 = static_cast<uint32_t>(t.seed >> 32);
+    dt.pad = 0;
+    const int e = launch_retrieve_static(plan->storage, out_dtype, plan->dev_layers.data(), plan->n_layers, plan->units.data(),
+                                         static_cast<uint32_t>(plan->units.size()), t.slot_of_pos.data(), base, out,
+                                         static_cast<const float*>(M), dt, lambda, stream);
+    if (e == -1) return fail(RANDES_CAPACITY, "tables exceed the built-in scratch");
+    if (e) return fail_cuda(static_cast<cudaError_t>(e), "randes_retrieve_static");
+    if (!plan->units.empty()) ++g_launches;
+    return RANDES_OK;
+}
+
 }  // extern "C"

@@ -90,4 +90,13 @@ int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void
 int retrieve_ctas_per_sm(int storage_dtype, int out_dtype);
 int accumulate_ctas_per_sm(int storage_dtype, bool single_task);
 
+
+// Retrieve with its tables in a fixed device array inside the library (no workspace).
+// Returns a cudaError_t as int, or -1 when the tables exceed kStaticScratchBytes.
+constexpr size_t kStaticScratchBytes = 1u << 20;
+size_t retrieve_static_bytes(uint32_t n_layers, uint32_t n_units);
+int launch_retrieve_static(int storage_dtype, int out_dtype, const DevLayer* layers, uint32_t n_layers, const DevUnit* units,
+                           uint32_t n_units, const uint32_t* slot_of_pos, const void* const* base, void* const* out,
+                           const float* M, const DevTask& task, float lambda, void* stream);
+
 }  // namespace randes

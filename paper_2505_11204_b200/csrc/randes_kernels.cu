@@ -20,6 +20,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "randes_internal.h"
 
 namespace randes {
@@ -726,6 +728,83 @@ int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void
         else accumulate_kernel<bf16, false><<<grid, kThreadsPerCta, AccConfig<bf16, false>::kSmemBytes, s>>>(a);
     }
     return static_cast<int>(cudaGetLastError());
+}
+
+// ---- retrieve without a caller-provided workspace ---------------------------------------------
+// The tables the retrieve kernel reads (layers, units, sigma^-1, pointer arrays) are
+// placed in this fixed array instead of a workspace the caller would have to allocate.
+// Every GPU that loads the library holds the array until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device
+int g_static_grid[kMaxDevices][2][2] = {};       // persistent grid size [storage][out dtype], per device
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+}  // namespace
+
+size_t retrieve_static_bytes(uint32_t n_layers, uint32_t n_units)
+{
+    return align256(n_layers * sizeof(DevLayer)) + align256(n_units * sizeof(DevUnit)) + align256(n_layers * sizeof(uint32_t)) +
+           2 * align256(n_layers * sizeof(void*));
+}
+
+int launch_retrieve_static(int storage_dtype, int out_dtype, const DevLayer* layers, uint32_t n_layers, const DevUnit* units,
+                           uint32_t n_units, const uint32_t* slot_of_pos, const void* const* base, void* const* out,
+                           const float* M, const DevTask& task, float lambda, void* stream)
+{
+    if (retrieve_static_bytes(n_layers, n_units) > kStaticScratchBytes) return -1;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return static_cast<int>(e);
+    if (dev < 0 || dev >= kMaxDevices) return static_cast<int>(cudaErrorInvalidDevice);
+    unsigned char* scratch = nullptr;
+    int grid = 0;
+    {
+        // once per device, with that device current: the array's name is only a host-side
+        // handle here; the kernel needs the address the symbol has on this device
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev]) {
+            void* p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_static_scratch);
+            if (e != cudaSuccess) return static_cast<int>(e);
+            int sms = 0;
+            e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess) return static_cast<int>(e);
+            for (int st = 0; st < 2; ++st)
+                for (int od = 0; od < 2; ++od) {
+                    const int occ = retrieve_ctas_per_sm(st, od);
+                    if (occ <= 0) return static_cast<int>(cudaErrorInvalidDeviceFunction);
+                    g_static_grid[dev][st][od] = sms * occ;
+                }
+            g_static_ptr[dev] = static_cast<unsigned char*>(p);
+        }
+        scratch = g_static_ptr[dev];
+        grid = g_static_grid[dev][storage_dtype][out_dtype];
+    }
+    size_t off = 0;
+    auto put = [&](const void* src, size_t bytes) -> unsigned char* {
+        unsigned char* dst = scratch + off;
+        off += align256(bytes);
+        if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s);
+        return dst;
+    };
+    RetrieveArgs a;
+    a.layers = reinterpret_cast<const DevLayer*>(put(layers, n_layers * sizeof(DevLayer)));
+    a.units = reinterpret_cast<const DevUnit*>(put(units, n_units * sizeof(DevUnit)));
+    a.slot_of_pos = reinterpret_cast<const uint32_t*>(put(slot_of_pos, n_layers * sizeof(uint32_t)));
+    a.base = reinterpret_cast<const void* const*>(put(base, n_layers * sizeof(void*)));
+    a.out = reinterpret_cast<void* const*>(put(out, n_layers * sizeof(void*)));
+    if (e != cudaSuccess) return static_cast<int>(e);
+    a.n_units = n_units;
+    a.n_layers = n_layers;
+    a.M = M;
+    a.task = task;
+    a.lambda = lambda;
+    if (n_units == 0) return 0;
+    return launch_retrieve(storage_dtype, out_dtype, a, grid < static_cast<int>(n_units) ? grid : static_cast<int>(n_units), stream);
 }
 
 int retrieve_ctas_per_sm(int storage_dtype, int out_dtype)

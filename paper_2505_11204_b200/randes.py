@@ -90,6 +90,8 @@ def lib():
         L.randes_remove_model.restype = ctypes.c_int
         L.randes_retrieve.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
         L.randes_retrieve.restype = ctypes.c_int
+        L.randes_retrieve_static.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
+        L.randes_retrieve_static.restype = ctypes.c_int
         L.randes_launch_count.argtypes = []
         L.randes_launch_count.restype = u64
         L.randes_last_error.argtypes = []
@@ -102,7 +104,7 @@ EXPORTS = [
     "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
     "randes_task_tables", "randes_compress", "randes_add_model", "randes_remove_model",
-    "randes_retrieve", "randes_launch_count", "randes_last_error",
+    "randes_retrieve", "randes_retrieve_static", "randes_launch_count", "randes_last_error",
 ]
 
 
@@ -174,6 +176,11 @@ def randes_remove_model(plan, task_id, base, task, M, stream) -> None:
 
 def randes_retrieve(plan, task_id, lam, out_dtype, base, M, out, stream) -> None:
     _check(lib().randes_retrieve(plan, task_id, lam, out_dtype, _addr(base), _addr(M), _addr(out), stream))
+
+
+def randes_retrieve_static(plan, task_id, lam, out_dtype, base, M, out, stream) -> None:
+    """retrieve with the kernel's tables in the library's built-in device array (no workspace)."""
+    _check(lib().randes_retrieve_static(plan, task_id, lam, out_dtype, _addr(base), _addr(M), _addr(out), stream))
 
 
 def randes_launch_count() -> int:

@@ -203,67 +203,72 @@ template <int CPL> __device__ __forceinline__ WarpTile warp_tile(const DevUnit& 
 // (Section 4, second display; Section 4.4, second display.)  The sign is folded
 // into lambda: fma(+-lambda, m, w) is bit-identical to fma(lambda, +-m, w).
 // =========================================================================================
-template <typename ST, typename OT, bool VEC>
+#ifndef RANDES_RET_U
+#define RANDES_RET_U 4
+#endif
+#ifndef RANDES_RET_MINB
+#define RANDES_RET_MINB 2
+#endif
+
+// Vector path: U rows per trip, all loads issued before the first use.
+template <typename ST, typename OT>
 __device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, const float* __restrict__ mp,
                                               const ST* __restrict__ wp, OT* __restrict__ op,
                                               const float (&lam)[Store<ST>::CPL])
 {
     constexpr int CPL = Store<ST>::CPL;
-    constexpr int U = CPL == 4 ? 4 : 2;
-    for (uint32_t r = t.r0; r < t.r_end; r += t.rstep * U) {
+    constexpr int U = CPL == 4 ? RANDES_RET_U : RANDES_RET_U / 2;
+    const uint32_t row_stride = t.rstep * cols;
+    uint32_t off = t.r0 * cols + t.c;               // layers hold < 2^32 elements
+    for (uint32_t r = t.r0; r < t.r_end; r += t.rstep * U, off += row_stride * U) {
         float4 m[U][CPL / 4];
         uint4 w[U];
-        float ms[U][CPL], wsc[U][CPL];
 #pragma unroll
         for (int j = 0; j < U; ++j) {
-            const uint32_t rr = r + j * t.rstep;
-            if (rr < t.r_end) {
-                const size_t off = static_cast<size_t>(rr) * cols + t.c;
-                if (VEC) {
+            if (r + j * t.rstep < t.r_end) {
+                const uint32_t o = off + j * row_stride;
 #pragma unroll
-                    for (int h = 0; h < CPL / 4; ++h) m[j][h] = __ldcs(reinterpret_cast<const float4*>(mp + off) + h);
-                    w[j] = __ldcs(reinterpret_cast<const uint4*>(wp + off));
-                } else {
-#pragma unroll
-                    for (int e = 0; e < CPL; ++e) {
-                        ms[j][e] = 0.f; wsc[j][e] = 0.f;
-                        if (t.c + e < cols) { ms[j][e] = mp[off + e]; wsc[j][e] = Store<ST>::load1(wp + off + e); }
-                    }
-                }
+                for (int h = 0; h < CPL / 4; ++h) m[j][h] = __ldcs(reinterpret_cast<const float4*>(mp + o) + h);
+                w[j] = __ldcs(reinterpret_cast<const uint4*>(wp + o));
             }
         }
 #pragma unroll
         for (int j = 0; j < U; ++j) {
-            const uint32_t rr = r + j * t.rstep;
-            if (rr < t.r_end) {
-                const size_t off = static_cast<size_t>(rr) * cols + t.c;
+            if (r + j * t.rstep < t.r_end) {
+                const uint32_t o = off + j * row_stride;
                 float mv[CPL], wv[CPL], y[CPL];
-                if (VEC) {
 #pragma unroll
-                    for (int h = 0; h < CPL / 4; ++h) {
-                        mv[4 * h] = m[j][h].x; mv[4 * h + 1] = m[j][h].y; mv[4 * h + 2] = m[j][h].z; mv[4 * h + 3] = m[j][h].w;
-                    }
-                    Store<ST>::widen(w[j], wv);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < CPL; ++e) { mv[e] = ms[j][e]; wv[e] = wsc[j][e]; }
+                for (int h = 0; h < CPL / 4; ++h) {
+                    mv[4 * h] = m[j][h].x; mv[4 * h + 1] = m[j][h].y; mv[4 * h + 2] = m[j][h].z; mv[4 * h + 3] = m[j][h].w;
                 }
+                Store<ST>::widen(w[j], wv);
 #pragma unroll
                 for (int e = 0; e < CPL; ++e) y[e] = __fmaf_rn(lam[e], mv[e], wv[e]);
-                if (VEC) {
-                    Out<OT>::template store<CPL>(op + off, y);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < CPL; ++e)
-                        if (t.c + e < cols) Out<OT>::store1(op + off + e, y[e]);
-                }
+                Out<OT>::template store<CPL>(op + o, y);
             }
         }
     }
 }
 
+// Element-at-a-time path for ragged widths and unaligned tensors; out of line so
+// that it does not set the register budget of the vector path.
 template <typename ST, typename OT>
-__global__ void __launch_bounds__(kThreadsPerCta) retrieve_kernel(const RetrieveArgs a)
+__device__ __noinline__ void retrieve_rows_scalar(WarpTile t, uint32_t cols, const float* mp, const ST* wp, OT* op, float lambda,
+                                                  uint32_t bits)
+{
+    constexpr int CPL = Store<ST>::CPL;
+    for (uint32_t r = t.r0; r < t.r_end; r += t.rstep) {
+        const size_t off = static_cast<size_t>(r) * cols + t.c;
+        for (int e = 0; e < CPL; ++e) {
+            if (t.c + e >= cols) break;
+            const float lam = flip(lambda, ((bits >> e) & 1u) << 31);
+            Out<OT>::store1(op + off + e, __fmaf_rn(lam, mp[off + e], Store<ST>::load1(wp + off + e)));
+        }
+    }
+}
+
+template <typename ST, typename OT>
+__global__ void __launch_bounds__(kThreadsPerCta, RANDES_RET_MINB) retrieve_kernel(const RetrieveArgs a)
 {
     constexpr int CPL = Store<ST>::CPL;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -281,16 +286,18 @@ __global__ void __launch_bounds__(kThreadsPerCta) retrieve_kernel(const Retrieve
             const uint4 blk = philox4x32_10(lane_block<CPL>(t.cb, lane), slot, kTagSign, a.task.id, a.task.key0, a.task.key1);
             bits = lane_bits<CPL>(blk, lane);
         }
-        float lam[CPL];
-#pragma unroll
-        for (int e = 0; e < CPL; ++e) lam[e] = flip(a.lambda, ((bits >> e) & 1u) << 31);
-
         const ST* wp = static_cast<const ST*>(a.base[p]);
         OT* op = static_cast<OT*>(a.out[p]);
         const float* mp = a.M + m_off;
         const bool vec = lp.cols % CPL == 0 && aligned16(wp) && Out<OT>::template aligned<CPL>(op);
-        if (vec) retrieve_rows<ST, OT, true>(t, lp.cols, mp, wp, op, lam);
-        else retrieve_rows<ST, OT, false>(t, lp.cols, mp, wp, op, lam);
+        if (vec) {
+            float lam[CPL];
+#pragma unroll
+            for (int e = 0; e < CPL; ++e) lam[e] = flip(a.lambda, ((bits >> e) & 1u) << 31);
+            retrieve_rows<ST, OT>(t, lp.cols, mp, wp, op, lam);
+        } else {
+            retrieve_rows_scalar<ST, OT>(t, lp.cols, mp, wp, op, a.lambda, bits);
+        }
     }
 }
 

@@ -184,6 +184,19 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda,
                     void* const* out, void* stream);
 
 /*
+ * Batched retrieve: rebuild n_tasks models in one pass (Section 4, second
+ * display, for several tasks at once; the multi-model serving case of the
+ * paper's introduction).  Equivalent, bit for bit, to n_tasks calls of
+ * randes_retrieve, but W_0 is read once instead of n_tasks times.
+ *   task_ids[n_tasks]           distinct registered ids, 1 <= n_tasks <= 32 and <= max_tasks
+ *   out[n_tasks * n_layers]     out[b*n_layers + l] = layer l of the b-th requested model
+ * One kernel launch.  Errors: as randes_retrieve, plus DUPLICATE_TASK, CAPACITY.
+ */
+int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_t n_tasks, float lambda,
+                          randes_dtype_t out_dtype, const void* const* base, const void* M,
+                          void* const* out, void* stream);
+
+/*
  * retrieve for callers that cannot provide a device workspace.  (The paper has
  * no counterpart: this entry point exists for deployment, not for the method.)
  *

@@ -173,6 +173,7 @@ struct randes_plan_s {
     int sm_count = 0;
     int grid_acc[2] = {0, 0};   // [0] compress, [1] one task (add / remove)
     int grid_ret[2] = {0, 0};
+    int grid_batch[2] = {0, 0};
     // host mirrors of what the device pointer tables currently hold
     std::vector<const void*> h_base, h_out, h_tasks;
     std::vector<DevTask> h_dev_tasks;
@@ -441,6 +442,8 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         p->grid_acc[1] = p->sm_count * occ_acc1;
         p->grid_ret[0] = p->sm_count * occ_r0;
         p->grid_ret[1] = p->sm_count * occ_r1;
+        p->grid_batch[0] = p->sm_count * std::max(1, retrieve_batch_ctas_per_sm(p->storage, RANDES_F32));
+        p->grid_batch[1] = p->sm_count * std::max(1, retrieve_batch_ctas_per_sm(p->storage, RANDES_BF16));
         e = cudaMemcpyAsync(p->ws + p->lay.layers, p->dev_layers.data(), n_layers * sizeof(DevLayer),
                             cudaMemcpyHostToDevice, s);
         if (e == cudaSuccess && !p->units.empty())
@@ -595,6 +598,61 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_
     const int grid = std::min<int>(plan->grid_ret[out_dtype], static_cast<int>(a.n_units));
     const int e = launch_retrieve(plan->storage, out_dtype, a, grid, s);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the retrieve kernel");
+    ++g_launches;
+    return RANDES_OK;
+}
+
+int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_t n_tasks, float lambda,
+                          randes_dtype_t out_dtype, const void* const* base, const void* M, void* const* out, void* stream)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
+    if (out_dtype != RANDES_F32 && out_dtype != RANDES_BF16)
+        return fail(RANDES_UNSUPPORTED_DTYPE, "output dtype %d is not supported", static_cast<int>(out_dtype));
+    if (!task_ids || n_tasks == 0) return fail(RANDES_INVALID_ARGUMENT, "task_ids is NULL or empty");
+    if (n_tasks > static_cast<uint32_t>(kTaskChunk) || n_tasks > plan->max_tasks)
+        return fail(RANDES_CAPACITY, "a batch holds at most %d tasks (and at most max_tasks = %u); got %u", kTaskChunk,
+                    plan->max_tasks, n_tasks);
+    int rc;
+    if ((rc = check_m(M))) return rc;
+    if ((rc = check_ptrs(*plan, base, "base", elem_size(plan->storage), false))) return rc;
+    if (!out) return fail(RANDES_INVALID_ARGUMENT, "out is NULL");
+    RetrieveBatchArgs a;
+    const char* m_lo = static_cast<const char*>(M);
+    const char* m_hi = m_lo + plan->m_bytes;
+    for (uint32_t b = 0; b < n_tasks; ++b) {
+        const int row = find_task(*plan, task_ids[b]);
+        if (row < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_ids[b]);
+        for (uint32_t c = 0; c < b; ++c)
+            if (task_ids[c] == task_ids[b]) return fail(RANDES_DUPLICATE_TASK, "task id %u appears twice in the batch", task_ids[b]);
+        a.task_rows[b] = static_cast<uint32_t>(row);
+        void* const* ob = out + static_cast<size_t>(b) * plan->n_layers;
+        if ((rc = check_ptrs(*plan, const_cast<const void* const*>(ob), "out", elem_size(out_dtype), false))) return rc;
+        for (uint32_t l = 0; l < plan->n_layers; ++l) {
+            const char* o = static_cast<const char*>(ob[l]);
+            if (ob[l] && (ob[l] == base[l] || (o >= m_lo && o < m_hi)))
+                return fail(RANDES_INVALID_ARGUMENT, "out[%u][%u] aliases base or M", b, l);
+        }
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if ((rc = stage_ptrs(*plan, plan->h_base, plan->base_valid, plan->lay.base_ptrs, base, s))) return rc;
+    // the batch's output tables share the device area of the task pointer tables
+    if ((rc = stage_task_ptrs(*plan, const_cast<const void* const*>(out), n_tasks, s))) return rc;
+    a.layers = plan->dev<DevLayer>(plan->lay.layers);
+    a.units = plan->dev<DevUnit>(plan->lay.units);
+    a.n_units = static_cast<uint32_t>(plan->units.size());
+    a.n_layers = plan->n_layers;
+    a.slot_of_pos = plan->dev<uint32_t>(plan->lay.slot_of_pos);
+    a.tasks = plan->dev<DevTask>(plan->lay.tasks);
+    a.n_tasks = n_tasks;
+    a.base = plan->dev<const void*>(plan->lay.base_ptrs);
+    a.out = plan->dev<void*>(plan->lay.task_ptrs);
+    a.M = static_cast<const float*>(M);
+    a.lambda = lambda;
+    if (a.n_units == 0) return RANDES_OK;
+    const int grid = std::min<int>(plan->grid_batch[out_dtype], static_cast<int>(a.n_units));
+    const int e = launch_retrieve_batch(plan->storage, out_dtype, a, grid, s);
+    if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the batched retrieve kernel");
     ++g_launches;
     return RANDES_OK;
 }

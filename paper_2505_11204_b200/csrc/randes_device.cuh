@@ -1,0 +1,188 @@
+// Device-side helpers shared by the kernels of the RanDeS library: Philox4x32-10,
+// packed fp32x2 arithmetic, element access for fp32 / bf16 storage and output,
+// the lane <-> column mapping and the geometry of a warp inside a unit of work.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "randes_internal.h"
+
+namespace randes {
+namespace device {
+
+
+typedef __nv_bfloat16 bf16;
+
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11): counter (c0..c3), key (k0,k1).
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                               uint32_t k1)
+{
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+__device__ __forceinline__ float flip(float x, uint32_t mask) { return __uint_as_float(__float_as_uint(x) ^ mask); }
+
+// Two fp32 values in one 64-bit register, for the packed add / sub / fma of sm_100.
+// Each half is rounded to nearest even exactly like the scalar instruction.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(uint32_t lo, uint32_t hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi)
+{
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
+// ---- storage types: a lane's 16 bytes hold CPL columns -------------------------------------
+template <typename T> struct Store;
+
+template <> struct Store<float> {
+    static constexpr int CPL = 4;
+    static __device__ __forceinline__ void widen(const uint4& raw, float (&v)[4])
+    {
+        v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y);
+        v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
+    }
+    static __device__ __forceinline__ void widen2(const uint4& raw, f32x2 (&v)[2])
+    {
+        v[0] = pack2(raw.x, raw.y);
+        v[1] = pack2(raw.z, raw.w);
+    }
+    static __device__ __forceinline__ float load1(const float* p) { return __ldg(p); }
+};
+
+template <> struct Store<bf16> {
+    static constexpr int CPL = 8;
+    static __device__ __forceinline__ void widen(const uint4& raw, float (&v)[8])
+    {
+        v[0] = __uint_as_float(raw.x << 16); v[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+        v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+        v[4] = __uint_as_float(raw.z << 16); v[5] = __uint_as_float(raw.z & 0xFFFF0000u);
+        v[6] = __uint_as_float(raw.w << 16); v[7] = __uint_as_float(raw.w & 0xFFFF0000u);
+    }
+    static __device__ __forceinline__ void widen2(const uint4& raw, f32x2 (&v)[4])
+    {
+        v[0] = pack2(raw.x << 16, raw.x & 0xFFFF0000u);
+        v[1] = pack2(raw.y << 16, raw.y & 0xFFFF0000u);
+        v[2] = pack2(raw.z << 16, raw.z & 0xFFFF0000u);
+        v[3] = pack2(raw.w << 16, raw.w & 0xFFFF0000u);
+    }
+    static __device__ __forceinline__ float load1(const bf16* p)
+    {
+        return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
+    }
+};
+
+// ---- output types: CPL consecutive values ---------------------------------------------------
+template <typename T> struct Out;
+
+template <> struct Out<float> {
+    template <int CPL> static __device__ __forceinline__ void store(float* p, const float (&y)[CPL])
+    {
+#pragma unroll
+        for (int j = 0; j < CPL / 4; ++j)
+            __stcs(reinterpret_cast<float4*>(p) + j, make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]));
+    }
+    static __device__ __forceinline__ void store1(float* p, float v) { *p = v; }
+    template <int CPL> static __device__ __forceinline__ bool aligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+};
+
+template <> struct Out<bf16> {
+    // round to nearest even, two values per conversion
+    static __device__ __forceinline__ uint32_t pack(float lo, float hi)
+    {
+        const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t*>(&v);
+    }
+    template <int CPL> static __device__ __forceinline__ void store(bf16* p, const float (&y)[CPL])
+    {
+        if (CPL == 4) {
+            __stcs(reinterpret_cast<uint2*>(p), make_uint2(pack(y[0], y[1]), pack(y[2], y[3])));
+        } else {
+            __stcs(reinterpret_cast<uint4*>(p),
+                   make_uint4(pack(y[0], y[1]), pack(y[2], y[3]), pack(y[4 % CPL], y[5 % CPL]), pack(y[6 % CPL], y[7 % CPL])));
+        }
+    }
+    static __device__ __forceinline__ void store1(bf16* p, float v) { *p = __float2bfloat16_rn(v); }
+    template <int CPL> static __device__ __forceinline__ bool aligned(const void* p)
+    {
+        return (reinterpret_cast<uintptr_t>(p) & (2 * CPL - 1)) == 0;
+    }
+};
+
+__device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// The sign bits of this lane's CPL columns (bit e = column c + e), out of the
+// Philox block that covers them.
+template <int CPL> __device__ __forceinline__ uint32_t lane_bits(const uint4& blk, int lane)
+{
+    if (CPL == 4) {
+        const int q = lane >> 3;
+        const uint32_t w = q == 0 ? blk.x : (q == 1 ? blk.y : (q == 2 ? blk.z : blk.w));
+        return (w >> ((lane & 7) * 4)) & 0xFu;
+    }
+    const int q = (lane & 15) >> 2;
+    const uint32_t w = q == 0 ? blk.x : (q == 1 ? blk.y : (q == 2 ? blk.z : blk.w));
+    return (w >> ((lane & 3) * 8)) & 0xFFu;
+}
+
+// Which 128-column Philox block holds this lane's columns.
+template <int CPL> __device__ __forceinline__ uint32_t lane_block(uint32_t cb, int lane)
+{
+    return CPL == 4 ? cb : cb * 2 + (lane >> 4);
+}
+
+// geometry of this warp inside a unit
+struct WarpTile {
+    uint32_t cb;      // warp-wide column block of the layer
+    uint32_t c;       // first of this lane's CPL columns
+    uint32_t r0;      // first row of this warp
+    uint32_t r_end;   // one past the last row of the unit
+    uint32_t rstep;   // row stride between this warp's rows
+};
+
+template <int CPL> __device__ __forceinline__ WarpTile warp_tile(const DevUnit& un, int warp, int lane)
+{
+    WarpTile t;
+    const uint32_t nbc = un.nbc;
+    t.cb = un.cb0 + (warp & (nbc - 1));
+    t.c = (t.cb * 32 + lane) * CPL;
+    t.rstep = kWarpsPerCta / nbc;
+    t.r0 = un.row0 + warp / nbc;
+    t.r_end = un.row0 + un.nrows;
+    return t;
+}
+
+
+}  // namespace device
+}  // namespace randes

@@ -12,7 +12,10 @@ constexpr uint32_t kFlagFlip = 2u;      // per-column sign flip on this slot
 
 constexpr int kWarpsPerCta = 8;
 constexpr int kThreadsPerCta = kWarpsPerCta * 32;
-constexpr int kRowsPerWarp = 16;        // rows one warp walks per unit
+#ifndef RANDES_ROWS_PER_WARP
+#define RANDES_ROWS_PER_WARP 16
+#endif
+constexpr int kRowsPerWarp = RANDES_ROWS_PER_WARP;   // rows one warp walks per unit
 constexpr int kTaskChunk = 32;          // tasks whose pointers / sign blocks a warp holds at once
 constexpr uint32_t kTagSign = 0x5349474Eu;  // counter word 2 of the sign stream ("SIGN")
 constexpr uint32_t kTagPerm = 0x5045524Du;  // counter word 2 of the permutation stream ("PERM")
@@ -81,6 +84,21 @@ struct AccumulateArgs {
     float* M;
 };
 
+struct RetrieveBatchArgs {
+    const DevLayer* layers;
+    const DevUnit* units;
+    uint32_t n_units;
+    uint32_t n_layers;
+    const uint32_t* slot_of_pos;   // all registered tasks' sigma^-1 rows, n_layers entries each
+    const DevTask* tasks;          // all registered tasks' descriptors
+    uint32_t task_rows[kTaskChunk];   // which rows to rebuild, in output order
+    uint32_t n_tasks;              // <= kTaskChunk
+    const void* const* base;       // device array [n_layers]
+    void* const* out;              // device array [n_tasks][n_layers]
+    const float* M;
+    float lambda;
+};
+
 // Launchers (randes_kernels.cu).  Return a cudaError_t as int.
 int launch_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, int grid, void* stream);
 int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void* stream);
@@ -89,6 +107,9 @@ int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void
 // dynamic shared memory they need: call once per device before launching.
 int retrieve_ctas_per_sm(int storage_dtype, int out_dtype);
 int accumulate_ctas_per_sm(int storage_dtype, bool single_task);
+// randes_batch.cu
+int launch_retrieve_batch(int storage_dtype, int out_dtype, const RetrieveBatchArgs& a, int grid, void* stream);
+int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype);
 
 
 // Retrieve with its tables in a fixed device array inside the library (no workspace).

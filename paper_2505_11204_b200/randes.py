@@ -90,6 +90,8 @@ def lib():
         L.randes_remove_model.restype = ctypes.c_int
         L.randes_retrieve.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
         L.randes_retrieve.restype = ctypes.c_int
+        L.randes_retrieve_batch.argtypes = [vp, vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
+        L.randes_retrieve_batch.restype = ctypes.c_int
         L.randes_retrieve_static.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
         L.randes_retrieve_static.restype = ctypes.c_int
         L.randes_launch_count.argtypes = []
@@ -104,7 +106,7 @@ EXPORTS = [
     "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
     "randes_task_tables", "randes_compress", "randes_add_model", "randes_remove_model",
-    "randes_retrieve", "randes_retrieve_static", "randes_launch_count", "randes_last_error",
+    "randes_retrieve", "randes_retrieve_batch", "randes_retrieve_static", "randes_launch_count", "randes_last_error",
 ]
 
 
@@ -176,6 +178,13 @@ def randes_remove_model(plan, task_id, base, task, M, stream) -> None:
 
 def randes_retrieve(plan, task_id, lam, out_dtype, base, M, out, stream) -> None:
     _check(lib().randes_retrieve(plan, task_id, lam, out_dtype, _addr(base), _addr(M), _addr(out), stream))
+
+
+def randes_retrieve_batch(plan, task_ids, lam, out_dtype, base, M, out, stream) -> None:
+    """Several tasks in one pass; ``out`` holds n_tasks * n_layers pointers, task-major."""
+    ids = (ctypes.c_uint32 * len(task_ids))(*[int(t) for t in task_ids])
+    _check(lib().randes_retrieve_batch(plan, ctypes.addressof(ids), len(task_ids), lam, out_dtype, _addr(base), _addr(M),
+                                       _addr(out), stream))
 
 
 def randes_retrieve_static(plan, task_id, lam, out_dtype, base, M, out, stream) -> None:
@@ -323,6 +332,16 @@ class Plan:
     def remove_model(self, task_id: int, base, task, M):
         randes_remove_model(self.handle, task_id, _as_ptrs(base), _as_ptrs(task), M, self._stream())
         return M
+
+    def retrieve_batch(self, task_ids, lam: float, base, M, out=None, out_dtype: int = F32):
+        """Rebuild several tasks in one launch; returns a list (per task) of lists of tensors."""
+        out_lists = None
+        if out is None:
+            out = out_lists = [self.new_output(out_dtype) for _ in task_ids]
+        elif not isinstance(out, ctypes.Array):
+            out_lists = out
+        randes_retrieve_batch(self.handle, task_ids, lam, out_dtype, _as_ptrs(base), M, _as_ptrs(out), self._stream())
+        return out_lists
 
     def retrieve(self, task_id: int, lam: float, base, M, out=None, out_dtype: int = F32):
         out_list = None

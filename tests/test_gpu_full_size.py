@@ -100,6 +100,17 @@ def run_full_size(storage, n_swap):
 
     for t, s in zip(ids, seeds):
         check_retrieve(t, s, "sweep")
+    if storage == wl.F32:
+        # all 20 tasks in one launch: the same sampled layers, against the same oracle results
+        outs = [plan.new_output(wl.F32) for _ in ids]
+        randes.randes_retrieve_batch(plan.handle, ids, w.lam, wl.F32, p_base, M, randes.ptr_array(outs), sh)
+        for b, (t, s) in enumerate(zip(ids, seeds)):
+            pos = sorted(set(int(src_of[t][l]) for l in slots))
+            ref = ro.retrieve(w.spec, storage, wl.F32, t, s, w.lam, base_h, M_ref, positions=pos)
+            for p in pos:
+                assert_bits_equal(from_dev(outs[b][p]), ref[p], "batched retrieve task %d layer %d" % (t, p))
+        del outs
+        torch.cuda.empty_cache()
     for t, s in zip(swap_ids, swap_seeds):
         randes.randes_add_model(plan.handle, t, s, p_base, randes.ptr_array(d_tasks[t]), M, sh)
         ro.add_model(w.spec, storage, t, s, base_h, tasks_h[t], M_ref, slots=slots)

@@ -195,6 +195,31 @@ def test_unaligned_tensors_take_the_scalar_path():
         plan.close()
 
 
+@pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
+def test_batched_retrieve_equals_single_retrieves(storage):
+    # several tasks rebuilt in one pass over W_0: bit-identical to one call per task
+    w = make_workload(RAGGED, storage=storage, n_tasks=6)
+    base, tasks = wl.model_set(w)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w)
+    M = plan.compress(d_base, d_tasks)
+    M_ref = ro.compress(w.spec, storage, w.task_ids, w.seeds, base, tasks)
+    for od in (wl.F32, wl.BF16):
+        for batch in ([4, 0, 5, 2, 1, 3], [3], [5, 1]):
+            outs = [[poison(o) for o in plan.new_output(od)] for _ in batch]
+            plan.retrieve_batch(batch, w.lam, d_base, M, out=outs, out_dtype=od)
+            for b, t in enumerate(batch):
+                ref = ro.retrieve(w.spec, storage, od, t, w.seeds[t], w.lam, base, M_ref)
+                check_model(outs[b], ref, "batched retrieve task %d dtype %d" % (t, od))
+    with pytest.raises(randes.RandesError) as e:
+        plan.retrieve_batch([1, 1], w.lam, d_base, M)
+    assert e.value.code == randes.DUPLICATE_TASK
+    with pytest.raises(randes.RandesError) as e:
+        plan.retrieve_batch([1, 77], w.lam, d_base, M)
+    assert e.value.code == randes.UNKNOWN_TASK
+    plan.close()
+
+
 def test_gpu_argument_validation():
     import torch
 

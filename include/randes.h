@@ -59,8 +59,18 @@ typedef struct randes_plan_s randes_plan_t; /* opaque, host memory, library-owne
 
 typedef enum { RANDES_F32 = 0, RANDES_BF16 = 1 } randes_dtype_t;
 
-/* per-group transform flags */
-enum { RANDES_SHUFFLE = 1, RANDES_FLIP = 2 };
+/* per-group transform flags.
+ *   RANDES_SHUFFLE  random permutation of the group's members per task (Section 4.3)
+ *   RANDES_FLIP     per-column +-1 sign flip (Section 4.4)
+ *   RANDES_SHIFT    deterministic alternative to SHUFFLE (appendix on the dynamics between
+ *                   shuffling and sign flips): the participating members are rotated
+ *                   towards higher index, task t by 1 + (t mod (n - 1)) of n positions.
+ *                   Mutually exclusive with RANDES_SHUFFLE.
+ *   RANDES_SKIP(k)  skip rate of the same appendix: only the members with index 0, k,
+ *                   2k, ... of the group (in layer order) are shuffled / shifted and
+ *                   flipped; k = 0 or 1 means all.  1 <= k <= 255. */
+enum { RANDES_SHUFFLE = 1, RANDES_FLIP = 2, RANDES_SHIFT = 4 };
+#define RANDES_SKIP(k) (((uint32_t)(k) & 0xFFu) << 8)
 
 typedef struct { uint32_t rows, cols, group; } randes_layer_t;
 typedef struct { uint32_t flags; } randes_group_t;

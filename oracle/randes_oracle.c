@@ -29,6 +29,15 @@
  *   - Random numbers: Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11),
  *     key = the task's 64-bit seed, counter = (index, layer-or-group, domain
  *     tag, task id).
+ *   - Skip rate k (appendix on the dynamics between shuffling and sign flips):
+ *     of the members of a group, in layer order, those with index 0, k, 2k, ...
+ *     take part in the shuffle (among themselves) and in the flip; the others
+ *     are left as they are.
+ *   - Layer shifting (same appendix): "one position deeper with wrap-around"
+ *     is read as a rotation of the participating members towards higher block
+ *     index; task t rotates by 1 + (t mod (n - 1)) positions (n participants),
+ *     so that different tasks are misaligned and no task gets the identity.
+ *     Slot k then receives member (k - shift) mod n.
  *   - Arithmetic: fp32; the subtraction W_i - W_0 and each accumulation are
  *     separately rounded; retrieval is one fused multiply-add; bf16 is
  *     round-to-nearest-even.
@@ -50,6 +59,8 @@
 #define RO_BF16 1
 #define RO_SHUFFLE 1u
 #define RO_FLIP 2u
+#define RO_SHIFT 4u                      /* deterministic rotation instead of a random permutation */
+#define RO_SKIP(flags) (((flags) >> 8) & 0xFFu) /* every k-th member of a group takes part; 0 and 1 = all */
 
 #define RO_TAG_PERM 0x5045524Du /* "PERM" */
 #define RO_TAG_SIGN 0x5349474Eu /* "SIGN" */
@@ -138,6 +149,21 @@ void ro_sign_row(uint64_t seed, uint32_t task_id, uint32_t slot, uint32_t cols, 
 /* Group members are the layers carrying that group id, in layer order.      */
 /* Returns 0, or -1 if a group id is out of range / allocation fails.        */
 /* ------------------------------------------------------------------------ */
+/* 1 if the layer's position inside its group is one the skip rate selects. */
+static int takes_part(uint32_t n_layers, const uint32_t *group, const uint32_t *gflags, uint32_t l)
+{
+    uint32_t j = 0, k = RO_SKIP(gflags[group[l]]);
+    for (uint32_t a = 0; a < l && a < n_layers; ++a)
+        if (group[a] == group[l]) ++j;
+    return k <= 1 || j % k == 0;
+}
+
+/* 1 if slot l is sign-flipped (Section 4.4, restricted by the skip rate). */
+int ro_layer_flips(uint32_t n_layers, const uint32_t *group, const uint32_t *gflags, uint32_t l)
+{
+    return (gflags[group[l]] & RO_FLIP) != 0 && takes_part(n_layers, group, gflags, l);
+}
+
 int ro_task_tables(uint32_t n_layers, const uint32_t *group, uint32_t n_groups,
                    const uint32_t *gflags, uint64_t seed, uint32_t task_id,
                    uint32_t *src_of_slot, uint32_t *slot_of_pos)
@@ -151,12 +177,20 @@ int ro_task_tables(uint32_t n_layers, const uint32_t *group, uint32_t n_groups,
         slot_of_pos[l] = l;
     }
     for (uint32_t g = 0; g < n_groups; ++g) {
-        uint32_t G = 0;
+        /* the participating members of the group, in layer order */
+        uint32_t n = 0;
         for (uint32_t l = 0; l < n_layers; ++l)
-            if (group[l] == g) members[G++] = l;
-        if (G < 2 || !(gflags[g] & RO_SHUFFLE)) continue;
-        ro_permutation(seed, task_id, g, G, sigma);
-        for (uint32_t k = 0; k < G; ++k) {
+            if (group[l] == g && takes_part(n_layers, group, gflags, l)) members[n++] = l;
+        if (n < 2) continue;
+        if (gflags[g] & RO_SHUFFLE) {
+            ro_permutation(seed, task_id, g, n, sigma);
+        } else if (gflags[g] & RO_SHIFT) {
+            uint32_t shift = 1u + task_id % (n - 1u);
+            for (uint32_t k = 0; k < n; ++k) sigma[k] = (k + n - shift) % n;
+        } else {
+            continue;
+        }
+        for (uint32_t k = 0; k < n; ++k) {
             src_of_slot[members[k]] = members[sigma[k]];
             slot_of_pos[members[sigma[k]]] = members[k];
         }
@@ -220,6 +254,8 @@ typedef struct {
 
 static int spec_check(const ro_spec_t *s)
 {
+    for (uint32_t g = 0; g < s->n_groups; ++g)
+        if ((s->gflags[g] & RO_SHUFFLE) && (s->gflags[g] & RO_SHIFT)) return -3;
     /* all members of a group must have one shape (Section 4.3: same type) */
     for (uint32_t a = 0; a < s->n_layers; ++a) {
         if (s->group[a] >= s->n_groups) return -1;
@@ -254,7 +290,7 @@ static int accumulate_one(const ro_spec_t *s, int dtype, int sign_op,
         if (slot_mask && !slot_mask[l]) continue;
         uint32_t rows = s->rows[l], cols = s->cols[l];
         uint32_t src = src_of_slot[l];
-        int flip = (s->gflags[s->group[l]] & RO_FLIP) != 0;
+        int flip = ro_layer_flips(L, s->group, s->gflags, l);
         int8_t *sg = (int8_t *)malloc(cols ? cols : 1);
         if (!sg) { free(src_of_slot); free(slot_of_pos); return -1; }
         if (flip) ro_sign_row(seed, task_id, l, cols, sg);
@@ -367,7 +403,7 @@ int ro_retrieve(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
         if (pos_mask && !pos_mask[p]) continue;
         uint32_t nr = rows[p], nc = cols[p];
         uint32_t l = slot_of_pos[p];
-        int flip = (gflags[group[p]] & RO_FLIP) != 0;
+        int flip = ro_layer_flips(L, group, gflags, l);
         int8_t *sg = (int8_t *)malloc(nc ? nc : 1);
         if (!sg) { free(src_of_slot); free(slot_of_pos); return -1; }
         if (flip) ro_sign_row(seed, task_id, l, nc, sg);

@@ -27,6 +27,12 @@ F32 = 0
 BF16 = 1
 SHUFFLE = 1
 FLIP = 2
+SHIFT = 4
+
+
+def SKIP(k: int) -> int:
+    """Group flag bits for 'only every k-th member takes part'."""
+    return (int(k) & 0xFF) << 8
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "randes_oracle.c")

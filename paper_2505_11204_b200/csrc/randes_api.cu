@@ -185,6 +185,15 @@ struct randes_plan_s {
 
 namespace {
 
+// the members of group g that the skip rate selects (every k-th, in layer order)
+std::vector<uint32_t> participants(const randes_plan_t& p, uint32_t g)
+{
+    const uint32_t k = std::max<uint32_t>(1, (p.gflags[g] >> 8) & 0xFFu);
+    std::vector<uint32_t> out;
+    for (size_t j = 0; j < p.members[g].size(); j += k) out.push_back(p.members[g][j]);
+    return out;
+}
+
 void make_task_tables(const randes_plan_t& p, TaskEntry& t)
 {
     t.src_of_slot.resize(p.n_layers);
@@ -192,9 +201,19 @@ void make_task_tables(const randes_plan_t& p, TaskEntry& t)
     for (uint32_t l = 0; l < p.n_layers; ++l) t.src_of_slot[l] = t.slot_of_pos[l] = l;
     std::vector<uint32_t> sigma;
     for (uint32_t g = 0; g < p.n_groups; ++g) {
-        const std::vector<uint32_t>& mem = p.members[g];
-        if (mem.size() < 2 || !(p.gflags[g] & RANDES_SHUFFLE)) continue;
-        draw_sigma(t.seed, t.id, g, static_cast<uint32_t>(mem.size()), sigma);
+        const std::vector<uint32_t> mem = participants(p, g);
+        if (mem.size() < 2) continue;
+        const uint32_t n = static_cast<uint32_t>(mem.size());
+        if (p.gflags[g] & RANDES_SHUFFLE) {
+            draw_sigma(t.seed, t.id, g, n, sigma);
+        } else if (p.gflags[g] & RANDES_SHIFT) {
+            // rotate towards higher index by `shift`: slot k receives member k - shift
+            const uint32_t shift = 1u + t.id % (n - 1u);
+            sigma.resize(n);
+            for (uint32_t k = 0; k < n; ++k) sigma[k] = (k + n - shift) % n;
+        } else {
+            continue;
+        }
         for (size_t k = 0; k < mem.size(); ++k) {
             t.src_of_slot[mem[k]] = mem[sigma[k]];     // slot k receives member sigma(k)
             t.slot_of_pos[mem[sigma[k]]] = mem[k];
@@ -347,8 +366,12 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         return fail(RANDES_INVALID_ARGUMENT, "max_tasks = %u must be >= max(1, n_tasks = %u)", max_tasks, n_tasks);
     if (n_tasks && (!task_ids || !seeds)) return fail(RANDES_INVALID_ARGUMENT, "task_ids / seeds is NULL");
     for (uint32_t g = 0; g < n_groups; ++g)
-        if (groups[g].flags & ~static_cast<uint32_t>(RANDES_SHUFFLE | RANDES_FLIP))
+    {
+        if (groups[g].flags & ~static_cast<uint32_t>(RANDES_SHUFFLE | RANDES_FLIP | RANDES_SHIFT | RANDES_SKIP(0xFF)))
             return fail(RANDES_INVALID_ARGUMENT, "group %u: unknown flag bits 0x%x", g, groups[g].flags);
+        if ((groups[g].flags & RANDES_SHUFFLE) && (groups[g].flags & RANDES_SHIFT))
+            return fail(RANDES_INVALID_ARGUMENT, "group %u: RANDES_SHUFFLE and RANDES_SHIFT exclude each other", g);
+    }
     for (uint32_t i = 0; i < n_tasks; ++i)
         for (uint32_t j = 0; j < i; ++j)
             if (task_ids[i] == task_ids[j]) return fail(RANDES_DUPLICATE_TASK, "task id %u appears twice", task_ids[i]);
@@ -389,10 +412,13 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
             d.m_off = off / sizeof(float);
             d.rows = layers[l].rows;
             d.cols = layers[l].cols;
-            d.flags = (p->gflags[g] & RANDES_FLIP ? kFlagFlip : 0u) |
-                      ((p->gflags[g] & RANDES_SHUFFLE) && mem.size() >= 2 ? kFlagShuffle : 0u);
             d.group = g;
             d.member = static_cast<uint32_t>(std::find(mem.begin(), mem.end(), l) - mem.begin());
+            const uint32_t skip = std::max<uint32_t>(1, (p->gflags[g] >> 8) & 0xFFu);
+            const bool takes_part = d.member % skip == 0;
+            const size_t n_part = (mem.size() + skip - 1) / skip;
+            d.flags = ((p->gflags[g] & RANDES_FLIP) && takes_part ? kFlagFlip : 0u) |
+                      ((p->gflags[g] & (RANDES_SHUFFLE | RANDES_SHIFT)) && takes_part && n_part >= 2 ? kFlagShuffle : 0u);
             d.group_size = static_cast<uint32_t>(mem.size());
             p->dev_layers[l] = d;
             p->m_off_bytes[l] = off;

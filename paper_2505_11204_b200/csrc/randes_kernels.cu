@@ -49,7 +49,9 @@ __device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, 
                                               const float (&lam)[Store<ST>::CPL])
 {
     constexpr int CPL = Store<ST>::CPL;
-    constexpr int U = CPL == 4 ? RANDES_RET_U : RANDES_RET_U / 2;
+    // rows per trip, measured best per type pair: bf16 weights with fp32 output move 80 B per lane
+    // and row and are fastest one row at a time; bf16 -> bf16 (48 B) wants four
+    constexpr int U = CPL == 4 ? RANDES_RET_U : (sizeof(OT) == 4 ? 1 : 4);
     const uint32_t row_stride = t.rstep * cols;
     uint32_t off = t.r0 * cols + t.c;               // layers hold < 2^32 elements
     for (uint32_t r = t.r0; r < t.r_end; r += t.rstep * U, off += row_stride * U) {
@@ -100,7 +102,11 @@ __device__ __noinline__ void retrieve_rows_scalar(WarpTile t, uint32_t cols, con
 }
 
 template <typename ST, typename OT>
-__global__ void __launch_bounds__(kThreadsPerCta, RANDES_RET_MINB) retrieve_kernel(const RetrieveArgs a)
+#ifndef RANDES_RET_MINB_BF16
+#define RANDES_RET_MINB_BF16 2
+#endif
+__global__ void __launch_bounds__(kThreadsPerCta, Store<ST>::CPL == 4 ? RANDES_RET_MINB : RANDES_RET_MINB_BF16)
+    retrieve_kernel(const RetrieveArgs a)
 {
     constexpr int CPL = Store<ST>::CPL;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

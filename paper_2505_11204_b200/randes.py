@@ -21,6 +21,12 @@ F32 = 0
 BF16 = 1
 SHUFFLE = 1
 FLIP = 2
+SHIFT = 4
+
+
+def SKIP(k: int) -> int:
+    """Group flag bits of RANDES_SKIP(k): only every k-th member of the group takes part."""
+    return (int(k) & 0xFF) << 8
 
 OK = 0
 INVALID_ARGUMENT = -1

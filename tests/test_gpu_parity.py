@@ -114,6 +114,14 @@ def test_mixed_group_flags():
     run_full_cycle(make_workload(shapes, flags=[S | F, S, F, 0], n_tasks=4), out_dtypes=(wl.F32,))
 
 
+def test_shift_and_skip_rate_variants():
+    # layer shifting and skip rates of the paper's appendix: plan-level variants of the same kernels
+    shapes = [(9, 132, 7), (1, 132, 7), (4, 256, 1), (6, 20, 5)]
+    SH, K = randes.SHIFT, randes.SKIP
+    for flags in ([SH | F, SH, F, SH | F | K(2)], [S | F | K(2), S | K(3), F | K(2), S | F | K(4)]):
+        run_full_cycle(make_workload(shapes, flags=flags, n_tasks=4), out_dtypes=(wl.F32,))
+
+
 def test_more_tasks_than_one_chunk():
     # 40 tasks: the kernel holds 32 task descriptors at a time
     run_full_cycle(make_workload([(5, 260, 3), (1, 33, 2), (24, 128, 2)], n_tasks=40), out_dtypes=(wl.F32,),

@@ -67,6 +67,24 @@ def test_sigma_agrees_for_many_seeds_and_group_sizes():
         p.close()
 
 
+def test_shift_and_skip_tables_match_oracle():
+    S, F, SH = randes.SHUFFLE, randes.FLIP, randes.SHIFT
+    rows = [2] * 9 + [1] * 7
+    cols = [8] * 9 + [5] * 7
+    group = [0] * 9 + [1] * 7
+    for gflags in ([SH | F, SH], [S | F | randes.SKIP(2), SH | randes.SKIP(3)], [F | randes.SKIP(4), S | randes.SKIP(2)]):
+        ids, seeds = [0, 1, 5, 11], [3, 4, 5, 6]
+        p = randes.Plan(rows, cols, group, gflags, task_ids=ids, seeds=seeds, host_only=True)
+        for t, s in zip(ids, seeds):
+            src, pos = p.task_tables(t)
+            osrc, opos = ro.task_tables((rows, cols, group, gflags), s, t)
+            assert src == osrc.tolist() and pos == opos.tolist()
+        p.close()
+    with pytest.raises(randes.RandesError) as e:
+        randes.Plan(rows, cols, group, [S | SH, 0], task_ids=[0], seeds=[0], host_only=True)
+    assert e.value.code == randes.INVALID_ARGUMENT
+
+
 def test_superposition_layout_is_one_fp32_copy_independent_of_task_count():
     w = wl.vit_b32()
     p1 = randes.Plan.from_workload(w.with_tasks(1), host_only=True)

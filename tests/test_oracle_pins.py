@@ -59,18 +59,26 @@ def dense_transform(spec, seed, task_id):
     P = np.zeros((d, d))
     # identity on every layer, then overwrite shuffled groups
     src_of_slot = list(range(L))
+    takes_part = [False] * L
     for g, fl in enumerate(gflags):
-        mem = members_of(spec, g)
+        skip = max(1, (fl >> 8) & 0xFF)
+        mem = members_of(spec, g)[::skip]          # every skip-th member of the group takes part
+        for m in mem:
+            takes_part[m] = True
         if len(mem) >= 2 and (fl & SHUFFLE):
             sigma = ro.permutation(seed, task_id, g, len(mem))
             for k, m in enumerate(mem):
                 src_of_slot[m] = mem[int(sigma[k])]
+        elif len(mem) >= 2 and (fl & ro.SHIFT):
+            shift = 1 + task_id % (len(mem) - 1)   # one or more positions deeper, with wrap-around
+            for k, m in enumerate(mem):
+                src_of_slot[mem[(k + shift) % len(mem)]] = m
     for l in range(L):
         s = src_of_slot[l]
         P[offs[l]:offs[l + 1], offs[s]:offs[s + 1]] = np.eye(sizes[l])
     D = np.zeros((d, d))
     for l in range(L):
-        if gflags[group[l]] & FLIP:
+        if (gflags[group[l]] & FLIP) and takes_part[l]:
             diag = ro.sign_row(seed, task_id, l, cols[l]).astype(np.float64)
         else:
             diag = np.ones(cols[l])
@@ -284,6 +292,51 @@ def test_transform_is_orthogonal_and_compress_retrieve_match_dense_matrices(flag
         # Section 4, second display: own delta unchanged + transformed interference
         interference = sum(Ts[t].T @ (Ts[j] @ deltas[j]) for j in range(K) if j != t)
         assert np.array_equal(flat(what) - flat(base) - lam * deltas[t], lam * interference)
+
+
+@pytest.mark.parametrize("flags", [ro.SHIFT | FLIP, ro.SHIFT, SHUFFLE | FLIP | ro.SKIP(2), ro.SHIFT | FLIP | ro.SKIP(3),
+                                   FLIP | ro.SKIP(2), SHUFFLE | ro.SKIP(4)])
+def test_shift_and_skip_rate_variants_match_dense_matrices(flags):
+    """The appendix's layer shifting and skip rate: still orthogonal, still exact on dyadic inputs."""
+    spec = tiny_spec(flags, n_a=7, n_b=5, shape_a=(2, 6), shape_b=(1, 5))
+    rng = np.random.default_rng(31)
+    ids, seeds = [0, 3, 4], [5, 6, 7]
+    base = rand_model(spec, rng, dyadic=True)
+    tasks = [rand_model(spec, rng, dyadic=True) for _ in ids]
+    Ts = []
+    for t, s in zip(ids, seeds):
+        T, _ = dense_transform(spec, s, t)
+        assert np.array_equal(T.T @ T, np.eye(T.shape[0]))
+        Ts.append(T)
+    deltas = [flat(t) - flat(base) for t in tasks]
+    M_dense = sum(T @ d for T, d in zip(Ts, deltas))
+    M = ro.compress(spec, ro.F32, ids, seeds, base, tasks)
+    assert np.array_equal(flat(M), M_dense)
+    for j in range(len(ids)):
+        what = ro.retrieve(spec, ro.F32, ro.F32, ids[j], seeds[j], 0.5, base, M)
+        assert np.array_equal(flat(what), flat(base) + 0.5 * (Ts[j].T @ M_dense))
+
+
+def test_shift_moves_layers_one_position_deeper_and_skip_leaves_the_rest():
+    rng = np.random.default_rng(32)
+    G = 5
+    spec = ([2] * G, [4] * G, [0] * G, [ro.SHIFT])
+    delta = rand_model(spec, rng)
+    M = ro.compress(spec, ro.F32, [0], [9], None, [delta])          # task 0: one position
+    for k in range(G):
+        assert np.array_equal(M[(k + 1) % G], delta[k])
+    M = ro.compress(spec, ro.F32, [2], [9], None, [delta])          # task 2: three positions
+    for k in range(G):
+        assert np.array_equal(M[(k + 3) % G], delta[k])
+    # skip rate 2: members 1 and 3 neither move nor flip
+    spec2 = ([2] * G, [4] * G, [0] * G, [SHUFFLE | FLIP | ro.SKIP(2)])
+    for seed in range(6):
+        M = ro.compress(spec2, ro.F32, [1], [seed], None, [delta])
+        assert np.array_equal(M[1], delta[1]) and np.array_equal(M[3], delta[3])
+        src, _ = ro.task_tables(spec2, seed, 1)
+        assert sorted(int(src[k]) for k in (0, 2, 4)) == [0, 2, 4]
+    with pytest.raises(ValueError):
+        ro.compress(([2, 2], [4, 4], [0, 0], [SHUFFLE | ro.SHIFT]), ro.F32, [0], [0], None, [delta[:2]])
 
 
 def test_gaussian_inputs_match_dense_matrices_within_rounding():

@@ -78,6 +78,33 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def kernel_source_hash():
+    import hashlib
+
+    h = hashlib.sha256()
+    for name in ("randes_kernels.cu", "randes_device.cuh"):
+        with open(os.path.join(ROOT, "paper_2505_11204_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def read_traffic():
+    """DRAM traffic figures taken with ncu (profiles/traffic.txt); empty once the kernels changed."""
+    out = {}
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.txt")) as f:
+            for line in f:
+                if line.startswith("#") or not line.strip():
+                    continue
+                k, v = line.split()[:2]
+                out[k] = v
+        if out.get("source_sha256") != kernel_source_hash():
+            return {}
+        return {k: float(v) for k, v in out.items() if k != "source_sha256"}
+    except Exception:
+        return {}
+
+
 def max_over_ranks(values, world, device=None):
     """Element-wise maximum of a list of floats over all ranks (identity when world == 1)."""
     if world <= 1:
@@ -348,20 +375,32 @@ def run_ours(args):
         ops[n] = {"ms_per_call": ms, "GBps": gbs, "Gparams_per_s": w.n_params / (ms * 1e-3) / 1e9,
                   "frac_of_%s_peak" % peak_kind: gbs / peak, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
                   "share_of_step": op_ms[n] / total_ms}
-    # dominant kernel by device time: retrieve_kernel vs accumulate_kernel (compress + add + remove)
-    acc_ms = op_ms["compress"] + op_ms.get("add", 0.0) + op_ms.get("remove", 0.0)
-    if op_ms["retrieve"] >= acc_ms:
-        dom, dom_bytes, dom_ms = "retrieve_kernel", b["retrieve"], ops["retrieve"]["ms_per_call"]
+    # dominant kernel = the kernel instantiation with the largest share of the step
+    shares = {"retrieve_kernel": op_ms["retrieve"],
+              "accumulate_kernel<single task> (add, remove)": op_ms.get("add", 0.0) + op_ms.get("remove", 0.0),
+              "accumulate_kernel<compress>": op_ms["compress"]}
+    dom = max(shares, key=shares.get)
+    traffic_tbl = read_traffic()
+    if dom == "retrieve_kernel":
+        dom_bytes, dom_ms = b["retrieve"], ops["retrieve"]["ms_per_call"]
+        traffic = traffic_tbl.get("retrieve_kernel_bytes_per_param")
+        traffic = traffic * w.n_params if traffic and w.storage == wl.F32 else None
+    elif dom.startswith("accumulate_kernel<single"):
+        dom_bytes, dom_ms = b["add"], (op_ms["add"] + op_ms["remove"]) / (2 * n_swap * args.steps)
+        traffic = traffic_tbl.get("accumulate_kernel_single_bytes_per_param")
+        traffic = traffic * w.n_params if traffic and w.storage == wl.F32 else None
     else:
-        dom = "accumulate_kernel (compress, add, remove launches)"
-        n_acc = (1 + 2 * n_swap) * args.steps
-        dom_bytes = (b["compress"] + n_swap * (b["add"] + b["remove"])) / (1 + 2 * n_swap)
-        dom_ms = acc_ms / n_acc
+        dom_bytes, dom_ms = b["compress"], ops["compress"]["ms_per_call"]
+        traffic = traffic_tbl.get("accumulate_kernel_compress_traffic_over_algorithmic")
+        traffic = traffic * dom_bytes if traffic and w.storage == wl.F32 else None
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak,
                 "peak_source": "%s copy bandwidth (MEASURED_PEAKS.json)" % peak_kind if peak_kind == "measured"
                                else "fallback copy bandwidth",
-                "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+                "traffic_source": "ncu dram bytes on the ViT-B/32-shaped case scaled by parameter count (profiles/)"
+                                  if traffic else "none valid for this build",
+                "share_of_step": shares[dom] / total_ms,
                 "per_kernel": {k: {"achieved": ops[k]["GBps"], "frac": ops[k]["GBps"] / peak, "bytes_per_launch": b[k]}
                                for k in ops}}
 

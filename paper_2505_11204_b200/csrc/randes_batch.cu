@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
 {
     constexpr int CPL = Store<ST>::CPL;
     constexpr int U = CPL == 4 ? 2 : 1;     // rows per trip
-    constexpr int TB = 2;                   // tasks whose loads are issued together
+    constexpr int TB = 4;                   // tasks whose loads are issued together
     __shared__ BatchScratch scratch[kWarpsPerCta];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     BatchScratch& ws = scratch[warp];

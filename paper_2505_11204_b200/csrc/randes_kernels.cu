@@ -159,46 +159,6 @@ constexpr int kNoBase = 0;        // the task tensors already hold deltas
 constexpr int kSharedBase = 1;    // no shuffle: every task subtracts the same W_0 tile, fetched once per row
 constexpr int kPerTaskBase = 2;   // shuffle: task i subtracts W_0[sigma_i(l)]; tiles repeat across slots and hit in L2
 
-constexpr uint32_t kSlotBytes = kThreadsPerCta * 16;   // one 16-byte slot of every thread of the CTA
-
-__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void prefetch_l2(const void* gmem) { asm volatile("prefetch.global.L2 [%0];" ::"l"(gmem)); }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ uint4 lds128(uint32_t saddr)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
-    return v;
-}
-__device__ __forceinline__ const char* lds_ptr(uint32_t saddr)
-{
-    unsigned long long v;
-    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(saddr));
-    return reinterpret_cast<const char*>(v);
-}
-__device__ __forceinline__ uint32_t lds_u16(uint32_t saddr)
-{
-    unsigned short v;
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(saddr));
-    return v;
-}
-__device__ __forceinline__ void sts128(uint32_t saddr, const uint4& v)
-{
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ void sts_u16(uint32_t saddr, uint32_t v)
-{
-    asm volatile("st.shared.u16 [%0], %1;" ::"r"(saddr), "h"(static_cast<unsigned short>(v)) : "memory");
-}
-__device__ __forceinline__ void sts_ptrs(uint32_t saddr, const void* a, const void* b)
-{
-    asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(saddr), "l"(a), "l"(b) : "memory");
-}
-
 // Shared memory of the accumulate kernel, per CTA:
 //   ring     kRingSlots slots x (256 threads x 16 B), cut into stages whose layout
 //            depends on how W_0 comes in (StageGeom)

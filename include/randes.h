@@ -207,6 +207,28 @@ int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_
                           void* const* out, void* stream);
 
 /*
+ * Interference diagnostics (Section 3, the equation for the norm of the
+ * interference; the paper's figures on pairwise cosine similarity among the
+ * interfering deltas during retrieval).  Computes, for the registered tasks in
+ * plan order, the Gram matrix of the transformed deltas
+ *     gram[i*n + j] = < T_i (W_i - W_0) , T_j (W_j - W_0) >     (fp64, n = number of tasks)
+ * summed over every parameter.  Because every T is orthogonal, the deltas that
+ * interfere when task t is retrieved, T_t^-1 T_j d_j (j != t), have exactly these
+ * inner products: cos(j, l) = gram[j][l] / sqrt(gram[j][j] gram[l][l]) and
+ * || lambda sum_{j != t} T_t^-1 T_j d_j || = lambda sqrt( sum_{j,l != t} gram[j][l] ).
+ *   base / tasks     as for randes_compress (base may be NULL: tasks hold deltas)
+ *   gram             DEVICE array of n*n doubles, written on `stream`
+ *   scratch          device memory of at least randes_delta_gram_scratch_bytes(plan) bytes
+ * Products are exact in fp64 and summed in a fixed order: the result is
+ * reproducible bit for bit.  At most 32 tasks.  ceil(n/4) passes over the
+ * weights, two kernel launches each.
+ * Errors: INVALID_ARGUMENT, CAPACITY, MISALIGNED, WORKSPACE_TOO_SMALL, CUDA_ERROR.
+ */
+size_t randes_delta_gram_scratch_bytes(const randes_plan_t* plan);
+int randes_delta_gram(randes_plan_t* plan, const void* const* base, const void* const* tasks,
+                      double* gram, void* scratch, size_t scratch_bytes, void* stream);
+
+/*
  * retrieve for callers that cannot provide a device workspace.  (The paper has
  * no counterpart: this entry point exists for deployment, not for the method.)
  *

@@ -429,6 +429,58 @@ int ro_retrieve(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
     return 0;
 }
 
+/*
+ * Gram matrix of the transformed deltas (Section 3: the interference norm is a
+ * function of the inner products of the deltas; Section 4: every O_i is
+ * orthogonal, so the deltas that interfere at retrieval have the inner products
+ * of the transformed deltas):
+ *   gram[i*n + j] = sum over slots l and elements (r,c) of x_i * x_j,
+ *   x_i = s_i(l,c) * (W_i[sigma_i(l)][r,c] - W_0[sigma_i(l)][r,c])   (the fp32 value compress sums)
+ * accumulated in double, element by element.
+ */
+int ro_delta_gram(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+                  const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
+                  int dtype, uint32_t n_tasks, const uint32_t *task_ids, const uint64_t *seeds,
+                  const void *const *base, const void *const *tasks, double *gram)
+{
+    ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
+    int rc = spec_check(&s);
+    if (rc) return rc;
+    uint32_t L = n_layers, n = n_tasks;
+    uint32_t *src = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)(L + 1) * (n + 1));
+    uint32_t *pos = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
+    float *x = (float *)malloc(sizeof(float) * (n + 1));
+    if (!src || !pos || !x) { free(src); free(pos); free(x); return -1; }
+    for (uint32_t i = 0; i < n; ++i)
+        if (ro_task_tables(L, group, n_groups, gflags, seeds[i], task_ids[i], src + (size_t)i * L, pos)) {
+            free(src); free(pos); free(x); return -1;
+        }
+    for (size_t e = 0; e < (size_t)n * n; ++e) gram[e] = 0.0;
+    for (uint32_t l = 0; l < L; ++l) {
+        uint32_t nr = rows[l], nc = cols[l];
+        int flip = ro_layer_flips(L, group, gflags, l);
+        int8_t *sg = (int8_t *)malloc((size_t)(nc ? nc : 1) * (n ? n : 1));
+        if (!sg) { free(src); free(pos); free(x); return -1; }
+        for (uint32_t i = 0; i < n; ++i) {
+            if (flip) ro_sign_row(seeds[i], task_ids[i], l, nc, sg + (size_t)i * nc);
+            else memset(sg + (size_t)i * nc, 1, nc);
+        }
+        for (uint32_t r = 0; r < nr; ++r)
+            for (uint32_t c = 0; c < nc; ++c) {
+                size_t idx = (size_t)r * nc + c;
+                for (uint32_t i = 0; i < n; ++i) {
+                    uint32_t sl = src[(size_t)i * L + l];
+                    x[i] = transformed_delta(tasks[(size_t)i * L + sl], base ? base[sl] : NULL, dtype, idx, sg[(size_t)i * nc + c]);
+                }
+                for (uint32_t i = 0; i < n; ++i)
+                    for (uint32_t j = 0; j < n; ++j) gram[(size_t)i * n + j] += (double)x[i] * (double)x[j];
+            }
+        free(sg);
+    }
+    free(src); free(pos); free(x);
+    return 0;
+}
+
 int ro_num_threads(void)
 {
 #ifdef _OPENMP

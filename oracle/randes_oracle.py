@@ -73,6 +73,7 @@ def _load():
         lib.ro_add_model.restype = ctypes.c_int
         lib.ro_remove_model.restype = ctypes.c_int
         lib.ro_retrieve.restype = ctypes.c_int
+        lib.ro_delta_gram.restype = ctypes.c_int
         lib.ro_num_threads.restype = ctypes.c_int
         lib.ro_set_num_threads.argtypes = [ctypes.c_int]
         _lib = lib
@@ -216,6 +217,30 @@ def compress(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
     if rc:
         raise ValueError("ro_compress failed: %d" % rc)
     return M
+
+
+def delta_gram(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
+               base: Optional[Sequence[np.ndarray]], tasks: Sequence[Sequence[np.ndarray]]) -> np.ndarray:
+    """gram[i, j] = <T_i d_i, T_j d_j> in float64 (Section 3; the interfering deltas' inner products)."""
+    lib = _load()
+    sargs, keep = _spec_args(spec)
+    K = len(task_ids)
+    if base is not None:
+        _check_layers(spec, base, dtype)
+    flat = []
+    for t in tasks:
+        _check_layers(spec, t, dtype)
+        flat.extend(t)
+    ids = _u32(task_ids)
+    sd = np.ascontiguousarray(np.asarray(seeds, dtype=np.uint64))
+    gram = np.zeros((K, K), dtype=np.float64)
+    p = ctypes.c_void_p
+    base_pa = _ptr_array(base) if base is not None else None
+    rc = lib.ro_delta_gram(*sargs, ctypes.c_int(dtype), ctypes.c_uint32(K), p(ids.ctypes.data), p(sd.ctypes.data),
+                           base_pa, _ptr_array(flat), p(gram.ctypes.data))
+    if rc:
+        raise ValueError("ro_delta_gram failed: %d" % rc)
+    return gram
 
 
 def _swap(fn_name, spec, dtype, task_id, seed, base, task, M, slots):

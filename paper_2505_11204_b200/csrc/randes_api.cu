@@ -174,6 +174,7 @@ struct randes_plan_s {
     int grid_acc[2] = {0, 0};   // [0] compress, [1] one task (add / remove)
     int grid_ret[2] = {0, 0};
     int grid_batch[2] = {0, 0};
+    int grid_gram = 0;
     // host mirrors of what the device pointer tables currently hold
     std::vector<const void*> h_base, h_out, h_tasks;
     std::vector<DevTask> h_dev_tasks;
@@ -468,6 +469,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         p->grid_acc[1] = p->sm_count * occ_acc1;
         p->grid_ret[0] = p->sm_count * occ_r0;
         p->grid_ret[1] = p->sm_count * occ_r1;
+        p->grid_gram = p->sm_count * std::max(1, gram_ctas_per_sm(p->storage));
         p->grid_batch[0] = p->sm_count * std::max(1, retrieve_batch_ctas_per_sm(p->storage, RANDES_F32));
         p->grid_batch[1] = p->sm_count * std::max(1, retrieve_batch_ctas_per_sm(p->storage, RANDES_BF16));
         e = cudaMemcpyAsync(p->ws + p->lay.layers, p->dev_layers.data(), n_layers * sizeof(DevLayer),
@@ -625,6 +627,57 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_
     const int e = launch_retrieve(plan->storage, out_dtype, a, grid, s);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the retrieve kernel");
     ++g_launches;
+    return RANDES_OK;
+}
+
+size_t randes_delta_gram_scratch_bytes(const randes_plan_t* plan)
+{
+    if (!plan || !plan->ws) return 0;
+    return static_cast<size_t>(plan->grid_gram) * kWarpsPerCta * kGramAnchors * kTaskChunk * sizeof(double);
+}
+
+int randes_delta_gram(randes_plan_t* plan, const void* const* base, const void* const* tasks, double* gram, void* scratch,
+                      size_t scratch_bytes, void* stream)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
+    const size_t n = plan->tasks.size();
+    if (n == 0) return fail(RANDES_INVALID_ARGUMENT, "no task is registered");
+    if (n > static_cast<size_t>(kTaskChunk)) return fail(RANDES_CAPACITY, "the Gram matrix is limited to %d tasks; the plan holds %zu", kTaskChunk, n);
+    if (!gram || reinterpret_cast<uintptr_t>(gram) % 8) return fail(RANDES_MISALIGNED, "gram = %p is NULL or not 8-byte aligned", (void*)gram);
+    if (!scratch || reinterpret_cast<uintptr_t>(scratch) % 8) return fail(RANDES_MISALIGNED, "scratch = %p is NULL or not 8-byte aligned", scratch);
+    if (scratch_bytes < randes_delta_gram_scratch_bytes(plan))
+        return fail(RANDES_WORKSPACE_TOO_SMALL, "scratch has %zu bytes, the Gram matrix needs %zu", scratch_bytes,
+                    randes_delta_gram_scratch_bytes(plan));
+    if (!tasks) return fail(RANDES_INVALID_ARGUMENT, "tasks is NULL");
+    int rc;
+    const size_t es = elem_size(plan->storage);
+    if ((rc = check_ptrs(*plan, base, "base", es, true))) return rc;
+    for (size_t i = 0; i < n; ++i)
+        if ((rc = check_ptrs(*plan, tasks + i * plan->n_layers, "tasks", es, false))) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (base && (rc = stage_ptrs(*plan, plan->h_base, plan->base_valid, plan->lay.base_ptrs, base, s))) return rc;
+    if ((rc = stage_task_ptrs(*plan, tasks, n, s))) return rc;
+    GramArgs a;
+    a.layers = plan->dev<DevLayer>(plan->lay.layers);
+    a.units = plan->dev<DevUnit>(plan->lay.units);
+    a.n_units = static_cast<uint32_t>(plan->units.size());
+    a.n_layers = plan->n_layers;
+    a.src_of_slot = plan->dev<uint32_t>(plan->lay.src_of_slot);
+    a.tasks = plan->dev<DevTask>(plan->lay.tasks);
+    a.n_tasks = static_cast<uint32_t>(n);
+    a.has_base = base != nullptr;
+    a.base = plan->dev<const void*>(plan->lay.base_ptrs);
+    a.task_ptrs = plan->dev<const void*>(plan->lay.task_ptrs);
+    a.partial = static_cast<double*>(scratch);
+    const int grid = std::max(1, std::min<int>(plan->grid_gram, static_cast<int>(a.n_units)));
+    for (uint32_t a0 = 0; a0 < n; a0 += kGramAnchors) {
+        a.a0 = a0;
+        a.na = std::min<uint32_t>(kGramAnchors, static_cast<uint32_t>(n) - a0);
+        const int e = launch_gram_pass(plan->storage, a, grid, gram, s);
+        if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the Gram kernels");
+        g_launches += 2;
+    }
     return RANDES_OK;
 }
 

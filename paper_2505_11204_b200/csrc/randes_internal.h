@@ -99,6 +99,23 @@ struct RetrieveBatchArgs {
     float lambda;
 };
 
+constexpr int kGramAnchors = 4;   // rows of the Gram matrix produced per pass
+
+struct GramArgs {
+    const DevLayer* layers;
+    const DevUnit* units;
+    uint32_t n_units;
+    uint32_t n_layers;
+    const uint32_t* src_of_slot;   // sigma rows of all registered tasks
+    const DevTask* tasks;
+    uint32_t n_tasks;              // <= kTaskChunk
+    uint32_t a0, na;               // this pass produces rows [a0, a0 + na), na <= kGramAnchors
+    uint32_t has_base;
+    const void* const* base;
+    const void* const* task_ptrs;  // [n_tasks][n_layers]
+    double* partial;               // [grid * kWarpsPerCta][kGramAnchors][kTaskChunk]
+};
+
 // Launchers (randes_kernels.cu).  Return a cudaError_t as int.
 int launch_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, int grid, void* stream);
 int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void* stream);
@@ -107,6 +124,9 @@ int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void
 // dynamic shared memory they need: call once per device before launching.
 int retrieve_ctas_per_sm(int storage_dtype, int out_dtype);
 int accumulate_ctas_per_sm(int storage_dtype, bool single_task);
+// randes_diag.cu: one pass = the Gram kernel plus the fixed-order reduction into gram[a0 .. a0+na)[*]
+int launch_gram_pass(int storage_dtype, const GramArgs& a, int grid, double* gram, void* stream);
+int gram_ctas_per_sm(int storage_dtype);
 // randes_batch.cu
 int launch_retrieve_batch(int storage_dtype, int out_dtype, const RetrieveBatchArgs& a, int grid, void* stream);
 int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype);

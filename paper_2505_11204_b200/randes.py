@@ -96,6 +96,10 @@ def lib():
         L.randes_remove_model.restype = ctypes.c_int
         L.randes_retrieve.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
         L.randes_retrieve.restype = ctypes.c_int
+        L.randes_delta_gram_scratch_bytes.argtypes = [vp]
+        L.randes_delta_gram_scratch_bytes.restype = sz
+        L.randes_delta_gram.argtypes = [vp, vp, vp, vp, vp, sz, vp]
+        L.randes_delta_gram.restype = ctypes.c_int
         L.randes_retrieve_batch.argtypes = [vp, vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
         L.randes_retrieve_batch.restype = ctypes.c_int
         L.randes_retrieve_static.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
@@ -112,7 +116,7 @@ EXPORTS = [
     "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
     "randes_task_tables", "randes_compress", "randes_add_model", "randes_remove_model",
-    "randes_retrieve", "randes_retrieve_batch", "randes_retrieve_static", "randes_launch_count", "randes_last_error",
+    "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_retrieve_batch", "randes_retrieve_static", "randes_launch_count", "randes_last_error",
 ]
 
 
@@ -186,6 +190,14 @@ def randes_retrieve(plan, task_id, lam, out_dtype, base, M, out, stream) -> None
     _check(lib().randes_retrieve(plan, task_id, lam, out_dtype, _addr(base), _addr(M), _addr(out), stream))
 
 
+def randes_delta_gram_scratch_bytes(plan) -> int:
+    return int(lib().randes_delta_gram_scratch_bytes(plan))
+
+
+def randes_delta_gram(plan, base, tasks, gram, scratch, scratch_bytes, stream) -> None:
+    _check(lib().randes_delta_gram(plan, _addr(base), _addr(tasks), _addr(gram), _addr(scratch), scratch_bytes, stream))
+
+
 def randes_retrieve_batch(plan, task_ids, lam, out_dtype, base, M, out, stream) -> None:
     """Several tasks in one pass; ``out`` holds n_tasks * n_layers pointers, task-major."""
     ids = (ctypes.c_uint32 * len(task_ids))(*[int(t) for t in task_ids])
@@ -220,6 +232,24 @@ def _as_ptrs(x):
     if x is None or isinstance(x, ctypes.Array):
         return x
     return ptr_array(x)
+
+
+def interference_norm(gram, t: int, lam: float) -> float:
+    """|| lam * sum_{j != t} T_t^-1 T_j d_j || from the Gram matrix (Section 3 of the paper)."""
+    import math
+
+    n = len(gram)
+    return lam * math.sqrt(max(0.0, sum(float(gram[j][l]) for j in range(n) for l in range(n) if j != t and l != t)))
+
+
+def mean_pairwise_cosine(gram, exclude=None) -> float:
+    """Average cosine over all pairs of distinct tasks, leaving `exclude` out (the retrieved task)."""
+    import math
+
+    n = len(gram)
+    idx = [i for i in range(n) if i != exclude]
+    pairs = [(i, j) for a, i in enumerate(idx) for j in idx[a + 1:]]
+    return sum(float(gram[i][j]) / math.sqrt(float(gram[i][i]) * float(gram[j][j])) for i, j in pairs) / max(len(pairs), 1)
 
 
 # ---- convenience object over torch tensors --------------------------------------------------
@@ -338,6 +368,17 @@ class Plan:
     def remove_model(self, task_id: int, base, task, M):
         randes_remove_model(self.handle, task_id, _as_ptrs(base), _as_ptrs(task), M, self._stream())
         return M
+
+    def delta_gram(self, base, tasks):
+        """Gram matrix of the transformed deltas as an [n, n] float64 CUDA tensor (see include/randes.h)."""
+        import torch
+
+        n = self.n_tasks
+        gram = torch.empty(n, n, dtype=torch.float64, device=self.device)
+        nbytes = randes_delta_gram_scratch_bytes(self.handle)
+        scratch = torch.empty(nbytes // 8, dtype=torch.float64, device=self.device)
+        randes_delta_gram(self.handle, _as_ptrs(base), _as_ptrs(tasks), gram, scratch, nbytes, self._stream())
+        return gram
 
     def retrieve_batch(self, task_ids, lam: float, base, M, out=None, out_dtype: int = F32):
         """Rebuild several tasks in one launch; returns a list (per task) of lists of tensors."""

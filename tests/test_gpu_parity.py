@@ -228,6 +228,40 @@ def test_batched_retrieve_equals_single_retrieves(storage):
     plan.close()
 
 
+@pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
+def test_delta_gram_matches_oracle(storage):
+    """Gram matrix of the transformed deltas (interference diagnostics).  Products are exact in fp64 on both
+    sides; only the order of the fp64 additions differs, so |dG_ij| <= N * 2^-53 * sum|x_i x_j|
+    <= N * 2^-53 * sqrt(G_ii G_jj) with N the number of parameters."""
+    import torch
+
+    w = make_workload(RAGGED, storage=storage, n_tasks=6)
+    base, tasks = wl.model_set(w)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w)
+    N = w.n_params
+    for use_base in (True, False):
+        G = plan.delta_gram(d_base if use_base else None, d_tasks).cpu().numpy()
+        ref = ro.delta_gram(w.spec, storage, w.task_ids, w.seeds, base if use_base else None, tasks)
+        scale = np.sqrt(np.outer(np.diag(ref), np.diag(ref)))
+        assert np.all(np.abs(G - ref) <= N * 2.0 ** -53 * scale), np.max(np.abs(G - ref) / scale)
+        G2 = plan.delta_gram(d_base if use_base else None, d_tasks).cpu().numpy()
+        assert np.array_equal(G, G2)                      # fixed summation order: reproducible bit for bit
+    # helpers on top of the matrix
+    M_ref = ro.compress(w.spec, storage, w.task_ids, w.seeds, base, tasks)
+    G = plan.delta_gram(d_base, d_tasks).cpu().numpy()
+    m2 = sum(float((m.astype(np.float64) ** 2).sum()) for m in M_ref)
+    assert abs(G.sum() - m2) <= 1e-5 * m2                  # ||M||^2 = sum_ij G_ij up to M's fp32 rounding
+    t = 2
+    out = ro.retrieve(w.spec, storage, wl.F32, t, w.seeds[t], 1.0, base, M_ref)
+    f32 = (lambda a: wl.bf16_bits_to_f32(a) if a.dtype == np.uint16 else a)
+    inter = np.concatenate([(o.astype(np.float64) - f32(b).astype(np.float64) - (f32(x).astype(np.float64) - f32(b).astype(np.float64))).ravel()
+                            for o, b, x in zip(out, base, tasks[t])])
+    assert abs(randes.interference_norm(G, t, 1.0) - float(np.sqrt(inter @ inter))) <= 1e-3 * float(np.sqrt(inter @ inter))
+    assert abs(randes.mean_pairwise_cosine(G)) < 0.2       # decorrelated (raw cosine of this recipe: 0.25)
+    plan.close()
+
+
 def test_gpu_argument_validation():
     import torch
 

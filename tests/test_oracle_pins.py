@@ -532,6 +532,38 @@ def test_shuffle_aligns_shared_component_only_when_slots_coincide():
         assert abs(got - want) < 1e-9
 
 
+def test_gram_of_transformed_deltas_matches_dense_matrices_and_the_interference_norm():
+    """Section 3: || lambda sum_{j != i} Delta_j ||^2 = lambda^2 sum_{j,l != i} <Delta_j, Delta_l>; under
+    RanDeS the interfering deltas are O_i^-1 O_j Delta_j, whose inner products are those of O_j Delta_j."""
+    spec = tiny_spec(SHUFFLE | FLIP)
+    rng = np.random.default_rng(33)
+    ids, seeds = [0, 1, 2, 3], [42, 43, 44, 45]
+    base = rand_model(spec, rng, dyadic=True)
+    tasks = [rand_model(spec, rng, dyadic=True) for _ in ids]
+    Ts = [dense_transform(spec, s, t)[0] for t, s in zip(ids, seeds)]
+    X = [T @ (flat(t) - flat(base)) for T, t in zip(Ts, tasks)]
+    want = np.array([[float(a @ b) for b in X] for a in X])
+    G = ro.delta_gram(spec, ro.F32, ids, seeds, base, tasks)
+    assert np.array_equal(G, want)              # dyadic inputs: every product and sum is exact in double
+    assert np.array_equal(G, G.T)
+    # the diagonal is the squared norm of the untouched delta (orthogonality)
+    for i, t in enumerate(tasks):
+        assert G[i, i] == float((flat(t) - flat(base)) @ (flat(t) - flat(base)))
+    # interference norm at retrieval, against the retrieved model itself
+    lam = 0.5
+    M = ro.compress(spec, ro.F32, ids, seeds, base, tasks)
+    for t in range(len(ids)):
+        what = ro.retrieve(spec, ro.F32, ro.F32, ids[t], seeds[t], lam, base, M)
+        interference = flat(what) - flat(base) - lam * (flat(tasks[t]) - flat(base))
+        others = [j for j in range(len(ids)) if j != t]
+        assert float(interference @ interference) == lam * lam * sum(G[j, l] for j in others for l in others)
+    # the same without transforms is the plain Gram matrix of the deltas
+    G0 = ro.delta_gram(tiny_spec(0), ro.F32, ids, seeds, base, tasks)
+    D = [flat(t) - flat(base) for t in tasks]
+    assert np.array_equal(G0, np.array([[float(a @ b) for b in D] for a in D]))
+    assert np.array_equal(np.diag(G0), np.diag(G))
+
+
 # --------------------------------------------------------------------------- bf16 storage
 def test_bf16_storage_and_output():
     rng = np.random.default_rng(23)

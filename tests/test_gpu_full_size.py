@@ -111,6 +111,25 @@ def run_full_size(storage, n_swap):
                 assert_bits_equal(from_dev(outs[b][p]), ref[p], "batched retrieve task %d layer %d" % (t, p))
         del outs
         torch.cuda.empty_cache()
+    if storage == wl.F32:
+        # Gram matrix of the transformed deltas at full size, checked through what holds at any size:
+        # orthogonality keeps every delta's norm, sum_ij G_ij = ||M||^2, and the transforms remove the
+        # cosine of 0.25 that the input recipe puts between any two deltas.
+        task_ptrs = randes.ptr_array([d_tasks[t] for t in ids])
+        G = plan.delta_gram(p_base, task_ptrs).cpu().numpy()
+        for i in (0, 7, 19):
+            n2 = sum(float(((a.double() - b.double()) ** 2).sum()) for a, b in zip(d_tasks[ids[i]], d_base))
+            assert abs(G[i, i] - n2) <= 1e-9 * n2
+        m2 = sum(float((plan.slot(M, l).double() ** 2).sum()) for l in range(L))
+        assert abs(G.sum() - m2) <= 1e-5 * m2
+        assert abs(randes.mean_pairwise_cosine(G)) < 2e-3
+        w0 = wl.Workload(**{**w.__dict__})
+        w0.gflags = [0] * len(w.gflags)
+        plain = randes.Plan.from_workload(w0)
+        G0 = plain.delta_gram(p_base, task_ptrs).cpu().numpy()
+        assert abs(randes.mean_pairwise_cosine(G0) - 0.25) < 5e-3
+        assert np.allclose(np.diag(G0), np.diag(G), rtol=1e-12)
+        plain.close()
     for t, s in zip(swap_ids, swap_seeds):
         randes.randes_add_model(plan.handle, t, s, p_base, randes.ptr_array(d_tasks[t]), M, sh)
         ro.add_model(w.spec, storage, t, s, base_h, tasks_h[t], M_ref, slots=slots)

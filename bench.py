@@ -43,7 +43,7 @@ def parse_args(argv=None):
     ap.add_argument("--swap", type=int, default=5, help="models streamed in and out per step")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=3)
     return ap.parse_args(argv)
 
 
@@ -280,27 +280,45 @@ def run_ours(args):
     swap_seeds = [w.seeds[0] + K + j for j in range(n_swap)]
     want_e2e = not args.no_e2e
 
-    # ---- inputs: generated on the host (seeded); pinned when the end-to-end leg needs them again
-    def host_tensor(a):
-        t = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
-        return t.pin_memory() if want_e2e else t
+    # ---- inputs: generated on the host (seeded), one flat arena per model (pinned when the
+    #      end-to-end leg needs it again), copied to a flat device arena; layers are views
+    tdt = torch.bfloat16 if w.storage == wl.BF16 else torch.float32
+    offs, total_el = [], 0
+    for r, c in zip(w.rows, w.cols):
+        offs.append(total_el)
+        total_el += (r * c + 63) // 64 * 64           # 256-byte aligned layer starts
+
+    def views(flat):
+        return [flat[o:o + r * c].view(r, c) for o, r, c in zip(offs, w.rows, w.cols)]
+
+    def host_arena(arrs):
+        flat = torch.zeros(total_el, dtype=tdt, pin_memory=want_e2e)
+        for v, a in zip(views(flat), arrs):
+            v.copy_(torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a))
+        return flat
 
     base_np, models_np = wl.model_set(w, ids, threads=os.cpu_count() or 1)
-    h_base = [host_tensor(a) for a in base_np]
-    h_models = [[host_tensor(a) for a in m] for m in models_np]
+    h_flat = [host_arena(base_np)] + [host_arena(m) for m in models_np]     # [0] = W_0, [1 + i] = model i
     del base_np, models_np
-    d_base = [t.to(dev, non_blocking=True) for t in h_base]
-    d_models = [[t.to(dev, non_blocking=True) for t in m] for m in h_models]
+
+    def device_set():
+        flats = [torch.empty(total_el, dtype=tdt, device=dev) for _ in h_flat]
+        vs = [views(f) for f in flats]
+        return {"flat": flats, "base": vs[0], "models": vs[1:], "p_base": randes.ptr_array(vs[0]),
+                "p_tasks": randes.ptr_array(vs[1:1 + K]), "p_swap": [randes.ptr_array(m) for m in vs[1 + K:]]}
+
+    dset = device_set()
+    for dst, src in zip(dset["flat"], h_flat):
+        dst.copy_(src, non_blocking=True)
     torch.cuda.synchronize()
+    d_base, d_models = dset["base"], dset["models"]
     if not want_e2e:
-        del h_base, h_models
+        del h_flat
 
     plan = randes.Plan.from_workload(w, max_tasks=K + n_swap, device=dev)
     M = plan.new_superposition()
     out = plan.new_output(wl.F32)
-    p_base = randes.ptr_array(d_base)
-    p_tasks = randes.ptr_array(d_models[:K])
-    p_swap = [randes.ptr_array(m) for m in d_models[K:]]
+    p_base, p_tasks, p_swap = dset["p_base"], dset["p_tasks"], dset["p_swap"]
     p_out = randes.ptr_array(out)
     stream = torch.cuda.current_stream(dev)
     sh = stream.cuda_stream
@@ -434,48 +452,81 @@ def run_ours(args):
         except torch.OutOfMemoryError:
             extras["retrieve_batch"] = None
 
-    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region.
+    #      Every step copies all its inputs from pinned host memory and all its results back.
+    #      Copies and kernels are pipelined: the next step's inputs arrive in a second set of
+    #      device buffers while this step computes, and retrieved models leave through two
+    #      alternating output buffers.
     e2e = None
     if want_e2e:
-        h_out = [torch.empty_like(o, device="cpu").pin_memory() for o in out]
+        del out, p_out
+        sets = [dset, device_set()]
+        out_el = sum((r * c + 63) // 64 * 64 for r, c in zip(w.rows, w.cols))
+        o_flat = [torch.empty(out_el, dtype=torch.float32, device=dev) for _ in range(2)]
+        o_ptrs = [randes.ptr_array(views(f)) for f in o_flat]
+        h_out = [torch.empty(out_el, dtype=torch.float32, pin_memory=True) for _ in range(2)]
         h_M = torch.empty_like(M, device="cpu").pin_memory()
+        s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        ev = lambda: torch.cuda.Event()
+        ev_in, ev_set_free = [ev(), ev()], [ev(), ev()]
+        ev_ret, ev_out_free, ev_m_free = [ev(), ev()], [ev(), ev()], ev()
+        for e_ in ev_set_free + ev_out_free + [ev_m_free]:
+            e_.record(stream)
 
-        def e2e_step():
-            for dst, src in zip(d_base, h_base):
-                dst.copy_(src, non_blocking=True)
-            for dm, hm in zip(d_models, h_models):
-                for dst, src in zip(dm, hm):
+        def e2e_step(i):
+            k = i % 2
+            ds = sets[k]
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_set_free[k])
+                for dst, src in zip(ds["flat"], h_flat):
                     dst.copy_(src, non_blocking=True)
-            randes.randes_compress(plan.handle, p_base, p_tasks, M, sh)
-            for ti in w.task_ids:
-                randes.randes_retrieve(plan.handle, ti, w.lam, wl.F32, p_base, M, p_out, sh)
-                for dst, src in zip(h_out, out):
-                    dst.copy_(src, non_blocking=True)
+                ev_in[k].record(s_in)
+            stream.wait_event(ev_in[k])
+            stream.wait_event(ev_m_free)
+            randes.randes_compress(plan.handle, ds["p_base"], ds["p_tasks"], M, sh)
+            for n_t, ti in enumerate(w.task_ids):
+                bfr = n_t % 2
+                stream.wait_event(ev_out_free[bfr])
+                randes.randes_retrieve(plan.handle, ti, w.lam, wl.F32, ds["p_base"], M, o_ptrs[bfr], sh)
+                ev_ret[bfr].record(stream)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_ret[bfr])
+                    h_out[bfr].copy_(o_flat[bfr], non_blocking=True)
+                    ev_out_free[bfr].record(s_out)
             for j in range(n_swap):
-                randes.randes_add_model(plan.handle, K + j, swap_seeds[j], p_base, p_swap[j], M, sh)
+                randes.randes_add_model(plan.handle, K + j, swap_seeds[j], ds["p_base"], ds["p_swap"][j], M, sh)
             for j in range(n_swap):
-                randes.randes_remove_model(plan.handle, K + j, p_base, p_swap[j], M, sh)
-            h_M.copy_(M, non_blocking=True)
+                randes.randes_remove_model(plan.handle, K + j, ds["p_base"], ds["p_swap"][j], M, sh)
+            ev_set_free[k].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_set_free[k])
+                h_M.copy_(M, non_blocking=True)
+                ev_m_free.record(s_out)
 
-        e2e_step()
+        e2e_step(0)
+        stream.wait_stream(s_out)
         barrier()
         a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
-        for _ in range(args.e2e_steps):
-            e2e_step()
+        s_in.wait_event(a)
+        for i in range(args.e2e_steps):
+            e2e_step(i + 1)
+        stream.wait_stream(s_out)
+        stream.wait_stream(s_in)
         z.record(stream)
         barrier()
         e2e_ms = max_over_ranks([a.elapsed_time(z)], world, dev)[0] / args.e2e_steps
-        s = 2 if w.storage == wl.BF16 else 4
+        s_b = 2 if w.storage == wl.BF16 else 4
         e2e = {"value": aggregate_value(total_bytes, e2e_ms, world), "unit": "GB/s", "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": (1 + K + n_swap) * w.n_params * s,
-               "d2h_bytes_per_step": (K + 1) * w.n_params * 4, "steps": args.e2e_steps}
-        del h_out, h_M, h_base, h_models
+               "h2d_bytes_per_step": (1 + K + n_swap) * w.n_params * s_b,
+               "d2h_bytes_per_step": (K + 1) * w.n_params * 4, "steps": args.e2e_steps,
+               "note": "copies and kernels pipelined over three streams; PCIe-bound"}
+        del h_out, h_M, h_flat, sets, o_flat
 
     plan.close()
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        del d_models, d_base, M, out
+        del d_models, d_base, M, dset
         torch.cuda.empty_cache()
         cpu = time_oracle(w, n_swap, 5, 1)
         cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}

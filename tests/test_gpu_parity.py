@@ -262,6 +262,86 @@ def test_delta_gram_matches_oracle(storage):
     plan.close()
 
 
+def test_empty_layers_and_degenerate_plans():
+    import torch
+
+    # a model with empty tensors (zero rows or zero columns) among ordinary ones
+    w = wl.Workload(name="empties", layer_names=list("abcde"), rows=[4, 0, 3, 5, 0], cols=[128, 64, 0, 20, 0], group=[0, 1, 2, 3, 4],
+                    gflags=[F, F, F, F, F], storage=wl.F32, n_tasks=2, task_ids=[0, 1], seeds=[5, 6], scale=1e-3,
+                    lam=0.5, data_seed=3)
+    base, tasks = wl.model_set(w)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w)
+    M = plan.compress(d_base, d_tasks)
+    M_ref = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, base, tasks)
+    check_superposition(plan, M, M_ref, "compress with empty layers")
+    out = plan.retrieve(1, w.lam, d_base, M)
+    check_model(out, ro.retrieve(w.spec, w.storage, wl.F32, 1, 6, w.lam, base, M_ref), "retrieve with empty layers")
+    plan.close()
+    # nothing but empty layers: every call succeeds and launches nothing
+    w0 = wl.Workload(name="nothing", layer_names=["x", "y"], rows=[0, 7], cols=[9, 0], group=[0, 1], gflags=[F, F],
+                     storage=wl.F32, n_tasks=1, task_ids=[0], seeds=[1], scale=1e-3, lam=1.0, data_seed=3)
+    base, tasks = wl.model_set(w0)
+    plan = randes.Plan.from_workload(w0)
+    before = randes.randes_launch_count()
+    M = torch.zeros(64, dtype=torch.float32, device="cuda")
+    plan.compress(model_to_dev(base), [model_to_dev(tasks[0])], M)
+    plan.retrieve(0, 1.0, model_to_dev(base), M, out=plan.new_output())
+    assert randes.randes_launch_count() == before
+    plan.close()
+
+
+def test_lambda_zero_and_bf16_ties():
+    import torch
+
+    # lambda = 0 gives back W_0 bit for bit; lambda = 1 on W_0 = 0 exposes +-M, whose values sit on
+    # bf16 rounding ties, just above and just below them
+    w = make_workload([(8, 128, 1)], flags=F, n_tasks=1)
+    base, tasks = wl.model_set(w)
+    plan = randes.Plan.from_workload(w)
+    d_base = model_to_dev(base)
+    M = plan.compress(d_base, [model_to_dev(tasks[0])])
+    out = plan.retrieve(0, 0.0, d_base, M)
+    assert_bits_equal(from_dev(out[0]), base[0], "lambda = 0")
+    rng = np.random.default_rng(4)
+    hi = rng.integers(0x3C00, 0x4400, size=(8, 128)).astype(np.uint32) << 16
+    lo = rng.choice(np.array([0x8000, 0x7FFF, 0x8001, 0x0000, 0xFFFF], dtype=np.uint32), size=(8, 128))
+    m_vals = (hi | lo).view(np.float32)
+    M_dev = plan.new_superposition().zero_()
+    plan.slot(M_dev, 0).copy_(to_dev(m_vals))
+    zero = [torch.zeros(8, 128, device="cuda")]
+    out = plan.retrieve(0, 1.0, zero, M_dev, out_dtype=wl.BF16)
+    ref = ro.retrieve(w.spec, wl.F32, wl.BF16, 0, w.seeds[0], 1.0, [np.zeros((8, 128), np.float32)], [m_vals])
+    assert_bits_equal(from_dev(out[0]), ref[0], "bf16 ties")
+    plan.close()
+
+
+def test_thirty_two_tasks_exactly_and_wide_single_row():
+    run_full_cycle(make_workload([(1, 100000, 1), (3, 4096, 2)], n_tasks=32), out_dtypes=(wl.F32,), extra_task=False)
+
+
+def test_random_plans():
+    """Seeded random models: shapes, group sizes, flags (shuffle / shift / flip / skip), task counts, ids,
+    seeds and storage types drawn at random; every step of the path against the oracle."""
+    rng = np.random.default_rng(2024)
+    SH, SK = randes.SHIFT, randes.SKIP
+    for case in range(12):
+        n_groups = int(rng.integers(1, 6))
+        shapes, flags = [], []
+        for _ in range(n_groups):
+            rows = int(rng.choice([1, 1, 2, 7, 16, 17, 40, 130]))
+            cols = int(rng.choice([1, 4, 8, 12, 100, 128, 132, 256, 384, 520, 1024, 1032]))
+            shapes.append((rows, cols, int(rng.integers(1, 7))))
+            f = int(rng.choice([0, S, SH])) | (F if rng.random() < 0.7 else 0)
+            if rng.random() < 0.3:
+                f |= SK(int(rng.integers(2, 4)))
+            flags.append(f)
+        w = make_workload(shapes, flags=flags, storage=int(rng.integers(0, 2)), n_tasks=int(rng.integers(1, 7)),
+                          seed0=int(rng.integers(0, 2**62)), data_seed=100 + case, interleave=bool(rng.integers(0, 2)))
+        w.task_ids = [int(x) for x in rng.choice(1000, size=w.n_tasks, replace=False)]
+        run_full_cycle(w, out_dtypes=(int(rng.integers(0, 2)),), lam=float(rng.choice([0.1, 0.3, 1.0, 2.0])))
+
+
 def test_gpu_argument_validation():
     import torch
 

@@ -29,9 +29,13 @@
  *   caller.  The library allocates no device memory and frees nothing it is
  *   handed.  Weight tensors must be aligned to their element size; 16-byte
  *   aligned tensors with cols % 4 == 0 take the vectorised path.
- * - M is one fp32 arena of randes_superposition_bytes() bytes, 256-byte
- *   aligned; slot l starts at byte randes_layer_offset(plan, l).  M is fp32
- *   whatever the storage type of the weights.
+ * - M is one arena of randes_superposition_bytes() bytes, 256-byte aligned;
+ *   slot l starts at byte randes_layer_offset(plan, l).  Its element type is
+ *   the plan's m_dtype: fp32 by default whatever the storage type of the
+ *   weights, or bf16 (half the footprint; the "further compression" the
+ *   paper's conclusion leaves open).  Sums always run in fp32: with a bf16 M,
+ *   compress rounds each element once at the end (nearest even), add / remove
+ *   widen the stored element, add in fp32 and round again, retrieve widens.
  * - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *   Calls enqueue work and return; results are ordered on `stream`.  All calls
  *   on one plan must be issued on one stream or otherwise ordered by the
@@ -103,6 +107,7 @@ size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_laye
  *
  *   layers[n_layers], groups[n_groups]  host arrays, copied.
  *   storage_dtype   element type of every W_0 / W_i tensor.
+ *   m_dtype         element type of the superposition arena M (RANDES_F32 or RANDES_BF16).
  *   task_ids/seeds[n_tasks]  the initially registered models, in the order in
  *                   which compress sums them.  Ids must be distinct.
  *   max_tasks       capacity of the registry (>= n_tasks, >= 1).
@@ -120,7 +125,7 @@ size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_laye
  */
 int randes_plan(const randes_layer_t* layers, uint32_t n_layers,
                 const randes_group_t* groups, uint32_t n_groups,
-                randes_dtype_t storage_dtype,
+                randes_dtype_t storage_dtype, randes_dtype_t m_dtype,
                 const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
                 uint32_t max_tasks,
                 void* dev_workspace, size_t dev_workspace_bytes, void* stream,
@@ -128,7 +133,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers,
 
 void randes_plan_destroy(randes_plan_t* plan); /* NULL is allowed; frees host memory only */
 
-/* Size of the fp32 arena M: sum of 4*rows*cols, each slot padded to 256 bytes.
+/* Size of the arena M: sum of rows*cols elements of m_dtype, each slot padded to 256 bytes.
  * Independent of the number of tasks (Section 4.1: a seed per added model). */
 size_t randes_superposition_bytes(const randes_plan_t* plan);
 
@@ -160,7 +165,9 @@ int randes_task_tables(const randes_plan_t* plan, uint32_t task_id,
  *                              themselves (adapter deltas, Section 5.8).
  *   tasks[n_tasks * n_layers]  tasks[i*n_layers + l] = layer l of the i-th
  *                              registered task.
- * One kernel launch.  Errors: INVALID_ARGUMENT, MISALIGNED, CUDA_ERROR.
+ * With a bf16 superposition at most 32 tasks can be summed in one call
+ * (CAPACITY otherwise): further models are added with randes_add_model.
+ * One kernel launch.  Errors: INVALID_ARGUMENT, MISALIGNED, CAPACITY, CUDA_ERROR.
  */
 int randes_compress(randes_plan_t* plan, const void* const* base, const void* const* tasks,
                     void* M, void* stream);

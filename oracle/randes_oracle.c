@@ -22,8 +22,12 @@
  *   - T_i = D_i o P_i: the layers of a delta are shuffled first, the sign flip
  *     is indexed by the position ("slot") the layer lands on in M.
  *   - Shuffle is the gather the paper prints: slot k receives member sigma(k).
- *   - lambda is applied at retrieval; M is kept in fp32 whatever the storage
- *     type of the weights.
+ *   - lambda is applied at retrieval; M is kept in fp32 by default, whatever the
+ *     storage type of the weights.  With m_dtype = bf16 (the "further
+ *     compression of the superposed delta" the conclusion leaves to future work)
+ *     compress sums in fp32 and rounds each element once at the end; add and
+ *     remove widen the stored element, add in fp32 and round again; retrieve
+ *     widens it.
  *   - "Column" is the second (contiguous) index of a row-major [rows, cols]
  *     array; a 1-D parameter is [1, cols].
  *   - Random numbers: Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11),
@@ -273,10 +277,18 @@ static int spec_check(const ro_spec_t *s)
  * remove (sign_op=-1).  slot_mask (may be NULL) limits the work to chosen
  * slots so that large cases can be spot-checked.
  */
-static int accumulate_one(const ro_spec_t *s, int dtype, int sign_op,
+static float load_m(const void *m, int m_dtype, size_t i) { return load_elem(m, m_dtype, i); }
+
+static void store_m(void *m, int m_dtype, size_t i, float v)
+{
+    if (m_dtype == RO_BF16) ((uint16_t *)m)[i] = ro_f32_to_bf16(v);
+    else ((float *)m)[i] = v;
+}
+
+static int accumulate_one(const ro_spec_t *s, int dtype, int m_dtype, int sign_op,
                           uint32_t task_id, uint64_t seed,
                           const void *const *base, const void *const *task,
-                          float *const *M, const uint8_t *slot_mask)
+                          void *const *M, const uint8_t *slot_mask)
 {
     uint32_t L = s->n_layers;
     uint32_t *src_of_slot = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
@@ -297,13 +309,15 @@ static int accumulate_one(const ro_spec_t *s, int dtype, int sign_op,
         else memset(sg, 1, cols);
         const void *wt = task[src];
         const void *wb = base ? base[src] : NULL;
-        float *m = M[l];
+        void *m = M[l];
 #pragma omp parallel for schedule(static)
         for (int64_t r = 0; r < (int64_t)rows; ++r) {
             for (uint32_t c = 0; c < cols; ++c) {
                 size_t idx = (size_t)r * cols + c;
                 float x = transformed_delta(wt, wb, dtype, idx, sg[c]);
-                m[idx] = sign_op < 0 ? m[idx] - x : m[idx] + x; /* one rounding */
+                float old = load_m(m, m_dtype, idx);
+                float sum = sign_op < 0 ? old - x : old + x; /* one fp32 rounding */
+                store_m(m, m_dtype, idx, sum);               /* and one more if M is bf16 */
             }
         }
         free(sg);
@@ -329,49 +343,66 @@ static ro_spec_t make_spec(uint32_t n_layers, const uint32_t *rows, const uint32
  */
 int ro_compress(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
                 const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
-                int dtype, uint32_t n_tasks, const uint32_t *task_ids, const uint64_t *seeds,
+                int dtype, int m_dtype, uint32_t n_tasks, const uint32_t *task_ids, const uint64_t *seeds,
                 const void *const *base, const void *const *tasks,
-                float *const *M, const uint8_t *slot_mask)
+                void *const *M, const uint8_t *slot_mask)
 {
     ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
     int rc = spec_check(&s);
     if (rc) return rc;
+    /* the sum always runs in fp32; a bf16 M receives it rounded once, at the end */
+    void **acc = (void **)calloc(n_layers ? n_layers : 1, sizeof(void *));
+    if (!acc) return -1;
     for (uint32_t l = 0; l < n_layers; ++l) {
         if (slot_mask && !slot_mask[l]) continue;
         size_t n = (size_t)rows[l] * cols[l];
-        for (size_t e = 0; e < n; ++e) M[l][e] = 0.0f;
+        if (m_dtype == RO_F32) {
+            acc[l] = M[l];
+        } else {
+            acc[l] = malloc(sizeof(float) * (n ? n : 1));
+            if (!acc[l]) { rc = -1; goto done; }
+        }
+        for (size_t e = 0; e < n; ++e) ((float *)acc[l])[e] = 0.0f;
     }
-    for (uint32_t i = 0; i < n_tasks; ++i) {
-        rc = accumulate_one(&s, dtype, +1, task_ids[i], seeds[i], base,
-                            tasks + (size_t)i * n_layers, M, slot_mask);
-        if (rc) return rc;
-    }
-    return 0;
+    for (uint32_t i = 0; i < n_tasks && !rc; ++i)
+        rc = accumulate_one(&s, dtype, RO_F32, +1, task_ids[i], seeds[i], base,
+                            tasks + (size_t)i * n_layers, acc, slot_mask);
+    if (!rc && m_dtype != RO_F32)
+        for (uint32_t l = 0; l < n_layers; ++l) {
+            if (slot_mask && !slot_mask[l]) continue;
+            size_t n = (size_t)rows[l] * cols[l];
+            for (size_t e = 0; e < n; ++e) store_m(M[l], m_dtype, e, ((float *)acc[l])[e]);
+        }
+done:
+    if (m_dtype != RO_F32)
+        for (uint32_t l = 0; l < n_layers; ++l) free(acc[l]);
+    free(acc);
+    return rc;
 }
 
 /* Model hot swapping (Section 5.7): M <- M + T_j(d_j)  /  M <- M - T_j(d_j). */
 int ro_add_model(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
                  const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
-                 int dtype, uint32_t task_id, uint64_t seed,
+                 int dtype, int m_dtype, uint32_t task_id, uint64_t seed,
                  const void *const *base, const void *const *task,
-                 float *const *M, const uint8_t *slot_mask)
+                 void *const *M, const uint8_t *slot_mask)
 {
     ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
     int rc = spec_check(&s);
     if (rc) return rc;
-    return accumulate_one(&s, dtype, +1, task_id, seed, base, task, M, slot_mask);
+    return accumulate_one(&s, dtype, m_dtype, +1, task_id, seed, base, task, M, slot_mask);
 }
 
 int ro_remove_model(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
                     const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
-                    int dtype, uint32_t task_id, uint64_t seed,
+                    int dtype, int m_dtype, uint32_t task_id, uint64_t seed,
                     const void *const *base, const void *const *task,
-                    float *const *M, const uint8_t *slot_mask)
+                    void *const *M, const uint8_t *slot_mask)
 {
     ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
     int rc = spec_check(&s);
     if (rc) return rc;
-    return accumulate_one(&s, dtype, -1, task_id, seed, base, task, M, slot_mask);
+    return accumulate_one(&s, dtype, m_dtype, -1, task_id, seed, base, task, M, slot_mask);
 }
 
 /*
@@ -385,8 +416,8 @@ int ro_remove_model(uint32_t n_layers, const uint32_t *rows, const uint32_t *col
  */
 int ro_retrieve(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
                 const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
-                int dtype, int out_dtype, uint32_t task_id, uint64_t seed, float lambda,
-                const void *const *base, const float *const *M,
+                int dtype, int m_dtype, int out_dtype, uint32_t task_id, uint64_t seed, float lambda,
+                const void *const *base, const void *const *M,
                 void *const *out, const uint8_t *pos_mask)
 {
     ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
@@ -408,14 +439,14 @@ int ro_retrieve(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
         if (!sg) { free(src_of_slot); free(slot_of_pos); return -1; }
         if (flip) ro_sign_row(seed, task_id, l, nc, sg);
         else memset(sg, 1, nc);
-        const float *m = M[l];
+        const void *m = M[l];
         const void *wb = base[p];
         void *o = out[p];
 #pragma omp parallel for schedule(static)
         for (int64_t r = 0; r < (int64_t)nr; ++r) {
             for (uint32_t c = 0; c < nc; ++c) {
                 size_t idx = (size_t)r * nc + c;
-                float mv = m[idx];
+                float mv = load_m(m, m_dtype, idx);
                 float signed_m = sg[c] < 0 ? -mv : mv;
                 float y = fmaf(lambda, signed_m, load_elem(wb, dtype, idx));
                 if (out_dtype == RO_BF16) ((uint16_t *)o)[idx] = ro_f32_to_bf16(y);

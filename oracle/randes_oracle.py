@@ -183,17 +183,19 @@ def task_tables(spec, seed: int, task_id: int) -> Tuple[np.ndarray, np.ndarray]:
     return src[:L], pos[:L]
 
 
-def new_superposition(spec, slots=None) -> List[np.ndarray]:
-    """One zeroed fp32 array per slot; with ``slots`` given, only those are allocated."""
+def new_superposition(spec, slots=None, m_dtype: int = F32) -> List[np.ndarray]:
+    """One zeroed array per slot (fp32, or uint16 bf16 bits); with ``slots`` given, only those are allocated."""
     keep = None if slots is None else set(int(x) for x in slots)
-    return [np.zeros((int(r), int(c)), dtype=np.float32) if keep is None or l in keep else None
+    mdt = np.uint16 if m_dtype == BF16 else np.float32
+    return [np.zeros((int(r), int(c)), dtype=mdt) if keep is None or l in keep else None
             for l, (r, c) in enumerate(zip(spec[0], spec[1]))]
 
 
 def compress(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
              base: Optional[Sequence[np.ndarray]], tasks: Sequence[Sequence[np.ndarray]],
-             slots=None, M: Optional[List[np.ndarray]] = None) -> List[np.ndarray]:
-    """M = sum_i T_i(W_i - W_0) in the given task order.  base=None: tasks hold deltas."""
+             slots=None, M: Optional[List[np.ndarray]] = None, m_dtype: int = F32) -> List[np.ndarray]:
+    """M = sum_i T_i(W_i - W_0) in the given task order.  base=None: tasks hold deltas.
+    m_dtype=BF16: the fp32 sum is rounded once to bf16 bit patterns."""
     lib = _load()
     sargs, keep = _spec_args(spec)
     L = keep[0].size
@@ -206,13 +208,13 @@ def compress(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
         _check_layers(spec, t, dtype)
         flat.extend(t)
     if M is None:
-        M = new_superposition(spec, slots)
+        M = new_superposition(spec, slots, m_dtype)
     ids = _u32(task_ids)
     sd = np.ascontiguousarray(np.asarray(seeds, dtype=np.uint64))
     mptr, mkeep = _mask(slots, L)
     p = ctypes.c_void_p
     base_pa = _ptr_array(base) if base is not None else None
-    rc = lib.ro_compress(*sargs, ctypes.c_int(dtype), ctypes.c_uint32(K), p(ids.ctypes.data),
+    rc = lib.ro_compress(*sargs, ctypes.c_int(dtype), ctypes.c_int(m_dtype), ctypes.c_uint32(K), p(ids.ctypes.data),
                          p(sd.ctypes.data), base_pa, _ptr_array(flat), _ptr_array(M), mptr)
     if rc:
         raise ValueError("ro_compress failed: %d" % rc)
@@ -243,7 +245,7 @@ def delta_gram(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
     return gram
 
 
-def _swap(fn_name, spec, dtype, task_id, seed, base, task, M, slots):
+def _swap(fn_name, spec, dtype, task_id, seed, base, task, M, slots, m_dtype):
     lib = _load()
     sargs, keep = _spec_args(spec)
     L = keep[0].size
@@ -252,7 +254,7 @@ def _swap(fn_name, spec, dtype, task_id, seed, base, task, M, slots):
     _check_layers(spec, task, dtype)
     mptr, mkeep = _mask(slots, L)
     base_pa = _ptr_array(base) if base is not None else None
-    rc = getattr(lib, fn_name)(*sargs, ctypes.c_int(dtype), ctypes.c_uint32(task_id),
+    rc = getattr(lib, fn_name)(*sargs, ctypes.c_int(dtype), ctypes.c_int(m_dtype), ctypes.c_uint32(task_id),
                                ctypes.c_uint64(seed), base_pa, _ptr_array(task),
                                _ptr_array(M), mptr)
     if rc:
@@ -260,30 +262,30 @@ def _swap(fn_name, spec, dtype, task_id, seed, base, task, M, slots):
     return M
 
 
-def add_model(spec, dtype, task_id, seed, base, task, M, slots=None):
+def add_model(spec, dtype, task_id, seed, base, task, M, slots=None, m_dtype: int = F32):
     """M <- M + T_j(W_j - W_0), in place (Section 5.7, model hot swapping)."""
-    return _swap("ro_add_model", spec, dtype, task_id, seed, base, task, M, slots)
+    return _swap("ro_add_model", spec, dtype, task_id, seed, base, task, M, slots, m_dtype)
 
 
-def remove_model(spec, dtype, task_id, seed, base, task, M, slots=None):
+def remove_model(spec, dtype, task_id, seed, base, task, M, slots=None, m_dtype: int = F32):
     """M <- M - T_j(W_j - W_0), in place."""
-    return _swap("ro_remove_model", spec, dtype, task_id, seed, base, task, M, slots)
+    return _swap("ro_remove_model", spec, dtype, task_id, seed, base, task, M, slots, m_dtype)
 
 
 def retrieve(spec, dtype: int, out_dtype: int, task_id: int, seed: int, lam: float,
-             base: Sequence[np.ndarray], M: Sequence[np.ndarray], positions=None) -> List[np.ndarray]:
+             base: Sequence[np.ndarray], M: Sequence[np.ndarray], positions=None, m_dtype: int = F32) -> List[np.ndarray]:
     """What_t = W_0 + lambda * T_t^-1(M) (Section 4); out fp32 or bf16 bit patterns."""
     lib = _load()
     sargs, keep = _spec_args(spec)
     L = keep[0].size
     _check_layers(spec, base, dtype)
-    _check_layers(spec, M, F32)
+    _check_layers(spec, M, m_dtype)
     odt = np.uint16 if out_dtype == BF16 else np.float32
     wanted = None if positions is None else set(int(x) for x in positions)
     out = [np.zeros((int(r), int(c)), dtype=odt) if wanted is None or l in wanted else None
            for l, (r, c) in enumerate(zip(spec[0], spec[1]))]
     mptr, mkeep = _mask(positions, L)
-    rc = lib.ro_retrieve(*sargs, ctypes.c_int(dtype), ctypes.c_int(out_dtype),
+    rc = lib.ro_retrieve(*sargs, ctypes.c_int(dtype), ctypes.c_int(m_dtype), ctypes.c_int(out_dtype),
                          ctypes.c_uint32(task_id), ctypes.c_uint64(seed), ctypes.c_float(lam),
                          _ptr_array(base), _ptr_array(M), _ptr_array(out), mptr)
     if rc:

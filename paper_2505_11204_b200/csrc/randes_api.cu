@@ -159,6 +159,7 @@ int check_layers(const randes_layer_t* layers, uint32_t n_layers)
 struct randes_plan_s {
     uint32_t n_layers = 0, n_groups = 0, max_tasks = 0;
     int storage = RANDES_F32;
+    int m_dtype = RANDES_F32;                     // element type of the superposition arena
     std::vector<randes_layer_t> layers;
     std::vector<uint32_t> gflags;
     std::vector<std::vector<uint32_t>> members;   // per group, in layer order
@@ -322,10 +323,10 @@ int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_
     a.has_base = base != nullptr;
     a.base = p.dev<const void*>(p.lay.base_ptrs);
     a.task_ptrs = p.dev<const void*>(p.lay.task_ptrs);
-    a.M = static_cast<float*>(M);
+    a.M = M;
     if (a.n_units == 0) return RANDES_OK;
     const int grid = std::min<int>(p.grid_acc[n_rows == 1], static_cast<int>(a.n_units));
-    const int e = launch_accumulate(p.storage, a, grid, s);
+    const int e = launch_accumulate(p.storage, p.m_dtype, a, grid, s);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the accumulate kernel");
     ++g_launches;
     return RANDES_OK;
@@ -352,7 +353,7 @@ size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_laye
 }
 
 int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_group_t* groups, uint32_t n_groups,
-                randes_dtype_t storage_dtype, const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
+                randes_dtype_t storage_dtype, randes_dtype_t m_dtype, const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
                 uint32_t max_tasks, void* dev_workspace, size_t dev_workspace_bytes, void* stream,
                 randes_plan_t** out_plan)
 {
@@ -363,6 +364,8 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
     if (!groups || n_groups == 0) return fail(RANDES_INVALID_ARGUMENT, "groups is NULL or empty");
     if (storage_dtype != RANDES_F32 && storage_dtype != RANDES_BF16)
         return fail(RANDES_UNSUPPORTED_DTYPE, "storage dtype %d is not supported", static_cast<int>(storage_dtype));
+    if (m_dtype != RANDES_F32 && m_dtype != RANDES_BF16)
+        return fail(RANDES_UNSUPPORTED_DTYPE, "superposition dtype %d is not supported", static_cast<int>(m_dtype));
     if (max_tasks == 0 || n_tasks > max_tasks)
         return fail(RANDES_INVALID_ARGUMENT, "max_tasks = %u must be >= max(1, n_tasks = %u)", max_tasks, n_tasks);
     if (n_tasks && (!task_ids || !seeds)) return fail(RANDES_INVALID_ARGUMENT, "task_ids / seeds is NULL");
@@ -384,6 +387,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         p->n_groups = n_groups;
         p->max_tasks = max_tasks;
         p->storage = storage_dtype;
+        p->m_dtype = m_dtype;
         p->layers.assign(layers, layers + n_layers);
         p->gflags.resize(n_groups);
         for (uint32_t g = 0; g < n_groups; ++g) p->gflags[g] = groups[g].flags;
@@ -410,7 +414,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
             const uint32_t g = layers[l].group;
             const std::vector<uint32_t>& mem = p->members[g];
             DevLayer d;
-            d.m_off = off / sizeof(float);
+            d.m_off = off / elem_size(m_dtype);
             d.rows = layers[l].rows;
             d.cols = layers[l].cols;
             d.group = g;
@@ -423,7 +427,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
             d.group_size = static_cast<uint32_t>(mem.size());
             p->dev_layers[l] = d;
             p->m_off_bytes[l] = off;
-            off = align_up(off + static_cast<size_t>(layers[l].rows) * layers[l].cols * sizeof(float), 256);
+            off = align_up(off + static_cast<size_t>(layers[l].rows) * layers[l].cols * elem_size(m_dtype), 256);
         }
         p->m_bytes = off;
         build_units(layers, n_layers, p->storage, p->units);
@@ -457,10 +461,10 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         cudaError_t e = cudaGetDevice(&dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) { delete p; return fail_cuda(e, "device query"); }
-        const int occ_acc = accumulate_ctas_per_sm(p->storage, false);
-        const int occ_acc1 = accumulate_ctas_per_sm(p->storage, true);
-        const int occ_r0 = retrieve_ctas_per_sm(p->storage, RANDES_F32);
-        const int occ_r1 = retrieve_ctas_per_sm(p->storage, RANDES_BF16);
+        const int occ_acc = accumulate_ctas_per_sm(p->storage, p->m_dtype, false);
+        const int occ_acc1 = accumulate_ctas_per_sm(p->storage, p->m_dtype, true);
+        const int occ_r0 = retrieve_ctas_per_sm(p->storage, RANDES_F32, p->m_dtype);
+        const int occ_r1 = retrieve_ctas_per_sm(p->storage, RANDES_BF16, p->m_dtype);
         if (occ_acc <= 0 || occ_acc1 <= 0 || occ_r0 <= 0 || occ_r1 <= 0) {
             delete p;
             return fail(RANDES_CUDA_ERROR, "kernels are not loadable on this device (built for sm_100a)");
@@ -470,8 +474,8 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         p->grid_ret[0] = p->sm_count * occ_r0;
         p->grid_ret[1] = p->sm_count * occ_r1;
         p->grid_gram = p->sm_count * std::max(1, gram_ctas_per_sm(p->storage));
-        p->grid_batch[0] = p->sm_count * std::max(1, retrieve_batch_ctas_per_sm(p->storage, RANDES_F32));
-        p->grid_batch[1] = p->sm_count * std::max(1, retrieve_batch_ctas_per_sm(p->storage, RANDES_BF16));
+        p->grid_batch[0] = p->sm_count * std::max(1, retrieve_batch_ctas_per_sm(p->storage, RANDES_F32, p->m_dtype));
+        p->grid_batch[1] = p->sm_count * std::max(1, retrieve_batch_ctas_per_sm(p->storage, RANDES_BF16, p->m_dtype));
         e = cudaMemcpyAsync(p->ws + p->lay.layers, p->dev_layers.data(), n_layers * sizeof(DevLayer),
                             cudaMemcpyHostToDevice, s);
         if (e == cudaSuccess && !p->units.empty())
@@ -526,6 +530,11 @@ int randes_compress(randes_plan_t* plan, const void* const* base, const void* co
     if ((rc = check_m(M))) return rc;
     if (plan->tasks.empty()) return fail(RANDES_INVALID_ARGUMENT, "no task is registered");
     if (!tasks) return fail(RANDES_INVALID_ARGUMENT, "tasks is NULL");
+    // Beyond kTaskChunk tasks the kernel carries the partial sum through M between chunks; a bf16 M
+    // would round it there, while compress promises one rounding at the end.
+    if (plan->m_dtype == RANDES_BF16 && plan->tasks.size() > static_cast<size_t>(kTaskChunk))
+        return fail(RANDES_CAPACITY, "with a bf16 superposition compress sums at most %d tasks per call (plan holds %zu); "
+                    "use an fp32 superposition or add the remaining models with randes_add_model", kTaskChunk, plan->tasks.size());
     const size_t es = elem_size(plan->storage);
     if ((rc = check_ptrs(*plan, base, "base", es, true))) return rc;
     for (size_t i = 0; i < plan->tasks.size(); ++i)
@@ -616,7 +625,7 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_
     a.slot_of_pos = plan->dev<uint32_t>(plan->lay.slot_of_pos) + static_cast<size_t>(row) * plan->n_layers;
     a.base = plan->dev<const void*>(plan->lay.base_ptrs);
     a.out = plan->dev<void*>(plan->lay.out_ptrs);
-    a.M = static_cast<const float*>(M);
+    a.M = M;
     a.task.id = plan->tasks[row].id;
     a.task.key0 = static_cast<uint32_t>(plan->tasks[row].seed);
     a.task.key1 = static_cast<uint32_t>(plan->tasks[row].seed >> 32);
@@ -624,7 +633,7 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_
     a.lambda = lambda;
     if (a.n_units == 0) return RANDES_OK;
     const int grid = std::min<int>(plan->grid_ret[out_dtype], static_cast<int>(a.n_units));
-    const int e = launch_retrieve(plan->storage, out_dtype, a, grid, s);
+    const int e = launch_retrieve(plan->storage, out_dtype, plan->m_dtype, a, grid, s);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the retrieve kernel");
     ++g_launches;
     return RANDES_OK;
@@ -726,11 +735,11 @@ int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_
     a.n_tasks = n_tasks;
     a.base = plan->dev<const void*>(plan->lay.base_ptrs);
     a.out = plan->dev<void*>(plan->lay.task_ptrs);
-    a.M = static_cast<const float*>(M);
+    a.M = M;
     a.lambda = lambda;
     if (a.n_units == 0) return RANDES_OK;
     const int grid = std::min<int>(plan->grid_batch[out_dtype], static_cast<int>(a.n_units));
-    const int e = launch_retrieve_batch(plan->storage, out_dtype, a, grid, s);
+    const int e = launch_retrieve_batch(plan->storage, out_dtype, plan->m_dtype, a, grid, s);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the batched retrieve kernel");
     ++g_launches;
     return RANDES_OK;
@@ -767,9 +776,9 @@ int randes_retrieve_static(const randes_plan_t* plan, uint32_t task_id, float la
     dt.key0 = static_cast<uint32_t>(t.seed);
     dt.key1 = static_cast<uint32_t>(t.seed >> 32);
     dt.pad = 0;
-    const int e = launch_retrieve_static(plan->storage, out_dtype, plan->dev_layers.data(), plan->n_layers, plan->units.data(),
-                                         static_cast<uint32_t>(plan->units.size()), t.slot_of_pos.data(), base, out,
-                                         static_cast<const float*>(M), dt, lambda, stream);
+    const int e = launch_retrieve_static(plan->storage, out_dtype, plan->m_dtype, plan->dev_layers.data(), plan->n_layers,
+                                         plan->units.data(), static_cast<uint32_t>(plan->units.size()), t.slot_of_pos.data(), base,
+                                         out, M, dt, lambda, stream);
     if (e == -1) return fail(RANDES_CAPACITY, "tables exceed the built-in scratch");
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "randes_retrieve_static");
     if (!plan->units.empty()) ++g_launches;

@@ -21,13 +21,13 @@ using namespace device;
 
 // per warp: what lane i resolved for task i, and every lane's own sign bits per task
 struct BatchScratch {
-    const float* m[kTaskChunk];      // M slot of task i for this layer
+    const void* m[kTaskChunk];       // M slot of task i for this layer
     void* out[kTaskChunk];           // output tensor of task i for this layer
     uint4 block[2][kTaskChunk];      // Philox blocks of task i (second one only for 256-column warps)
     unsigned short bits[kTaskChunk][32];
 };
 
-template <typename ST, typename OT>
+template <typename ST, typename OT, typename MT>
 __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const RetrieveBatchArgs a)
 {
     constexpr int CPL = Store<ST>::CPL;
@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
         if (lane < n) {
             const uint32_t row = a.task_rows[lane];
             const uint32_t slot = (lp.flags & kFlagShuffle) ? a.slot_of_pos[static_cast<size_t>(row) * L + p] : p;   // sigma^-1
-            ws.m[lane] = a.M + a.layers[slot].m_off;
+            ws.m[lane] = static_cast<const MT*>(a.M) + a.layers[slot].m_off;
             void* o = a.out[static_cast<size_t>(lane) * L + p];
             ws.out[lane] = o;
             ok = ok && Out<OT>::template aligned<CPL>(o);
@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
                     const float w = Store<ST>::load1(wp + off + e);
                     for (uint32_t i = 0; i < n; ++i) {
                         const float lam = flip(a.lambda, ((static_cast<uint32_t>(ws.bits[i][lane]) >> e) & 1u) << 31);
-                        Out<OT>::store1(static_cast<OT*>(ws.out[i]) + off + e, __fmaf_rn(lam, ws.m[i][off + e], w));
+                        Out<OT>::store1(static_cast<OT*>(ws.out[i]) + off + e, __fmaf_rn(lam, MTile<MT, CPL>::load1(static_cast<const MT*>(ws.m[i]) + off + e), w));
                     }
                 }
             }
@@ -95,18 +95,14 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
                 if (on[j]) Store<ST>::widen(__ldcs(reinterpret_cast<const uint4*>(wp + off + j * row_stride)), wv[j]);
             }
             for (uint32_t i0 = 0; i0 < n; i0 += TB) {
-                float4 m[TB][U][CPL / 4];
+                float m[TB][U][CPL];
 #pragma unroll
                 for (int b = 0; b < TB; ++b) {
                     if (i0 + b < n) {
-                        const float* mp = ws.m[i0 + b];
+                        const MT* mp = static_cast<const MT*>(ws.m[i0 + b]);
 #pragma unroll
                         for (int j = 0; j < U; ++j)
-                            if (on[j]) {
-#pragma unroll
-                                for (int h = 0; h < CPL / 4; ++h)
-                                    m[b][j][h] = __ldg(reinterpret_cast<const float4*>(mp + off + j * row_stride) + h);
-                            }
+                            if (on[j]) MTile<MT, CPL>::template load<false>(mp + off + j * row_stride, m[b][j]);
                     }
                 }
 #pragma unroll
@@ -122,12 +118,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
                             if (on[j]) {
                                 float y[CPL];
 #pragma unroll
-                                for (int h = 0; h < CPL / 4; ++h) {
-                                    y[4 * h] = __fmaf_rn(lam[4 * h], m[b][j][h].x, wv[j][4 * h]);
-                                    y[4 * h + 1] = __fmaf_rn(lam[4 * h + 1], m[b][j][h].y, wv[j][4 * h + 1]);
-                                    y[4 * h + 2] = __fmaf_rn(lam[4 * h + 2], m[b][j][h].z, wv[j][4 * h + 2]);
-                                    y[4 * h + 3] = __fmaf_rn(lam[4 * h + 3], m[b][j][h].w, wv[j][4 * h + 3]);
-                                }
+                                for (int e = 0; e < CPL; ++e) y[e] = __fmaf_rn(lam[e], m[b][j][e], wv[j][e]);
                                 Out<OT>::template store<CPL>(op + off + j * row_stride, y);
                             }
                     }
@@ -147,24 +138,34 @@ template <typename K> int occupancy(K kernel)
     return n;
 }
 
+template <typename T> struct Tag { typedef T type; };
+template <typename F> int with_type(int dtype, F&& f) { return dtype == 0 ? f(Tag<float>{}) : f(Tag<__nv_bfloat16>{}); }
+
 }  // namespace
 
-int launch_retrieve_batch(int storage_dtype, int out_dtype, const RetrieveBatchArgs& a, int grid, void* stream)
+int launch_retrieve_batch(int storage_dtype, int out_dtype, int m_dtype, const RetrieveBatchArgs& a, int grid, void* stream)
 {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (storage_dtype == 0 && out_dtype == 0) retrieve_batch_kernel<float, float><<<grid, kThreadsPerCta, 0, s>>>(a);
-    else if (storage_dtype == 0 && out_dtype == 1) retrieve_batch_kernel<float, __nv_bfloat16><<<grid, kThreadsPerCta, 0, s>>>(a);
-    else if (storage_dtype == 1 && out_dtype == 0) retrieve_batch_kernel<__nv_bfloat16, float><<<grid, kThreadsPerCta, 0, s>>>(a);
-    else retrieve_batch_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, kThreadsPerCta, 0, s>>>(a);
-    return static_cast<int>(cudaGetLastError());
+    return with_type(storage_dtype, [&](auto st) {
+        return with_type(out_dtype, [&](auto ot) {
+            return with_type(m_dtype, [&](auto mt) {
+                retrieve_batch_kernel<typename decltype(st)::type, typename decltype(ot)::type, typename decltype(mt)::type>
+                    <<<grid, kThreadsPerCta, 0, s>>>(a);
+                return static_cast<int>(cudaGetLastError());
+            });
+        });
+    });
 }
 
-int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype)
+int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype)
 {
-    if (storage_dtype == 0 && out_dtype == 0) return occupancy(retrieve_batch_kernel<float, float>);
-    if (storage_dtype == 0 && out_dtype == 1) return occupancy(retrieve_batch_kernel<float, __nv_bfloat16>);
-    if (storage_dtype == 1 && out_dtype == 0) return occupancy(retrieve_batch_kernel<__nv_bfloat16, float>);
-    return occupancy(retrieve_batch_kernel<__nv_bfloat16, __nv_bfloat16>);
+    return with_type(storage_dtype, [&](auto st) {
+        return with_type(out_dtype, [&](auto ot) {
+            return with_type(m_dtype, [&](auto mt) {
+                return occupancy(retrieve_batch_kernel<typename decltype(st)::type, typename decltype(ot)::type, typename decltype(mt)::type>);
+            });
+        });
+    });
 }
 
 }  // namespace randes

@@ -184,12 +184,86 @@ template <int CPL> __device__ __forceinline__ WarpTile warp_tile(const DevUnit& 
 }
 
 
+// ---- a lane's CPL consecutive elements of the superposition M (fp32 or bf16) ------------------
+template <typename MT, int CPL> struct MTile;
+
+template <int CPL> struct MTile<float, CPL> {
+    static constexpr int kBytes = 4 * CPL;
+    // STREAM: the tile is read once (evict-first); otherwise other CTAs will want it from L2
+    template <bool STREAM = true> static __device__ __forceinline__ void load(const float* p, float (&v)[CPL])
+    {
+#pragma unroll
+        for (int h = 0; h < CPL / 4; ++h) {
+            const float4 m = STREAM ? __ldcs(reinterpret_cast<const float4*>(p) + h) : __ldg(reinterpret_cast<const float4*>(p) + h);
+            v[4 * h] = m.x; v[4 * h + 1] = m.y; v[4 * h + 2] = m.z; v[4 * h + 3] = m.w;
+        }
+    }
+    static __device__ __forceinline__ void store(float* p, const float (&v)[CPL])
+    {
+#pragma unroll
+        for (int h = 0; h < CPL / 4; ++h)
+            reinterpret_cast<float4*>(p)[h] = make_float4(v[4 * h], v[4 * h + 1], v[4 * h + 2], v[4 * h + 3]);
+    }
+    // from 16-byte words as they sit in memory (word h = elements 4h .. 4h+3)
+    static __device__ __forceinline__ void unpack(const uint4 (&raw)[(kBytes + 15) / 16], float (&v)[CPL])
+    {
+#pragma unroll
+        for (int h = 0; h < CPL / 4; ++h) {
+            v[4 * h] = __uint_as_float(raw[h].x); v[4 * h + 1] = __uint_as_float(raw[h].y);
+            v[4 * h + 2] = __uint_as_float(raw[h].z); v[4 * h + 3] = __uint_as_float(raw[h].w);
+        }
+    }
+    static __device__ __forceinline__ float load1(const float* p) { return *p; }
+    static __device__ __forceinline__ void store1(float* p, float v) { *p = v; }
+};
+
+template <int CPL> struct MTile<__nv_bfloat16, CPL> {
+    static constexpr int kBytes = 2 * CPL;
+    static __device__ __forceinline__ float lo(uint32_t w) { return __uint_as_float(w << 16); }
+    static __device__ __forceinline__ float hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+    static __device__ __forceinline__ uint32_t pack(float a, float b)
+    {
+        const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);   // round to nearest even
+        return *reinterpret_cast<const uint32_t*>(&v);
+    }
+    template <bool STREAM = true> static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[CPL])
+    {
+        if (CPL == 4) {
+            const uint2 m = STREAM ? __ldcs(reinterpret_cast<const uint2*>(p)) : __ldg(reinterpret_cast<const uint2*>(p));
+            v[0] = lo(m.x); v[1] = hi(m.x); v[2] = lo(m.y); v[3] = hi(m.y);
+        } else {
+            const uint4 m = STREAM ? __ldcs(reinterpret_cast<const uint4*>(p)) : __ldg(reinterpret_cast<const uint4*>(p));
+            v[0] = lo(m.x); v[1] = hi(m.x); v[2] = lo(m.y); v[3] = hi(m.y);
+            v[4 % CPL] = lo(m.z); v[5 % CPL] = hi(m.z); v[6 % CPL] = lo(m.w); v[7 % CPL] = hi(m.w);
+        }
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&v)[CPL])
+    {
+        if (CPL == 4) *reinterpret_cast<uint2*>(p) = make_uint2(pack(v[0], v[1]), pack(v[2], v[3]));
+        else *reinterpret_cast<uint4*>(p) = make_uint4(pack(v[0], v[1]), pack(v[2], v[3]), pack(v[4 % CPL], v[5 % CPL]), pack(v[6 % CPL], v[7 % CPL]));
+    }
+    static __device__ __forceinline__ void unpack(const uint4 (&raw)[1], float (&v)[CPL])
+    {
+        v[0] = lo(raw[0].x); v[1] = hi(raw[0].x); v[2] = lo(raw[0].y); v[3] = hi(raw[0].y);
+        if (CPL == 8) { v[4 % CPL] = lo(raw[0].z); v[5 % CPL] = hi(raw[0].z); v[6 % CPL] = lo(raw[0].w); v[7 % CPL] = hi(raw[0].w); }
+    }
+    static __device__ __forceinline__ float load1(const __nv_bfloat16* p)
+    {
+        return __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(p)) << 16);
+    }
+    static __device__ __forceinline__ void store1(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
 // ---- asynchronous copies into shared memory and 32-bit shared-window accesses ----------------
 constexpr uint32_t kSlotBytes = kThreadsPerCta * 16;   // one 16-byte slot of every thread of the CTA
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gmem_src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(uint32_t smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void prefetch_l2(const void* gmem) { asm volatile("prefetch.global.L2 [%0];" ::"l"(gmem)); }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }

@@ -63,7 +63,7 @@ struct RetrieveArgs {
     const uint32_t* slot_of_pos;   // this task's sigma^-1, n_layers entries
     const void* const* base;       // device array of n_layers device pointers
     void* const* out;
-    const float* M;
+    const void* M;                 // fp32 or bf16 arena
     DevTask task;
     float lambda;
 };
@@ -81,7 +81,7 @@ struct AccumulateArgs {
     uint32_t has_base;             // 0: task tensors already hold deltas
     const void* const* base;       // device array [n_layers]
     const void* const* task_ptrs;  // device array [n_tasks][n_layers]
-    float* M;
+    void* M;                       // fp32 or bf16 arena
 };
 
 struct RetrieveBatchArgs {
@@ -95,7 +95,7 @@ struct RetrieveBatchArgs {
     uint32_t n_tasks;              // <= kTaskChunk
     const void* const* base;       // device array [n_layers]
     void* const* out;              // device array [n_tasks][n_layers]
-    const float* M;
+    const void* M;
     float lambda;
 };
 
@@ -117,27 +117,27 @@ struct GramArgs {
 };
 
 // Launchers (randes_kernels.cu).  Return a cudaError_t as int.
-int launch_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, int grid, void* stream);
-int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void* stream);
+int launch_retrieve(int storage_dtype, int out_dtype, int m_dtype, const RetrieveArgs& a, int grid, void* stream);
+int launch_accumulate(int storage_dtype, int m_dtype, const AccumulateArgs& a, int grid, void* stream);
 // Resident CTAs per SM of each kernel (for sizing persistent grids); 0 if the
 // kernels cannot run on the current device.  Also opts the kernels into the
 // dynamic shared memory they need: call once per device before launching.
-int retrieve_ctas_per_sm(int storage_dtype, int out_dtype);
-int accumulate_ctas_per_sm(int storage_dtype, bool single_task);
+int retrieve_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype);
+int accumulate_ctas_per_sm(int storage_dtype, int m_dtype, bool single_task);
 // randes_diag.cu: one pass = the Gram kernel plus the fixed-order reduction into gram[a0 .. a0+na)[*]
 int launch_gram_pass(int storage_dtype, const GramArgs& a, int grid, double* gram, void* stream);
 int gram_ctas_per_sm(int storage_dtype);
 // randes_batch.cu
-int launch_retrieve_batch(int storage_dtype, int out_dtype, const RetrieveBatchArgs& a, int grid, void* stream);
-int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype);
+int launch_retrieve_batch(int storage_dtype, int out_dtype, int m_dtype, const RetrieveBatchArgs& a, int grid, void* stream);
+int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype);
 
 
 // Retrieve with its tables in a fixed device array inside the library (no workspace).
 // Returns a cudaError_t as int, or -1 when the tables exceed kStaticScratchBytes.
 constexpr size_t kStaticScratchBytes = 1u << 20;
 size_t retrieve_static_bytes(uint32_t n_layers, uint32_t n_units);
-int launch_retrieve_static(int storage_dtype, int out_dtype, const DevLayer* layers, uint32_t n_layers, const DevUnit* units,
+int launch_retrieve_static(int storage_dtype, int out_dtype, int m_dtype, const DevLayer* layers, uint32_t n_layers, const DevUnit* units,
                            uint32_t n_units, const uint32_t* slot_of_pos, const void* const* base, void* const* out,
-                           const float* M, const DevTask& task, float lambda, void* stream);
+                           const void* M, const DevTask& task, float lambda, void* stream);
 
 }  // namespace randes

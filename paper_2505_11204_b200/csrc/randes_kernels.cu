@@ -43,8 +43,8 @@ using namespace device;
 #endif
 
 // Vector path: U rows per trip, all loads issued before the first use.
-template <typename ST, typename OT>
-__device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, const float* __restrict__ mp,
+template <typename ST, typename OT, typename MT>
+__device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, const MT* __restrict__ mp,
                                               const ST* __restrict__ wp, OT* __restrict__ op,
                                               const float (&lam)[Store<ST>::CPL])
 {
@@ -55,14 +55,13 @@ __device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, 
     const uint32_t row_stride = t.rstep * cols;
     uint32_t off = t.r0 * cols + t.c;               // layers hold < 2^32 elements
     for (uint32_t r = t.r0; r < t.r_end; r += t.rstep * U, off += row_stride * U) {
-        float4 m[U][CPL / 4];
+        float m[U][CPL];
         uint4 w[U];
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             if (r + j * t.rstep < t.r_end) {
                 const uint32_t o = off + j * row_stride;
-#pragma unroll
-                for (int h = 0; h < CPL / 4; ++h) m[j][h] = __ldcs(reinterpret_cast<const float4*>(mp + o) + h);
+                MTile<MT, CPL>::load(mp + o, m[j]);
                 w[j] = __ldcs(reinterpret_cast<const uint4*>(wp + o));
             }
         }
@@ -70,14 +69,10 @@ __device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, 
         for (int j = 0; j < U; ++j) {
             if (r + j * t.rstep < t.r_end) {
                 const uint32_t o = off + j * row_stride;
-                float mv[CPL], wv[CPL], y[CPL];
-#pragma unroll
-                for (int h = 0; h < CPL / 4; ++h) {
-                    mv[4 * h] = m[j][h].x; mv[4 * h + 1] = m[j][h].y; mv[4 * h + 2] = m[j][h].z; mv[4 * h + 3] = m[j][h].w;
-                }
+                float wv[CPL], y[CPL];
                 Store<ST>::widen(w[j], wv);
 #pragma unroll
-                for (int e = 0; e < CPL; ++e) y[e] = __fmaf_rn(lam[e], mv[e], wv[e]);
+                for (int e = 0; e < CPL; ++e) y[e] = __fmaf_rn(lam[e], m[j][e], wv[e]);
                 Out<OT>::template store<CPL>(op + o, y);
             }
         }
@@ -86,8 +81,8 @@ __device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, 
 
 // Element-at-a-time path for ragged widths and unaligned tensors; out of line so
 // that it does not set the register budget of the vector path.
-template <typename ST, typename OT>
-__device__ __noinline__ void retrieve_rows_scalar(WarpTile t, uint32_t cols, const float* mp, const ST* wp, OT* op, float lambda,
+template <typename ST, typename OT, typename MT>
+__device__ __noinline__ void retrieve_rows_scalar(WarpTile t, uint32_t cols, const MT* mp, const ST* wp, OT* op, float lambda,
                                                   uint32_t bits)
 {
     constexpr int CPL = Store<ST>::CPL;
@@ -96,12 +91,12 @@ __device__ __noinline__ void retrieve_rows_scalar(WarpTile t, uint32_t cols, con
         for (int e = 0; e < CPL; ++e) {
             if (t.c + e >= cols) break;
             const float lam = flip(lambda, ((bits >> e) & 1u) << 31);
-            Out<OT>::store1(op + off + e, __fmaf_rn(lam, mp[off + e], Store<ST>::load1(wp + off + e)));
+            Out<OT>::store1(op + off + e, __fmaf_rn(lam, MTile<MT, CPL>::load1(mp + off + e), Store<ST>::load1(wp + off + e)));
         }
     }
 }
 
-template <typename ST, typename OT>
+template <typename ST, typename OT, typename MT>
 #ifndef RANDES_RET_MINB_BF16
 #define RANDES_RET_MINB_BF16 2
 #endif
@@ -126,15 +121,15 @@ __global__ void __launch_bounds__(kThreadsPerCta, Store<ST>::CPL == 4 ? RANDES_R
         }
         const ST* wp = static_cast<const ST*>(a.base[p]);
         OT* op = static_cast<OT*>(a.out[p]);
-        const float* mp = a.M + m_off;
-        const bool vec = lp.cols % CPL == 0 && aligned16(wp) && Out<OT>::template aligned<CPL>(op);
+        const MT* mp = static_cast<const MT*>(a.M) + m_off;
+        const bool vec = lp.cols % CPL == 0 && aligned16(wp) && Out<OT>::template aligned<CPL>(op);   // M slots are 256-byte aligned
         if (vec) {
             float lam[CPL];
 #pragma unroll
             for (int e = 0; e < CPL; ++e) lam[e] = flip(a.lambda, ((bits >> e) & 1u) << 31);
-            retrieve_rows<ST, OT>(t, lp.cols, mp, wp, op, lam);
+            retrieve_rows<ST, OT, MT>(t, lp.cols, mp, wp, op, lam);
         } else {
-            retrieve_rows_scalar<ST, OT>(t, lp.cols, mp, wp, op, a.lambda, bits);
+            retrieve_rows_scalar<ST, OT, MT>(t, lp.cols, mp, wp, op, a.lambda, bits);
         }
     }
 }
@@ -197,28 +192,31 @@ template <typename ST, bool SINGLE> struct AccConfig {
 //   kPerTaskBase: next U*NB   W_0[sigma_i(l)] tiles, same order (L2 hits, staged as deep as the W_i)
 //   kSharedBase:  next U      W_0 tile of row u, filled with the rows' first batch
 //   add / remove: next U*CPL/4  M tiles of the rows, filled likewise
-template <typename ST, bool SINGLE, int BASE> struct StageGeom {
+template <typename ST, bool SINGLE, int BASE, typename MT> struct StageGeom {
     typedef AccConfig<ST, SINGLE> C;
     static constexpr int kW = 0;
     static constexpr int kB = C::U * C::NB;
     static constexpr int kM = kB + (BASE == kPerTaskBase ? C::U * C::NB : (BASE == kSharedBase ? C::U : 0));
-    // A lane's M tile is 16 B for fp32 storage and travels through the ring; for bf16 storage it
-    // is 32 B, which one 16-byte copy per lane can only fetch with a 32-byte stride between lanes
-    // (slow for cp.async): there M is prefetched into L2 and loaded into registers one step ahead.
-    static constexpr bool kInitViaRing = C::kAsyncInit && C::CPL == 4;
-    static constexpr bool kInitViaRegs = C::kAsyncInit && C::CPL == 8;
-    static constexpr int SLOTS = kM + (kInitViaRing ? C::U * C::CPL / 4 : 0);
+    // A lane's M tile (CPL elements) is 8, 16 or 32 bytes.  Up to 16 bytes it travels through the
+    // ring, one slot per row.  32 bytes (fp32 M under bf16 weights) could only be fetched by two
+    // 16-byte copies with a 32-byte stride between lanes, which cp.async handles badly: there M is
+    // prefetched into L2 and loaded into registers one step ahead.
+    static constexpr int kMBytes = static_cast<int>(sizeof(MT)) * C::CPL;
+    static constexpr bool kInitViaRing = C::kAsyncInit && kMBytes <= 16;
+    static constexpr bool kInitViaRegs = C::kAsyncInit && kMBytes == 32;
+    static constexpr int SLOTS = kM + (kInitViaRing ? C::U : 0);
     static constexpr int NSTAGE = (kRingSlots / SLOTS) > 8 ? 8 : (kRingSlots / SLOTS);
     static constexpr uint32_t kStageBytes = SLOTS * kSlotBytes;
     static_assert(NSTAGE >= 2, "ring too small");
 };
 
-template <typename ST, bool SINGLE, int BASE, bool FULL>
+template <typename ST, bool SINGLE, int BASE, bool FULL, typename MT>
 __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_t cols, uint32_t nt, bool init_plain, bool init_async,
-                                                      float* __restrict__ mp, uint32_t ring, uint32_t sptr, uint32_t sbits)
+                                                      MT* __restrict__ mp, uint32_t ring, uint32_t sptr, uint32_t sbits)
 {
     typedef AccConfig<ST, SINGLE> C;
-    typedef StageGeom<ST, SINGLE, BASE> G;
+    typedef StageGeom<ST, SINGLE, BASE, MT> G;
+    typedef MTile<MT, C::CPL> MTl;
     constexpr int CPL = C::CPL, U = C::U, NB = C::NB, NSTAGE = G::NSTAGE;
     constexpr uint32_t ES = sizeof(ST);
     const uint32_t nrows = (t.r_end - t.r0 + t.rstep - 1) / t.rstep;
@@ -259,9 +257,8 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
                     const uint32_t off = off_i + u * row_stride;
                     if (BASE == kSharedBase) cp_async16(stage_i + (G::kB + u) * kSlotBytes, pb0 + static_cast<size_t>(off) * ES);
                     if (G::kInitViaRing && init_async) {
-#pragma unroll
-                        for (int h = 0; h < CPL / 4; ++h)
-                            cp_async16(stage_i + (G::kM + u * (CPL / 4) + h) * kSlotBytes, mp + off + 4 * h);
+                        if (G::kMBytes == 16) cp_async16(stage_i + (G::kM + u) * kSlotBytes, mp + off);
+                        else cp_async8(stage_i + (G::kM + u) * kSlotBytes, mp + off);
                     }
                     if (G::kInitViaRegs && init_async) prefetch_l2(mp + off);
                 }
@@ -283,15 +280,15 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
     const uint32_t one = 0x3F800000u;
 
     // M tiles of the next row group, when they come through registers
-    uint4 m_next[U][CPL / 4];
+    uint4 m_next[U][2];
     uint32_t off_m = off0, left_m = nrows;
     auto load_m_next = [&]() {
 #pragma unroll
         for (int u = 0; u < U; ++u)
             if (u == 0 || left_m > u) {
 #pragma unroll
-                for (int h = 0; h < CPL / 4; ++h)
-                    m_next[u][h] = *reinterpret_cast<const uint4*>(mp + off_m + u * row_stride + 4 * h);
+                for (int h = 0; h < 2; ++h)
+                    m_next[u][h] = reinterpret_cast<const uint4*>(mp + off_m + u * row_stride)[h];
             }
         off_m += U * row_stride;
         left_m -= U;
@@ -309,26 +306,22 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
 #pragma unroll
                 for (int e = 0; e < CPL / 2; ++e) { acc[u][e] = 0ull; w0row[u][e] = 0ull; }
                 if (u == 0 || left_c > u) {
+                    bool have = false;
+                    float mv[CPL];
                     if (G::kInitViaRing && init_async) {
-#pragma unroll
-                        for (int h = 0; h < CPL / 4; ++h) {
-                            const uint4 raw = lds128(stage_c + (G::kM + u * (CPL / 4) + h) * kSlotBytes);
-                            acc[u][2 * h] = pack2(raw.x, raw.y);
-                            acc[u][2 * h + 1] = pack2(raw.z, raw.w);
-                        }
+                        const uint4 raw[1] = {lds128(stage_c + (G::kM + u) * kSlotBytes)};
+                        MTile<MT, CPL>::unpack(reinterpret_cast<const uint4(&)[(G::kMBytes + 15) / 16]>(raw), mv);
+                        have = true;
                     } else if (G::kInitViaRegs && init_async) {
-#pragma unroll
-                        for (int h = 0; h < CPL / 4; ++h) {
-                            acc[u][2 * h] = pack2(m_next[u][h].x, m_next[u][h].y);
-                            acc[u][2 * h + 1] = pack2(m_next[u][h].z, m_next[u][h].w);
-                        }
+                        MTile<MT, CPL>::unpack(reinterpret_cast<const uint4(&)[(G::kMBytes + 15) / 16]>(m_next[u]), mv);
+                        have = true;
                     } else if (init_plain) {
+                        MTl::load(mp + off_c + u * row_stride, mv);
+                        have = true;
+                    }
+                    if (have) {
 #pragma unroll
-                        for (int h = 0; h < CPL / 4; ++h) {
-                            const uint4 raw = *reinterpret_cast<const uint4*>(mp + off_c + u * row_stride + 4 * h);
-                            acc[u][2 * h] = pack2(raw.x, raw.y);
-                            acc[u][2 * h + 1] = pack2(raw.z, raw.w);
-                        }
+                        for (int e = 0; e < CPL / 2; ++e) acc[u][e] = pack2(__float_as_uint(mv[2 * e]), __float_as_uint(mv[2 * e + 1]));
                     }
                     if (BASE == kSharedBase) Store<ST>::widen2(lds128(stage_c + (G::kB + u) * kSlotBytes), w0row[u]);
                 }
@@ -369,13 +362,10 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 if (u == 0 || left_c > u) {
+                    float v[CPL];
 #pragma unroll
-                    for (int h = 0; h < CPL / 4; ++h) {
-                        float4 v;
-                        unpack2(acc[u][2 * h], v.x, v.y);
-                        unpack2(acc[u][2 * h + 1], v.z, v.w);
-                        *reinterpret_cast<float4*>(mp + off_c + u * row_stride + 4 * h) = v;
-                    }
+                    for (int e = 0; e < CPL / 2; ++e) unpack2(acc[u][e], v[2 * e], v[2 * e + 1]);
+                    MTl::store(mp + off_c + u * row_stride, v);
                 }
             }
             b_c = 0;
@@ -393,8 +383,8 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
 // Element-at-a-time path for layers whose width is not a multiple of the lane
 // width or whose tensors are not 16-byte aligned.  Kept out of line: it is rare
 // and must not set the register budget of the vector path.
-template <typename ST, int NB>
-__device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, uint32_t nt, bool init, float* mp, int base_mode,
+template <typename ST, int NB, typename MT>
+__device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, uint32_t nt, bool init, MT* mp, int base_mode,
                                                     uint32_t sptr, uint32_t sbits)
 {
     constexpr int CPL = Store<ST>::CPL;
@@ -402,21 +392,21 @@ __device__ __noinline__ void accumulate_rows_scalar(WarpTile t, uint32_t cols, u
         const size_t off = static_cast<size_t>(r) * cols + t.c;
         for (int e = 0; e < CPL; ++e) {
             if (t.c + e >= cols) break;
-            float acc = init ? mp[off + e] : 0.f;
+            float acc = init ? MTile<MT, CPL>::load1(mp + off + e) : 0.f;
             for (uint32_t i = 0; i < nt; ++i) {
                 float d = Store<ST>::load1(reinterpret_cast<const ST*>(lds_ptr(sptr + i * 16)) + off + e);
                 if (base_mode != kNoBase) d = __fsub_rn(d, Store<ST>::load1(reinterpret_cast<const ST*>(lds_ptr(sptr + i * 16 + 8)) + off + e));
                 const uint32_t bit = (lds_u16(sbits + (i / NB) * 64) >> ((i % NB) * CPL + e)) & 1u;
                 acc = __fadd_rn(acc, flip(d, bit << 31));
             }
-            mp[off + e] = acc;
+            MTile<MT, CPL>::store1(mp + off + e, acc);
         }
     }
 }
 
 // SINGLE: one task per launch (add / remove): a deep ring of single rows, M staged
 // with the weights.  Otherwise (compress): 2 rows x 2 tasks per stage.
-template <typename ST, bool SINGLE>
+template <typename ST, bool SINGLE, typename MT>
 __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const AccumulateArgs a)
 {
     typedef AccConfig<ST, SINGLE> C;
@@ -440,7 +430,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const Acc
         const bool lane_on = t.c < ls.cols;
         const bool shuffled = (ls.flags & kFlagShuffle) != 0;
         const bool flipped = (ls.flags & kFlagFlip) != 0;
-        float* mp = a.M + ls.m_off;
+        MT* mp = static_cast<MT*>(a.M) + ls.m_off;
         const int base_mode = !a.has_base ? kNoBase : ((shuffled && !SINGLE) ? kPerTaskBase : kSharedBase);
 
         for (uint32_t chunk0 = 0; chunk0 < a.n_tasks; chunk0 += MAXT) {
@@ -484,16 +474,16 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const Acc
                 const bool init_async = SINGLE && chunk0 == 0 && a.init_from_m;
                 const bool full = nt % NB == 0;
                 if (!vec)
-                    accumulate_rows_scalar<ST, NB>(t, ls.cols, nt, init_plain || a.init_from_m, mp, base_mode, sptr, sbits);
+                    accumulate_rows_scalar<ST, NB, MT>(t, ls.cols, nt, init_plain || a.init_from_m, mp, base_mode, sptr, sbits);
                 else if (base_mode == kNoBase) {
-                    if (full) accumulate_rows_async<ST, SINGLE, kNoBase, true>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
-                    else accumulate_rows_async<ST, SINGLE, kNoBase, false>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
+                    if (full) accumulate_rows_async<ST, SINGLE, kNoBase, true, MT>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
+                    else accumulate_rows_async<ST, SINGLE, kNoBase, false, MT>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
                 } else if (base_mode == kSharedBase) {
-                    if (full) accumulate_rows_async<ST, SINGLE, kSharedBase, true>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
-                    else accumulate_rows_async<ST, SINGLE, kSharedBase, false>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
+                    if (full) accumulate_rows_async<ST, SINGLE, kSharedBase, true, MT>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
+                    else accumulate_rows_async<ST, SINGLE, kSharedBase, false, MT>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
                 } else {
-                    if (full) accumulate_rows_async<ST, SINGLE, kPerTaskBase, true>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
-                    else accumulate_rows_async<ST, SINGLE, kPerTaskBase, false>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
+                    if (full) accumulate_rows_async<ST, SINGLE, kPerTaskBase, true, MT>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
+                    else accumulate_rows_async<ST, SINGLE, kPerTaskBase, false, MT>(t, ls.cols, nt, init_plain, init_async, mp, ring, sptr, sbits);
                 }
             }
         }
@@ -517,28 +507,37 @@ template <typename K> int ctas_per_sm(K kernel, size_t smem)
 
 }  // namespace
 
-int launch_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, int grid, void* stream)
+// dtype code -> element type, for the launch and occupancy dispatch below
+template <typename T> struct Tag { typedef T type; };
+template <typename F> int with_type(int dtype, F&& f) { return dtype == 0 ? f(Tag<float>{}) : f(Tag<bf16>{}); }
+
+int launch_retrieve(int storage_dtype, int out_dtype, int m_dtype, const RetrieveArgs& a, int grid, void* stream)
 {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (storage_dtype == 0 && out_dtype == 0) retrieve_kernel<float, float><<<grid, kThreadsPerCta, 0, s>>>(a);
-    else if (storage_dtype == 0 && out_dtype == 1) retrieve_kernel<float, bf16><<<grid, kThreadsPerCta, 0, s>>>(a);
-    else if (storage_dtype == 1 && out_dtype == 0) retrieve_kernel<bf16, float><<<grid, kThreadsPerCta, 0, s>>>(a);
-    else retrieve_kernel<bf16, bf16><<<grid, kThreadsPerCta, 0, s>>>(a);
-    return static_cast<int>(cudaGetLastError());
+    return with_type(storage_dtype, [&](auto st) {
+        return with_type(out_dtype, [&](auto ot) {
+            return with_type(m_dtype, [&](auto mt) {
+                retrieve_kernel<typename decltype(st)::type, typename decltype(ot)::type, typename decltype(mt)::type>
+                    <<<grid, kThreadsPerCta, 0, s>>>(a);
+                return static_cast<int>(cudaGetLastError());
+            });
+        });
+    });
 }
 
-int launch_accumulate(int storage_dtype, const AccumulateArgs& a, int grid, void* stream)
+int launch_accumulate(int storage_dtype, int m_dtype, const AccumulateArgs& a, int grid, void* stream)
 {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool single = a.n_tasks == 1;
-    if (storage_dtype == 0) {
-        if (single) accumulate_kernel<float, true><<<grid, kThreadsPerCta, AccConfig<float, true>::kSmemBytes, s>>>(a);
-        else accumulate_kernel<float, false><<<grid, kThreadsPerCta, AccConfig<float, false>::kSmemBytes, s>>>(a);
-    } else {
-        if (single) accumulate_kernel<bf16, true><<<grid, kThreadsPerCta, AccConfig<bf16, true>::kSmemBytes, s>>>(a);
-        else accumulate_kernel<bf16, false><<<grid, kThreadsPerCta, AccConfig<bf16, false>::kSmemBytes, s>>>(a);
-    }
-    return static_cast<int>(cudaGetLastError());
+    return with_type(storage_dtype, [&](auto st) {
+        return with_type(m_dtype, [&](auto mt) {
+            typedef typename decltype(st)::type ST;
+            typedef typename decltype(mt)::type MT;
+            if (single) accumulate_kernel<ST, true, MT><<<grid, kThreadsPerCta, AccConfig<ST, true>::kSmemBytes, s>>>(a);
+            else accumulate_kernel<ST, false, MT><<<grid, kThreadsPerCta, AccConfig<ST, false>::kSmemBytes, s>>>(a);
+            return static_cast<int>(cudaGetLastError());
+        });
+    });
 }
 
 // ---- retrieve without a caller-provided workspace ---------------------------------------------
@@ -561,9 +560,9 @@ size_t retrieve_static_bytes(uint32_t n_layers, uint32_t n_units)
            2 * align256(n_layers * sizeof(void*));
 }
 
-int launch_retrieve_static(int storage_dtype, int out_dtype, const DevLayer* layers, uint32_t n_layers, const DevUnit* units,
+int launch_retrieve_static(int storage_dtype, int out_dtype, int m_dtype, const DevLayer* layers, uint32_t n_layers, const DevUnit* units,
                            uint32_t n_units, const uint32_t* slot_of_pos, const void* const* base, void* const* out,
-                           const float* M, const DevTask& task, float lambda, void* stream)
+                           const void* M, const DevTask& task, float lambda, void* stream)
 {
     if (retrieve_static_bytes(n_layers, n_units) > kStaticScratchBytes) return -1;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -586,7 +585,7 @@ int launch_retrieve_static(int storage_dtype, int out_dtype, const DevLayer* lay
             if (e != cudaSuccess) return static_cast<int>(e);
             for (int st = 0; st < 2; ++st)
                 for (int od = 0; od < 2; ++od) {
-                    const int occ = retrieve_ctas_per_sm(st, od);
+                    const int occ = retrieve_ctas_per_sm(st, od, 0);
                     if (occ <= 0) return static_cast<int>(cudaErrorInvalidDeviceFunction);
                     g_static_grid[dev][st][od] = sms * occ;
                 }
@@ -615,24 +614,30 @@ int launch_retrieve_static(int storage_dtype, int out_dtype, const DevLayer* lay
     a.task = task;
     a.lambda = lambda;
     if (n_units == 0) return 0;
-    return launch_retrieve(storage_dtype, out_dtype, a, grid < static_cast<int>(n_units) ? grid : static_cast<int>(n_units), stream);
+    return launch_retrieve(storage_dtype, out_dtype, m_dtype, a, grid < static_cast<int>(n_units) ? grid : static_cast<int>(n_units), stream);
 }
 
-int retrieve_ctas_per_sm(int storage_dtype, int out_dtype)
+int retrieve_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype)
 {
-    if (storage_dtype == 0 && out_dtype == 0) return ctas_per_sm(retrieve_kernel<float, float>, 0);
-    if (storage_dtype == 0 && out_dtype == 1) return ctas_per_sm(retrieve_kernel<float, bf16>, 0);
-    if (storage_dtype == 1 && out_dtype == 0) return ctas_per_sm(retrieve_kernel<bf16, float>, 0);
-    return ctas_per_sm(retrieve_kernel<bf16, bf16>, 0);
+    return with_type(storage_dtype, [&](auto st) {
+        return with_type(out_dtype, [&](auto ot) {
+            return with_type(m_dtype, [&](auto mt) {
+                return ctas_per_sm(retrieve_kernel<typename decltype(st)::type, typename decltype(ot)::type, typename decltype(mt)::type>, 0);
+            });
+        });
+    });
 }
 
-int accumulate_ctas_per_sm(int storage_dtype, bool single)
+int accumulate_ctas_per_sm(int storage_dtype, int m_dtype, bool single)
 {
-    if (storage_dtype == 0)
-        return single ? ctas_per_sm(accumulate_kernel<float, true>, AccConfig<float, true>::kSmemBytes)
-                      : ctas_per_sm(accumulate_kernel<float, false>, AccConfig<float, false>::kSmemBytes);
-    return single ? ctas_per_sm(accumulate_kernel<bf16, true>, AccConfig<bf16, true>::kSmemBytes)
-                  : ctas_per_sm(accumulate_kernel<bf16, false>, AccConfig<bf16, false>::kSmemBytes);
+    return with_type(storage_dtype, [&](auto st) {
+        return with_type(m_dtype, [&](auto mt) {
+            typedef typename decltype(st)::type ST;
+            typedef typename decltype(mt)::type MT;
+            return single ? ctas_per_sm(accumulate_kernel<ST, true, MT>, AccConfig<ST, true>::kSmemBytes)
+                          : ctas_per_sm(accumulate_kernel<ST, false, MT>, AccConfig<ST, false>::kSmemBytes);
+        });
+    });
 }
 
 }  // namespace randes

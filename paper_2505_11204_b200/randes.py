@@ -71,7 +71,7 @@ def lib():
         vp, u32, u64, sz = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_size_t
         L.randes_plan_workspace_bytes.argtypes = [vp, u32, u32]
         L.randes_plan_workspace_bytes.restype = sz
-        L.randes_plan.argtypes = [vp, u32, vp, u32, ctypes.c_int, vp, vp, u32, u32, vp, sz, vp,
+        L.randes_plan.argtypes = [vp, u32, vp, u32, ctypes.c_int, ctypes.c_int, vp, vp, u32, u32, vp, sz, vp,
                                   ctypes.POINTER(vp)]
         L.randes_plan.restype = ctypes.c_int
         L.randes_plan_destroy.argtypes = [vp]
@@ -144,11 +144,11 @@ def randes_plan_workspace_bytes(layers, n_layers: int, max_tasks: int) -> int:
     return int(lib().randes_plan_workspace_bytes(_addr(layers), n_layers, max_tasks))
 
 
-def randes_plan(layers, n_layers, groups, n_groups, storage_dtype, task_ids, seeds, n_tasks, max_tasks,
+def randes_plan(layers, n_layers, groups, n_groups, storage_dtype, m_dtype, task_ids, seeds, n_tasks, max_tasks,
                 dev_workspace, dev_workspace_bytes, stream) -> int:
     """Returns the plan handle (an address); raises RandesError on failure."""
     out = ctypes.c_void_p()
-    _check(lib().randes_plan(_addr(layers), n_layers, _addr(groups), n_groups, storage_dtype,
+    _check(lib().randes_plan(_addr(layers), n_layers, _addr(groups), n_groups, storage_dtype, m_dtype,
                              _addr(task_ids), _addr(seeds), n_tasks, max_tasks, _addr(dev_workspace),
                              dev_workspace_bytes, stream, ctypes.byref(out)))
     return out.value
@@ -262,7 +262,7 @@ class Plan:
     """
 
     def __init__(self, rows, cols, group, gflags, storage: int = F32, task_ids=(), seeds=(),
-                 max_tasks: Optional[int] = None, device="cuda", host_only: bool = False):
+                 max_tasks: Optional[int] = None, device="cuda", host_only: bool = False, m_dtype: int = F32):
         n_layers, n_groups = len(rows), len(gflags)
         self._layers = (Layer * max(n_layers, 1))()
         for l in range(n_layers):
@@ -278,6 +278,7 @@ class Plan:
         self.n_layers = n_layers
         self.rows, self.cols = [int(r) for r in rows], [int(c) for c in cols]
         self.storage = storage
+        self.m_dtype = m_dtype
         self.handle = None
         self.workspace = None
         self.device = device
@@ -291,7 +292,7 @@ class Plan:
             self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
             ws_ptr = self.workspace.data_ptr()
             stream = self._stream()
-        self.handle = randes_plan(self._layers, n_layers, self._groups, n_groups, storage, ids, sds, n_tasks,
+        self.handle = randes_plan(self._layers, n_layers, self._groups, n_groups, storage, m_dtype, ids, sds, n_tasks,
                                   max_tasks, ws_ptr, ws_bytes, stream)
         self.m_bytes = randes_superposition_bytes(self.handle)
         self.offsets = [randes_layer_offset(self.handle, l) for l in range(n_layers)]
@@ -340,11 +341,13 @@ class Plan:
     def new_superposition(self):
         import torch
 
+        if self.m_dtype == BF16:
+            return torch.empty(self.m_bytes // 2, dtype=torch.bfloat16, device=self.device)
         return torch.empty(self.m_bytes // 4, dtype=torch.float32, device=self.device)
 
     def slot(self, M, layer: int):
         """View of slot ``layer`` of the arena M as a [rows, cols] tensor."""
-        o = self.offsets[layer] // 4
+        o = self.offsets[layer] // (2 if self.m_dtype == BF16 else 4)
         n = self.rows[layer] * self.cols[layer]
         return M[o:o + n].view(self.rows[layer], self.cols[layer])
 

@@ -38,7 +38,7 @@ def make_workload(shapes, flags=S | F, storage=wl.F32, n_tasks=3, seed0=42, data
                        seeds=[seed0 + i for i in range(n_tasks)], scale=1e-3, lam=0.3, data_seed=data_seed)
 
 
-def run_full_cycle(w, out_dtypes=(wl.F32, wl.BF16), lam=None, extra_task=True):
+def run_full_cycle(w, out_dtypes=(wl.F32, wl.BF16), lam=None, extra_task=True, m_dtype=wl.F32):
     """compress -> retrieve all -> add -> retrieve -> remove -> retrieve, each
     step compared with the oracle replaying the same calls."""
     import torch
@@ -48,18 +48,19 @@ def run_full_cycle(w, out_dtypes=(wl.F32, wl.BF16), lam=None, extra_task=True):
     all_ids = ids + ([max(ids) + 5] if extra_task else [])
     base, tasks = wl.model_set(w, all_ids)
     d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
-    plan = randes.Plan.from_workload(w, max_tasks=len(all_ids) + 1)
+    plan = randes.Plan.from_workload(w, max_tasks=len(all_ids) + 1, m_dtype=m_dtype)
     K = len(ids)
+    msz = 2 if m_dtype == wl.BF16 else 4
 
     M_dev = poison(plan.new_superposition())
     plan.compress(d_base, d_tasks[:K], M_dev)
-    M_ref = ro.compress(w.spec, w.storage, ids, seeds, base, tasks[:K])
+    M_ref = ro.compress(w.spec, w.storage, ids, seeds, base, tasks[:K], m_dtype=m_dtype)
     check_superposition(plan, M_dev, M_ref, "compress")
     # padding between slots is never written
-    raw = M_dev.view(torch.int32)
+    raw = M_dev.view(torch.int16 if m_dtype == wl.BF16 else torch.int32)
     for l in range(w.n_layers):
-        end = plan.offsets[l] // 4 + w.rows[l] * w.cols[l]
-        nxt = plan.offsets[l + 1] // 4 if l + 1 < w.n_layers else plan.m_bytes // 4
+        end = plan.offsets[l] // msz + w.rows[l] * w.cols[l]
+        nxt = plan.offsets[l + 1] // msz if l + 1 < w.n_layers else plan.m_bytes // msz
         assert bool((raw[end:nxt] == -1).all()), "padding after slot %d was written" % l
 
     def retrieve_all(tag):
@@ -68,21 +69,21 @@ def run_full_cycle(w, out_dtypes=(wl.F32, wl.BF16), lam=None, extra_task=True):
             for t, s in zip(cur_ids, cur_seeds):
                 out = [poison(o) for o in plan.new_output(od)]
                 plan.retrieve(t, lam, d_base, M_dev, out=out, out_dtype=od)
-                ref = ro.retrieve(w.spec, w.storage, od, t, s, lam, base, M_ref)
+                ref = ro.retrieve(w.spec, w.storage, od, t, s, lam, base, M_ref, m_dtype=m_dtype)
                 check_model(out, ref, "%s retrieve task %d dtype %d" % (tag, t, od))
 
     retrieve_all("after compress")
     if extra_task:
         new_id, new_seed = all_ids[-1], 100
         plan.add_model(new_id, new_seed, d_base, d_tasks[K], M_dev)
-        ro.add_model(w.spec, w.storage, new_id, new_seed, base, tasks[K], M_ref)
+        ro.add_model(w.spec, w.storage, new_id, new_seed, base, tasks[K], M_ref, m_dtype=m_dtype)
         check_superposition(plan, M_dev, M_ref, "add")
         assert plan.task_list() == (ids + [new_id], seeds + [new_seed])
         retrieve_all("after add")
         gone = ids[len(ids) // 2]
         j = ids.index(gone)
         plan.remove_model(gone, d_base, d_tasks[j], M_dev)
-        ro.remove_model(w.spec, w.storage, gone, seeds[j], base, tasks[j], M_ref)
+        ro.remove_model(w.spec, w.storage, gone, seeds[j], base, tasks[j], M_ref, m_dtype=m_dtype)
         check_superposition(plan, M_dev, M_ref, "remove")
         assert gone not in plan.task_list()[0]
         retrieve_all("after remove")
@@ -102,6 +103,41 @@ RAGGED = [(1, 1, 3), (5, 3, 3), (37, 12, 2), (3, 127, 3), (2, 129, 4), (7, 130, 
 @pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
 def test_ragged_shapes_span_tiles_and_tails(storage):
     run_full_cycle(make_workload(RAGGED, storage=storage, n_tasks=3))
+
+
+@pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
+def test_bf16_superposition(storage):
+    # M stored as bf16: sums in fp32, one rounding per element at the end of compress, again after add / remove
+    run_full_cycle(make_workload(RAGGED, storage=storage, n_tasks=4), m_dtype=wl.BF16)
+    # more than 32 tasks would need the partial sum to pass through the bf16 arena: refused
+    w = make_workload([(5, 260, 3), (1, 33, 2)], storage=storage, n_tasks=35)
+    base, tasks = wl.model_set(w)
+    plan = randes.Plan.from_workload(w, m_dtype=wl.BF16)
+    with pytest.raises(randes.RandesError) as e:
+        plan.compress(model_to_dev(base), [model_to_dev(t) for t in tasks])
+    assert e.value.code == randes.CAPACITY
+    plan.close()
+
+
+def test_bf16_superposition_batched_and_static_retrieve():
+    import torch
+
+    w = make_workload(RAGGED, storage=wl.BF16, n_tasks=5)
+    base, tasks = wl.model_set(w)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, m_dtype=wl.BF16)
+    assert plan.m_bytes <= 2 * w.n_params + 256 * w.n_layers
+    M = plan.compress(d_base, d_tasks)
+    M_ref = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, base, tasks, m_dtype=wl.BF16)
+    outs = plan.retrieve_batch([3, 0, 4], w.lam, d_base, M, out_dtype=wl.BF16)
+    for b, t in enumerate([3, 0, 4]):
+        check_model(outs[b], ro.retrieve(w.spec, w.storage, wl.BF16, t, w.seeds[t], w.lam, base, M_ref, m_dtype=wl.BF16),
+                    "batched retrieve from bf16 M, task %d" % t)
+    got = plan.new_output(wl.F32)
+    randes.randes_retrieve_static(plan.handle, 2, w.lam, wl.F32, randes.ptr_array(d_base), M, randes.ptr_array(got),
+                                  torch.cuda.current_stream().cuda_stream)
+    check_model(got, ro.retrieve(w.spec, w.storage, wl.F32, 2, w.seeds[2], w.lam, base, M_ref, m_dtype=wl.BF16), "static retrieve from bf16 M")
+    plan.close()
 
 
 @pytest.mark.parametrize("flags", [0, S, F])
@@ -373,7 +409,7 @@ def test_gpu_argument_validation():
     assert randes.randes_launch_count() == before + 1      # only the valid add launched
     small = torch.empty(256, dtype=torch.uint8, device="cuda")
     with pytest.raises(randes.RandesError) as e:
-        randes.randes_plan(plan._layers, 2, plan._groups, 1, 0, None, None, 0, 1, small, 256, None)
+        randes.randes_plan(plan._layers, 2, plan._groups, 1, 0, 0, None, None, 0, 1, small, 256, None)
     assert e.value.code == randes.WORKSPACE_TOO_SMALL
     plan.close()
 

@@ -97,6 +97,9 @@ def test_superposition_layout_is_one_fp32_copy_independent_of_task_count():
     for l in range(w.n_layers - 1):
         assert p8.offsets[l + 1] - p8.offsets[l] >= 4 * w.rows[l] * w.cols[l]
     assert randes.randes_layer_offset(p8.handle, w.n_layers) == 2**64 - 1
+    # a bf16 superposition takes half the bytes (up to slot padding)
+    ph = randes.Plan.from_workload(w, host_only=True, m_dtype=randes.BF16)
+    assert 2 * w.n_params <= ph.m_bytes <= 2 * w.n_params + 256 * w.n_layers and all(o % 256 == 0 for o in ph.offsets)
     # memory figures of the paper's first results table: 0.564 -> 0.89 (GiB) is one fp32 copy of the encoder
     assert abs(0.564 + raw / 2**30 - 0.89) < 0.005
 
@@ -132,6 +135,9 @@ def test_plan_argument_validation():
     _expect(randes.INVALID_ARGUMENT, lambda: mk(max_tasks=0, ids=[], seeds=[]))
     _expect(randes.INVALID_ARGUMENT, lambda: mk(ids=[0, 1, 2], seeds=[0, 1, 2], max_tasks=2))
     _expect(randes.UNSUPPORTED_DTYPE, lambda: mk(storage=7))
+    with pytest.raises(randes.RandesError) as e:
+        randes.Plan([2], [4], [0], [0], task_ids=[0], seeds=[1], host_only=True, m_dtype=5)
+    assert e.value.code == randes.UNSUPPORTED_DTYPE
     p = mk()
     _expect(randes.UNKNOWN_TASK, lambda: p.task_tables(99))
     # a host-only plan cannot compute

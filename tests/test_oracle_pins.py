@@ -585,6 +585,33 @@ def test_bf16_storage_and_output():
         assert np.array_equal(a, wl.to_bf16_bits(b))
 
 
+def test_bf16_superposition_is_the_fp32_sum_rounded_once():
+    # the further compression of M that the paper's conclusion leaves open: M stored as bf16
+    rng = np.random.default_rng(41)
+    spec = tiny_spec(SHUFFLE | FLIP, shape_a=(3, 40))
+    base = rand_model(spec, rng, 0.02)
+    tasks = [[b + d for b, d in zip(base, rand_model(spec, rng, 1e-3))] for _ in range(4)]
+    ids, seeds = [0, 1, 2], [4, 5, 6]
+    M32 = ro.compress(spec, ro.F32, ids, seeds, base, tasks[:3])
+    M16 = ro.compress(spec, ro.F32, ids, seeds, base, tasks[:3], m_dtype=ro.BF16)
+    for a, b in zip(M16, M32):
+        assert a.dtype == np.uint16 and np.array_equal(a, wl.to_bf16_bits(b))
+    # retrieve widens the stored element: same as retrieving from the widened copy
+    wide = [wl.bf16_bits_to_f32(m) for m in M16]
+    out16 = ro.retrieve(spec, ro.F32, ro.F32, 1, 5, 0.3, base, M16, m_dtype=ro.BF16)
+    out32 = ro.retrieve(spec, ro.F32, ro.F32, 1, 5, 0.3, base, wide)
+    assert all(np.array_equal(a, b) for a, b in zip(out16, out32))
+    # add: widen, add the transformed delta in fp32, round again
+    x = ro.compress(spec, ro.F32, [7], [70], base, [tasks[3]])             # T_7(delta) alone
+    ro.add_model(spec, ro.F32, 7, 70, base, tasks[3], M16, m_dtype=ro.BF16)
+    for m, w_, xx in zip(M16, wide, x):
+        assert np.array_equal(m, wl.to_bf16_bits((w_ + xx).astype(np.float32)))
+    wide2 = [wl.bf16_bits_to_f32(m) for m in M16]
+    ro.remove_model(spec, ro.F32, 7, 70, base, tasks[3], M16, m_dtype=ro.BF16)
+    for m, w_, xx in zip(M16, wide2, x):
+        assert np.array_equal(m, wl.to_bf16_bits((w_ - xx).astype(np.float32)))
+
+
 # --------------------------------------------------------------------------- masks, errors
 def test_slot_mask_limits_work_and_matches_full_result():
     rng = np.random.default_rng(24)

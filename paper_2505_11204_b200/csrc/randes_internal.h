@@ -12,10 +12,7 @@ constexpr uint32_t kFlagFlip = 2u;      // per-column sign flip on this slot
 
 constexpr int kWarpsPerCta = 8;
 constexpr int kThreadsPerCta = kWarpsPerCta * 32;
-#ifndef RANDES_ROWS_PER_WARP
-#define RANDES_ROWS_PER_WARP 16
-#endif
-constexpr int kRowsPerWarp = RANDES_ROWS_PER_WARP;   // rows one warp walks per unit
+constexpr int kRowsPerWarp = 16;        // rows one warp walks per unit (8 to 16 measured best; 32 and 64 slower)
 constexpr int kTaskChunk = 32;          // tasks whose pointers / sign blocks a warp holds at once
 constexpr uint32_t kTagSign = 0x5349474Eu;  // counter word 2 of the sign stream ("SIGN")
 constexpr uint32_t kTagPerm = 0x5045524Du;  // counter word 2 of the permutation stream ("PERM")

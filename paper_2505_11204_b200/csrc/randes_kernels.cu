@@ -35,12 +35,6 @@ using namespace device;
 // (Section 4, second display; Section 4.4, second display.)  The sign is folded
 // into lambda: fma(+-lambda, m, w) is bit-identical to fma(lambda, +-m, w).
 // =========================================================================================
-#ifndef RANDES_RET_U
-#define RANDES_RET_U 4
-#endif
-#ifndef RANDES_RET_MINB
-#define RANDES_RET_MINB 2
-#endif
 
 // Vector path: U rows per trip, all loads issued before the first use.
 template <typename ST, typename OT, typename MT>
@@ -51,7 +45,7 @@ __device__ __forceinline__ void retrieve_rows(const WarpTile& t, uint32_t cols, 
     constexpr int CPL = Store<ST>::CPL;
     // rows per trip, measured best per type pair: bf16 weights with fp32 output move 80 B per lane
     // and row and are fastest one row at a time; bf16 -> bf16 (48 B) wants four
-    constexpr int U = CPL == 4 ? RANDES_RET_U : (sizeof(OT) == 4 ? 1 : 4);
+    constexpr int U = CPL == 4 ? 4 : (sizeof(OT) == 4 ? 1 : 4);
     const uint32_t row_stride = t.rstep * cols;
     uint32_t off = t.r0 * cols + t.c;               // layers hold < 2^32 elements
     for (uint32_t r = t.r0; r < t.r_end; r += t.rstep * U, off += row_stride * U) {
@@ -97,11 +91,7 @@ __device__ __noinline__ void retrieve_rows_scalar(WarpTile t, uint32_t cols, con
 }
 
 template <typename ST, typename OT, typename MT>
-#ifndef RANDES_RET_MINB_BF16
-#define RANDES_RET_MINB_BF16 2
-#endif
-__global__ void __launch_bounds__(kThreadsPerCta, Store<ST>::CPL == 4 ? RANDES_RET_MINB : RANDES_RET_MINB_BF16)
-    retrieve_kernel(const RetrieveArgs a)
+__global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_kernel(const RetrieveArgs a)
 {
     constexpr int CPL = Store<ST>::CPL;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -163,20 +153,9 @@ constexpr int kRingSlots = 24;    // 16-byte slots per thread: 96 KiB per CTA, t
 
 template <typename ST, bool SINGLE> struct AccConfig {
     static constexpr int CPL = Store<ST>::CPL;
-#ifndef RANDES_SINGLE_U
-#define RANDES_SINGLE_U 1
-#endif
-#ifndef RANDES_COMPRESS_U_BF16
-#define RANDES_COMPRESS_U_BF16 1
-#endif
-#ifndef RANDES_COMPRESS_U_F32
-#define RANDES_COMPRESS_U_F32 2
-#endif
-#ifndef RANDES_COMPRESS_NB
-#define RANDES_COMPRESS_NB 2
-#endif
-    static constexpr int U = SINGLE ? RANDES_SINGLE_U : (CPL == 8 ? RANDES_COMPRESS_U_BF16 : RANDES_COMPRESS_U_F32);   // rows per stage
-    static constexpr int NB = SINGLE ? 1 : (CPL == 8 ? 2 : RANDES_COMPRESS_NB);         // tasks per stage
+    // measured best: fp32 weights 2 rows x 2 tasks per stage, bf16 weights 1 row x 2 tasks, add / remove 1 row
+    static constexpr int U = (SINGLE || CPL == 8) ? 1 : 2;   // rows per stage
+    static constexpr int NB = SINGLE ? 1 : 2;                // tasks per stage
     static constexpr int MAXT = SINGLE ? 1 : kTaskChunk;
     static constexpr bool kAsyncInit = SINGLE;        // add / remove start from M
     static constexpr uint32_t kRingBytes = kRingSlots * kSlotBytes;

@@ -112,7 +112,7 @@ __device__ __forceinline__ void gram_rows(const WarpTile& t, uint32_t cols, Gram
 }
 
 template <typename ST>
-__global__ void __launch_bounds__(kThreadsPerCta, 2) gram_kernel(const GramArgs a)
+__global__ void __launch_bounds__(kThreadsPerCta, 4) gram_kernel(const GramArgs a)
 {
     constexpr int CPL = Store<ST>::CPL;
     __shared__ GramScratch scratch[kWarpsPerCta];

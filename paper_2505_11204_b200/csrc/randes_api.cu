@@ -148,9 +148,15 @@ int check_layers(const randes_layer_t* layers, uint32_t n_layers)
 {
     if (!layers || n_layers == 0) return fail(RANDES_INVALID_ARGUMENT, "layers is NULL or empty");
     for (uint32_t l = 0; l < n_layers; ++l)
+    {
         if (layers[l].cols > 65535u * 128u)
             return fail(RANDES_INVALID_ARGUMENT, "layer %u: cols %u exceeds the supported %u", l, layers[l].cols,
                         65535u * 128u);
+        // the kernels index inside a layer with 32-bit element offsets
+        if (static_cast<unsigned long long>(layers[l].rows) * layers[l].cols > 0xFFFFFFFFull)
+            return fail(RANDES_INVALID_ARGUMENT, "layer %u: %u x %u elements exceed the supported 2^32 - 1 per layer", l,
+                        layers[l].rows, layers[l].cols);
+    }
     return RANDES_OK;
 }
 
@@ -330,6 +336,18 @@ int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the accumulate kernel");
     ++g_launches;
     return RANDES_OK;
+}
+
+// Runs the body of an entry point; nothing may cross the C ABI as an exception.
+template <typename F> int guarded(F&& body)
+{
+    try {
+        return body();
+    } catch (const std::bad_alloc&) {
+        return fail(RANDES_OUT_OF_MEMORY, "host allocation failed");
+    } catch (...) {
+        return fail(RANDES_INVALID_ARGUMENT, "unexpected internal error");
+    }
 }
 
 }  // namespace
@@ -522,7 +540,7 @@ int randes_task_tables(const randes_plan_t* plan, uint32_t task_id, uint32_t* sr
     return RANDES_OK;
 }
 
-int randes_compress(randes_plan_t* plan, const void* const* base, const void* const* tasks, void* M, void* stream)
+static int randes_compress_impl(randes_plan_t* plan, const void* const* base, const void* const* tasks, void* M, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
     if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
@@ -542,7 +560,7 @@ int randes_compress(randes_plan_t* plan, const void* const* base, const void* co
     return run_accumulate(*plan, 0, plan->tasks.size(), false, false, base, tasks, M, static_cast<cudaStream_t>(stream));
 }
 
-int randes_add_model(randes_plan_t* plan, uint32_t task_id, uint64_t seed, const void* const* base,
+static int randes_add_model_impl(randes_plan_t* plan, uint32_t task_id, uint64_t seed, const void* const* base,
                      const void* const* task, void* M, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
@@ -574,7 +592,7 @@ int randes_add_model(randes_plan_t* plan, uint32_t task_id, uint64_t seed, const
     return RANDES_OK;
 }
 
-int randes_remove_model(randes_plan_t* plan, uint32_t task_id, const void* const* base, const void* const* task,
+static int randes_remove_model_impl(randes_plan_t* plan, uint32_t task_id, const void* const* base, const void* const* task,
                         void* M, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
@@ -593,7 +611,7 @@ int randes_remove_model(randes_plan_t* plan, uint32_t task_id, const void* const
     return upload_task_rows(*plan, row, s);
 }
 
-int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
+static int randes_retrieve_impl(randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
                     const void* const* base, const void* M, void* const* out, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
@@ -645,7 +663,7 @@ size_t randes_delta_gram_scratch_bytes(const randes_plan_t* plan)
     return static_cast<size_t>(plan->grid_gram) * kWarpsPerCta * kGramAnchors * kTaskChunk * sizeof(double);
 }
 
-int randes_delta_gram(randes_plan_t* plan, const void* const* base, const void* const* tasks, double* gram, void* scratch,
+static int randes_delta_gram_impl(randes_plan_t* plan, const void* const* base, const void* const* tasks, double* gram, void* scratch,
                       size_t scratch_bytes, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
@@ -690,7 +708,7 @@ int randes_delta_gram(randes_plan_t* plan, const void* const* base, const void* 
     return RANDES_OK;
 }
 
-int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_t n_tasks, float lambda,
+static int randes_retrieve_batch_impl(randes_plan_t* plan, const uint32_t* task_ids, uint32_t n_tasks, float lambda,
                           randes_dtype_t out_dtype, const void* const* base, const void* M, void* const* out, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
@@ -745,7 +763,7 @@ int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_
     return RANDES_OK;
 }
 
-int randes_retrieve_static(const randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
+static int randes_retrieve_static_impl(const randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
                            const void* const* base, const void* M, void* const* out, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
@@ -783,6 +801,47 @@ int randes_retrieve_static(const randes_plan_t* plan, uint32_t task_id, float la
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "randes_retrieve_static");
     if (!plan->units.empty()) ++g_launches;
     return RANDES_OK;
+}
+
+int randes_compress(randes_plan_t* plan, const void* const* base, const void* const* tasks, void* M, void* stream)
+{
+    return guarded([&] { return randes_compress_impl(plan, base, tasks, M, stream); });
+}
+
+int randes_add_model(randes_plan_t* plan, uint32_t task_id, uint64_t seed, const void* const* base,
+                     const void* const* task, void* M, void* stream)
+{
+    return guarded([&] { return randes_add_model_impl(plan, task_id, seed, base, task, M, stream); });
+}
+
+int randes_remove_model(randes_plan_t* plan, uint32_t task_id, const void* const* base, const void* const* task,
+                        void* M, void* stream)
+{
+    return guarded([&] { return randes_remove_model_impl(plan, task_id, base, task, M, stream); });
+}
+
+int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
+                    const void* const* base, const void* M, void* const* out, void* stream)
+{
+    return guarded([&] { return randes_retrieve_impl(plan, task_id, lambda, out_dtype, base, M, out, stream); });
+}
+
+int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_t n_tasks, float lambda,
+                          randes_dtype_t out_dtype, const void* const* base, const void* M, void* const* out, void* stream)
+{
+    return guarded([&] { return randes_retrieve_batch_impl(plan, task_ids, n_tasks, lambda, out_dtype, base, M, out, stream); });
+}
+
+int randes_delta_gram(randes_plan_t* plan, const void* const* base, const void* const* tasks, double* gram, void* scratch,
+                      size_t scratch_bytes, void* stream)
+{
+    return guarded([&] { return randes_delta_gram_impl(plan, base, tasks, gram, scratch, scratch_bytes, stream); });
+}
+
+int randes_retrieve_static(const randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
+                           const void* const* base, const void* M, void* const* out, void* stream)
+{
+    return guarded([&] { return randes_retrieve_static_impl(plan, task_id, lambda, out_dtype, base, M, out, stream); });
 }
 
 }  // extern "C"

@@ -135,6 +135,7 @@ def test_plan_argument_validation():
     _expect(randes.INVALID_ARGUMENT, lambda: mk(max_tasks=0, ids=[], seeds=[]))
     _expect(randes.INVALID_ARGUMENT, lambda: mk(ids=[0, 1, 2], seeds=[0, 1, 2], max_tasks=2))
     _expect(randes.UNSUPPORTED_DTYPE, lambda: mk(storage=7))
+    _expect(randes.INVALID_ARGUMENT, lambda: mk(rows=[70000, 70000], cols=[70000, 70000]))   # >= 2^32 elements per layer
     with pytest.raises(randes.RandesError) as e:
         randes.Plan([2], [4], [0], [0], task_ids=[0], seeds=[1], host_only=True, m_dtype=5)
     assert e.value.code == randes.UNSUPPORTED_DTYPE

@@ -148,6 +148,22 @@ uint32_t randes_num_tasks(const randes_plan_t* plan);
 int randes_task_list(const randes_plan_t* plan, uint32_t* task_ids, uint64_t* seeds);
 
 /*
+ * Persistence.  What RanDeS keeps per model is a seed (Section 4.1), so a plan
+ * is fully described by its layer shapes, group flags, element types and the
+ * registered (id, seed) pairs in summation order; M itself is the caller's
+ * buffer to save.  serialize writes that description as a self-contained blob
+ * (host memory; pass buffer = NULL to get the size) and returns the number of
+ * bytes, 0 on error.  deserialize rebuilds an equivalent plan from a blob; the
+ * workspace arguments are those of randes_plan (NULL workspace = host-only),
+ * and max_tasks is raised to the number of stored tasks if it is smaller.
+ * Errors: INVALID_ARGUMENT (not a blob, truncated), plus those of randes_plan.
+ */
+size_t randes_plan_serialize(const randes_plan_t* plan, void* buffer, size_t buffer_bytes);
+int randes_plan_deserialize(const void* buffer, size_t buffer_bytes, uint32_t max_tasks,
+                            void* dev_workspace, size_t dev_workspace_bytes, void* stream,
+                            randes_plan_t** out_plan);
+
+/*
  * Host copies of one task's layer tables (n_layers entries each, either may be
  * NULL):  src_of_slot[l] = layer whose delta lands on slot l (sigma);
  * slot_of_pos[p] = slot holding layer p's delta (sigma^-1).   (Section 4.3)

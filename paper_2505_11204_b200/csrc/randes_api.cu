@@ -529,6 +529,66 @@ int randes_task_list(const randes_plan_t* plan, uint32_t* task_ids, uint64_t* se
     return RANDES_OK;
 }
 
+// ---- persistence: what the paper stores per model is a seed; a plan is its shapes, flags and seeds ----
+namespace {
+constexpr uint32_t kBlobMagic = 0x53444E52u;   // "RNDS"
+constexpr uint32_t kBlobVersion = 1;
+struct BlobHeader {
+    uint32_t magic, version, n_layers, n_groups, storage, m_dtype, n_tasks, reserved;
+};
+size_t blob_bytes(uint32_t n_layers, uint32_t n_groups, uint32_t n_tasks)
+{
+    return sizeof(BlobHeader) + n_layers * sizeof(randes_layer_t) + n_groups * sizeof(uint32_t) + n_tasks * (sizeof(uint32_t) + sizeof(uint64_t));
+}
+}  // namespace
+
+size_t randes_plan_serialize(const randes_plan_t* plan, void* buffer, size_t buffer_bytes)
+{
+    if (!plan) { fail(RANDES_INVALID_ARGUMENT, "plan is NULL"); return 0; }
+    const uint32_t n_tasks = static_cast<uint32_t>(plan->tasks.size());
+    const size_t need = blob_bytes(plan->n_layers, plan->n_groups, n_tasks);
+    if (!buffer) return need;
+    if (buffer_bytes < need) { fail(RANDES_WORKSPACE_TOO_SMALL, "buffer has %zu bytes, the plan needs %zu", buffer_bytes, need); return 0; }
+    char* out = static_cast<char*>(buffer);
+    const BlobHeader h = {kBlobMagic, kBlobVersion, plan->n_layers, plan->n_groups, static_cast<uint32_t>(plan->storage),
+                          static_cast<uint32_t>(plan->m_dtype), n_tasks, 0};
+    std::memcpy(out, &h, sizeof h); out += sizeof h;
+    std::memcpy(out, plan->layers.data(), plan->n_layers * sizeof(randes_layer_t)); out += plan->n_layers * sizeof(randes_layer_t);
+    std::memcpy(out, plan->gflags.data(), plan->n_groups * sizeof(uint32_t)); out += plan->n_groups * sizeof(uint32_t);
+    for (const TaskEntry& t : plan->tasks) { std::memcpy(out, &t.id, sizeof t.id); out += sizeof t.id; }
+    for (const TaskEntry& t : plan->tasks) { std::memcpy(out, &t.seed, sizeof t.seed); out += sizeof t.seed; }
+    return need;
+}
+
+int randes_plan_deserialize(const void* buffer, size_t buffer_bytes, uint32_t max_tasks, void* dev_workspace,
+                            size_t dev_workspace_bytes, void* stream, randes_plan_t** out_plan)
+{
+    if (!out_plan) return fail(RANDES_INVALID_ARGUMENT, "out_plan is NULL");
+    *out_plan = nullptr;
+    if (!buffer || buffer_bytes < sizeof(BlobHeader)) return fail(RANDES_INVALID_ARGUMENT, "buffer is NULL or shorter than a header");
+    BlobHeader h;
+    std::memcpy(&h, buffer, sizeof h);
+    if (h.magic != kBlobMagic || h.version != kBlobVersion)
+        return fail(RANDES_INVALID_ARGUMENT, "not a serialized plan (magic 0x%x, version %u)", h.magic, h.version);
+    if (h.n_layers > (1u << 24) || h.n_groups > (1u << 24) || h.n_tasks > (1u << 24) ||
+        buffer_bytes < blob_bytes(h.n_layers, h.n_groups, h.n_tasks))
+        return fail(RANDES_INVALID_ARGUMENT, "serialized plan is truncated or corrupt");
+    return guarded([&] {
+        const char* in = static_cast<const char*>(buffer) + sizeof h;
+        std::vector<randes_layer_t> layers(h.n_layers);
+        std::memcpy(layers.data(), in, h.n_layers * sizeof(randes_layer_t)); in += h.n_layers * sizeof(randes_layer_t);
+        std::vector<randes_group_t> groups(h.n_groups);
+        for (uint32_t g = 0; g < h.n_groups; ++g) { std::memcpy(&groups[g].flags, in, sizeof(uint32_t)); in += sizeof(uint32_t); }
+        std::vector<uint32_t> ids(h.n_tasks);
+        std::vector<uint64_t> seeds(h.n_tasks);
+        std::memcpy(ids.data(), in, h.n_tasks * sizeof(uint32_t)); in += h.n_tasks * sizeof(uint32_t);
+        std::memcpy(seeds.data(), in, h.n_tasks * sizeof(uint64_t));
+        return randes_plan(layers.data(), h.n_layers, groups.data(), h.n_groups, static_cast<randes_dtype_t>(h.storage),
+                           static_cast<randes_dtype_t>(h.m_dtype), ids.data(), seeds.data(), h.n_tasks,
+                           std::max(max_tasks, std::max(1u, h.n_tasks)), dev_workspace, dev_workspace_bytes, stream, out_plan);
+    });
+}
+
 int randes_task_tables(const randes_plan_t* plan, uint32_t task_id, uint32_t* src_of_slot, uint32_t* slot_of_pos)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");

@@ -96,6 +96,10 @@ def lib():
         L.randes_remove_model.restype = ctypes.c_int
         L.randes_retrieve.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
         L.randes_retrieve.restype = ctypes.c_int
+        L.randes_plan_serialize.argtypes = [vp, vp, sz]
+        L.randes_plan_serialize.restype = sz
+        L.randes_plan_deserialize.argtypes = [vp, sz, u32, vp, sz, vp, ctypes.POINTER(vp)]
+        L.randes_plan_deserialize.restype = ctypes.c_int
         L.randes_delta_gram_scratch_bytes.argtypes = [vp]
         L.randes_delta_gram_scratch_bytes.restype = sz
         L.randes_delta_gram.argtypes = [vp, vp, vp, vp, vp, sz, vp]
@@ -115,7 +119,7 @@ def lib():
 EXPORTS = [
     "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
-    "randes_task_tables", "randes_compress", "randes_add_model", "randes_remove_model",
+    "randes_task_tables", "randes_plan_serialize", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_remove_model",
     "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_retrieve_batch", "randes_retrieve_static", "randes_launch_count", "randes_last_error",
 ]
 
@@ -151,6 +155,26 @@ def randes_plan(layers, n_layers, groups, n_groups, storage_dtype, m_dtype, task
     _check(lib().randes_plan(_addr(layers), n_layers, _addr(groups), n_groups, storage_dtype, m_dtype,
                              _addr(task_ids), _addr(seeds), n_tasks, max_tasks, _addr(dev_workspace),
                              dev_workspace_bytes, stream, ctypes.byref(out)))
+    return out.value
+
+
+def randes_plan_serialize(plan) -> bytes:
+    """The plan's shapes, flags, element types and (id, seed) pairs as a self-contained blob."""
+    n = int(lib().randes_plan_serialize(plan, None, 0))
+    if n == 0:
+        raise RandesError(INVALID_ARGUMENT, randes_last_error())
+    buf = ctypes.create_string_buffer(n)
+    if int(lib().randes_plan_serialize(plan, ctypes.addressof(buf), n)) != n:
+        raise RandesError(INVALID_ARGUMENT, randes_last_error())
+    return buf.raw
+
+
+def randes_plan_deserialize(blob: bytes, max_tasks: int = 0, dev_workspace=None, dev_workspace_bytes: int = 0, stream=None) -> int:
+    """A plan handle rebuilt from randes_plan_serialize's blob (host-only without a workspace)."""
+    out = ctypes.c_void_p()
+    buf = ctypes.create_string_buffer(blob, len(blob))
+    _check(lib().randes_plan_deserialize(ctypes.addressof(buf), len(blob), max_tasks, _addr(dev_workspace), dev_workspace_bytes,
+                                         stream, ctypes.byref(out)))
     return out.value
 
 

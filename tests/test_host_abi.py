@@ -114,6 +114,32 @@ def test_workspace_size_grows_with_capacity_and_rejects_bad_input():
     assert randes.randes_plan_workspace_bytes(None, 3, 4) == 0
 
 
+def test_plan_round_trips_through_its_serialized_form():
+    w = wl.gpt2_small()
+    gflags = list(w.gflags)
+    gflags[2] |= randes.SKIP(2)
+    p = randes.Plan(w.rows, w.cols, w.group, gflags, storage=w.storage, task_ids=[3, 0, 9], seeds=[2**63 + 1, 42, 7],
+                    host_only=True, m_dtype=randes.BF16)
+    blob = randes.randes_plan_serialize(p.handle)
+    q = randes.randes_plan_deserialize(blob)
+    try:
+        assert randes.randes_num_layers(q) == w.n_layers and randes.randes_num_tasks(q) == 3
+        assert randes.randes_superposition_bytes(q) == p.m_bytes
+        L = w.n_layers
+        for t in (3, 0, 9):
+            a = (ctypes.c_uint32 * L)(); b = (ctypes.c_uint32 * L)()
+            assert randes.lib().randes_task_tables(q, t, ctypes.addressof(a), ctypes.addressof(b)) == 0
+            assert (list(a), list(b)) == p.task_tables(t)
+        assert randes.randes_plan_serialize(q) == blob
+    finally:
+        randes.randes_plan_destroy(q)
+    for bad in (blob[:20], b"\0" * len(blob), blob[:-8]):
+        with pytest.raises(randes.RandesError) as e:
+            randes.randes_plan_deserialize(bad)
+        assert e.value.code == randes.INVALID_ARGUMENT
+    p.close()
+
+
 def _expect(code, fn):
     with pytest.raises(randes.RandesError) as e:
         fn()

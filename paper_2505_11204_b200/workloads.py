@@ -254,6 +254,25 @@ def subset(w: Workload, layers: Sequence[int], name: Optional[str] = None) -> Wo
     return out
 
 
+def row_slice(w: Workload, part: int, parts: int) -> Tuple[Workload, List[Tuple[int, int]]]:
+    """The workload one of ``parts`` devices holds when every layer is cut into row slices.
+
+    Returns the sliced workload (same layers, groups, flags, tasks and seeds; fewer rows)
+    and, per layer, the (first row, one past last row) it covers.  The transforms move
+    data across layers and flip by column, never across rows, so each slice can be
+    compressed and retrieved on its own: no exchange between devices is needed.
+    """
+    bounds = []
+    out = Workload(**{**w.__dict__})
+    out.rows = []
+    for r in w.rows:
+        lo, hi = (r * part) // parts, (r * (part + 1)) // parts
+        bounds.append((lo, hi))
+        out.rows.append(hi - lo)
+    out.name = "%s:rows %d/%d" % (w.name, part, parts)
+    return out, bounds
+
+
 CONFIGS = {
     0: toy,
     1: vit_b32,

@@ -378,6 +378,27 @@ def test_random_plans():
         run_full_cycle(w, out_dtypes=(int(rng.integers(0, 2)),), lam=float(rng.choice([0.1, 0.3, 1.0, 2.0])))
 
 
+def test_row_slices_shard_without_exchange():
+    # what each of several GPUs would hold under row-slice sharding, run here one slice after the other
+    w = make_workload([(37, 256, 3), (1, 256, 3), (50, 132, 2)], n_tasks=3)
+    base, tasks = wl.model_set(w)
+    M_ref = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, base, tasks)
+    out_ref = ro.retrieve(w.spec, w.storage, wl.F32, 2, w.seeds[2], w.lam, base, M_ref)
+    parts = 2
+    for part in range(parts):
+        ws, bounds = wl.row_slice(w, part, parts)
+        cut = lambda model: [np.ascontiguousarray(a[lo:hi]) for a, (lo, hi) in zip(model, bounds)]
+        plan = randes.Plan.from_workload(ws)
+        d_base = model_to_dev(cut(base))
+        M = plan.compress(d_base, [model_to_dev(cut(t)) for t in tasks])
+        out = plan.retrieve(2, w.lam, d_base, M)
+        for l, (lo, hi) in enumerate(bounds):
+            if hi > lo:
+                assert_bits_equal(from_dev(plan.slot(M, l)), M_ref[l][lo:hi], "slice %d of M, slot %d" % (part, l))
+                assert_bits_equal(from_dev(out[l]), out_ref[l][lo:hi], "slice %d of the retrieved model, layer %d" % (part, l))
+        plan.close()
+
+
 def test_gpu_argument_validation():
     import torch
 

@@ -85,3 +85,25 @@ def test_workload_parameter_counts():
         w = wl.CONFIGS[k]()
         assert (w.n_params, w.n_layers, len(w.gflags)) == (P, L, G), w.name
     assert len(wl.flan_t5_lora_targets(wl.flan_t5_base())) == 72
+
+
+def test_row_slices_of_every_layer_are_independent_problems():
+    """Sharding by row slices needs no collective: the oracle on each slice equals the slice of the oracle."""
+    import numpy as np
+
+    from oracle import randes_oracle as ro
+    from paper_2505_11204_b200 import workloads as wl
+
+    w = wl.subset(wl.toy(n_tasks=3, width=40, n_blocks=5), list(range(10)))
+    w.rows = [7 if r > 1 else 1 for r in w.rows]           # odd row counts: uneven slices, vectors stay whole on part 0
+    base, tasks = wl.model_set(w)
+    M = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, base, tasks)
+    out = ro.retrieve(w.spec, w.storage, wl.F32, 1, w.seeds[1], 0.3, base, M)
+    parts = 3
+    for part in range(parts):
+        ws, bounds = wl.row_slice(w, part, parts)
+        cut = lambda model: [np.ascontiguousarray(a[lo:hi]) for a, (lo, hi) in zip(model, bounds)]
+        Ms = ro.compress(ws.spec, ws.storage, ws.task_ids, ws.seeds, cut(base), [cut(t) for t in tasks])
+        outs = ro.retrieve(ws.spec, ws.storage, wl.F32, 1, ws.seeds[1], 0.3, cut(base), Ms)
+        for l, (lo, hi) in enumerate(bounds):
+            assert np.array_equal(Ms[l], M[l][lo:hi]) and np.array_equal(outs[l], out[l][lo:hi])

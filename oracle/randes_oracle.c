@@ -337,15 +337,14 @@ static ro_spec_t make_spec(uint32_t n_layers, const uint32_t *rows, const uint32
 }
 
 /*
- * compress (Section 4, first display; Section 4.4 first display):
- *   M = sum_{i in given order} T_i(W_i - W_0), every slot started from +0.0f.
- * tasks is a flattened [n_tasks][n_layers] array of host pointers.
+ * The sum of several transformed deltas, either from +0.0f (compress) or on top of
+ * what M already holds (adding several models at once).
  */
-int ro_compress(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
-                const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
-                int dtype, int m_dtype, uint32_t n_tasks, const uint32_t *task_ids, const uint64_t *seeds,
-                const void *const *base, const void *const *tasks,
-                void *const *M, const uint8_t *slot_mask)
+static int sum_models(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+                      const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
+                      int dtype, int m_dtype, int from_m, uint32_t n_tasks, const uint32_t *task_ids,
+                      const uint64_t *seeds, const void *const *base, const void *const *tasks,
+                      void *const *M, const uint8_t *slot_mask)
 {
     ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
     int rc = spec_check(&s);
@@ -362,7 +361,8 @@ int ro_compress(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
             acc[l] = malloc(sizeof(float) * (n ? n : 1));
             if (!acc[l]) { rc = -1; goto done; }
         }
-        for (size_t e = 0; e < n; ++e) ((float *)acc[l])[e] = 0.0f;
+        for (size_t e = 0; e < n; ++e)
+            ((float *)acc[l])[e] = from_m ? load_m(M[l], m_dtype, e) : 0.0f;
     }
     for (uint32_t i = 0; i < n_tasks && !rc; ++i)
         rc = accumulate_one(&s, dtype, RO_F32, +1, task_ids[i], seeds[i], base,
@@ -378,6 +378,37 @@ done:
         for (uint32_t l = 0; l < n_layers; ++l) free(acc[l]);
     free(acc);
     return rc;
+}
+
+/*
+ * compress (Section 4, first display; Section 4.4 first display):
+ *   M = sum_{i in given order} T_i(W_i - W_0), every slot started from +0.0f.
+ * tasks is a flattened [n_tasks][n_layers] array of host pointers.
+ */
+int ro_compress(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+                const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
+                int dtype, int m_dtype, uint32_t n_tasks, const uint32_t *task_ids, const uint64_t *seeds,
+                const void *const *base, const void *const *tasks,
+                void *const *M, const uint8_t *slot_mask)
+{
+    return sum_models(n_layers, rows, cols, group, n_groups, gflags, dtype, m_dtype, 0, n_tasks, task_ids, seeds,
+                      base, tasks, M, slot_mask);
+}
+
+/*
+ * Several models added in one step (Section 5.7, the hot swap applied to a set):
+ *   M <- M + T_a(d_a) + T_b(d_b) + ...   summed in fp32 in the given order, starting from M.
+ * With an fp32 M this is what the same ro_add_model calls give one after the other; a bf16 M
+ * is widened once, summed in fp32 and rounded once at the end.
+ */
+int ro_add_models(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+                  const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
+                  int dtype, int m_dtype, uint32_t n_tasks, const uint32_t *task_ids, const uint64_t *seeds,
+                  const void *const *base, const void *const *tasks,
+                  void *const *M, const uint8_t *slot_mask)
+{
+    return sum_models(n_layers, rows, cols, group, n_groups, gflags, dtype, m_dtype, 1, n_tasks, task_ids, seeds,
+                      base, tasks, M, slot_mask);
 }
 
 /* Model hot swapping (Section 5.7): M <- M + T_j(d_j)  /  M <- M - T_j(d_j). */

@@ -71,6 +71,7 @@ def _load():
         lib.ro_task_tables.restype = ctypes.c_int
         lib.ro_compress.restype = ctypes.c_int
         lib.ro_add_model.restype = ctypes.c_int
+        lib.ro_add_models.restype = ctypes.c_int
         lib.ro_remove_model.restype = ctypes.c_int
         lib.ro_retrieve.restype = ctypes.c_int
         lib.ro_delta_gram.restype = ctypes.c_int
@@ -191,11 +192,7 @@ def new_superposition(spec, slots=None, m_dtype: int = F32) -> List[np.ndarray]:
             for l, (r, c) in enumerate(zip(spec[0], spec[1]))]
 
 
-def compress(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
-             base: Optional[Sequence[np.ndarray]], tasks: Sequence[Sequence[np.ndarray]],
-             slots=None, M: Optional[List[np.ndarray]] = None, m_dtype: int = F32) -> List[np.ndarray]:
-    """M = sum_i T_i(W_i - W_0) in the given task order.  base=None: tasks hold deltas.
-    m_dtype=BF16: the fp32 sum is rounded once to bf16 bit patterns."""
+def _sum_models(fn_name, spec, dtype, task_ids, seeds, base, tasks, slots, M, m_dtype):
     lib = _load()
     sargs, keep = _spec_args(spec)
     L = keep[0].size
@@ -214,11 +211,27 @@ def compress(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
     mptr, mkeep = _mask(slots, L)
     p = ctypes.c_void_p
     base_pa = _ptr_array(base) if base is not None else None
-    rc = lib.ro_compress(*sargs, ctypes.c_int(dtype), ctypes.c_int(m_dtype), ctypes.c_uint32(K), p(ids.ctypes.data),
-                         p(sd.ctypes.data), base_pa, _ptr_array(flat), _ptr_array(M), mptr)
+    rc = getattr(lib, fn_name)(*sargs, ctypes.c_int(dtype), ctypes.c_int(m_dtype), ctypes.c_uint32(K), p(ids.ctypes.data),
+                               p(sd.ctypes.data), base_pa, _ptr_array(flat), _ptr_array(M), mptr)
     if rc:
-        raise ValueError("ro_compress failed: %d" % rc)
+        raise ValueError("%s failed: %d" % (fn_name, rc))
     return M
+
+
+def compress(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
+             base: Optional[Sequence[np.ndarray]], tasks: Sequence[Sequence[np.ndarray]],
+             slots=None, M: Optional[List[np.ndarray]] = None, m_dtype: int = F32) -> List[np.ndarray]:
+    """M = sum_i T_i(W_i - W_0) in the given task order.  base=None: tasks hold deltas.
+    m_dtype=BF16: the fp32 sum is rounded once to bf16 bit patterns."""
+    return _sum_models("ro_compress", spec, dtype, task_ids, seeds, base, tasks, slots, M, m_dtype)
+
+
+def add_models(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],
+               base: Optional[Sequence[np.ndarray]], tasks: Sequence[Sequence[np.ndarray]], M: List[np.ndarray],
+               slots=None, m_dtype: int = F32) -> List[np.ndarray]:
+    """M <- M + sum_i T_i(W_i - W_0), in place: several models added in one step (Section 5.7).  The sum runs in
+    fp32 from M's values in the given order; a bf16 M is rounded once, at the end."""
+    return _sum_models("ro_add_models", spec, dtype, task_ids, seeds, base, tasks, slots, M, m_dtype)
 
 
 def delta_gram(spec, dtype: int, task_ids: Sequence[int], seeds: Sequence[int],

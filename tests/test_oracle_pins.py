@@ -486,6 +486,47 @@ def test_add_remove_on_gaussian_inputs_within_one_rounding():
         assert np.all(np.abs(a - b) <= 2.0 ** -23 * (np.abs(b) + xx))
 
 
+def test_adding_several_models_at_once_matches_dense_matrices_and_left_to_right_sums():
+    # Section 5.7 applied to a set of models: M <- M + T_a d_a + T_b d_b + ..., in the given order
+    rng = np.random.default_rng(23)
+    spec = tiny_spec(SHUFFLE | FLIP)
+    base = rand_model(spec, rng, dyadic=True)
+    tasks = [rand_model(spec, rng, dyadic=True) for _ in range(5)]
+    ids, seeds = [4, 0, 8, 2, 6], [40, 41, 2**35, 43, 44]
+    M = ro.compress(spec, ro.F32, ids[:2], seeds[:2], base, tasks[:2])
+    M_before = flat(M)
+    ro.add_models(spec, ro.F32, ids[2:], seeds[2:], base, tasks[2:], M)
+    dense = sum(dense_transform(spec, seeds[i], ids[i])[0] @ (flat(tasks[i]) - flat(base)) for i in range(2, 5))
+    assert np.array_equal(flat(M), M_before + dense)              # exact on the dyadic grid
+    M_all = ro.compress(spec, ro.F32, ids, seeds, base, tasks)
+    assert np.array_equal(flat(M), flat(M_all))
+    # Gaussian inputs: one fp32 rounding per term, left to right, starting from M
+    base = rand_model(spec, rng, 0.02)
+    tasks = [[b + d for b, d in zip(base, rand_model(spec, rng, 1e-3))] for _ in range(4)]
+    M = ro.compress(spec, ro.F32, [1], [5], base, tasks[:1])
+    terms = [ro.compress(spec, ro.F32, [i], [s], base, [t]) for i, s, t in zip([2, 3, 9], [6, 7, 8], tasks[1:])]
+    want = [m.copy() for m in M]
+    for x in terms:
+        want = [(w + xx).astype(np.float32) for w, xx in zip(want, x)]
+    ro.add_models(spec, ro.F32, [2, 3, 9], [6, 7, 8], base, tasks[1:], M)
+    assert all(np.array_equal(a, b) for a, b in zip(M, want))
+    # a bf16 M is widened once, summed in fp32 and rounded once: not what three separate adds give
+    M16 = ro.compress(spec, ro.F32, [1], [5], base, tasks[:1], m_dtype=ro.BF16)
+    want = [wl.bf16_bits_to_f32(m) for m in M16]
+    for x in terms:
+        want = [(w + xx).astype(np.float32) for w, xx in zip(want, x)]
+    one_by_one = [m.copy() for m in M16]
+    for i, s_, t in zip([2, 3, 9], [6, 7, 8], tasks[1:]):
+        ro.add_model(spec, ro.F32, i, s_, base, t, one_by_one, m_dtype=ro.BF16)
+    ro.add_models(spec, ro.F32, [2, 3, 9], [6, 7, 8], base, tasks[1:], M16, m_dtype=ro.BF16)
+    assert all(np.array_equal(a, wl.to_bf16_bits(b)) for a, b in zip(M16, want))
+    assert any(not np.array_equal(a, b) for a, b in zip(M16, one_by_one))
+    # an empty set leaves M alone
+    keep = [m.copy() for m in M]
+    ro.add_models(spec, ro.F32, [], [], base, [], M)
+    assert all(np.array_equal(a, b) for a, b in zip(M, keep))
+
+
 # --------------------------------------------------------------------------- decorrelation
 def test_sign_flip_decorrelates_with_the_predicted_variance():
     """For one m x n layer and tasks i != j: <A D_i, B D_j> = sum_c eps_c g_c with

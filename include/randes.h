@@ -205,6 +205,24 @@ int randes_remove_model(randes_plan_t* plan, uint32_t task_id,
                         const void* const* base, const void* const* task, void* M, void* stream);
 
 /*
+ * Several models added in one pass over M (Section 5.7 applied to a set):
+ *   M <- M + T_a(W_a - W_0) + T_b(W_b - W_0) + ...      in the order given,
+ * each term rounded once in fp32, starting from M's values; the tasks are
+ * registered at the end of the summation order, in that order.  With an fp32
+ * superposition the result equals, bit for bit, n_tasks calls of
+ * randes_add_model, but M is read and written once instead of n_tasks times.
+ * A bf16 superposition is widened once and rounded once, at the end (so the
+ * result may differ in the last bit from separate adds, which round each time);
+ * it takes at most 32 models per call.
+ *   task_ids[n_tasks], seeds[n_tasks]   new, distinct ids; n_tasks may be 0 (nothing happens)
+ *   base[n_layers] or NULL; tasks[n_tasks * n_layers] as for randes_compress
+ * Either every model is added or, on error, none.  One kernel launch.
+ * Errors: DUPLICATE_TASK, CAPACITY, INVALID_ARGUMENT, MISALIGNED, CUDA_ERROR.
+ */
+int randes_add_models(randes_plan_t* plan, const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
+                      const void* const* base, const void* const* tasks, void* M, void* stream);
+
+/*
  * retrieve (Section 4, second display; Section 4.4, second display):
  *   out[p][r,c] = fma(lambda, s_t(l,c) * M[l][r,c], W_0[p][r,c]),  l = sigma_t^-1(p)
  * written as out_dtype (fp32, or bf16 rounded to nearest even).

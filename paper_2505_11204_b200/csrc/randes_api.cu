@@ -652,6 +652,50 @@ static int randes_add_model_impl(randes_plan_t* plan, uint32_t task_id, uint64_t
     return RANDES_OK;
 }
 
+static int randes_add_models_impl(randes_plan_t* plan, const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
+                                  const void* const* base, const void* const* tasks, void* M, void* stream)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
+    int rc;
+    if ((rc = check_m(M))) return rc;
+    if (n_tasks == 0) return RANDES_OK;
+    if (!task_ids || !seeds || !tasks) return fail(RANDES_INVALID_ARGUMENT, "task_ids / seeds / tasks is NULL");
+    for (uint32_t i = 0; i < n_tasks; ++i) {
+        if (find_task(*plan, task_ids[i]) >= 0) return fail(RANDES_DUPLICATE_TASK, "task id %u is already registered", task_ids[i]);
+        for (uint32_t j = 0; j < i; ++j)
+            if (task_ids[i] == task_ids[j]) return fail(RANDES_DUPLICATE_TASK, "task id %u appears twice", task_ids[i]);
+    }
+    if (plan->tasks.size() + n_tasks > plan->max_tasks)
+        return fail(RANDES_CAPACITY, "plan holds %zu tasks, %u more exceed max_tasks = %u", plan->tasks.size(), n_tasks, plan->max_tasks);
+    // beyond kTaskChunk terms the kernel carries the partial sum through M, where a bf16 M would round it
+    if (plan->m_dtype == RANDES_BF16 && n_tasks > static_cast<uint32_t>(kTaskChunk))
+        return fail(RANDES_CAPACITY, "with a bf16 superposition at most %d models are added per call (got %u)", kTaskChunk, n_tasks);
+    const size_t es = elem_size(plan->storage);
+    if ((rc = check_ptrs(*plan, base, "base", es, true))) return rc;
+    for (uint32_t i = 0; i < n_tasks; ++i)
+        if ((rc = check_ptrs(*plan, tasks + static_cast<size_t>(i) * plan->n_layers, "tasks", es, false))) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t first = plan->tasks.size();
+    try {
+        for (uint32_t i = 0; i < n_tasks; ++i) {
+            TaskEntry t;
+            t.id = task_ids[i];
+            t.seed = seeds[i];
+            make_task_tables(*plan, t);
+            plan->tasks.push_back(std::move(t));
+        }
+    } catch (const std::bad_alloc&) {
+        plan->tasks.resize(first);
+        return fail(RANDES_OUT_OF_MEMORY, "host allocation failed");
+    }
+    if ((rc = upload_task_rows(*plan, first, s)) || (rc = run_accumulate(*plan, first, n_tasks, true, false, base, tasks, M, s))) {
+        plan->tasks.resize(first);
+        return rc;
+    }
+    return RANDES_OK;
+}
+
 static int randes_remove_model_impl(randes_plan_t* plan, uint32_t task_id, const void* const* base, const void* const* task,
                         void* M, void* stream)
 {
@@ -872,6 +916,12 @@ int randes_add_model(randes_plan_t* plan, uint32_t task_id, uint64_t seed, const
                      const void* const* task, void* M, void* stream)
 {
     return guarded([&] { return randes_add_model_impl(plan, task_id, seed, base, task, M, stream); });
+}
+
+int randes_add_models(randes_plan_t* plan, const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
+                      const void* const* base, const void* const* tasks, void* M, void* stream)
+{
+    return guarded([&] { return randes_add_models_impl(plan, task_ids, seeds, n_tasks, base, tasks, M, stream); });
 }
 
 int randes_remove_model(randes_plan_t* plan, uint32_t task_id, const void* const* base, const void* const* task,

@@ -295,7 +295,10 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
                         MTile<MT, CPL>::unpack(reinterpret_cast<const uint4(&)[(G::kMBytes + 15) / 16]>(m_next[u]), mv);
                         have = true;
                     } else if (init_plain) {
+                        // a sum that starts from M (several models added at once; a later chunk of a
+                        // long compress): the next row group's M tile is pulled into L2 meanwhile
                         MTl::load(mp + off_c + u * row_stride, mv);
+                        if (left_c > U + u) prefetch_l2(mp + off_c + (U + u) * row_stride);
                         have = true;
                     }
                     if (have) {

@@ -92,6 +92,8 @@ def lib():
         L.randes_compress.restype = ctypes.c_int
         L.randes_add_model.argtypes = [vp, u32, u64, vp, vp, vp, vp]
         L.randes_add_model.restype = ctypes.c_int
+        L.randes_add_models.argtypes = [vp, vp, vp, u32, vp, vp, vp, vp]
+        L.randes_add_models.restype = ctypes.c_int
         L.randes_remove_model.argtypes = [vp, u32, vp, vp, vp, vp]
         L.randes_remove_model.restype = ctypes.c_int
         L.randes_retrieve.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
@@ -119,7 +121,7 @@ def lib():
 EXPORTS = [
     "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
-    "randes_task_tables", "randes_plan_serialize", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_remove_model",
+    "randes_task_tables", "randes_plan_serialize", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_add_models", "randes_remove_model",
     "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_retrieve_batch", "randes_retrieve_static", "randes_launch_count", "randes_last_error",
 ]
 
@@ -204,6 +206,14 @@ def randes_compress(plan, base, tasks, M, stream) -> None:
 
 def randes_add_model(plan, task_id, seed, base, task, M, stream) -> None:
     _check(lib().randes_add_model(plan, task_id, seed, _addr(base), _addr(task), _addr(M), stream))
+
+
+def randes_add_models(plan, task_ids, seeds, base, tasks, M, stream) -> None:
+    """Several models added in one pass over M; ``tasks`` holds n_tasks * n_layers pointers, task-major."""
+    n = len(task_ids)
+    ids = (ctypes.c_uint32 * max(n, 1))(*[int(t) for t in task_ids])
+    sds = (ctypes.c_uint64 * max(n, 1))(*[int(t) for t in seeds])
+    _check(lib().randes_add_models(plan, ctypes.addressof(ids), ctypes.addressof(sds), n, _addr(base), _addr(tasks), _addr(M), stream))
 
 
 def randes_remove_model(plan, task_id, base, task, M, stream) -> None:
@@ -390,6 +400,10 @@ class Plan:
 
     def add_model(self, task_id: int, seed: int, base, task, M):
         randes_add_model(self.handle, task_id, seed, _as_ptrs(base), _as_ptrs(task), M, self._stream())
+        return M
+
+    def add_models(self, task_ids, seeds, base, tasks, M):
+        randes_add_models(self.handle, task_ids, seeds, _as_ptrs(base), _as_ptrs(tasks), M, self._stream())
         return M
 
     def remove_model(self, task_id: int, base, task, M):

@@ -1,6 +1,6 @@
 """Full-size parity on the ViT-L/14-shaped set (304 M parameters, K = 20), in the launch
 configuration the benchmark times: compress all 20, a retrieve sweep over all tasks, then a
-streaming add / remove of further models.
+streaming add / remove of further models, one by one and all in one pass.
 
 The oracle cannot redo 26 models x 304 M parameters in seconds, so it computes whole sampled
 slots of M (one or two of every kind of tensor) and the layers that those slots feed at
@@ -140,6 +140,15 @@ def run_full_size(storage, n_swap):
         randes.randes_remove_model(plan.handle, t, p_base, randes.ptr_array(d_tasks[t]), M, sh)
         ro.remove_model(w.spec, storage, t, s, base_h, tasks_h[t], M_ref, slots=slots)
         check_m("remove %d" % t)
+    if len(swap_ids) > 1:
+        # the same models again, now in one pass over M
+        randes.randes_add_models(plan.handle, swap_ids, swap_seeds, p_base, randes.ptr_array([d_tasks[t] for t in swap_ids]), M, sh)
+        ro.add_models(w.spec, storage, swap_ids, swap_seeds, base_h, [tasks_h[t] for t in swap_ids], M_ref, slots=slots)
+        check_m("add_models")
+        for t, s in zip(swap_ids, swap_seeds):
+            randes.randes_remove_model(plan.handle, t, p_base, randes.ptr_array(d_tasks[t]), M, sh)
+            ro.remove_model(w.spec, storage, t, s, base_h, tasks_h[t], M_ref, slots=slots)
+        check_m("removes after add_models")
     check_retrieve(ids[7], seeds[7], "after removes")
     # properties that hold at any size: M is finite everywhere and no slot was left untouched
     assert bool(torch.isfinite(M).all())

@@ -298,6 +298,56 @@ def test_delta_gram_matches_oracle(storage):
     plan.close()
 
 
+@pytest.mark.parametrize("storage,m_dtype,n_new", [(wl.F32, wl.F32, 3), (wl.F32, wl.F32, 1), (wl.BF16, wl.F32, 5),
+                                                   (wl.F32, wl.BF16, 4), (wl.BF16, wl.BF16, 2), (wl.F32, wl.F32, 37)])
+def test_adding_several_models_in_one_pass(storage, m_dtype, n_new):
+    """M <- M + sum of the new models' transformed deltas, one launch; with an fp32 M also equal to separate adds."""
+    import torch
+
+    shapes = RAGGED if n_new < 10 else [(19, 260, 3), (1, 4100, 2), (37, 12, 2), (5, 3, 3)]
+    w = make_workload(shapes, storage=storage, n_tasks=2)
+    new_ids = [10 + 3 * j for j in range(n_new)]
+    new_seeds = [1000 + j for j in range(n_new)]
+    base, tasks = wl.model_set(w, list(w.task_ids) + new_ids)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, max_tasks=2 + n_new, m_dtype=m_dtype)
+    M_dev = poison(plan.new_superposition())
+    plan.compress(d_base, d_tasks[:2], M_dev)
+    M_ref = ro.compress(w.spec, storage, w.task_ids, w.seeds, base, tasks[:2], m_dtype=m_dtype)
+    if m_dtype == wl.F32:
+        one_by_one = M_dev.clone()
+    plan.add_models(new_ids, new_seeds, d_base, d_tasks[2:], M_dev)
+    ro.add_models(w.spec, storage, new_ids, new_seeds, base, tasks[2:], M_ref, m_dtype=m_dtype)
+    check_superposition(plan, M_dev, M_ref, "add_models")
+    assert plan.task_list() == (list(w.task_ids) + new_ids, list(w.seeds) + new_seeds)
+    # the new tasks are retrievable and removable like any other
+    t, s_ = new_ids[-1], new_seeds[-1]
+    out = plan.retrieve(t, 0.3, d_base, M_dev)
+    check_model(out, ro.retrieve(w.spec, storage, wl.F32, t, s_, 0.3, base, M_ref, m_dtype=m_dtype), "retrieve of an added model")
+    if m_dtype == wl.F32:
+        other = randes.Plan.from_workload(w, max_tasks=2 + n_new)
+        for i, sd, dt in zip(new_ids, new_seeds, d_tasks[2:]):
+            other.add_model(i, sd, d_base, dt, one_by_one)
+        assert torch.equal(one_by_one.view(torch.int32), M_dev.view(torch.int32))
+        other.close()
+    # nothing is registered when the call is refused
+    before = plan.task_list()
+    with pytest.raises(randes.RandesError) as e:
+        plan.add_models([500, new_ids[0]], [1, 2], d_base, d_tasks[:2], M_dev)
+    assert e.value.code == randes.DUPLICATE_TASK
+    with pytest.raises(randes.RandesError) as e:
+        plan.add_models([500, 500], [1, 2], d_base, d_tasks[:2], M_dev)
+    assert e.value.code == randes.DUPLICATE_TASK
+    with pytest.raises(randes.RandesError) as e:
+        plan.add_models([500], [1], d_base, d_tasks[:1], M_dev)
+    assert e.value.code == randes.CAPACITY
+    plan.add_models([], [], d_base, [], M_dev)
+    assert plan.task_list() == before
+    check_superposition(plan, M_dev, M_ref, "after refused calls")
+    torch.cuda.synchronize()
+    plan.close()
+
+
 def test_empty_layers_and_degenerate_plans():
     import torch
 

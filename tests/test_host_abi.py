@@ -173,6 +173,7 @@ def test_plan_argument_validation():
     _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_retrieve(p.handle, 0, 1.0, randes.F32, arr, 256, arr, None))
     _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_add_model(p.handle, 5, 5, arr, arr, 256, None))
     _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_remove_model(p.handle, 0, arr, arr, 256, None))
+    _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_add_models(p.handle, [5, 6], [5, 6], arr, arr, 256, None))
     p.close()
 
 

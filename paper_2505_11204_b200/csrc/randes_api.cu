@@ -90,10 +90,10 @@ struct TaskEntry {
 };
 
 struct WorkspaceLayout {
-    size_t layers, units, tasks, src_of_slot, slot_of_pos, base_ptrs, out_ptrs, task_ptrs, total;
+    size_t layers, units, tasks, src_of_slot, slot_of_pos, base_ptrs, out_ptrs, task_ptrs, members, staged_units, total;
 };
 
-WorkspaceLayout layout_workspace(size_t n_layers, size_t n_units, size_t max_tasks)
+WorkspaceLayout layout_workspace(size_t n_layers, size_t n_units, size_t n_staged_units, size_t max_tasks)
 {
     WorkspaceLayout w;
     size_t off = 0;
@@ -106,6 +106,8 @@ WorkspaceLayout layout_workspace(size_t n_layers, size_t n_units, size_t max_tas
     w.base_ptrs = take(n_layers * sizeof(void*));
     w.out_ptrs = take(n_layers * sizeof(void*));
     w.task_ptrs = take(max_tasks * n_layers * sizeof(void*));
+    w.members = take(n_layers * sizeof(uint32_t));
+    w.staged_units = take(n_staged_units * sizeof(DevUnit));
     w.total = off;
     return w;
 }
@@ -113,7 +115,17 @@ WorkspaceLayout layout_workspace(size_t n_layers, size_t n_units, size_t max_tas
 // Units in group order; inside a group, all members at one (row block, column
 // chunk) are adjacent, so that tiles of W_0 which several slots read (under a
 // shuffle) are touched close together in time and stay in L2.
-void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, std::vector<DevUnit>& units)
+//
+// With `staged` (one flag per group) the flagged groups are cut into group units
+// instead: one unit = a few rows x one warp-wide column block of every member,
+// whose W_0 tiles the CTA stages in shared memory (`member_base[g]` = index of
+// the group's first entry in the member table).  `which` selects the groups that
+// are listed at all.  `per_group`, if given, receives the number of units of each
+// group (indexed by group id).
+enum { kAllGroups = 0, kStagedGroups = 1, kOtherGroups = 2 };
+void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, std::vector<DevUnit>& units,
+                 const std::vector<char>* staged = nullptr, const std::vector<uint32_t>* member_base = nullptr,
+                 int which = kAllGroups, std::vector<size_t>* per_group = nullptr)
 {
     const uint32_t wcols = cols_per_warp(storage);
     units.clear();
@@ -121,27 +133,74 @@ void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, s
     std::vector<uint32_t> members;
     for (uint32_t first = 0; first < n_layers; ++first) {
         if (done[first]) continue;
+        const uint32_t g = layers[first].group;
         members.clear();
         for (uint32_t l = first; l < n_layers; ++l)
-            if (!done[l] && layers[l].group == layers[first].group) { members.push_back(l); done[l] = 1; }
+            if (!done[l] && layers[l].group == g) { members.push_back(l); done[l] = 1; }
         const uint32_t rows = layers[first].rows, cols = layers[first].cols;
         if (rows == 0 || cols == 0) continue;
+        const bool is_staged = staged && (*staged)[g];
+        if ((which == kStagedGroups && !is_staged) || (which == kOtherGroups && is_staged)) continue;
+        const size_t before = units.size();
         const uint32_t nb = (cols + wcols - 1) / wcols;
-        uint32_t nbc = 1;
-        while (nbc < static_cast<uint32_t>(kWarpsPerCta) && nb % (nbc * 2) == 0) nbc *= 2;
-        const uint32_t rows_per_unit = kRowsPerWarp * (kWarpsPerCta / nbc);
-        for (uint32_t r0 = 0; r0 < rows; r0 += rows_per_unit)
-            for (uint32_t cb0 = 0; cb0 < nb; cb0 += nbc)
-                for (uint32_t l : members) {
+        if (is_staged) {
+            const uint32_t R = group_unit_rows(static_cast<uint32_t>(members.size()));
+            for (uint32_t r0 = 0; r0 < rows; r0 += R)
+                for (uint32_t cb0 = 0; cb0 < nb; ++cb0) {
                     DevUnit u;
-                    u.layer = l;
+                    u.layer = (*member_base)[g];
                     u.row0 = r0;
-                    u.nrows = std::min(rows_per_unit, rows - r0);
+                    u.nrows = std::min(R, rows - r0);
                     u.cb0 = static_cast<uint16_t>(cb0);
-                    u.nbc = static_cast<uint16_t>(nbc);
+                    u.nbc = 0;
                     units.push_back(u);
                 }
+        } else {
+            uint32_t nbc = 1;
+            while (nbc < static_cast<uint32_t>(kWarpsPerCta) && nb % (nbc * 2) == 0) nbc *= 2;
+            const uint32_t rows_per_unit = kRowsPerWarp * (kWarpsPerCta / nbc);
+            for (uint32_t r0 = 0; r0 < rows; r0 += rows_per_unit)
+                for (uint32_t cb0 = 0; cb0 < nb; cb0 += nbc)
+                    for (uint32_t l : members) {
+                        DevUnit u;
+                        u.layer = l;
+                        u.row0 = r0;
+                        u.nrows = std::min(rows_per_unit, rows - r0);
+                        u.cb0 = static_cast<uint16_t>(cb0);
+                        u.nbc = static_cast<uint16_t>(nbc);
+                        units.push_back(u);
+                    }
+        }
+        if (per_group) {
+            if (per_group->size() <= g) per_group->resize(g + 1, 0);
+            (*per_group)[g] += units.size() - before;
+        }
     }
+}
+
+// Could group g (of `size` members, `cols` wide) be cut into group units at all?
+bool group_fits_stash(size_t size, uint32_t cols, int storage)
+{
+    return size >= 2 && cols % cols_per_lane(storage) == 0 && group_unit_rows(static_cast<uint32_t>(size)) >= 1;
+}
+
+// Upper bound of the length of a unit list in which any subset of the groups is staged.
+size_t max_mixed_units(const randes_layer_t* layers, uint32_t n_layers, int storage)
+{
+    uint32_t n_groups = 0;
+    for (uint32_t l = 0; l < n_layers; ++l) n_groups = std::max(n_groups, layers[l].group + 1);
+    std::vector<size_t> size(n_groups, 0);
+    std::vector<uint32_t> cols(n_groups, 0), base(n_groups, 0);
+    for (uint32_t l = 0; l < n_layers; ++l) { ++size[layers[l].group]; cols[layers[l].group] = layers[l].cols; }
+    std::vector<char> staged(n_groups, 0);
+    for (uint32_t g = 0; g < n_groups; ++g) staged[g] = group_fits_stash(size[g], cols[g], storage);
+    std::vector<DevUnit> units;
+    std::vector<size_t> plain(n_groups, 0), mixed(n_groups, 0);
+    build_units(layers, n_layers, storage, units, nullptr, nullptr, kAllGroups, &plain);
+    build_units(layers, n_layers, storage, units, &staged, &base, kAllGroups, &mixed);
+    size_t total = 0;
+    for (uint32_t g = 0; g < n_groups; ++g) total += std::max(g < plain.size() ? plain[g] : 0, g < mixed.size() ? mixed[g] : 0);
+    return total;
 }
 
 int check_layers(const randes_layer_t* layers, uint32_t n_layers)
@@ -171,6 +230,13 @@ struct randes_plan_s {
     std::vector<std::vector<uint32_t>> members;   // per group, in layer order
     std::vector<DevLayer> dev_layers;
     std::vector<DevUnit> units;
+    // compress: the shuffled groups cut into group units (their W_0 tiles are staged in shared
+    // memory), the other groups as in `units`; both empty when no group qualifies.
+    // member table = layers of every group, group after group
+    std::vector<DevUnit> group_units, other_units;
+    std::vector<char> group_staged;
+    std::vector<uint32_t> member_table;
+    uint32_t max_staged_group = 0;
     std::vector<size_t> m_off_bytes;
     size_t m_bytes = 0;
     std::vector<TaskEntry> tasks;                 // summation order
@@ -320,6 +386,19 @@ int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_
     a.layers = p.dev<DevLayer>(p.lay.layers);
     a.units = p.dev<DevUnit>(p.lay.units);
     a.n_units = static_cast<uint32_t>(p.units.size());
+    // Compress from zero under a shuffle: the shuffled groups go to the group kernel, which needs W_0,
+    // all tasks in one chunk, room for its tables, and 16-byte aligned tensors in those groups.
+    bool staged = !init_from_m && n_rows >= 2 && n_rows <= static_cast<size_t>(kTaskChunk) && base != nullptr &&
+                  !p.group_units.empty() && compress_group_fits(p.storage, p.max_staged_group, static_cast<uint32_t>(n_rows));
+    for (uint32_t l = 0; staged && l < p.n_layers; ++l) {
+        if (!p.group_staged[p.layers[l].group]) continue;
+        staged = reinterpret_cast<uintptr_t>(base[l]) % 16 == 0;
+        for (size_t i = 0; staged && i < n_rows; ++i) staged = reinterpret_cast<uintptr_t>(task_ptrs[i * p.n_layers + l]) % 16 == 0;
+    }
+    if (staged) {
+        a.units = p.dev<DevUnit>(p.lay.staged_units);
+        a.n_units = static_cast<uint32_t>(p.other_units.size());
+    }
     a.n_layers = p.n_layers;
     a.src_of_slot = p.dev<uint32_t>(p.lay.src_of_slot) + first_row * p.n_layers;
     a.tasks = p.dev<DevTask>(p.lay.tasks) + first_row;
@@ -330,6 +409,23 @@ int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_
     a.base = p.dev<const void*>(p.lay.base_ptrs);
     a.task_ptrs = p.dev<const void*>(p.lay.task_ptrs);
     a.M = M;
+    if (staged) {
+        CompressGroupArgs g;
+        g.layers = a.layers;
+        g.units = p.dev<DevUnit>(p.lay.staged_units) + p.other_units.size();
+        g.n_units = static_cast<uint32_t>(p.group_units.size());
+        g.n_layers = p.n_layers;
+        g.src_of_slot = a.src_of_slot;
+        g.tasks = a.tasks;
+        g.n_tasks = a.n_tasks;
+        g.base = a.base;
+        g.task_ptrs = a.task_ptrs;
+        g.M = M;
+        g.members = p.dev<uint32_t>(p.lay.members);
+        const int e = launch_compress_groups(p.storage, p.m_dtype, g, p.max_staged_group, p.sm_count, s);
+        if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the group compress kernel");
+        ++g_launches;
+    }
     if (a.n_units == 0) return RANDES_OK;
     const int grid = std::min<int>(p.grid_acc[n_rows == 1], static_cast<int>(a.n_units));
     const int e = launch_accumulate(p.storage, p.m_dtype, a, grid, s);
@@ -367,7 +463,8 @@ size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_laye
     size_t n_units = units.size();
     build_units(layers, n_layers, RANDES_BF16, units);
     n_units = std::max(n_units, units.size());
-    return layout_workspace(n_layers, n_units, max_tasks).total;
+    const size_t n_staged = std::max(max_mixed_units(layers, n_layers, RANDES_F32), max_mixed_units(layers, n_layers, RANDES_BF16));
+    return layout_workspace(n_layers, n_units, n_staged, max_tasks).total;
 }
 
 int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_group_t* groups, uint32_t n_groups,
@@ -449,13 +546,35 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         }
         p->m_bytes = off;
         build_units(layers, n_layers, p->storage, p->units);
+        {
+            std::vector<uint32_t> member_base(n_groups, 0);
+            p->group_staged.assign(n_groups, 0);
+            bool any = false;
+            for (uint32_t g = 0; g < n_groups; ++g) {
+                const std::vector<uint32_t>& mem = p->members[g];
+                member_base[g] = static_cast<uint32_t>(p->member_table.size());
+                p->member_table.insert(p->member_table.end(), mem.begin(), mem.end());
+                if (mem.empty() || !group_fits_stash(mem.size(), layers[mem[0]].cols, p->storage)) continue;
+                bool shuffled = false;
+                for (uint32_t l : mem) shuffled = shuffled || (p->dev_layers[l].flags & kFlagShuffle);
+                p->group_staged[g] = shuffled;
+                any = any || shuffled;
+                if (shuffled) p->max_staged_group = std::max<uint32_t>(p->max_staged_group, static_cast<uint32_t>(mem.size()));
+            }
+            // fp32 weights only: with bf16 weights the row loop is bound by instruction issue (two
+            // elements to widen per 4 bytes), and the per-layer kernel was measured faster
+            if (any && p->storage == RANDES_F32) {
+                build_units(layers, n_layers, p->storage, p->group_units, &p->group_staged, &member_base, kStagedGroups);
+                build_units(layers, n_layers, p->storage, p->other_units, &p->group_staged, &member_base, kOtherGroups);
+            }
+        }
         p->tasks.resize(n_tasks);
         for (uint32_t i = 0; i < n_tasks; ++i) {
             p->tasks[i].id = task_ids[i];
             p->tasks[i].seed = seeds[i];
             make_task_tables(*p, p->tasks[i]);
         }
-        p->lay = layout_workspace(n_layers, p->units.size(), max_tasks);
+        p->lay = layout_workspace(n_layers, p->units.size(), p->group_units.size() + p->other_units.size(), max_tasks);
     } catch (const std::bad_alloc&) {
         delete p;
         return fail(RANDES_OUT_OF_MEMORY, "host allocation failed");
@@ -499,6 +618,20 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         if (e == cudaSuccess && !p->units.empty())
             e = cudaMemcpyAsync(p->ws + p->lay.units, p->units.data(), p->units.size() * sizeof(DevUnit),
                                 cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(p->ws + p->lay.members, p->member_table.data(), p->member_table.size() * sizeof(uint32_t),
+                                cudaMemcpyHostToDevice, s);
+        // [other units][group units]
+        if (e == cudaSuccess && !p->other_units.empty())
+            e = cudaMemcpyAsync(p->ws + p->lay.staged_units, p->other_units.data(), p->other_units.size() * sizeof(DevUnit),
+                                cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess && !p->group_units.empty())
+            e = cudaMemcpyAsync(p->dev<DevUnit>(p->lay.staged_units) + p->other_units.size(), p->group_units.data(),
+                                p->group_units.size() * sizeof(DevUnit), cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess && !p->group_units.empty()) {
+            const int ge = compress_group_prepare(p->storage, p->m_dtype);
+            if (ge) { delete p; return fail_cuda(static_cast<cudaError_t>(ge), "set-up of the group compress kernel"); }
+        }
         if (e != cudaSuccess) { delete p; return fail_cuda(e, "copy of plan tables"); }
         if ((rc = upload_task_rows(*p, 0, s))) { delete p; return rc; }
     }

@@ -1,0 +1,296 @@
+// Compress under a layer shuffle, one group of same-shape layers at a time.
+//
+//   M[l] = sum_i s_i(l, c) * ( W_i[sigma_i(l)] - W_0[sigma_i(l)] )        (Section 4, first display;
+//                                                                           Section 4.3 for sigma, 4.4 for s)
+//
+// Under a shuffle slot l needs W_0[sigma_i(l)] for every task i: each W_0 tile of a
+// group is wanted by every slot of the group and K times per slot.  A CTA therefore takes a
+// group unit -- a few rows x one warp-wide column block of EVERY member of the group --,
+// copies the W_0 tiles of all members into a shared-memory stash once, and resolves, for all
+// (slot, task) pairs of the unit at once and in parallel over its threads, the source tensor
+// sigma_i(l) and the Philox block of sign bits.  After that only the task tensors stream from
+// HBM, through a per-thread cp.async ring (each lane reads back only what it copied, so the
+// row loop needs no barrier), and W_0 and the signs come from shared memory.
+//
+// A warp takes (slot, block of kItemRows rows) items in turn and runs ONE software pipeline
+// over all its items: stage = one task x two rows.  Sums run in task order, every output
+// element is written by one thread: results are bit-reproducible and equal to the per-layer
+// kernel's.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <type_traits>
+
+#include "randes_device.cuh"
+#include "randes_internal.h"
+
+namespace randes {
+namespace {
+
+using namespace device;
+
+constexpr uint32_t kMaxGroup = kStashBytes / kStashTileBytes;   // members whose tiles fit the stash at one row each
+constexpr uint32_t kOffTableBytes = kMaxGroup * 8;
+
+__device__ __forceinline__ void sts_u64(uint32_t saddr, unsigned long long v)
+{
+    asm volatile("st.shared.u64 [%0], %1;" ::"r"(saddr), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long lds_u64(uint32_t saddr)
+{
+    unsigned long long v;
+    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(saddr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t saddr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
+    return v;
+}
+
+// Position of a warp in its sequence of stages: item -> row pair -> task.
+struct Cursor {
+    uint32_t item;      // (slot, row block) index inside the unit
+    uint32_t ms;        // member index of the slot
+    uint32_t row;       // first row of the current row pair, relative to the unit
+    uint32_t rows_left; // rows of the item from `row` on (1 or more)
+    uint32_t i;         // task
+};
+
+__device__ __forceinline__ void cursor_set(Cursor& c, uint32_t item, uint32_t n_chunks, uint32_t Rn)
+{
+    c.item = item;
+    c.ms = item / n_chunks;
+    const uint32_t chunk = item - c.ms * n_chunks;
+    c.row = chunk * kItemRows;
+    c.rows_left = min(kItemRows, Rn - c.row);
+    c.i = 0;
+}
+
+__device__ __forceinline__ void cursor_next(Cursor& c, uint32_t nt, uint32_t n_chunks, uint32_t Rn)
+{
+    if (++c.i < nt) return;
+    c.i = 0;
+    if (c.rows_left > 2) {
+        c.row += 2;
+        c.rows_left -= 2;
+    } else {
+        cursor_set(c, c.item + kWarpsPerCta, n_chunks, Rn);   // may run past the last item: never used then
+    }
+}
+
+template <typename ST, typename MT, int NSTAGE>
+__global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const CompressGroupArgs a, const uint32_t pair_cap)
+{
+    constexpr int CPL = Store<ST>::CPL;
+    constexpr int HB = CPL / 4;                          // Philox blocks under a warp-wide column block
+    constexpr uint32_t ES = sizeof(ST);
+    constexpr uint32_t kRingBytes = NSTAGE * 2 * kSlotBytes;
+    constexpr uint32_t kStageBytes = 2 * kSlotBytes;
+    typedef MTile<MT, CPL> MTl;
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_s = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
+    const uint32_t ring = smem_s + threadIdx.x * 16;
+    const uint32_t stash = smem_s + kRingBytes;
+    const uint32_t s_off = stash + kStashBytes;          // per member: first element of its slot in M
+    const uint32_t s_ptr = s_off + kOffTableBytes;       // per (slot, task): {W_i[sigma_i(l)], member index of sigma_i(l)}
+    const uint32_t s_blk = s_ptr + pair_cap * 16;        // per (slot, task): HB Philox blocks of sign bits
+    const uint32_t L = a.n_layers, nt = a.n_tasks;
+    // where this lane's sign bits sit inside a pair's blocks
+    const uint32_t sign_word = CPL == 4 ? (lane >> 3) * 4u : (lane >> 4) * 16u + ((lane & 15) >> 2) * 4u;
+    const uint32_t sign_shift = CPL == 4 ? (lane & 7) * 4u : (lane & 3) * 8u;
+    const uint32_t one = 0x3F800000u;
+
+    for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+        const DevUnit un = a.units[u];
+        const uint32_t* mem = a.members + un.layer;
+        const DevLayer l0 = a.layers[mem[0]];
+        const uint32_t G = l0.group_size, cols = l0.cols, Rn = un.nrows, row0 = un.row0;
+        const uint32_t c = (un.cb0 * 32u + lane) * CPL;
+        const bool lane_on = c < cols;
+
+        // ---- prologue, all threads: W_0 tiles of every member into the stash ...
+        if (lane_on) {
+            const uint32_t ntiles = G * Rn;
+            for (uint32_t q = warp; q < ntiles; q += kWarpsPerCta) {
+                const uint32_t m = q / Rn, r = q - m * Rn;
+                const char* pb = static_cast<const char*>(a.base[mem[m]]);
+                cp_async16(stash + q * kStashTileBytes + lane * 16, pb + (static_cast<size_t>(row0 + r) * cols + c) * ES);
+            }
+        }
+        cp_async_commit();
+        // ... and, per (slot, task) pair, the source tensor and the sign bits
+        const uint32_t npairs = G * nt;
+        for (uint32_t p = threadIdx.x; p < npairs; p += kThreadsPerCta) {
+            const uint32_t ms = p / nt, i = p - ms * nt;
+            const uint32_t slot = mem[ms];
+            const uint32_t fl = a.layers[slot].flags;
+            const uint32_t src = (fl & kFlagShuffle) ? a.src_of_slot[static_cast<size_t>(i) * L + slot] : slot;   // sigma_i(l)
+            const void* pw = a.task_ptrs[static_cast<size_t>(i) * L + src];
+            sts_ptrs(s_ptr + p * 16, pw, reinterpret_cast<const void*>(static_cast<uintptr_t>(a.layers[src].member)));
+            const DevTask tk = a.tasks[i];
+#pragma unroll
+            for (int h = 0; h < HB; ++h) {
+                uint4 blk = make_uint4(0, 0, 0, 0);
+                if (fl & kFlagFlip) blk = philox4x32_10(un.cb0 * HB + h, slot, kTagSign, tk.id, tk.key0, tk.key1);
+                sts128(s_blk + (p * HB + h) * 16, blk);
+            }
+        }
+        for (uint32_t ms = threadIdx.x; ms < G; ms += kThreadsPerCta) sts_u64(s_off + ms * 8, a.layers[mem[ms]].m_off);
+        cp_async_wait<0>();
+        __syncthreads();   // stash and tables are complete and visible to every warp
+
+        if (lane_on) {
+            const uint32_t n_chunks = (Rn + kItemRows - 1) / kItemRows;
+            const uint32_t n_items = G * n_chunks;
+            uint32_t N = 0;   // stages of this warp
+            for (uint32_t item = warp; item < n_items; item += kWarpsPerCta) {
+                const uint32_t chunk = item % n_chunks;
+                N += (min(kItemRows, Rn - chunk * kItemRows) + 1) / 2 * nt;
+            }
+            Cursor ci, cc;
+            cursor_set(ci, warp, n_chunks, Rn);
+            cc = ci;
+            uint32_t issued = 0, stage_i = ring, stage_c = ring;
+            const uint32_t ring_end = ring + kRingBytes;
+            const uint32_t stash_lane = stash + lane * 16;
+
+            auto issue = [&]() {
+                const char* pw = lds_ptr(s_ptr + (ci.ms * nt + ci.i) * 16);
+                const size_t off = (static_cast<size_t>(row0 + ci.row) * cols + c) * ES;
+                cp_async16(stage_i, pw + off);
+                if (ci.rows_left > 1) cp_async16(stage_i + kSlotBytes, pw + off + static_cast<size_t>(cols) * ES);
+                cursor_next(ci, nt, n_chunks, Rn);
+                stage_i += kStageBytes;
+                if (stage_i == ring_end) stage_i = ring;
+                ++issued;
+            };
+
+#pragma unroll
+            for (int s = 0; s < NSTAGE - 1; ++s) {
+                if (issued < N) issue();
+                cp_async_commit();
+            }
+            f32x2 acc[2][CPL / 2];
+            for (uint32_t it = 0; it < N; ++it) {
+                if (issued < N) issue();
+                cp_async_commit();
+                cp_async_wait<NSTAGE - 1>();   // all but the newest NSTAGE-1 groups have landed: stage_c is ready
+                if (cc.i == 0) {
+#pragma unroll
+                    for (int r = 0; r < 2; ++r)
+#pragma unroll
+                        for (int e = 0; e < CPL / 2; ++e) acc[r][e] = 0ull;
+                }
+                const uint32_t pair = cc.ms * nt + cc.i;
+                const uint32_t member = lds_u32(s_ptr + pair * 16 + 8);
+                const uint32_t bits = lds_u32(s_blk + pair * (HB * 16) + sign_word) >> sign_shift;
+                f32x2 sg[CPL / 2];   // +-1.0f per column
+#pragma unroll
+                for (int e = 0; e < CPL / 2; ++e)
+                    sg[e] = pack2(((bits << (31 - 2 * e)) & 0x80000000u) | one, ((bits << (30 - 2 * e)) & 0x80000000u) | one);
+                const uint32_t b0 = stash_lane + (member * Rn + cc.row) * kStashTileBytes;
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    if (r == 0 || cc.rows_left > 1) {
+                        f32x2 d[CPL / 2], b[CPL / 2];
+                        Store<ST>::widen2(lds128(stage_c + r * kSlotBytes), d);
+                        Store<ST>::widen2(lds128(b0 + r * kStashTileBytes), b);
+#pragma unroll
+                        for (int e = 0; e < CPL / 2; ++e) acc[r][e] = fma2(sub2(d[e], b[e]), sg[e], acc[r][e]);
+                    }
+                }
+                if (cc.i + 1 == nt) {
+                    MT* mp = static_cast<MT*>(a.M) + lds_u64(s_off + cc.ms * 8) + (static_cast<size_t>(row0 + cc.row) * cols + c);
+#pragma unroll
+                    for (int r = 0; r < 2; ++r) {
+                        if (r == 0 || cc.rows_left > 1) {
+                            float v[CPL];
+#pragma unroll
+                            for (int e = 0; e < CPL / 2; ++e) unpack2(acc[r][e], v[2 * e], v[2 * e + 1]);
+                            MTl::store(mp + static_cast<size_t>(r) * cols, v);
+                        }
+                    }
+                }
+                cursor_next(cc, nt, n_chunks, Rn);
+                stage_c += kStageBytes;
+                if (stage_c == ring_end) stage_c = ring;
+            }
+            cp_async_wait<0>();
+        }
+        __syncthreads();   // every warp is done with the stash and the tables before the next unit overwrites them
+    }
+}
+
+template <typename T> struct Tag { typedef T type; };
+template <typename F> int with_type(int dtype, F&& f) { return dtype == 0 ? f(Tag<float>{}) : f(Tag<bf16>{}); }
+template <typename F> int with_stages(int nstage, F&& f)
+{
+    return nstage >= 6 ? f(std::integral_constant<int, 6>{}) : (nstage == 5 ? f(std::integral_constant<int, 5>{}) : f(std::integral_constant<int, 4>{}));
+}
+
+constexpr size_t kMaxDynamicSmem = 227 * 1024;
+constexpr size_t kTwoCtaSmem = (228 * 1024 - 2 * 1024) / 2;   // two CTAs per SM, 1 KiB reserved for each
+
+size_t group_smem_bytes(int storage_dtype, int nstage, uint32_t pair_cap)
+{
+    const size_t hb = storage_dtype == 1 ? 2 : 1;
+    return static_cast<size_t>(nstage) * 2 * kSlotBytes + kStashBytes + kOffTableBytes + static_cast<size_t>(pair_cap) * 16 * (1 + hb);
+}
+
+}  // namespace
+
+int compress_group_prepare(int storage_dtype, int m_dtype)
+{
+    return with_type(storage_dtype, [&](auto st) {
+        return with_type(m_dtype, [&](auto mt) {
+            typedef typename decltype(st)::type ST;
+            typedef typename decltype(mt)::type MT;
+            cudaError_t e = cudaFuncSetAttribute(compress_group_kernel<ST, MT, 6>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynamicSmem));
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(compress_group_kernel<ST, MT, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynamicSmem));
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(compress_group_kernel<ST, MT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynamicSmem));
+            if (e != cudaSuccess) (void)cudaGetLastError();
+            return static_cast<int>(e);
+        });
+    });
+}
+
+bool compress_group_fits(int storage_dtype, uint32_t max_group, uint32_t n_tasks)
+{
+    return max_group >= 1 && max_group <= kMaxGroup && group_smem_bytes(storage_dtype, 4, max_group * n_tasks) <= kMaxDynamicSmem;
+}
+
+int launch_compress_groups(int storage_dtype, int m_dtype, const CompressGroupArgs& a, uint32_t max_group, int sm_count, void* stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint32_t pair_cap = max_group * a.n_tasks;
+    // the deepest ring that still leaves room for two CTAs per SM; failing that, the deepest ring with one
+    int nstage = 0;
+    for (int n = 6; n >= 4 && !nstage; --n)
+        if (group_smem_bytes(storage_dtype, n, pair_cap) <= kTwoCtaSmem) nstage = n;
+    for (int n = 6; n >= 4 && !nstage; --n)
+        if (group_smem_bytes(storage_dtype, n, pair_cap) <= kMaxDynamicSmem) nstage = n;
+    if (!nstage) return static_cast<int>(cudaErrorInvalidConfiguration);
+    const size_t smem = group_smem_bytes(storage_dtype, nstage, pair_cap);
+    return with_type(storage_dtype, [&](auto st) {
+        return with_type(m_dtype, [&](auto mt) {
+            return with_stages(nstage, [&](auto ns) {
+                typedef typename decltype(st)::type ST;
+                typedef typename decltype(mt)::type MT;
+                constexpr int NS = decltype(ns)::value;
+                int per_sm = 0;
+                cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_group_kernel<ST, MT, NS>, kThreadsPerCta, smem);
+                if (e != cudaSuccess) { (void)cudaGetLastError(); return static_cast<int>(e); }
+                if (per_sm <= 0) return static_cast<int>(cudaErrorInvalidConfiguration);
+                const int grid = static_cast<int>(std::min<uint64_t>(static_cast<uint64_t>(sm_count) * per_sm, a.n_units));
+                compress_group_kernel<ST, MT, NS><<<grid, kThreadsPerCta, smem, s>>>(a, pair_cap);
+                return static_cast<int>(cudaGetLastError());
+            });
+        });
+    });
+}
+
+}  // namespace randes

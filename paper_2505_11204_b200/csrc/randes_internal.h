@@ -46,6 +46,20 @@ struct DevUnit {
 };
 static_assert(sizeof(DevUnit) == 16, "DevUnit layout");
 
+// A group unit (nbc == 0) covers `nrows` rows x one warp-wide column block of EVERY member of a
+// shuffled group: the CTA first stashes the W_0 tiles of all members in shared memory, then its
+// warps sum the tasks' deltas slot by slot, subtracting W_0[sigma_i(l)] from the stash.  `layer`
+// is then the index of the group's first entry in the member table.
+constexpr uint32_t kStashTileBytes = 512;             // 32 lanes x 16 bytes
+constexpr uint32_t kStashBytes = 48 * 1024;
+constexpr uint32_t kItemRows = 4;                     // rows of one slot a warp sums in one go
+// rows per group unit for a group of G members (0: the group is too large for the stash)
+constexpr uint32_t group_unit_rows(uint32_t G)
+{
+    const uint32_t fit = G ? kStashBytes / kStashTileBytes / G : 0;
+    return fit >= 4 * kItemRows ? 4 * kItemRows : (fit >= kItemRows ? fit / kItemRows * kItemRows : fit);
+}
+
 struct DevTask {
     uint32_t id;
     uint32_t key0, key1;       // low / high half of the 64-bit seed
@@ -79,6 +93,21 @@ struct AccumulateArgs {
     const void* const* base;       // device array [n_layers]
     const void* const* task_ptrs;  // device array [n_tasks][n_layers]
     void* M;                       // fp32 or bf16 arena
+};
+
+// compress over group units (randes_group.cu)
+struct CompressGroupArgs {
+    const DevLayer* layers;
+    const DevUnit* units;          // group units only (nbc == 0; `layer` indexes `members`)
+    uint32_t n_units;
+    uint32_t n_layers;
+    const uint32_t* src_of_slot;   // rows of sigma, one per task to sum
+    const DevTask* tasks;
+    uint32_t n_tasks;              // 2 .. kTaskChunk
+    const void* const* base;       // device array [n_layers]
+    const void* const* task_ptrs;  // device array [n_tasks][n_layers]
+    void* M;
+    const uint32_t* members;       // layers of every group, group after group, in member order
 };
 
 struct RetrieveBatchArgs {
@@ -116,6 +145,10 @@ struct GramArgs {
 // Launchers (randes_kernels.cu).  Return a cudaError_t as int.
 int launch_retrieve(int storage_dtype, int out_dtype, int m_dtype, const RetrieveArgs& a, int grid, void* stream);
 int launch_accumulate(int storage_dtype, int m_dtype, const AccumulateArgs& a, int grid, void* stream);
+// randes_group.cu: compress over group units.  `max_group` = the largest staged group.
+int compress_group_prepare(int storage_dtype, int m_dtype);   // once per device: opts into the shared memory the kernel needs
+bool compress_group_fits(int storage_dtype, uint32_t max_group, uint32_t n_tasks);
+int launch_compress_groups(int storage_dtype, int m_dtype, const CompressGroupArgs& a, uint32_t max_group, int sm_count, void* stream);
 // Resident CTAs per SM of each kernel (for sizing persistent grids); 0 if the
 // kernels cannot run on the current device.  Also opts the kernels into the
 // dynamic shared memory they need: call once per device before launching.

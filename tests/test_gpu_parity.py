@@ -406,6 +406,17 @@ def test_thirty_two_tasks_exactly_and_wide_single_row():
     run_full_cycle(make_workload([(1, 100000, 1), (3, 4096, 2)], n_tasks=32), out_dtypes=(wl.F32,), extra_task=False)
 
 
+@pytest.mark.parametrize("n_tasks", [2, 5, 32])
+def test_large_and_partly_shuffled_groups(n_tasks):
+    """Compress of shuffled groups runs over group units (W_0 of all members staged in shared memory):
+    groups of 30, 48 and 50 members (3, 2 and 1 rows per unit), 97 members (too large: per-layer path),
+    a group where only every second member is shuffled, ragged rows and widths; 2 to 32 tasks (32 tasks
+    x 48 members exceed the tables that fit beside two resident CTAs)."""
+    shapes = [(9, 132, 30), (5, 256, 50), (3, 128, 97), (6, 260, 48), (11, 520, 7), (21, 128, 4), (2, 4, 24)]
+    flags = [S | F, S | F, S | F, S, S | F | randes.SKIP(2), S | F, S | F]
+    run_full_cycle(make_workload(shapes, flags=flags, n_tasks=n_tasks), out_dtypes=(wl.F32,), extra_task=False)
+
+
 def test_random_plans():
     """Seeded random models: shapes, group sizes, flags (shuffle / shift / flip / skip), task counts, ids,
     seeds and storage types drawn at random; every step of the path against the oracle."""

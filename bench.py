@@ -82,7 +82,7 @@ def kernel_source_hash():
     import hashlib
 
     h = hashlib.sha256()
-    for name in ("randes_kernels.cu", "randes_device.cuh"):
+    for name in ("randes_kernels.cu", "randes_group.cu", "randes_device.cuh"):
         with open(os.path.join(ROOT, "paper_2505_11204_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()
@@ -429,7 +429,7 @@ def run_ours(args):
     # dominant kernel = the kernel instantiation with the largest share of the step
     shares = {"retrieve_kernel": op_ms["retrieve"],
               "accumulate_kernel<single task> (add, remove)": op_ms.get("add", 0.0) + op_ms.get("remove", 0.0),
-              "accumulate_kernel<compress>": op_ms["compress"]}
+              "compress_group_kernel + accumulate_kernel<compress>": op_ms["compress"]}
     dom = max(shares, key=shares.get)
     traffic_tbl = read_traffic()
     if dom == "retrieve_kernel":
@@ -442,7 +442,7 @@ def run_ours(args):
         traffic = traffic * w.n_params if traffic and w.storage == wl.F32 else None
     else:
         dom_bytes, dom_ms = b["compress"], ops["compress"]["ms_per_call"]
-        traffic = traffic_tbl.get("accumulate_kernel_compress_traffic_over_algorithmic")
+        traffic = traffic_tbl.get("compress_kernels_traffic_over_algorithmic")
         traffic = traffic * dom_bytes if traffic and w.storage == wl.F32 else None
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak,

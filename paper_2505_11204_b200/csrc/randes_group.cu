@@ -50,42 +50,66 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t saddr)
     return v;
 }
 
-// Position of a warp in its sequence of stages: item -> row pair -> task.
-struct Cursor {
-    uint32_t item;      // (slot, row block) index inside the unit
-    uint32_t ms;        // member index of the slot
-    uint32_t row;       // first row of the current row pair, relative to the unit
-    uint32_t rows_left; // rows of the item from `row` on (1 or more)
-    uint32_t i;         // task
+// Per (slot, task) pair of a unit, in shared memory: the task's source tensor W_i[sigma_i(l)],
+// which member of the group that source layer is (-> its W_0 tile in the stash), and the
+// Philox blocks with the sign bits of the unit's columns.
+template <int HB> struct PairRecord {
+    static constexpr uint32_t kBytes = 16 + 16 * HB;
+    static constexpr uint32_t kPtr = 0, kMember = 8, kBlocks = 16;
 };
 
-__device__ __forceinline__ void cursor_set(Cursor& c, uint32_t item, uint32_t n_chunks, uint32_t Rn)
+// Position of a warp in its sequence of stages: item (slot, block of rows) -> row pair -> task.
+// Everything a stage needs is kept incrementally so that the common step (next task of the
+// same row pair) is one addition and one comparison.
+struct Cursor {
+    uint32_t rec;        // shared address of the current pair's record
+    uint32_t rec_begin;  // record of task 0 of the current slot
+    uint32_t rec_end;    // one past the record of the last task
+    uint32_t off;        // element offset of the row pair's first row inside a layer (+ this lane's column)
+    uint32_t row;        // that row, relative to the unit (-> stash)
+    uint32_t rows_left;  // rows of the item from `row` on
+    uint32_t item;       // index of the (slot, block of rows) item
+    uint32_t m_off;      // shared address of the slot's offset in M
+};
+
+template <uint32_t REC>
+__device__ __forceinline__ void cursor_set(Cursor& c, uint32_t item, uint32_t n_chunks, uint32_t Rn, uint32_t nt, uint32_t s_rec,
+                                           uint32_t off0, uint32_t cols)
 {
     c.item = item;
-    c.ms = item / n_chunks;
-    const uint32_t chunk = item - c.ms * n_chunks;
+    const uint32_t ms = item / n_chunks;
+    c.m_off = s_rec - kOffTableBytes + ms * 8;
+    const uint32_t chunk = item - ms * n_chunks;
     c.row = chunk * kItemRows;
     c.rows_left = min(kItemRows, Rn - c.row);
-    c.i = 0;
+    c.off = off0 + c.row * cols;
+    c.rec_begin = c.rec = s_rec + ms * nt * REC;
+    c.rec_end = c.rec_begin + nt * REC;
 }
 
-__device__ __forceinline__ void cursor_next(Cursor& c, uint32_t nt, uint32_t n_chunks, uint32_t Rn)
+template <uint32_t REC>
+__device__ __forceinline__ void cursor_next(Cursor& c, uint32_t n_chunks, uint32_t Rn, uint32_t nt, uint32_t s_rec, uint32_t off0,
+                                            uint32_t cols)
 {
-    if (++c.i < nt) return;
-    c.i = 0;
-    if (c.rows_left > 2) {
+    c.rec += REC;
+    if (c.rec != c.rec_end) return;
+    if (c.rows_left > 2) {          // next row pair of the same slot
+        c.rec = c.rec_begin;
         c.row += 2;
         c.rows_left -= 2;
-    } else {
-        cursor_set(c, c.item + kWarpsPerCta, n_chunks, Rn);   // may run past the last item: never used then
+        c.off += 2 * cols;
+    } else {                        // next item; may run past the last one: never used then
+        cursor_set<REC>(c, c.item + kWarpsPerCta, n_chunks, Rn, nt, s_rec, off0, cols);
     }
 }
 
 template <typename ST, typename MT, int NSTAGE>
-__global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const CompressGroupArgs a, const uint32_t pair_cap)
+__global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const CompressGroupArgs a)
 {
     constexpr int CPL = Store<ST>::CPL;
     constexpr int HB = CPL / 4;                          // Philox blocks under a warp-wide column block
+    typedef PairRecord<HB> Rec;
+    constexpr uint32_t REC = Rec::kBytes;
     constexpr uint32_t ES = sizeof(ST);
     constexpr uint32_t kRingBytes = NSTAGE * 2 * kSlotBytes;
     constexpr uint32_t kStageBytes = 2 * kSlotBytes;
@@ -94,13 +118,13 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_s = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
     const uint32_t ring = smem_s + threadIdx.x * 16;
+    const uint32_t ring_end = ring + kRingBytes;
     const uint32_t stash = smem_s + kRingBytes;
     const uint32_t s_off = stash + kStashBytes;          // per member: first element of its slot in M
-    const uint32_t s_ptr = s_off + kOffTableBytes;       // per (slot, task): {W_i[sigma_i(l)], member index of sigma_i(l)}
-    const uint32_t s_blk = s_ptr + pair_cap * 16;        // per (slot, task): HB Philox blocks of sign bits
+    const uint32_t s_rec = s_off + kOffTableBytes;       // per (slot, task): PairRecord
     const uint32_t L = a.n_layers, nt = a.n_tasks;
-    // where this lane's sign bits sit inside a pair's blocks
-    const uint32_t sign_word = CPL == 4 ? (lane >> 3) * 4u : (lane >> 4) * 16u + ((lane & 15) >> 2) * 4u;
+    // where this lane's sign bits sit inside a record
+    const uint32_t sign_word = Rec::kBlocks + (CPL == 4 ? (lane >> 3) * 4u : (lane >> 4) * 16u + ((lane & 15) >> 2) * 4u);
     const uint32_t sign_shift = CPL == 4 ? (lane & 7) * 4u : (lane & 3) * 8u;
     const uint32_t one = 0x3F800000u;
 
@@ -111,6 +135,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
         const uint32_t G = l0.group_size, cols = l0.cols, Rn = un.nrows, row0 = un.row0;
         const uint32_t c = (un.cb0 * 32u + lane) * CPL;
         const bool lane_on = c < cols;
+        const uint32_t off0 = row0 * cols + c;           // layers hold < 2^32 elements
 
         // ---- prologue, all threads: W_0 tiles of every member into the stash ...
         if (lane_on) {
@@ -118,7 +143,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
             for (uint32_t q = warp; q < ntiles; q += kWarpsPerCta) {
                 const uint32_t m = q / Rn, r = q - m * Rn;
                 const char* pb = static_cast<const char*>(a.base[mem[m]]);
-                cp_async16(stash + q * kStashTileBytes + lane * 16, pb + (static_cast<size_t>(row0 + r) * cols + c) * ES);
+                cp_async16(stash + q * kStashTileBytes + lane * 16, pb + static_cast<size_t>(off0 + r * cols) * ES);
             }
         }
         cp_async_commit();
@@ -130,13 +155,13 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
             const uint32_t fl = a.layers[slot].flags;
             const uint32_t src = (fl & kFlagShuffle) ? a.src_of_slot[static_cast<size_t>(i) * L + slot] : slot;   // sigma_i(l)
             const void* pw = a.task_ptrs[static_cast<size_t>(i) * L + src];
-            sts_ptrs(s_ptr + p * 16, pw, reinterpret_cast<const void*>(static_cast<uintptr_t>(a.layers[src].member)));
+            sts_ptrs(s_rec + p * REC + Rec::kPtr, pw, reinterpret_cast<const void*>(static_cast<uintptr_t>(a.layers[src].member)));
             const DevTask tk = a.tasks[i];
 #pragma unroll
             for (int h = 0; h < HB; ++h) {
                 uint4 blk = make_uint4(0, 0, 0, 0);
                 if (fl & kFlagFlip) blk = philox4x32_10(un.cb0 * HB + h, slot, kTagSign, tk.id, tk.key0, tk.key1);
-                sts128(s_blk + (p * HB + h) * 16, blk);
+                sts128(s_rec + p * REC + Rec::kBlocks + h * 16, blk);
             }
         }
         for (uint32_t ms = threadIdx.x; ms < G; ms += kThreadsPerCta) sts_u64(s_off + ms * 8, a.layers[mem[ms]].m_off);
@@ -152,50 +177,50 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
                 N += (min(kItemRows, Rn - chunk * kItemRows) + 1) / 2 * nt;
             }
             Cursor ci, cc;
-            cursor_set(ci, warp, n_chunks, Rn);
+            cursor_set<REC>(ci, warp, n_chunks, Rn, nt, s_rec, off0, cols);
             cc = ci;
-            uint32_t issued = 0, stage_i = ring, stage_c = ring;
-            const uint32_t ring_end = ring + kRingBytes;
+            uint32_t to_issue = N, stage_i = ring, stage_c = ring;
             const uint32_t stash_lane = stash + lane * 16;
+            const uint32_t member_bytes = Rn * kStashTileBytes;
+            const size_t row_bytes = static_cast<size_t>(cols) * ES;
 
             auto issue = [&]() {
-                const char* pw = lds_ptr(s_ptr + (ci.ms * nt + ci.i) * 16);
-                const size_t off = (static_cast<size_t>(row0 + ci.row) * cols + c) * ES;
-                cp_async16(stage_i, pw + off);
-                if (ci.rows_left > 1) cp_async16(stage_i + kSlotBytes, pw + off + static_cast<size_t>(cols) * ES);
-                cursor_next(ci, nt, n_chunks, Rn);
+                const char* src = lds_ptr(ci.rec + Rec::kPtr) + static_cast<size_t>(ci.off) * ES;
+                cp_async16(stage_i, src);
+                if (ci.rows_left > 1) cp_async16(stage_i + kSlotBytes, src + row_bytes);
+                cursor_next<REC>(ci, n_chunks, Rn, nt, s_rec, off0, cols);
                 stage_i += kStageBytes;
                 if (stage_i == ring_end) stage_i = ring;
-                ++issued;
+                --to_issue;
             };
 
 #pragma unroll
             for (int s = 0; s < NSTAGE - 1; ++s) {
-                if (issued < N) issue();
+                if (to_issue) issue();
                 cp_async_commit();
             }
             f32x2 acc[2][CPL / 2];
             for (uint32_t it = 0; it < N; ++it) {
-                if (issued < N) issue();
+                if (to_issue) issue();
                 cp_async_commit();
                 cp_async_wait<NSTAGE - 1>();   // all but the newest NSTAGE-1 groups have landed: stage_c is ready
-                if (cc.i == 0) {
+                if (cc.rec == cc.rec_begin) {
 #pragma unroll
                     for (int r = 0; r < 2; ++r)
 #pragma unroll
                         for (int e = 0; e < CPL / 2; ++e) acc[r][e] = 0ull;
                 }
-                const uint32_t pair = cc.ms * nt + cc.i;
-                const uint32_t member = lds_u32(s_ptr + pair * 16 + 8);
-                const uint32_t bits = lds_u32(s_blk + pair * (HB * 16) + sign_word) >> sign_shift;
+                const uint32_t member = lds_u32(cc.rec + Rec::kMember);
+                const uint32_t bits = lds_u32(cc.rec + sign_word) >> sign_shift;
                 f32x2 sg[CPL / 2];   // +-1.0f per column
 #pragma unroll
                 for (int e = 0; e < CPL / 2; ++e)
                     sg[e] = pack2(((bits << (31 - 2 * e)) & 0x80000000u) | one, ((bits << (30 - 2 * e)) & 0x80000000u) | one);
-                const uint32_t b0 = stash_lane + (member * Rn + cc.row) * kStashTileBytes;
+                const uint32_t b0 = stash_lane + member * member_bytes + cc.row * kStashTileBytes;
+                const bool two = cc.rows_left > 1;
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
-                    if (r == 0 || cc.rows_left > 1) {
+                    if (r == 0 || two) {
                         f32x2 d[CPL / 2], b[CPL / 2];
                         Store<ST>::widen2(lds128(stage_c + r * kSlotBytes), d);
                         Store<ST>::widen2(lds128(b0 + r * kStashTileBytes), b);
@@ -203,11 +228,11 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
                         for (int e = 0; e < CPL / 2; ++e) acc[r][e] = fma2(sub2(d[e], b[e]), sg[e], acc[r][e]);
                     }
                 }
-                if (cc.i + 1 == nt) {
-                    MT* mp = static_cast<MT*>(a.M) + lds_u64(s_off + cc.ms * 8) + (static_cast<size_t>(row0 + cc.row) * cols + c);
+                if (cc.rec + REC == cc.rec_end) {   // last task: the rows of this slot are complete
+                    MT* mp = static_cast<MT*>(a.M) + lds_u64(cc.m_off) + cc.off;
 #pragma unroll
                     for (int r = 0; r < 2; ++r) {
-                        if (r == 0 || cc.rows_left > 1) {
+                        if (r == 0 || two) {
                             float v[CPL];
 #pragma unroll
                             for (int e = 0; e < CPL / 2; ++e) unpack2(acc[r][e], v[2 * e], v[2 * e + 1]);
@@ -215,7 +240,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
                         }
                     }
                 }
-                cursor_next(cc, nt, n_chunks, Rn);
+                cursor_next<REC>(cc, n_chunks, Rn, nt, s_rec, off0, cols);
                 stage_c += kStageBytes;
                 if (stage_c == ring_end) stage_c = ring;
             }
@@ -238,7 +263,7 @@ constexpr size_t kTwoCtaSmem = (228 * 1024 - 2 * 1024) / 2;   // two CTAs per SM
 size_t group_smem_bytes(int storage_dtype, int nstage, uint32_t pair_cap)
 {
     const size_t hb = storage_dtype == 1 ? 2 : 1;
-    return static_cast<size_t>(nstage) * 2 * kSlotBytes + kStashBytes + kOffTableBytes + static_cast<size_t>(pair_cap) * 16 * (1 + hb);
+    return static_cast<size_t>(nstage) * 2 * kSlotBytes + kStashBytes + kOffTableBytes + static_cast<size_t>(pair_cap) * (16 + 16 * hb);
 }
 
 }  // namespace
@@ -286,7 +311,7 @@ int launch_compress_groups(int storage_dtype, int m_dtype, const CompressGroupAr
                 if (e != cudaSuccess) { (void)cudaGetLastError(); return static_cast<int>(e); }
                 if (per_sm <= 0) return static_cast<int>(cudaErrorInvalidConfiguration);
                 const int grid = static_cast<int>(std::min<uint64_t>(static_cast<uint64_t>(sm_count) * per_sm, a.n_units));
-                compress_group_kernel<ST, MT, NS><<<grid, kThreadsPerCta, smem, s>>>(a, pair_cap);
+                compress_group_kernel<ST, MT, NS><<<grid, kThreadsPerCta, smem, s>>>(a);
                 return static_cast<int>(cudaGetLastError());
             });
         });

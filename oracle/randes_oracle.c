@@ -492,6 +492,65 @@ int ro_retrieve(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
 }
 
 /*
+ * A linear layer applied with a retrieved weight that is never formed
+ * (Section 4, second display, inserted into y = x What^T; Section 1 motivates
+ * serving many models from one store):
+ *   y[b][r] = sum_c x[b][c] * ( W_0[p][r,c] + lambda * s_t(l,c) * M[l][r,c] ),   l = sigma_t^-1(p).
+ * Everything is widened to double and summed in double, columns ascending: this
+ * is the definition, not a model of any particular arithmetic.  x is
+ * [n_tokens, cols] in the storage type; y and y_abs are [n_tokens, rows]
+ * doubles; y_abs (may be NULL) receives sum_c |x| * (|W_0| + |lambda * M|), the
+ * scale against which a finite-precision result is judged.
+ */
+int ro_linear(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
+              const uint32_t *group, uint32_t n_groups, const uint32_t *gflags,
+              int dtype, int m_dtype, uint32_t task_id, uint64_t seed, float lambda, uint32_t p,
+              const void *x, uint32_t n_tokens, const void *const *base, const void *const *M,
+              double *y, double *y_abs)
+{
+    ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
+    int rc = spec_check(&s);
+    if (rc) return rc;
+    uint32_t L = n_layers;
+    if (p >= L) return -1;
+    uint32_t *src_of_slot = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
+    uint32_t *slot_of_pos = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
+    if (!src_of_slot || !slot_of_pos) { free(src_of_slot); free(slot_of_pos); return -1; }
+    if (ro_task_tables(L, group, n_groups, gflags, seed, task_id, src_of_slot, slot_of_pos)) {
+        free(src_of_slot); free(slot_of_pos); return -1;
+    }
+    uint32_t nr = rows[p], nc = cols[p];
+    uint32_t l = slot_of_pos[p];
+    int8_t *sg = (int8_t *)malloc(nc ? nc : 1);
+    if (!sg) { free(src_of_slot); free(slot_of_pos); return -1; }
+    if (ro_layer_flips(L, group, gflags, l)) ro_sign_row(seed, task_id, l, nc, sg);
+    else memset(sg, 1, nc);
+    const void *m = M[l];
+    const void *wb = base[p];
+    const double lam = (double)lambda;
+#pragma omp parallel for schedule(static)
+    for (int64_t b = 0; b < (int64_t)n_tokens; ++b) {
+        for (uint32_t r = 0; r < nr; ++r) {
+            double acc = 0.0, mag = 0.0;
+            for (uint32_t c = 0; c < nc; ++c) {
+                size_t idx = (size_t)r * nc + c;
+                double xv = (double)load_elem(x, dtype, (size_t)b * nc + c);
+                double w0 = (double)load_elem(wb, dtype, idx);
+                double mv = (double)load_m(m, m_dtype, idx);
+                acc += xv * (w0 + lam * (sg[c] < 0 ? -mv : mv));
+                mag += fabs(xv) * (fabs(w0) + fabs(lam * mv));
+            }
+            y[(size_t)b * nr + r] = acc;
+            if (y_abs) y_abs[(size_t)b * nr + r] = mag;
+        }
+    }
+    free(sg);
+    free(src_of_slot);
+    free(slot_of_pos);
+    return 0;
+}
+
+/*
  * Gram matrix of the transformed deltas (Section 3: the interference norm is a
  * function of the inner products of the deltas; Section 4: every O_i is
  * orthogonal, so the deltas that interfere at retrieval have the inner products

@@ -74,6 +74,7 @@ def _load():
         lib.ro_add_models.restype = ctypes.c_int
         lib.ro_remove_model.restype = ctypes.c_int
         lib.ro_retrieve.restype = ctypes.c_int
+        lib.ro_linear.restype = ctypes.c_int
         lib.ro_delta_gram.restype = ctypes.c_int
         lib.ro_num_threads.restype = ctypes.c_int
         lib.ro_set_num_threads.argtypes = [ctypes.c_int]
@@ -304,3 +305,29 @@ def retrieve(spec, dtype: int, out_dtype: int, task_id: int, seed: int, lam: flo
     if rc:
         raise ValueError("ro_retrieve failed: %d" % rc)
     return out
+
+
+def linear(spec, dtype: int, task_id: int, seed: int, lam: float, layer: int, x: np.ndarray,
+           base: Sequence[np.ndarray], M: Sequence[np.ndarray], m_dtype: int = F32) -> Tuple[np.ndarray, np.ndarray]:
+    """y = x What_t[layer]^T with What = W_0 + lambda * T_t^-1(M) (Section 4) never formed: fp64 from the
+    definition.  x is [n_tokens, cols] in the storage type.  Returns (y, y_abs), both [n_tokens, rows] float64;
+    y_abs = sum_c |x| (|W_0| + |lambda M|) is the scale for judging a finite-precision result."""
+    lib = _load()
+    sargs, keep = _spec_args(spec)
+    _check_layers(spec, base, dtype)
+    _check_layers(spec, M, m_dtype)
+    rows, cols = int(spec[0][layer]), int(spec[1][layer])
+    want = np.uint16 if dtype == BF16 else np.float32
+    x = np.ascontiguousarray(x)
+    if x.dtype != want or x.ndim != 2 or x.shape[1] != cols:
+        raise ValueError("x must be [n_tokens, %d] of %s" % (cols, want))
+    y = np.zeros((x.shape[0], rows), dtype=np.float64)
+    y_abs = np.zeros_like(y)
+    rc = lib.ro_linear(*sargs, ctypes.c_int(dtype), ctypes.c_int(m_dtype), ctypes.c_uint32(task_id),
+                       ctypes.c_uint64(seed), ctypes.c_float(lam), ctypes.c_uint32(layer),
+                       x.ctypes.data_as(ctypes.c_void_p), ctypes.c_uint32(x.shape[0]),
+                       _ptr_array(base), _ptr_array(M),
+                       y.ctypes.data_as(ctypes.c_void_p), y_abs.ctypes.data_as(ctypes.c_void_p))
+    if rc:
+        raise ValueError("ro_linear failed: %d" % rc)
+    return y, y_abs

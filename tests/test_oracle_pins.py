@@ -674,3 +674,56 @@ def test_group_with_unequal_shapes_is_rejected():
     base = [np.zeros((4, 8), np.float32), np.zeros((4, 9), np.float32)]
     with pytest.raises(ValueError):
         ro.compress(spec, ro.F32, [0], [0], base, [base])
+
+
+# --------------------------------------------------------------------------- linear layer on the retrieved weight
+@pytest.mark.parametrize("flags", [SHUFFLE | FLIP, FLIP, SHUFFLE, 0])
+def test_linear_matches_dense_matrices_and_the_retrieved_weight(flags):
+    """y = x What^T with What = W_0 + lambda O_t^T M (Section 4, second display) taken from d x d matrices:
+    on dyadic inputs every product and sum is exact in double, so the oracle must agree bit for bit; it must
+    also agree with a matrix product on the oracle's own retrieved weights."""
+    spec = tiny_spec(flags)
+    rng = np.random.default_rng(77)
+    ids, seeds = [4, 1, 8], [11, 2**40 + 3, 5]
+    base = rand_model(spec, rng, dyadic=True)
+    tasks = [rand_model(spec, rng, dyadic=True) for _ in ids]
+    M = ro.compress(spec, ro.F32, ids, seeds, base, tasks)
+    lam = 0.25
+    for t, s in zip(ids, seeds):
+        T, offs = dense_transform(spec, s, t)
+        what_dense = unflat(flat(base) + lam * (T.T @ flat(M)), spec, offs)
+        what = ro.retrieve(spec, ro.F32, ro.F32, t, s, lam, base, M)
+        for p in range(len(spec[0])):
+            x = (rng.integers(-64, 65, size=(5, spec[1][p])) / 64.0).astype(np.float32)
+            y, y_abs = ro.linear(spec, ro.F32, t, s, lam, p, x, base, M)
+            assert np.array_equal(y, x.astype(np.float64) @ what_dense[p].T)
+            assert np.array_equal(y, x.astype(np.float64) @ what[p].astype(np.float64).T)
+            assert np.all(y_abs >= np.abs(y))
+
+
+def test_linear_on_bf16_inputs_and_superposition_stays_close_to_the_retrieved_weight():
+    """bf16 weights and a bf16 superposition: the unformed weight W_0 + lambda s M differs from the retrieved
+    fp32 weight by one fp32 rounding per element, so the two products agree to 2^-24 of the magnitude sum; a
+    single column with the wrong sign would move the result far beyond that."""
+    rng = np.random.default_rng(78)
+    spec = ([6] * 3, [40] * 3, [0] * 3, [SHUFFLE | FLIP])
+    to_b = lambda a: np.array([ro.f32_to_bf16(float(v)) for v in a.ravel()], dtype=np.uint16).reshape(a.shape)
+    widen = lambda b: (b.astype(np.uint32) << 16).view(np.float32)
+    base = [to_b(a * 0.02) for a in rand_model(spec, rng)]
+    M = [to_b(a * 0.003) for a in rand_model(spec, rng)]
+    x = to_b(rng.standard_normal((7, 40)).astype(np.float32))
+    lam, t, s = 0.3, 3, 99
+    for p in range(3):
+        y, y_abs = ro.linear(spec, ro.BF16, t, s, lam, p, x, base, M, m_dtype=ro.BF16)
+        what = ro.retrieve(spec, ro.BF16, ro.F32, t, s, lam, base, M, positions=[p], m_dtype=ro.BF16)[p]
+        y_ret = widen(x).astype(np.float64) @ what.astype(np.float64).T
+        assert np.all(np.abs(y - y_ret) <= 2.0 ** -23 * y_abs)
+        # flipping the sign of one column's superposition term changes y by 2 |x_c| lambda |M_c|
+        _, slot_of_pos = ro.task_tables(spec, s, t)
+        l = int(slot_of_pos[p])
+        Mw = [m.copy() for m in M]
+        Mw[l][:, 17] ^= 0x8000
+        y_wrong, _ = ro.linear(spec, ro.BF16, t, s, lam, p, x, base, Mw, m_dtype=ro.BF16)
+        want = -2.0 * float(np.float32(lam)) * ro.sign(s, t, l, 17) * np.outer(widen(x)[:, 17].astype(np.float64), widen(M[l])[:, 17].astype(np.float64))
+        assert np.allclose(y_wrong - y, want, rtol=0, atol=1e-12)
+        assert np.abs(y_wrong - y).max() > 2.0 ** -14 * y_abs.max()

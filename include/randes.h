@@ -235,6 +235,36 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda,
                     void* const* out, void* stream);
 
 /*
+ * A linear layer on the retrieved weight of one layer, without writing that
+ * weight to memory (Section 4, second display, inside y = x What^T; the serving
+ * case of the paper's introduction):
+ *   y[b][r] = sum_c x[b][c] * ( W_0[p][r,c] + lambda * s_t(l,c) * M[l][r,c] ),  l = sigma_t^-1(p)
+ * computed as x W_0[p]^T + lambda * (x D_t) M[l]^T: the inverse sign flip acts on the
+ * activations' columns, the inverse shuffle is the choice of the slot l.  Two bf16
+ * products on the tensor cores with fp32 accumulation; lambda is applied once per
+ * output in fp32.  Needs a plan with bf16 weights AND a bf16 superposition.
+ *   layer                 position p; its shape [rows, cols] must have cols % 8 == 0
+ *   x                     device, [n_tokens, cols] bf16 row-major, 16-byte aligned
+ *   base[n_layers]        host array of device pointers (only base[layer] is used, 16-byte aligned)
+ *   M                     device, the superposition arena
+ *   y                     device, [n_tokens, rows] fp32 row-major; must not alias the inputs
+ * Needs no workspace (the plan may have been built without one).  One kernel launch;
+ * asynchronous on `stream`.  The result equals the fp64 definition within
+ * 2 * cols * 2^-24 * sum_c |x| (|W_0| + |lambda M|) per output (fp32 accumulation of 2 * cols
+ * exact products in any order).  Errors: UNSUPPORTED_DTYPE, UNKNOWN_TASK, INVALID_ARGUMENT,
+ * MISALIGNED, CUDA_ERROR.
+ */
+int randes_linear(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x,
+                  uint32_t n_tokens, const void* const* base, const void* M, void* y, void* stream);
+
+/*
+ * Every wait inside the randes_linear kernel is bounded; a thread block whose wait runs out
+ * skips its tile and counts itself here.  *count = number of such blocks since the library was
+ * loaded on the current device (0 in a healthy run).  Synchronises with the device.
+ */
+int randes_linear_giveups(unsigned int* count);
+
+/*
  * Batched retrieve: rebuild n_tasks models in one pass (Section 4, second
  * display, for several tasks at once; the multi-model serving case of the
  * paper's introduction).  Equivalent, bit for bit, to n_tasks calls of

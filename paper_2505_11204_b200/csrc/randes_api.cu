@@ -1069,6 +1069,56 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_
     return guarded([&] { return randes_retrieve_impl(plan, task_id, lambda, out_dtype, base, M, out, stream); });
 }
 
+static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x,
+                              uint32_t n_tokens, const void* const* base, const void* M, void* y, void* stream)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (plan->storage != RANDES_BF16 || plan->m_dtype != RANDES_BF16)
+        return fail(RANDES_UNSUPPORTED_DTYPE, "randes_linear needs bf16 weights and a bf16 superposition (tensor-core operands)");
+    if (layer >= plan->n_layers) return fail(RANDES_INVALID_ARGUMENT, "layer %u out of range (n_layers = %u)", layer, plan->n_layers);
+    const int row = find_task(*plan, task_id);
+    if (row < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_id);
+    int rc;
+    if ((rc = check_m(M))) return rc;
+    if (!base || !base[layer]) return fail(RANDES_INVALID_ARGUMENT, "base or base[%u] is NULL", layer);
+    if (!x || !y) return fail(RANDES_INVALID_ARGUMENT, "x or y is NULL");
+    const uint32_t rows = plan->layers[layer].rows, cols = plan->layers[layer].cols;
+    if (n_tokens == 0 || rows == 0 || cols == 0) return RANDES_OK;
+    if (cols % 8) return fail(RANDES_INVALID_ARGUMENT, "layer %u: cols = %u is not a multiple of 8 (16-byte rows for the tensor maps)", layer, cols);
+    if (reinterpret_cast<uintptr_t>(x) % 16 || reinterpret_cast<uintptr_t>(base[layer]) % 16)
+        return fail(RANDES_MISALIGNED, "x and base[%u] must be 16-byte aligned", layer);
+    if (reinterpret_cast<uintptr_t>(y) % 4) return fail(RANDES_MISALIGNED, "y = %p is not aligned to 4 bytes", y);
+    const TaskEntry& t = plan->tasks[row];
+    const uint32_t slot = t.slot_of_pos[layer];                    // sigma_t^-1(p)
+    const bool flip = (plan->dev_layers[slot].flags & kFlagFlip) != 0;
+    DevTask d;
+    d.id = t.id;
+    d.key0 = static_cast<uint32_t>(t.seed);
+    d.key1 = static_cast<uint32_t>(t.seed >> 32);
+    d.pad = 0;
+    int e = linear_prepare();
+    if (e) return fail_cuda(static_cast<cudaError_t>(e), "set-up of the linear kernel");
+    e = launch_linear(x, n_tokens, base[layer], static_cast<const char*>(M) + plan->m_off_bytes[slot], rows, cols, flip, slot, d, lambda,
+                      static_cast<float*>(y), stream);
+    if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the linear kernel");
+    ++g_launches;
+    return RANDES_OK;
+}
+
+int randes_linear(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x, uint32_t n_tokens,
+                  const void* const* base, const void* M, void* y, void* stream)
+{
+    return guarded([&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, stream); });
+}
+
+int randes_linear_giveups(unsigned int* count)
+{
+    if (!count) return fail(RANDES_INVALID_ARGUMENT, "count is NULL");
+    const int e = linear_giveups(count);
+    if (e) return fail_cuda(static_cast<cudaError_t>(e), "read of the give-up counter");
+    return RANDES_OK;
+}
+
 int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_t n_tasks, float lambda,
                           randes_dtype_t out_dtype, const void* const* base, const void* M, void* const* out, void* stream)
 {

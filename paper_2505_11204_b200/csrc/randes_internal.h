@@ -162,6 +162,13 @@ int launch_retrieve_batch(int storage_dtype, int out_dtype, int m_dtype, const R
 int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype);
 
 
+// randes_linear.cu: y = x W_0^T + lambda (x D) M_slot^T on the tensor cores (bf16 operands, fp32 accumulators).
+// All return a cudaError_t as int.
+int linear_prepare();   // opts the kernel into its shared memory on the current device
+int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* m_slot, uint32_t rows, uint32_t cols, bool flip,
+                  uint32_t slot, const DevTask& task, float lambda, float* y, void* stream);
+int linear_giveups(unsigned int* count);   // CTAs that gave up on a bounded wait since the library was loaded (synchronises)
+
 // Retrieve with its tables in a fixed device array inside the library (no workspace).
 // Returns a cudaError_t as int, or -1 when the tables exceed kStaticScratchBytes.
 constexpr size_t kStaticScratchBytes = 1u << 20;

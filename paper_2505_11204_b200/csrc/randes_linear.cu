@@ -1,0 +1,381 @@
+// A linear layer on a retrieved weight that is never written to memory:
+//
+//   y[b][r] = sum_c x[b][c] * ( W_0[p][r,c] + lambda * s_t(l,c) * M[l][r,c] ),     l = sigma_t^-1(p)
+//           = ( x W_0[p]^T )[b][r] + lambda * ( (x D_t) M[l]^T )[b][r]
+//
+// (Section 4, second display, put inside y = x What^T; D_t is the sign diagonal of Section 4.4,
+// so the inverse transform becomes a sign flip on the activations' columns, and the inverse
+// shuffle of Section 4.3 is the choice of the slot l.)  Two bf16 GEMMs that share the activation
+// tile, on the fifth-generation tensor cores:
+//
+//   * operands are staged in shared memory by TMA (128-byte swizzle), three stages deep:
+//     x tile [128 tokens x 64], W_0 tile [128 features x 64], M tile [128 features x 64];
+//   * four warps copy the x tile to a second buffer with the sign bits of its 64 columns
+//     flipped (bf16 sign bit XOR: exact), Philox bits generated in registers;
+//   * one thread issues tcgen05.mma (M = 128, N = 128, K = 16) into two fp32 accumulators in
+//     tensor memory: acc0 += x W_0^T, acc1 += (x D) M^T;
+//   * the epilogue reads both accumulators with tcgen05.ld and stores fma(lambda, acc1, acc0).
+//
+// lambda stays in fp32 and is applied once per output, so the operands keep their stored bits.
+// Every wait on an mbarrier is bounded: a CTA that gives up raises a shared flag, every role
+// leaves its loop, tensor memory is freed, and a device counter records the event.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <mutex>
+
+#include "randes_device.cuh"
+#include "randes_internal.h"
+
+namespace randes {
+
+static __device__ unsigned int g_linear_giveups;   // CTAs that gave up waiting (0 in a healthy run)
+
+namespace {
+
+using namespace device;
+
+constexpr int kBM = 128;          // tokens per CTA tile
+constexpr int kBN = 128;          // output features per CTA tile
+constexpr int kBK = 64;           // bf16 columns per stage: one 128-byte swizzle row
+constexpr int kStages = 3;
+constexpr int kTileBytes = kBM * kBK * 2;                    // 16 KiB, also for the kBN x kBK tiles
+constexpr int kStageBytes = 4 * kTileBytes;                  // x, flipped x, W_0, M
+constexpr int kLinearThreads = 192;                          // warp 0 TMA, warp 1 MMA, warps 2-5 flip + epilogue
+constexpr int kFlipThreads = 128;
+constexpr uint32_t kTmemCols = 256;                          // two accumulators of kBN fp32 columns
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr size_t kLinearSmem = 1024 + kStages * kStageBytes + 256;   // alignment slack + stages + barriers
+
+struct LinearArgs {
+    uint32_t n_tokens, rows, cols;
+    float lambda;
+    uint32_t flip;                 // 0: no sign flip on this slot (one activation buffer serves both products)
+    uint32_t slot;                 // l = sigma_t^-1(p): counter word 1 of the sign stream
+    DevTask task;
+    float* y;                      // [n_tokens, rows]
+};
+
+// ---- mbarrier, TMA, tcgen05 wrappers --------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA has given up (here or in another role).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag)
+{
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    if (atomicExch(const_cast<uint32_t*>(abort_flag), 1u) == 0u) atomicAdd(&g_linear_giveups, 1u);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_load32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a [128 rows x 64 bf16] K-major tile written by TMA with the
+// 128-byte swizzle: rows are 128 bytes apart, groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
+{
+    return static_cast<uint64_t>((saddr >> 4) & 0x3FFFu)      // start address, 16-byte units
+           | (1ull << 16)                                     // leading byte offset: unused with this layout
+           | (static_cast<uint64_t>(1024 >> 4) << 32)         // stride byte offset: 8 rows x 128 bytes
+           | (1ull << 46)                                     // descriptor version of this architecture
+           | (2ull << 61);                                    // 128-byte swizzle
+}
+
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = kBN.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kBN >> 3) << 17) | (static_cast<uint32_t>(kBM >> 4) << 24);
+
+__global__ void __launch_bounds__(kLinearThreads, 1)
+linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+              const __grid_constant__ CUtensorMap map_m, const LinearArgs a)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t smem_base = (static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw)) + 1023u) & ~1023u;
+    const uint32_t bars = smem_base + kStages * kStageBytes;
+    // barriers: full[s], flipped[s], empty[s], then acc_full; then the tensor-memory address and the give-up flag
+    auto bar_full = [&](int s) { return bars + 8u * s; };
+    auto bar_flipped = [&](int s) { return bars + 8u * (kStages + s); };
+    auto bar_empty = [&](int s) { return bars + 8u * (2 * kStages + s); };
+    const uint32_t bar_acc = bars + 8u * (3 * kStages);
+    const uint32_t tmem_slot = bar_acc + 8;
+    unsigned char* gen_base = smem_raw + (smem_base - static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw)));
+    volatile uint32_t* tmem_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + kStages * kStageBytes + 8 * (3 * kStages + 1));
+    volatile uint32_t* abort_flag = tmem_ptr + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * kBN, m0 = blockIdx.y * kBM;
+    const uint32_t n_k = (a.cols + kBK - 1) / kBK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full(s), 1);
+            mbar_init(bar_flipped(s), kFlipThreads);
+            mbar_init(bar_empty(s), 1);
+        }
+        mbar_init(bar_acc, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_ptr;
+
+    if (warp == 0) {
+        // ---- TMA producer
+        if (lane == 0) {
+            uint32_t issued = 0;
+            for (uint32_t kk = 0; kk < n_k; ++kk) {
+                const int s = kk % kStages;
+                const uint32_t ph = (kk / kStages) & 1u;
+                if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag)) break;
+                const uint32_t st = smem_base + s * kStageBytes;
+                mbar_expect_tx(bar_full(s), 3 * kTileBytes);
+                tma_load_2d(st, &map_x, bar_full(s), kk * kBK, m0);
+                tma_load_2d(st + 2 * kTileBytes, &map_w, bar_full(s), kk * kBK, n0);
+                tma_load_2d(st + 3 * kTileBytes, &map_m, bar_full(s), kk * kBK, n0);
+                issued = kk + 1;
+            }
+            if (*abort_flag) {
+                // gave up: let the copies already issued land before the CTA's shared memory is released
+                const uint32_t first = issued > kStages ? issued - kStages : 0;
+                for (uint32_t kk = first; kk < issued; ++kk)
+                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar_full(kk % kStages), (kk / kStages) & 1u); ++it) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            for (uint32_t kk = 0; kk < n_k && ok; ++kk) {
+                const int s = kk % kStages;
+                const uint32_t ph = (kk / kStages) & 1u;
+                ok = mbar_wait(bar_full(s), ph, abort_flag);
+                if (ok && a.flip) ok = mbar_wait(bar_flipped(s), ph, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t st = smem_base + s * kStageBytes;
+                const uint64_t dx = smem_desc_sw128(st);
+                const uint64_t dxf = smem_desc_sw128(st + (a.flip ? kTileBytes : 0));
+                const uint64_t dw = smem_desc_sw128(st + 2 * kTileBytes);
+                const uint64_t dm = smem_desc_sw128(st + 3 * kTileBytes);
+#pragma unroll
+                for (int k = 0; k < kBK / 16; ++k) {
+                    const uint32_t acc = (kk | k) ? 1u : 0u;
+                    // 16 bf16 columns = 32 bytes = 2 units of the descriptor's start address
+                    tc_mma_bf16(tmem, dx + 2 * k, dw + 2 * k, kIdesc, acc);
+                    tc_mma_bf16(tmem + kBN, dxf + 2 * k, dm + 2 * k, kIdesc, acc);
+                }
+                tc_commit(bar_empty(s));     // the stage is free once these products have read it
+            }
+            tc_commit(bar_acc);              // both accumulators are final (or, after giving up, quiescent)
+            if (!ok) {
+                for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar_acc, 0); ++it) {}
+            }
+        }
+    } else {
+        // ---- warps 2-5: flipped copy of the activation tile, then the epilogue
+        const int t = threadIdx.x - 64;                       // 0 .. 127
+        bool ok = true;
+        if (a.flip) {
+            // 16-byte chunk q = t + 128 j of the tile sits in row q / 8 at physical position q % 8, which the
+            // 128-byte swizzle maps to logical chunk (q % 8) ^ (row % 8): the same for all j of a thread
+            const uint32_t lc = static_cast<uint32_t>((t & 7) ^ ((t >> 3) & 7));   // columns 8 lc .. 8 lc + 7 of the stage
+            uint4 blk = make_uint4(0, 0, 0, 0);
+            for (uint32_t kk = 0; kk < n_k; ++kk) {
+                const int s = kk % kStages;
+                const uint32_t ph = (kk / kStages) & 1u;
+                if ((kk & 1u) == 0) blk = philox4x32_10(kk >> 1, a.slot, kTagSign, a.task.id, a.task.key0, a.task.key1);
+                // column c = 64 kk + 8 lc: word (c >> 5) & 3 of the block, bits (c & 31) .. + 7
+                const uint32_t wsel = (kk & 1u) * 2u + (lc >> 2);
+                const uint32_t word = wsel == 0 ? blk.x : (wsel == 1 ? blk.y : (wsel == 2 ? blk.z : blk.w));
+                const uint32_t bits = (word >> ((lc & 3u) * 8u)) & 0xFFu;
+                uint32_t mask[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) mask[j] = (((bits >> (2 * j)) & 1u) << 15) | (((bits >> (2 * j + 1)) & 1u) << 31);
+                ok = mbar_wait(bar_full(s), ph, abort_flag);
+                if (!ok) break;
+                const uint32_t src = smem_base + s * kStageBytes + t * 16;
+#pragma unroll
+                for (int j = 0; j < kTileBytes / (16 * kFlipThreads); ++j) {
+                    uint4 v = lds128(src + j * kFlipThreads * 16);
+                    v.x ^= mask[0]; v.y ^= mask[1]; v.z ^= mask[2]; v.w ^= mask[3];
+                    sts128(src + kTileBytes + j * kFlipThreads * 16, v);
+                }
+                fence_proxy_async();          // the tensor core reads the copy through the async proxy
+                mbar_arrive(bar_flipped(s));
+            }
+        }
+        if (ok) ok = mbar_wait(bar_acc, 0, abort_flag);
+        if (ok) {
+            tc_fence_after();
+            const int quarter = warp & 3;                     // tensor-memory lanes 32 q .. 32 q + 31
+            const uint32_t token = m0 + quarter * 32 + lane;
+            const uint32_t tlane = static_cast<uint32_t>(quarter * 32) << 16;
+            const bool vec = (a.rows & 3u) == 0 && (reinterpret_cast<uintptr_t>(a.y) & 15u) == 0;
+#pragma unroll 1
+            for (int cchunk = 0; cchunk < kBN / 32; ++cchunk) {
+                uint32_t v0[32], v1[32];
+                tc_load32(tmem + tlane + cchunk * 32, v0);
+                tc_load32(tmem + tlane + kBN + cchunk * 32, v1);
+                tc_wait_ld();
+                if (token < a.n_tokens) {
+                    float* yp = a.y + static_cast<size_t>(token) * a.rows + n0 + cchunk * 32;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        float o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) o[e] = __fmaf_rn(a.lambda, __uint_as_float(v1[j + e]), __uint_as_float(v0[j + e]));
+                        const uint32_t f = n0 + cchunk * 32 + j;
+                        if (vec && f + 3 < a.rows) {
+                            *reinterpret_cast<float4*>(yp + j) = make_float4(o[0], o[1], o[2], o[3]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (f + e < a.rows) yp[j + e] = o[e];
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+std::mutex g_encode_mutex;
+EncodeTiledFn g_encode = nullptr;
+
+EncodeTiledFn encode_fn()
+{
+    std::lock_guard<std::mutex> lock(g_encode_mutex);
+    if (!g_encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult st;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &st) != cudaSuccess || st != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    return g_encode;
+}
+
+// row-major [outer, inner] bf16 matrix, tiles of [box_outer, 64] with the 128-byte swizzle; out-of-range elements read as zero
+bool make_map(EncodeTiledFn enc, CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_outer)
+{
+    const cuuint64_t dims[2] = {inner, outer};
+    const cuuint64_t strides[1] = {inner * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK), box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int linear_prepare()
+{
+    cudaError_t e = cudaFuncSetAttribute(linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kLinearSmem));
+    if (e != cudaSuccess) (void)cudaGetLastError();
+    return static_cast<int>(e);
+}
+
+int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* m_slot, uint32_t rows, uint32_t cols, bool flip,
+                  uint32_t slot, const DevTask& task, float lambda, float* y, void* stream)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return static_cast<int>(cudaErrorNotSupported);
+    CUtensorMap mx, mw, mm;
+    if (!make_map(enc, &mx, x, cols, n_tokens, kBM) || !make_map(enc, &mw, w0, cols, rows, kBN) || !make_map(enc, &mm, m_slot, cols, rows, kBN))
+        return static_cast<int>(cudaErrorInvalidValue);
+    LinearArgs a;
+    a.n_tokens = n_tokens;
+    a.rows = rows;
+    a.cols = cols;
+    a.lambda = lambda;
+    a.flip = flip ? 1u : 0u;
+    a.slot = slot;
+    a.task = task;
+    a.y = y;
+    const dim3 grid((rows + kBN - 1) / kBN, (n_tokens + kBM - 1) / kBM);
+    linear_kernel<<<grid, kLinearThreads, kLinearSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
+    return static_cast<int>(cudaGetLastError());
+}
+
+int linear_giveups(unsigned int* count)
+{
+    return static_cast<int>(cudaMemcpyFromSymbol(count, g_linear_giveups, sizeof(unsigned int)));
+}
+
+}  // namespace randes

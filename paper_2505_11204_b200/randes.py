@@ -110,6 +110,10 @@ def lib():
         L.randes_retrieve_batch.restype = ctypes.c_int
         L.randes_retrieve_static.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
         L.randes_retrieve_static.restype = ctypes.c_int
+        L.randes_linear.argtypes = [vp, u32, ctypes.c_float, u32, vp, u32, vp, vp, vp, vp]
+        L.randes_linear.restype = ctypes.c_int
+        L.randes_linear_giveups.argtypes = [ctypes.POINTER(ctypes.c_uint)]
+        L.randes_linear_giveups.restype = ctypes.c_int
         L.randes_launch_count.argtypes = []
         L.randes_launch_count.restype = u64
         L.randes_last_error.argtypes = []
@@ -122,7 +126,7 @@ EXPORTS = [
     "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
     "randes_task_tables", "randes_plan_serialize", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_add_models", "randes_remove_model",
-    "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_retrieve_batch", "randes_retrieve_static", "randes_launch_count", "randes_last_error",
+    "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_retrieve_batch", "randes_retrieve_static", "randes_linear", "randes_linear_giveups", "randes_launch_count", "randes_last_error",
 ]
 
 
@@ -242,6 +246,18 @@ def randes_retrieve_batch(plan, task_ids, lam, out_dtype, base, M, out, stream) 
 def randes_retrieve_static(plan, task_id, lam, out_dtype, base, M, out, stream) -> None:
     """retrieve with the kernel's tables in the library's built-in device array (no workspace)."""
     _check(lib().randes_retrieve_static(plan, task_id, lam, out_dtype, _addr(base), _addr(M), _addr(out), stream))
+
+
+def randes_linear(plan, task_id, lam, layer, x, n_tokens, base, M, y, stream) -> None:
+    """y = x What_t[layer]^T on the tensor cores, the retrieved weight never written to memory."""
+    _check(lib().randes_linear(plan, task_id, lam, layer, _addr(x), n_tokens, _addr(base), _addr(M), _addr(y), stream))
+
+
+def randes_linear_giveups() -> int:
+    """Thread blocks of randes_linear that gave up on a bounded wait (0 in a healthy run); synchronises."""
+    n = ctypes.c_uint(0)
+    _check(lib().randes_linear_giveups(ctypes.byref(n)))
+    return int(n.value)
 
 
 def randes_launch_count() -> int:
@@ -430,6 +446,15 @@ class Plan:
             out_lists = out
         randes_retrieve_batch(self.handle, task_ids, lam, out_dtype, _as_ptrs(base), M, _as_ptrs(out), self._stream())
         return out_lists
+
+    def linear(self, task_id: int, lam: float, layer: int, x, base, M, y=None):
+        """x: [n_tokens, cols] bf16 CUDA tensor; returns y [n_tokens, rows] fp32."""
+        import torch
+
+        if y is None:
+            y = torch.empty((x.shape[0], self.rows[layer]), dtype=torch.float32, device=x.device)
+        randes_linear(self.handle, task_id, lam, layer, x, int(x.shape[0]), _as_ptrs(base), M, y, self._stream())
+        return y
 
     def retrieve(self, task_id: int, lam: float, base, M, out=None, out_dtype: int = F32):
         out_list = None

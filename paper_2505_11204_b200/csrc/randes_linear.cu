@@ -8,13 +8,14 @@
 // shuffle of Section 4.3 is the choice of the slot l.)  Two bf16 GEMMs that share the activation
 // tile, on the fifth-generation tensor cores:
 //
-//   * operands are staged in shared memory by TMA (128-byte swizzle), three stages deep:
-//     x tile [128 tokens x 64], W_0 tile [128 features x 64], M tile [128 features x 64];
-//   * four warps copy the x tile to a second buffer with the sign bits of its 64 columns
-//     flipped (bf16 sign bit XOR: exact), Philox bits generated in registers;
-//   * one thread issues tcgen05.mma (M = 128, N = 128, K = 16) into two fp32 accumulators in
-//     tensor memory: acc0 += x W_0^T, acc1 += (x D) M^T;
-//   * the epilogue reads both accumulators with tcgen05.ld and stores fma(lambda, acc1, acc0).
+//   * operands are staged in shared memory by TMA (128-byte swizzle), three or four stages deep:
+//     x tile [128 or 256 tokens x 64], W_0 tile [128 features x 64], M tile [128 features x 64];
+//   * (x D) M^T = x (M D)^T: four warps flip, in place, the sign bits of the M tile's 64 columns
+//     (bf16 sign bit XOR: exact), Philox bits generated in registers -- no second buffer;
+//   * one thread issues tcgen05.mma (M = 128, N = 128, K = 16) into fp32 accumulators in tensor
+//     memory, per block of 128 tokens: acc0 += x W_0^T, acc1 += x (M D)^T; with 256 tokens per
+//     CTA each weight tile feeds two products (1.5 x the flops per byte staged);
+//   * the epilogue reads the accumulators with tcgen05.ld and stores fma(lambda, acc1, acc0).
 //
 // lambda stays in fp32 and is applied once per output, so the operands keep their stored bits.
 // Every wait on an mbarrier is bounded: a CTA that gives up raises a shared flag, every role
@@ -36,22 +37,27 @@ namespace {
 
 using namespace device;
 
-constexpr int kBM = 128;          // tokens per CTA tile
+constexpr int kBM = 128;          // tokens per block of accumulators (the M of one tcgen05.mma)
 constexpr int kBN = 128;          // output features per CTA tile
 constexpr int kBK = 64;           // bf16 columns per stage: one 128-byte swizzle row
-constexpr int kStages = 3;
 constexpr int kTileBytes = kBM * kBK * 2;                    // 16 KiB, also for the kBN x kBK tiles
-constexpr int kStageBytes = 4 * kTileBytes;                  // x, flipped x, W_0, M
 constexpr int kLinearThreads = 192;                          // warp 0 TMA, warp 1 MMA, warps 2-5 flip + epilogue
 constexpr int kFlipThreads = 128;
-constexpr uint32_t kTmemCols = 256;                          // two accumulators of kBN fp32 columns
 constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr size_t kLinearSmem = 1024 + kStages * kStageBytes + 256;   // alignment slack + stages + barriers
+constexpr int kMaxStages = 4;
+
+// HALVES = blocks of 128 tokens per CTA (1 or 2)
+template <int HALVES> struct LinearGeom {
+    static constexpr int kStages = HALVES == 1 ? 4 : 3;
+    static constexpr int kStageBytes = (HALVES + 2) * kTileBytes;            // x block(s), W_0, M
+    static constexpr uint32_t kTmemCols = HALVES * 2 * kBN;                  // two accumulators per token block
+    static constexpr size_t kSmem = 1024 + kStages * kStageBytes + 256;      // alignment slack + stages + barriers
+};
 
 struct LinearArgs {
     uint32_t n_tokens, rows, cols;
     float lambda;
-    uint32_t flip;                 // 0: no sign flip on this slot (one activation buffer serves both products)
+    uint32_t flip;                 // 0: no sign flip on this slot
     uint32_t slot;                 // l = sigma_t^-1(p): counter word 1 of the sign stream
     DevTask task;
     float* y;                      // [n_tokens, rows]
@@ -143,25 +149,30 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = kBN.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kBN >> 3) << 17) | (static_cast<uint32_t>(kBM >> 4) << 24);
 
+template <int HALVES>
 __global__ void __launch_bounds__(kLinearThreads, 1)
 linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
               const __grid_constant__ CUtensorMap map_m, const LinearArgs a)
 {
+    typedef LinearGeom<HALVES> Geo;
+    constexpr int kStages = Geo::kStages;
+    constexpr int kStageBytes = Geo::kStageBytes;
+    constexpr int kOffW = HALVES * kTileBytes, kOffM = kOffW + kTileBytes;   // inside a stage: x block(s), W_0, M
     extern __shared__ unsigned char smem_raw[];
     const uint32_t smem_base = (static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw)) + 1023u) & ~1023u;
     const uint32_t bars = smem_base + kStages * kStageBytes;
-    // barriers: full[s], flipped[s], empty[s], then acc_full; then the tensor-memory address and the give-up flag
+    // barriers: full[s], flipped[s], empty[s] (kMaxStages each), then acc_full; then the tensor-memory address and the give-up flag
     auto bar_full = [&](int s) { return bars + 8u * s; };
-    auto bar_flipped = [&](int s) { return bars + 8u * (kStages + s); };
-    auto bar_empty = [&](int s) { return bars + 8u * (2 * kStages + s); };
-    const uint32_t bar_acc = bars + 8u * (3 * kStages);
+    auto bar_flipped = [&](int s) { return bars + 8u * (kMaxStages + s); };
+    auto bar_empty = [&](int s) { return bars + 8u * (2 * kMaxStages + s); };
+    const uint32_t bar_acc = bars + 8u * (3 * kMaxStages);
     const uint32_t tmem_slot = bar_acc + 8;
     unsigned char* gen_base = smem_raw + (smem_base - static_cast<uint32_t>(__cvta_generic_to_shared(smem_raw)));
-    volatile uint32_t* tmem_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + kStages * kStageBytes + 8 * (3 * kStages + 1));
+    volatile uint32_t* tmem_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + kStages * kStageBytes + 8 * (3 * kMaxStages + 1));
     volatile uint32_t* abort_flag = tmem_ptr + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * kBN, m0 = blockIdx.y * kBM;
+    const int n0 = blockIdx.x * kBN, m0 = blockIdx.y * (HALVES * kBM);
     const uint32_t n_k = (a.cols + kBK - 1) / kBK;
 
     if (threadIdx.x == 0) {
@@ -175,7 +186,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(Geo::kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -192,15 +203,15 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 const uint32_t ph = (kk / kStages) & 1u;
                 if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag)) break;
                 const uint32_t st = smem_base + s * kStageBytes;
-                mbar_expect_tx(bar_full(s), 3 * kTileBytes);
-                tma_load_2d(st, &map_x, bar_full(s), kk * kBK, m0);
-                tma_load_2d(st + 2 * kTileBytes, &map_w, bar_full(s), kk * kBK, n0);
-                tma_load_2d(st + 3 * kTileBytes, &map_m, bar_full(s), kk * kBK, n0);
+                mbar_expect_tx(bar_full(s), kStageBytes);
+                tma_load_2d(st, &map_x, bar_full(s), kk * kBK, m0);             // HALVES x 128 tokens in one box
+                tma_load_2d(st + kOffW, &map_w, bar_full(s), kk * kBK, n0);
+                tma_load_2d(st + kOffM, &map_m, bar_full(s), kk * kBK, n0);
                 issued = kk + 1;
             }
             if (*abort_flag) {
                 // gave up: let the copies already issued land before the CTA's shared memory is released
-                const uint32_t first = issued > kStages ? issued - kStages : 0;
+                const uint32_t first = issued > static_cast<uint32_t>(kStages) ? issued - kStages : 0;
                 for (uint32_t kk = first; kk < issued; ++kk)
                     for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar_full(kk % kStages), (kk / kStages) & 1u); ++it) {}
             }
@@ -213,30 +224,40 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 const int s = kk % kStages;
                 const uint32_t ph = (kk / kStages) & 1u;
                 ok = mbar_wait(bar_full(s), ph, abort_flag);
-                if (ok && a.flip) ok = mbar_wait(bar_flipped(s), ph, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t st = smem_base + s * kStageBytes;
-                const uint64_t dx = smem_desc_sw128(st);
-                const uint64_t dxf = smem_desc_sw128(st + (a.flip ? kTileBytes : 0));
-                const uint64_t dw = smem_desc_sw128(st + 2 * kTileBytes);
-                const uint64_t dm = smem_desc_sw128(st + 3 * kTileBytes);
+                const uint64_t dw = smem_desc_sw128(st + kOffW);
+                const uint64_t dm = smem_desc_sw128(st + kOffM);
+                // x W_0^T first: it does not depend on the flip
 #pragma unroll
-                for (int k = 0; k < kBK / 16; ++k) {
-                    const uint32_t acc = (kk | k) ? 1u : 0u;
-                    // 16 bf16 columns = 32 bytes = 2 units of the descriptor's start address
-                    tc_mma_bf16(tmem, dx + 2 * k, dw + 2 * k, kIdesc, acc);
-                    tc_mma_bf16(tmem + kBN, dxf + 2 * k, dm + 2 * k, kIdesc, acc);
+                for (int h = 0; h < HALVES; ++h) {
+                    const uint64_t dx = smem_desc_sw128(st + h * kTileBytes);
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k)   // 16 bf16 columns = 32 bytes = 2 units of the descriptor's start address
+                        tc_mma_bf16(tmem + h * 2 * kBN, dx + 2 * k, dw + 2 * k, kIdesc, (kk | k) ? 1u : 0u);
+                }
+                if (a.flip) {
+                    ok = mbar_wait(bar_flipped(s), ph, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+#pragma unroll
+                for (int h = 0; h < HALVES; ++h) {
+                    const uint64_t dx = smem_desc_sw128(st + h * kTileBytes);
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k)
+                        tc_mma_bf16(tmem + h * 2 * kBN + kBN, dx + 2 * k, dm + 2 * k, kIdesc, (kk | k) ? 1u : 0u);
                 }
                 tc_commit(bar_empty(s));     // the stage is free once these products have read it
             }
-            tc_commit(bar_acc);              // both accumulators are final (or, after giving up, quiescent)
+            tc_commit(bar_acc);              // the accumulators are final (or, after giving up, quiescent)
             if (!ok) {
                 for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar_acc, 0); ++it) {}
             }
         }
     } else {
-        // ---- warps 2-5: flipped copy of the activation tile, then the epilogue
+        // ---- warps 2-5: sign flip of the M tile's columns, in place; then the epilogue
         const int t = threadIdx.x - 64;                       // 0 .. 127
         bool ok = true;
         if (a.flip) {
@@ -257,14 +278,16 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 for (int j = 0; j < 4; ++j) mask[j] = (((bits >> (2 * j)) & 1u) << 15) | (((bits >> (2 * j + 1)) & 1u) << 31);
                 ok = mbar_wait(bar_full(s), ph, abort_flag);
                 if (!ok) break;
-                const uint32_t src = smem_base + s * kStageBytes + t * 16;
+                const uint32_t tile = smem_base + s * kStageBytes + kOffM + t * 16;
+                uint4 v[kTileBytes / (16 * kFlipThreads)];
+#pragma unroll
+                for (int j = 0; j < kTileBytes / (16 * kFlipThreads); ++j) v[j] = lds128(tile + j * kFlipThreads * 16);
 #pragma unroll
                 for (int j = 0; j < kTileBytes / (16 * kFlipThreads); ++j) {
-                    uint4 v = lds128(src + j * kFlipThreads * 16);
-                    v.x ^= mask[0]; v.y ^= mask[1]; v.z ^= mask[2]; v.w ^= mask[3];
-                    sts128(src + kTileBytes + j * kFlipThreads * 16, v);
+                    v[j].x ^= mask[0]; v[j].y ^= mask[1]; v[j].z ^= mask[2]; v[j].w ^= mask[3];
+                    sts128(tile + j * kFlipThreads * 16, v[j]);
                 }
-                fence_proxy_async();          // the tensor core reads the copy through the async proxy
+                fence_proxy_async();          // the tensor core reads the tile through the async proxy
                 mbar_arrive(bar_flipped(s));
             }
         }
@@ -272,29 +295,32 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         if (ok) {
             tc_fence_after();
             const int quarter = warp & 3;                     // tensor-memory lanes 32 q .. 32 q + 31
-            const uint32_t token = m0 + quarter * 32 + lane;
             const uint32_t tlane = static_cast<uint32_t>(quarter * 32) << 16;
             const bool vec = (a.rows & 3u) == 0 && (reinterpret_cast<uintptr_t>(a.y) & 15u) == 0;
 #pragma unroll 1
-            for (int cchunk = 0; cchunk < kBN / 32; ++cchunk) {
-                uint32_t v0[32], v1[32];
-                tc_load32(tmem + tlane + cchunk * 32, v0);
-                tc_load32(tmem + tlane + kBN + cchunk * 32, v1);
-                tc_wait_ld();
-                if (token < a.n_tokens) {
-                    float* yp = a.y + static_cast<size_t>(token) * a.rows + n0 + cchunk * 32;
+            for (int h = 0; h < HALVES; ++h) {
+                const uint32_t token = m0 + h * kBM + quarter * 32 + lane;
+#pragma unroll 1
+                for (int cchunk = 0; cchunk < kBN / 32; ++cchunk) {
+                    uint32_t v0[32], v1[32];
+                    tc_load32(tmem + tlane + h * 2 * kBN + cchunk * 32, v0);
+                    tc_load32(tmem + tlane + h * 2 * kBN + kBN + cchunk * 32, v1);
+                    tc_wait_ld();
+                    if (token < a.n_tokens) {
+                        float* yp = a.y + static_cast<size_t>(token) * a.rows + n0 + cchunk * 32;
 #pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        float o[4];
+                        for (int j = 0; j < 32; j += 4) {
+                            float o[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) o[e] = __fmaf_rn(a.lambda, __uint_as_float(v1[j + e]), __uint_as_float(v0[j + e]));
-                        const uint32_t f = n0 + cchunk * 32 + j;
-                        if (vec && f + 3 < a.rows) {
-                            *reinterpret_cast<float4*>(yp + j) = make_float4(o[0], o[1], o[2], o[3]);
-                        } else {
+                            for (int e = 0; e < 4; ++e) o[e] = __fmaf_rn(a.lambda, __uint_as_float(v1[j + e]), __uint_as_float(v0[j + e]));
+                            const uint32_t f = n0 + cchunk * 32 + j;
+                            if (vec && f + 3 < a.rows) {
+                                *reinterpret_cast<float4*>(yp + j) = make_float4(o[0], o[1], o[2], o[3]);
+                            } else {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                if (f + e < a.rows) yp[j + e] = o[e];
+                                for (int e = 0; e < 4; ++e)
+                                    if (f + e < a.rows) yp[j + e] = o[e];
+                            }
                         }
                     }
                 }
@@ -305,7 +331,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(Geo::kTmemCols) : "memory");
     }
 }
 
@@ -346,7 +372,9 @@ bool make_map(EncodeTiledFn enc, CUtensorMap* map, const void* ptr, uint64_t inn
 
 int linear_prepare()
 {
-    cudaError_t e = cudaFuncSetAttribute(linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kLinearSmem));
+    cudaError_t e = cudaFuncSetAttribute(linear_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(LinearGeom<1>::kSmem));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(linear_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(LinearGeom<2>::kSmem));
     if (e != cudaSuccess) (void)cudaGetLastError();
     return static_cast<int>(e);
 }
@@ -356,8 +384,15 @@ int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* 
 {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return static_cast<int>(cudaErrorNotSupported);
+    // 256 tokens per CTA (each staged weight tile then feeds two products) once that still gives every SM a tile
+    int dev = 0, sms = 0;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (ce != cudaSuccess) return static_cast<int>(ce);
+    const uint64_t tiles256 = static_cast<uint64_t>((rows + kBN - 1) / kBN) * ((n_tokens + 2 * kBM - 1) / (2 * kBM));
+    const int halves = (n_tokens > static_cast<uint32_t>(kBM) && tiles256 >= static_cast<uint64_t>(sms)) ? 2 : 1;
     CUtensorMap mx, mw, mm;
-    if (!make_map(enc, &mx, x, cols, n_tokens, kBM) || !make_map(enc, &mw, w0, cols, rows, kBN) || !make_map(enc, &mm, m_slot, cols, rows, kBN))
+    if (!make_map(enc, &mx, x, cols, n_tokens, halves * kBM) || !make_map(enc, &mw, w0, cols, rows, kBN) || !make_map(enc, &mm, m_slot, cols, rows, kBN))
         return static_cast<int>(cudaErrorInvalidValue);
     LinearArgs a;
     a.n_tokens = n_tokens;
@@ -368,8 +403,9 @@ int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* 
     a.slot = slot;
     a.task = task;
     a.y = y;
-    const dim3 grid((rows + kBN - 1) / kBN, (n_tokens + kBM - 1) / kBM);
-    linear_kernel<<<grid, kLinearThreads, kLinearSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
+    const dim3 grid((rows + kBN - 1) / kBN, (n_tokens + halves * kBM - 1) / (halves * kBM));
+    if (halves == 1) linear_kernel<1><<<grid, kLinearThreads, LinearGeom<1>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
+    else linear_kernel<2><<<grid, kLinearThreads, LinearGeom<2>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
     return static_cast<int>(cudaGetLastError());
 }
 

@@ -507,6 +507,55 @@ def run_ours(args):
                                 "GBps": byts / (ms * 1e-3) / 1e9, "frac_of_%s_peak" % peak_kind: byts / (ms * 1e-3) / 1e9 / peak,
                                 "speedup_per_model_vs_add": ops["add"]["ms_per_call"] / (ms / n_swap)}
 
+    # ---- a linear layer on the retrieved weight, the weight never written (tensor cores): the largest
+    #      repeated matrix of the set, bf16 weights and a bf16 superposition, 8192 tokens, timed alone
+    try:
+        reps_by_group = {}
+        for l, g in enumerate(w.group):
+            if w.rows[l] > 1 and w.cols[l] % 8 == 0:
+                reps_by_group.setdefault(g, []).append(l)
+        cand = [ls for ls in reps_by_group.values() if len(ls) > 1] or list(reps_by_group.values())
+        grp = max(cand, key=lambda ls: w.rows[ls[0]] * w.cols[ls[0]])[:4]
+        wl_lin = wl.subset(w, grp, w.name + ":linear").with_storage(wl.BF16).with_tasks(min(K, 4))
+        g_lin = torch.Generator(device=dev).manual_seed(1234)
+        lin_base = [(torch.randn(r, c, device=dev, generator=g_lin) * 0.02).to(torch.bfloat16) for r, c in zip(wl_lin.rows, wl_lin.cols)]
+        lin_tasks = [[(b.float() + 1e-3 * torch.randn(b.shape, device=dev, generator=g_lin)).to(torch.bfloat16) for b in lin_base]
+                     for _ in range(wl_lin.n_tasks)]
+        plan_lin = randes.Plan.from_workload(wl_lin, max_tasks=wl_lin.n_tasks, device=dev, m_dtype=wl.BF16)
+        M_lin = plan_lin.compress(lin_base, lin_tasks)
+        n_tok = 8192
+        rows_l, cols_l = wl_lin.rows[0], wl_lin.cols[0]
+        x_lin = torch.randn(n_tok, cols_l, device=dev, generator=g_lin).to(torch.bfloat16)
+        y_lin = torch.empty(n_tok, rows_l, device=dev, dtype=torch.float32)
+        pb_lin = randes.ptr_array(lin_base)
+        for _ in range(3):
+            randes.randes_linear(plan_lin.handle, 0, w.lam, 0, x_lin, n_tok, pb_lin, M_lin, y_lin, sh)
+        barrier()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        a.record(stream)
+        for i in range(reps):
+            randes.randes_linear(plan_lin.handle, i % wl_lin.n_tasks, w.lam, i % len(grp), x_lin, n_tok, pb_lin, M_lin, y_lin, sh)
+        z.record(stream)
+        barrier()
+        ms = max_over_ranks([a.elapsed_time(z)], world, dev)[0] / reps
+        flops = 4.0 * n_tok * rows_l * cols_l            # two products of 2 * tokens * rows * cols each
+        try:
+            with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+                tc_peak, tc_kind = float(json.load(f)["bf16_tflops"]), "measured burst"
+        except Exception:
+            tc_peak, tc_kind = 1590.0, "fallback"
+        extras["linear"] = {"layer_shape": [rows_l, cols_l], "tokens": n_tok, "ms_per_call": ms, "TFLOPs": flops / (ms * 1e-3) / 1e12,
+                            "bound": "tensor", "peak_TFLOPs": tc_peak, "peak_source": "%s bf16 GEMM (MEASURED_PEAKS.json)" % tc_kind
+                            if tc_kind != "fallback" else "fallback bf16 GEMM",
+                            "frac": flops / (ms * 1e-3) / 1e12 / tc_peak, "giveups": randes.randes_linear_giveups(),
+                            "note": "y = x W_0^T + lambda (x D) M^T, bf16 operands, fp32 accumulators; flops count both products"}
+        plan_lin.close()
+        del lin_base, lin_tasks, M_lin, x_lin, y_lin
+        torch.cuda.empty_cache()
+    except torch.OutOfMemoryError:
+        extras["linear"] = None
+
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region.
     #      Every step copies all its inputs from pinned host memory and all its results back.
     #      Copies and kernels are pipelined: the next step's inputs arrive in a second set of

@@ -992,6 +992,28 @@ static int randes_retrieve_batch_impl(randes_plan_t* plan, const uint32_t* task_
     a.out = plan->dev<void*>(plan->lay.task_ptrs);
     a.M = M;
     a.lambda = lambda;
+    a.members = plan->dev<uint32_t>(plan->lay.members);
+    // fp32 weights and superposition: the shuffled groups go through the kernel that stages M and W_0 of a
+    // whole group in shared memory (needs 16-byte aligned tensors there); the rest as before
+    bool staged = plan->storage == RANDES_F32 && plan->m_dtype == RANDES_F32 && !plan->group_units.empty() &&
+                  retrieve_batch_group_fits(plan->max_staged_group, n_tasks);
+    for (uint32_t l = 0; staged && l < plan->n_layers; ++l) {
+        if (!plan->group_staged[plan->layers[l].group]) continue;
+        staged = reinterpret_cast<uintptr_t>(base[l]) % 16 == 0;
+        for (uint32_t b = 0; staged && b < n_tasks; ++b) staged = reinterpret_cast<uintptr_t>(out[static_cast<size_t>(b) * plan->n_layers + l]) % 16 == 0;
+    }
+    if (staged) {
+        int ge = retrieve_batch_group_prepare();
+        if (ge) return fail_cuda(static_cast<cudaError_t>(ge), "set-up of the grouped batched retrieve kernel");
+        RetrieveBatchArgs g = a;
+        g.units = plan->dev<DevUnit>(plan->lay.staged_units) + plan->other_units.size();
+        g.n_units = static_cast<uint32_t>(plan->group_units.size());
+        ge = launch_retrieve_batch_groups(out_dtype, g, plan->max_staged_group, plan->sm_count, s);
+        if (ge) return fail_cuda(static_cast<cudaError_t>(ge), "launch of the grouped batched retrieve kernel");
+        ++g_launches;
+        a.units = plan->dev<DevUnit>(plan->lay.staged_units);
+        a.n_units = static_cast<uint32_t>(plan->other_units.size());
+    }
     if (a.n_units == 0) return RANDES_OK;
     const int grid = std::min<int>(plan->grid_batch[out_dtype], static_cast<int>(a.n_units));
     const int e = launch_retrieve_batch(plan->storage, out_dtype, plan->m_dtype, a, grid, s);

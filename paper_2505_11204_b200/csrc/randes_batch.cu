@@ -128,6 +128,113 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
     }
 }
 
+// Batched retrieve of a shuffled group, fp32 weights and superposition.  Task b needs, for layer
+// position p, the slot M[sigma_b^-1(p)]: every slot of the group is wanted by several tasks.  A
+// CTA takes a group unit (a few rows x one warp-wide column block of every member), copies the M
+// tiles of all slots and the W_0 tiles of all positions into shared memory once, and resolves
+// one record per (position, task) -- output tensor, which member the wanted slot is, Philox block
+// of sign bits -- in parallel over its threads.  After that the row loop only reads shared memory
+// and streams 16-byte stores: the call is bound by HBM writes, as it should be.
+constexpr uint32_t kBatchRecBytes = 32;   // {out pointer, slot member, pad, Philox block}
+
+__device__ __forceinline__ void store_plain(float* p, const float (&y)[4])
+{
+    *reinterpret_cast<float4*>(p) = make_float4(y[0], y[1], y[2], y[3]);
+}
+__device__ __forceinline__ void store_plain(__nv_bfloat16* p, const float (&y)[4])
+{
+    *reinterpret_cast<uint2*>(p) = make_uint2(Out<__nv_bfloat16>::pack(y[0], y[1]), Out<__nv_bfloat16>::pack(y[2], y[3]));
+}
+
+template <typename OT>
+__global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_group_kernel(const RetrieveBatchArgs a)
+{
+    constexpr int CPL = 4;
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_s = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
+    const uint32_t m_stash = smem_s, w_stash = smem_s + kStashBytes, s_rec = smem_s + 2 * kStashBytes;
+    const uint32_t L = a.n_layers, n = a.n_tasks;
+    const uint32_t sign_word = 16 + (lane >> 3) * 4u, sign_shift = (lane & 7) * 4u;
+    for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+        const DevUnit un = a.units[u];
+        const uint32_t* mem = a.members + un.layer;
+        const DevLayer l0 = a.layers[mem[0]];
+        const uint32_t G = l0.group_size, cols = l0.cols, Rn = un.nrows;
+        const uint32_t c = (un.cb0 * 32u + lane) * CPL;
+        const bool lane_on = c < cols;
+        const uint32_t off0 = un.row0 * cols + c;          // layers hold < 2^32 elements
+
+        if (lane_on) {
+            const uint32_t ntiles = G * Rn;
+            for (uint32_t q = warp; q < ntiles; q += kWarpsPerCta) {
+                const uint32_t m = q / Rn, r = q - m * Rn;
+                const uint32_t layer = mem[m];
+                const uint32_t off = off0 + r * cols;
+                cp_async16(m_stash + q * kStashTileBytes + lane * 16, static_cast<const float*>(a.M) + a.layers[layer].m_off + off);
+                cp_async16(w_stash + q * kStashTileBytes + lane * 16, static_cast<const float*>(a.base[layer]) + off);
+            }
+        }
+        cp_async_commit();
+        const uint32_t npairs = G * n;
+        for (uint32_t p = threadIdx.x; p < npairs; p += kThreadsPerCta) {
+            const uint32_t mp = p / n, b = p - mp * n;
+            const uint32_t pos = mem[mp];
+            const uint32_t fl = a.layers[pos].flags;
+            const uint32_t row = a.task_rows[b];
+            const uint32_t slot = (fl & kFlagShuffle) ? a.slot_of_pos[static_cast<size_t>(row) * L + pos] : pos;   // sigma_b^-1(p)
+            sts_ptrs(s_rec + p * kBatchRecBytes, a.out[static_cast<size_t>(b) * L + pos],
+                     reinterpret_cast<const void*>(static_cast<uintptr_t>(a.layers[slot].member)));
+            uint4 blk = make_uint4(0, 0, 0, 0);
+            if (fl & kFlagFlip) {
+                const DevTask tk = a.tasks[row];
+                blk = philox4x32_10(un.cb0, slot, kTagSign, tk.id, tk.key0, tk.key1);
+            }
+            sts128(s_rec + p * kBatchRecBytes + 16, blk);
+        }
+        cp_async_wait<0>();
+        __syncthreads();   // stashes and records are complete and visible to every warp
+
+        if (lane_on) {
+            const uint32_t n_chunks = (Rn + kItemRows - 1) / kItemRows;
+            const uint32_t n_items = G * n_chunks;
+            for (uint32_t item = warp; item < n_items; item += kWarpsPerCta) {
+                const uint32_t mp = item / n_chunks;
+                const uint32_t r0 = (item - mp * n_chunks) * kItemRows;
+                const uint32_t nr = min(kItemRows, Rn - r0);
+                float wv[kItemRows][CPL];
+#pragma unroll
+                for (int r = 0; r < static_cast<int>(kItemRows); ++r)
+                    if (r < static_cast<int>(nr)) Store<float>::widen(lds128(w_stash + (mp * Rn + r0 + r) * kStashTileBytes + lane * 16), wv[r]);
+                const uint32_t off = off0 + r0 * cols;
+                uint32_t rec = s_rec + mp * n * kBatchRecBytes;
+                for (uint32_t b = 0; b < n; ++b, rec += kBatchRecBytes) {
+                    OT* op = reinterpret_cast<OT*>(const_cast<char*>(lds_ptr(rec))) + off;
+                    const uint32_t member = lds_u32(rec + 8);
+                    const uint32_t bits = lds_u32(rec + sign_word) >> sign_shift;
+                    float lam[CPL];
+#pragma unroll
+                    for (int e = 0; e < CPL; ++e) lam[e] = flip(a.lambda, ((bits >> e) & 1u) << 31);
+                    const uint32_t mb = m_stash + (member * Rn + r0) * kStashTileBytes + lane * 16;
+#pragma unroll
+                    for (int r = 0; r < static_cast<int>(kItemRows); ++r) {
+                        if (r < static_cast<int>(nr)) {
+                            float m[CPL], y[CPL];
+                            Store<float>::widen(lds128(mb + r * kStashTileBytes), m);
+#pragma unroll
+                            for (int e = 0; e < CPL; ++e) y[e] = __fmaf_rn(lam[e], m[e], wv[r][e]);
+                            store_plain(op + static_cast<size_t>(r) * cols, y);
+                        }
+                    }
+                }
+            }
+        }
+        __syncthreads();   // every warp is done with the stashes and records before the next unit overwrites them
+    }
+}
+
+size_t batch_group_smem(uint32_t pairs) { return 2 * static_cast<size_t>(kStashBytes) + static_cast<size_t>(pairs) * kBatchRecBytes; }
+
 template <typename K> int occupancy(K kernel)
 {
     int n = 0;
@@ -154,6 +261,37 @@ int launch_retrieve_batch(int storage_dtype, int out_dtype, int m_dtype, const R
                 return static_cast<int>(cudaGetLastError());
             });
         });
+    });
+}
+
+int retrieve_batch_group_prepare()
+{
+    cudaError_t e = cudaFuncSetAttribute(retrieve_batch_group_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(retrieve_batch_group_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) (void)cudaGetLastError();
+    return static_cast<int>(e);
+}
+
+bool retrieve_batch_group_fits(uint32_t max_group, uint32_t n_tasks)
+{
+    return max_group >= 1 && max_group * kStashTileBytes <= kStashBytes && batch_group_smem(max_group * n_tasks) <= 227 * 1024;
+}
+
+int launch_retrieve_batch_groups(int out_dtype, const RetrieveBatchArgs& a, uint32_t max_group, int sm_count, void* stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t smem = batch_group_smem(max_group * a.n_tasks);
+    return with_type(out_dtype, [&](auto ot) {
+        typedef typename decltype(ot)::type OT;
+        int per_sm = 0;
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, retrieve_batch_group_kernel<OT>, kThreadsPerCta, smem);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return static_cast<int>(e); }
+        if (per_sm <= 0) return static_cast<int>(cudaErrorInvalidConfiguration);
+        const uint64_t want = static_cast<uint64_t>(sm_count) * per_sm;
+        const int grid = static_cast<int>(want < a.n_units ? want : a.n_units);
+        retrieve_batch_group_kernel<OT><<<grid, kThreadsPerCta, smem, s>>>(a);
+        return static_cast<int>(cudaGetLastError());
     });
 }
 

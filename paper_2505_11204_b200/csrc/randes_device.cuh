@@ -280,6 +280,12 @@ __device__ __forceinline__ const char* lds_ptr(uint32_t saddr)
     asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(saddr));
     return reinterpret_cast<const char*>(v);
 }
+__device__ __forceinline__ uint32_t lds_u32(uint32_t saddr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
+    return v;
+}
 __device__ __forceinline__ uint32_t lds_u16(uint32_t saddr)
 {
     unsigned short v;

@@ -43,12 +43,6 @@ __device__ __forceinline__ unsigned long long lds_u64(uint32_t saddr)
     asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(saddr));
     return v;
 }
-__device__ __forceinline__ uint32_t lds_u32(uint32_t saddr)
-{
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
-    return v;
-}
 
 // Per (slot, task) pair of a unit, in shared memory: the task's source tensor W_i[sigma_i(l)],
 // which member of the group that source layer is (-> its W_0 tile in the stash), and the

@@ -123,6 +123,7 @@ struct RetrieveBatchArgs {
     void* const* out;              // device array [n_tasks][n_layers]
     const void* M;
     float lambda;
+    const uint32_t* members;       // layers of every group, group after group, in member order (group units only)
 };
 
 constexpr int kGramAnchors = 4;   // rows of the Gram matrix produced per pass
@@ -160,6 +161,10 @@ int gram_ctas_per_sm(int storage_dtype);
 // randes_batch.cu
 int launch_retrieve_batch(int storage_dtype, int out_dtype, int m_dtype, const RetrieveBatchArgs& a, int grid, void* stream);
 int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype);
+// batched retrieve over group units (fp32 weights and superposition): M and W_0 tiles of a whole group staged in shared memory
+int retrieve_batch_group_prepare();
+bool retrieve_batch_group_fits(uint32_t max_group, uint32_t n_tasks);
+int launch_retrieve_batch_groups(int out_dtype, const RetrieveBatchArgs& a, uint32_t max_group, int sm_count, void* stream);
 
 
 // randes_linear.cu: y = x W_0^T + lambda (x D) M_slot^T on the tensor cores (bf16 operands, fp32 accumulators).

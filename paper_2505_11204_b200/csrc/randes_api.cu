@@ -1103,9 +1103,9 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
     int rc;
     if ((rc = check_m(M))) return rc;
     if (!base || !base[layer]) return fail(RANDES_INVALID_ARGUMENT, "base or base[%u] is NULL", layer);
-    if (!x || !y) return fail(RANDES_INVALID_ARGUMENT, "x or y is NULL");
     const uint32_t rows = plan->layers[layer].rows, cols = plan->layers[layer].cols;
-    if (n_tokens == 0 || rows == 0 || cols == 0) return RANDES_OK;
+    if (n_tokens == 0 || rows == 0 || cols == 0) return RANDES_OK;   // nothing to compute (x and y may be NULL then)
+    if (!x || !y) return fail(RANDES_INVALID_ARGUMENT, "x or y is NULL");
     if (cols % 8) return fail(RANDES_INVALID_ARGUMENT, "layer %u: cols = %u is not a multiple of 8 (16-byte rows for the tensor maps)", layer, cols);
     if (reinterpret_cast<uintptr_t>(x) % 16 || reinterpret_cast<uintptr_t>(base[layer]) % 16)
         return fail(RANDES_MISALIGNED, "x and base[%u] must be 16-byte aligned", layer);

@@ -83,6 +83,36 @@ def test_linear_wide_layer_many_k_steps():
     _run(w, [257], layers=[1])
 
 
+def test_linear_unaligned_output_zero_tokens_and_host_only_plan():
+    """y only 4-byte aligned (element-wise stores), no tokens (nothing launched), and a plan built without a device
+    workspace (the call needs none)."""
+    w = _workload([(136, 128, 2)], [S | F], n_tasks=2)
+    ids, seeds = list(w.task_ids), list(w.seeds)
+    base, tasks = wl.model_set(w, ids)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, max_tasks=2, m_dtype=wl.BF16)
+    M_dev = plan.compress(d_base, d_tasks)
+    M_ref = ro.compress(w.spec, w.storage, ids, seeds, base, tasks, m_dtype=wl.BF16)
+    host_plan = randes.Plan.from_workload(w, max_tasks=2, m_dtype=wl.BF16, host_only=True)
+    x = _bf16_normal(np.random.default_rng(9), (45, 128))
+    buf = torch.full((45 * 136 + 1,), float("nan"), dtype=torch.float32, device="cuda")
+    y = buf[1:].view(45, 136)                                  # 4 bytes past a 16-byte boundary
+    before = randes.randes_launch_count()
+    host_plan.linear(ids[1], 0.3, 1, to_dev(x), d_base, M_dev, y=y)
+    assert randes.randes_launch_count() == before + 1
+    y_ref, y_abs = ro.linear(w.spec, w.storage, ids[1], seeds[1], 0.3, 1, x, base, M_ref, m_dtype=wl.BF16)
+    assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - y_ref) <= (2 * 128 + 2) * 2.0 ** -24 * y_abs + 1e-30)
+    assert bool(torch.isnan(buf[0]))                           # nothing before y was written
+    empty = torch.zeros((0, 128), dtype=torch.bfloat16, device="cuda")
+    randes.randes_linear(plan.handle, ids[0], 0.3, 0, empty, 0, randes.ptr_array(d_base), M_dev, y, torch.cuda.current_stream().cuda_stream)
+    assert randes.randes_launch_count() == before + 1          # no tokens: no launch
+    with pytest.raises(randes.RandesError) as e:
+        plan.linear(77, 0.3, 0, to_dev(x), d_base, M_dev)
+    assert e.value.code == randes.UNKNOWN_TASK
+    assert randes.randes_linear_giveups() == 0
+    plan.close(); host_plan.close()
+
+
 def test_linear_rejects_what_it_cannot_run():
     w = _workload([(16, 12, 1)], [F], n_tasks=1)           # cols not a multiple of 8
     base, tasks = wl.model_set(w, w.task_ids)

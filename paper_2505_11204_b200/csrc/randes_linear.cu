@@ -12,9 +12,11 @@
 //     x tile [128 or 256 tokens x 64], W_0 tile [128 features x 64], M tile [128 features x 64];
 //   * (x D) M^T = x (M D)^T: four warps flip, in place, the sign bits of the M tile's 64 columns
 //     (bf16 sign bit XOR: exact), Philox bits generated in registers -- no second buffer;
-//   * one thread issues tcgen05.mma (M = 128, N = 128, K = 16) into fp32 accumulators in tensor
-//     memory, per block of 128 tokens: acc0 += x W_0^T, acc1 += x (M D)^T; with 256 tokens per
-//     CTA each weight tile feeds two products (1.5 x the flops per byte staged);
+//   * the W_0 tile and the flipped M tile lie back to back in shared memory and form one
+//     [256 x 64] operand: one thread issues tcgen05.mma with M = 128, N = 256, K = 16, which fills
+//     both fp32 accumulators of a block of 128 tokens in tensor memory (columns 0-127: x W_0^T,
+//     128-255: x (M D)^T) and reads the x tile once; with 256 tokens per CTA each weight tile
+//     feeds two such products (1.5 x the flops per byte staged);
 //   * the epilogue reads the accumulators with tcgen05.ld and stores fma(lambda, acc1, acc0).
 //
 // lambda stays in fp32 and is applied once per output, so the operands keep their stored bits.
@@ -146,8 +148,8 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
            | (2ull << 61);                                    // 128-byte swizzle
 }
 
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = kBN.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kBN >> 3) << 17) | (static_cast<uint32_t>(kBM >> 4) << 24);
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 2 kBN (both accumulators at once).
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>((2 * kBN) >> 3) << 17) | (static_cast<uint32_t>(kBM >> 4) << 24);
 
 template <int HALVES>
 __global__ void __launch_bounds__(kLinearThreads, 1)
@@ -226,28 +228,21 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 ok = mbar_wait(bar_full(s), ph, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t st = smem_base + s * kStageBytes;
-                const uint64_t dw = smem_desc_sw128(st + kOffW);
-                const uint64_t dm = smem_desc_sw128(st + kOffM);
-                // x W_0^T first: it does not depend on the flip
-#pragma unroll
-                for (int h = 0; h < HALVES; ++h) {
-                    const uint64_t dx = smem_desc_sw128(st + h * kTileBytes);
-#pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k)   // 16 bf16 columns = 32 bytes = 2 units of the descriptor's start address
-                        tc_mma_bf16(tmem + h * 2 * kBN, dx + 2 * k, dw + 2 * k, kIdesc, (kk | k) ? 1u : 0u);
-                }
                 if (a.flip) {
                     ok = mbar_wait(bar_flipped(s), ph, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                 }
+                // The W_0 tile and the (flipped) M tile lie back to back: one [256 x 64] B operand, so ONE product
+                // x [W_0; M D]^T with N = 256 fills both accumulators (columns 0-127 and 128-255) and reads the x tile once.
+                const uint32_t st = smem_base + s * kStageBytes;
+                const uint64_t dwm = smem_desc_sw128(st + kOffW);
 #pragma unroll
                 for (int h = 0; h < HALVES; ++h) {
                     const uint64_t dx = smem_desc_sw128(st + h * kTileBytes);
 #pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k)
-                        tc_mma_bf16(tmem + h * 2 * kBN + kBN, dx + 2 * k, dm + 2 * k, kIdesc, (kk | k) ? 1u : 0u);
+                    for (int k = 0; k < kBK / 16; ++k)   // 16 bf16 columns = 32 bytes = 2 units of the descriptor's start address
+                        tc_mma_bf16(tmem + h * 2 * kBN, dx + 2 * k, dwm + 2 * k, kIdesc, (kk | k) ? 1u : 0u);
                 }
                 tc_commit(bar_empty(s));     // the stage is free once these products have read it
             }

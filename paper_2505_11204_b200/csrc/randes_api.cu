@@ -144,7 +144,7 @@ void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, s
         const size_t before = units.size();
         const uint32_t nb = (cols + wcols - 1) / wcols;
         if (is_staged) {
-            const uint32_t R = group_unit_rows(static_cast<uint32_t>(members.size()));
+            const uint32_t R = group_unit_rows(static_cast<uint32_t>(members.size()), storage);
             for (uint32_t r0 = 0; r0 < rows; r0 += R)
                 for (uint32_t cb0 = 0; cb0 < nb; ++cb0) {
                     DevUnit u;
@@ -181,7 +181,7 @@ void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, s
 // Could group g (of `size` members, `cols` wide) be cut into group units at all?
 bool group_fits_stash(size_t size, uint32_t cols, int storage)
 {
-    return size >= 2 && cols % cols_per_lane(storage) == 0 && group_unit_rows(static_cast<uint32_t>(size)) >= 1;
+    return size >= 2 && cols % cols_per_lane(storage) == 0 && group_unit_rows(static_cast<uint32_t>(size), storage) >= 1;
 }
 
 // Upper bound of the length of a unit list in which any subset of the groups is staged.
@@ -561,9 +561,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
                 any = any || shuffled;
                 if (shuffled) p->max_staged_group = std::max<uint32_t>(p->max_staged_group, static_cast<uint32_t>(mem.size()));
             }
-            // fp32 weights only: with bf16 weights the row loop is bound by instruction issue (two
-            // elements to widen per 4 bytes), and the per-layer kernel was measured faster
-            if (any && p->storage == RANDES_F32) {
+            if (any) {
                 build_units(layers, n_layers, p->storage, p->group_units, &p->group_staged, &member_base, kStagedGroups);
                 build_units(layers, n_layers, p->storage, p->other_units, &p->group_staged, &member_base, kOtherGroups);
             }

@@ -12,8 +12,9 @@
 // HBM, through a per-thread cp.async ring (each lane reads back only what it copied, so the
 // row loop needs no barrier), and W_0 and the signs come from shared memory.
 //
-// A warp takes (slot, block of kItemRows rows) items in turn and runs ONE software pipeline
-// over all its items: stage = one task x two rows.  Sums run in task order, every output
+// A warp takes (slot, block of rows) items in turn and runs ONE software pipeline over all its
+// items: stage = one task x two rows (fp32 weights, items of four rows) or one task x three rows
+// (bf16 weights, items of three rows: the sign decode is shared by more rows).  Sums run in task order, every output
 // element is written by one thread: results are bit-reproducible and equal to the per-layer
 // kernel's.
 #include <cuda_bf16.h>
@@ -30,8 +31,18 @@ namespace {
 
 using namespace device;
 
-constexpr uint32_t kMaxGroup = kStashBytes / kStashTileBytes;   // members whose tiles fit the stash at one row each
+constexpr uint32_t kMaxGroup = kStashBytes / kStashTileBytes;   // members whose tiles fit the largest stash at one row each
 constexpr uint32_t kOffTableBytes = kMaxGroup * 8;
+
+// rows per stage (SR), rows per item (IR) and stash size per weight type
+template <typename ST> struct GroupGeom;
+template <> struct GroupGeom<float> {
+    static constexpr uint32_t SR = 2, IR = item_rows(0), kStash = stash_bytes(0);
+};
+template <> struct GroupGeom<__nv_bfloat16> {
+    static constexpr uint32_t SR = 3, IR = item_rows(1), kStash = stash_bytes(1);
+};
+constexpr uint32_t stage_rows(int storage_dtype) { return storage_dtype == 1 ? 3u : 2u; }
 
 __device__ __forceinline__ void sts_u64(uint32_t saddr, unsigned long long v)
 {
@@ -66,7 +77,7 @@ struct Cursor {
     uint32_t m_off;      // shared address of the slot's offset in M
 };
 
-template <uint32_t REC>
+template <uint32_t REC, uint32_t IR>
 __device__ __forceinline__ void cursor_set(Cursor& c, uint32_t item, uint32_t n_chunks, uint32_t Rn, uint32_t nt, uint32_t s_rec,
                                            uint32_t off0, uint32_t cols)
 {
@@ -74,26 +85,26 @@ __device__ __forceinline__ void cursor_set(Cursor& c, uint32_t item, uint32_t n_
     const uint32_t ms = item / n_chunks;
     c.m_off = s_rec - kOffTableBytes + ms * 8;
     const uint32_t chunk = item - ms * n_chunks;
-    c.row = chunk * kItemRows;
-    c.rows_left = min(kItemRows, Rn - c.row);
+    c.row = chunk * IR;
+    c.rows_left = min(IR, Rn - c.row);
     c.off = off0 + c.row * cols;
     c.rec_begin = c.rec = s_rec + ms * nt * REC;
     c.rec_end = c.rec_begin + nt * REC;
 }
 
-template <uint32_t REC>
+template <uint32_t REC, uint32_t IR, uint32_t SR>
 __device__ __forceinline__ void cursor_next(Cursor& c, uint32_t n_chunks, uint32_t Rn, uint32_t nt, uint32_t s_rec, uint32_t off0,
                                             uint32_t cols)
 {
     c.rec += REC;
     if (c.rec != c.rec_end) return;
-    if (c.rows_left > 2) {          // next row pair of the same slot
+    if (c.rows_left > SR) {         // next rows of the same slot
         c.rec = c.rec_begin;
-        c.row += 2;
-        c.rows_left -= 2;
-        c.off += 2 * cols;
+        c.row += SR;
+        c.rows_left -= SR;
+        c.off += SR * cols;
     } else {                        // next item; may run past the last one: never used then
-        cursor_set<REC>(c, c.item + kWarpsPerCta, n_chunks, Rn, nt, s_rec, off0, cols);
+        cursor_set<REC, IR>(c, c.item + kWarpsPerCta, n_chunks, Rn, nt, s_rec, off0, cols);
     }
 }
 
@@ -105,8 +116,11 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
     typedef PairRecord<HB> Rec;
     constexpr uint32_t REC = Rec::kBytes;
     constexpr uint32_t ES = sizeof(ST);
-    constexpr uint32_t kRingBytes = NSTAGE * 2 * kSlotBytes;
-    constexpr uint32_t kStageBytes = 2 * kSlotBytes;
+    constexpr uint32_t SR = GroupGeom<ST>::SR;             // rows per stage
+    constexpr uint32_t IR = GroupGeom<ST>::IR;             // rows per item
+    constexpr uint32_t kStash = GroupGeom<ST>::kStash;
+    constexpr uint32_t kRingBytes = NSTAGE * SR * kSlotBytes;
+    constexpr uint32_t kStageBytes = SR * kSlotBytes;
     typedef MTile<MT, CPL> MTl;
     extern __shared__ __align__(16) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -114,7 +128,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
     const uint32_t ring = smem_s + threadIdx.x * 16;
     const uint32_t ring_end = ring + kRingBytes;
     const uint32_t stash = smem_s + kRingBytes;
-    const uint32_t s_off = stash + kStashBytes;          // per member: first element of its slot in M
+    const uint32_t s_off = stash + kStash;               // per member: first element of its slot in M
     const uint32_t s_rec = s_off + kOffTableBytes;       // per (slot, task): PairRecord
     const uint32_t L = a.n_layers, nt = a.n_tasks;
     // where this lane's sign bits sit inside a record
@@ -163,15 +177,15 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
         __syncthreads();   // stash and tables are complete and visible to every warp
 
         if (lane_on) {
-            const uint32_t n_chunks = (Rn + kItemRows - 1) / kItemRows;
+            const uint32_t n_chunks = (Rn + IR - 1) / IR;
             const uint32_t n_items = G * n_chunks;
             uint32_t N = 0;   // stages of this warp
             for (uint32_t item = warp; item < n_items; item += kWarpsPerCta) {
                 const uint32_t chunk = item % n_chunks;
-                N += (min(kItemRows, Rn - chunk * kItemRows) + 1) / 2 * nt;
+                N += (min(IR, Rn - chunk * IR) + SR - 1) / SR * nt;
             }
             Cursor ci, cc;
-            cursor_set<REC>(ci, warp, n_chunks, Rn, nt, s_rec, off0, cols);
+            cursor_set<REC, IR>(ci, warp, n_chunks, Rn, nt, s_rec, off0, cols);
             cc = ci;
             uint32_t to_issue = N, stage_i = ring, stage_c = ring;
             const uint32_t stash_lane = stash + lane * 16;
@@ -180,9 +194,10 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
 
             auto issue = [&]() {
                 const char* src = lds_ptr(ci.rec + Rec::kPtr) + static_cast<size_t>(ci.off) * ES;
-                cp_async16(stage_i, src);
-                if (ci.rows_left > 1) cp_async16(stage_i + kSlotBytes, src + row_bytes);
-                cursor_next<REC>(ci, n_chunks, Rn, nt, s_rec, off0, cols);
+#pragma unroll
+                for (uint32_t r = 0; r < SR; ++r)
+                    if (r == 0 || ci.rows_left > r) cp_async16(stage_i + r * kSlotBytes, src + r * row_bytes);
+                cursor_next<REC, IR, SR>(ci, n_chunks, Rn, nt, s_rec, off0, cols);
                 stage_i += kStageBytes;
                 if (stage_i == ring_end) stage_i = ring;
                 --to_issue;
@@ -193,14 +208,14 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
                 if (to_issue) issue();
                 cp_async_commit();
             }
-            f32x2 acc[2][CPL / 2];
+            f32x2 acc[SR][CPL / 2];
             for (uint32_t it = 0; it < N; ++it) {
                 if (to_issue) issue();
                 cp_async_commit();
                 cp_async_wait<NSTAGE - 1>();   // all but the newest NSTAGE-1 groups have landed: stage_c is ready
                 if (cc.rec == cc.rec_begin) {
 #pragma unroll
-                    for (int r = 0; r < 2; ++r)
+                    for (uint32_t r = 0; r < SR; ++r)
 #pragma unroll
                         for (int e = 0; e < CPL / 2; ++e) acc[r][e] = 0ull;
                 }
@@ -211,10 +226,10 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
                 for (int e = 0; e < CPL / 2; ++e)
                     sg[e] = pack2(((bits << (31 - 2 * e)) & 0x80000000u) | one, ((bits << (30 - 2 * e)) & 0x80000000u) | one);
                 const uint32_t b0 = stash_lane + member * member_bytes + cc.row * kStashTileBytes;
-                const bool two = cc.rows_left > 1;
+                const uint32_t rows_here = cc.rows_left;
 #pragma unroll
-                for (int r = 0; r < 2; ++r) {
-                    if (r == 0 || two) {
+                for (uint32_t r = 0; r < SR; ++r) {
+                    if (r == 0 || rows_here > r) {
                         f32x2 d[CPL / 2], b[CPL / 2];
                         Store<ST>::widen2(lds128(stage_c + r * kSlotBytes), d);
                         Store<ST>::widen2(lds128(b0 + r * kStashTileBytes), b);
@@ -225,8 +240,8 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
                 if (cc.rec + REC == cc.rec_end) {   // last task: the rows of this slot are complete
                     MT* mp = static_cast<MT*>(a.M) + lds_u64(cc.m_off) + cc.off;
 #pragma unroll
-                    for (int r = 0; r < 2; ++r) {
-                        if (r == 0 || two) {
+                    for (uint32_t r = 0; r < SR; ++r) {
+                        if (r == 0 || rows_here > r) {
                             float v[CPL];
 #pragma unroll
                             for (int e = 0; e < CPL / 2; ++e) unpack2(acc[r][e], v[2 * e], v[2 * e + 1]);
@@ -234,7 +249,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
                         }
                     }
                 }
-                cursor_next<REC>(cc, n_chunks, Rn, nt, s_rec, off0, cols);
+                cursor_next<REC, IR, SR>(cc, n_chunks, Rn, nt, s_rec, off0, cols);
                 stage_c += kStageBytes;
                 if (stage_c == ring_end) stage_c = ring;
             }
@@ -248,7 +263,9 @@ template <typename T> struct Tag { typedef T type; };
 template <typename F> int with_type(int dtype, F&& f) { return dtype == 0 ? f(Tag<float>{}) : f(Tag<bf16>{}); }
 template <typename F> int with_stages(int nstage, F&& f)
 {
-    return nstage >= 6 ? f(std::integral_constant<int, 6>{}) : (nstage == 5 ? f(std::integral_constant<int, 5>{}) : f(std::integral_constant<int, 4>{}));
+    return nstage >= 6 ? f(std::integral_constant<int, 6>{})
+                       : (nstage == 5 ? f(std::integral_constant<int, 5>{})
+                                      : (nstage == 4 ? f(std::integral_constant<int, 4>{}) : f(std::integral_constant<int, 3>{})));
 }
 
 constexpr size_t kMaxDynamicSmem = 227 * 1024;
@@ -257,8 +274,12 @@ constexpr size_t kTwoCtaSmem = (228 * 1024 - 2 * 1024) / 2;   // two CTAs per SM
 size_t group_smem_bytes(int storage_dtype, int nstage, uint32_t pair_cap)
 {
     const size_t hb = storage_dtype == 1 ? 2 : 1;
-    return static_cast<size_t>(nstage) * 2 * kSlotBytes + kStashBytes + kOffTableBytes + static_cast<size_t>(pair_cap) * (16 + 16 * hb);
+    return static_cast<size_t>(nstage) * stage_rows(storage_dtype) * kSlotBytes + stash_bytes(storage_dtype) + kOffTableBytes +
+           static_cast<size_t>(pair_cap) * (16 + 16 * hb);
 }
+// ring depths tried, deepest first: 12 slots per thread at most
+int max_stages(int storage_dtype) { return storage_dtype == 1 ? 4 : 6; }
+int min_stages(int storage_dtype) { return storage_dtype == 1 ? 3 : 4; }
 
 }  // namespace
 
@@ -271,6 +292,7 @@ int compress_group_prepare(int storage_dtype, int m_dtype)
             cudaError_t e = cudaFuncSetAttribute(compress_group_kernel<ST, MT, 6>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynamicSmem));
             if (e == cudaSuccess) e = cudaFuncSetAttribute(compress_group_kernel<ST, MT, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynamicSmem));
             if (e == cudaSuccess) e = cudaFuncSetAttribute(compress_group_kernel<ST, MT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynamicSmem));
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(compress_group_kernel<ST, MT, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kMaxDynamicSmem));
             if (e != cudaSuccess) (void)cudaGetLastError();
             return static_cast<int>(e);
         });
@@ -279,7 +301,8 @@ int compress_group_prepare(int storage_dtype, int m_dtype)
 
 bool compress_group_fits(int storage_dtype, uint32_t max_group, uint32_t n_tasks)
 {
-    return max_group >= 1 && max_group <= kMaxGroup && group_smem_bytes(storage_dtype, 4, max_group * n_tasks) <= kMaxDynamicSmem;
+    return max_group >= 1 && max_group * kStashTileBytes <= stash_bytes(storage_dtype) &&
+           group_smem_bytes(storage_dtype, min_stages(storage_dtype), max_group * n_tasks) <= kMaxDynamicSmem;
 }
 
 int launch_compress_groups(int storage_dtype, int m_dtype, const CompressGroupArgs& a, uint32_t max_group, int sm_count, void* stream)
@@ -288,9 +311,9 @@ int launch_compress_groups(int storage_dtype, int m_dtype, const CompressGroupAr
     const uint32_t pair_cap = max_group * a.n_tasks;
     // the deepest ring that still leaves room for two CTAs per SM; failing that, the deepest ring with one
     int nstage = 0;
-    for (int n = 6; n >= 4 && !nstage; --n)
+    for (int n = max_stages(storage_dtype); n >= min_stages(storage_dtype) && !nstage; --n)
         if (group_smem_bytes(storage_dtype, n, pair_cap) <= kTwoCtaSmem) nstage = n;
-    for (int n = 6; n >= 4 && !nstage; --n)
+    for (int n = max_stages(storage_dtype); n >= min_stages(storage_dtype) && !nstage; --n)
         if (group_smem_bytes(storage_dtype, n, pair_cap) <= kMaxDynamicSmem) nstage = n;
     if (!nstage) return static_cast<int>(cudaErrorInvalidConfiguration);
     const size_t smem = group_smem_bytes(storage_dtype, nstage, pair_cap);

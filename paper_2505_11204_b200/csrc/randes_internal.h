@@ -51,13 +51,19 @@ static_assert(sizeof(DevUnit) == 16, "DevUnit layout");
 // warps sum the tasks' deltas slot by slot, subtracting W_0[sigma_i(l)] from the stash.  `layer`
 // is then the index of the group's first entry in the member table.
 constexpr uint32_t kStashTileBytes = 512;             // 32 lanes x 16 bytes
-constexpr uint32_t kStashBytes = 48 * 1024;
-constexpr uint32_t kItemRows = 4;                     // rows of one slot a warp sums in one go
+constexpr uint32_t kStashBytes = 48 * 1024;           // fp32 weights
+constexpr uint32_t kItemRows = 4;                     // rows of one slot a warp sums in one go, fp32 weights
+// With bf16 weights a lane's 16 bytes hold twice the columns, so the sign records are twice as large and the
+// row loop is bound by instruction issue: items are 3 rows taken as one stage (more rows per sign decode), and
+// the stash is 36 KiB so that records for 20 tasks x 24 members still fit beside two resident CTAs.
+constexpr uint32_t stash_bytes(int storage_dtype) { return storage_dtype == 1 ? 36u * 1024u : kStashBytes; }
+constexpr uint32_t item_rows(int storage_dtype) { return storage_dtype == 1 ? 3u : kItemRows; }
 // rows per group unit for a group of G members (0: the group is too large for the stash)
-constexpr uint32_t group_unit_rows(uint32_t G)
+constexpr uint32_t group_unit_rows(uint32_t G, int storage_dtype)
 {
-    const uint32_t fit = G ? kStashBytes / kStashTileBytes / G : 0;
-    return fit >= 4 * kItemRows ? 4 * kItemRows : (fit >= kItemRows ? fit / kItemRows * kItemRows : fit);
+    const uint32_t ir = item_rows(storage_dtype);
+    const uint32_t fit = G ? stash_bytes(storage_dtype) / kStashTileBytes / G : 0;
+    return fit >= 4 * ir ? 4 * ir : (fit >= ir ? fit / ir * ir : fit);
 }
 
 struct DevTask {

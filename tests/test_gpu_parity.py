@@ -406,15 +406,17 @@ def test_thirty_two_tasks_exactly_and_wide_single_row():
     run_full_cycle(make_workload([(1, 100000, 1), (3, 4096, 2)], n_tasks=32), out_dtypes=(wl.F32,), extra_task=False)
 
 
+@pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
 @pytest.mark.parametrize("n_tasks", [2, 5, 32])
-def test_large_and_partly_shuffled_groups(n_tasks):
+def test_large_and_partly_shuffled_groups(n_tasks, storage):
     """Compress of shuffled groups runs over group units (W_0 of all members staged in shared memory):
-    groups of 30, 48 and 50 members (3, 2 and 1 rows per unit), 97 members (too large: per-layer path),
-    a group where only every second member is shuffled, ragged rows and widths; 2 to 32 tasks (32 tasks
-    x 48 members exceed the tables that fit beside two resident CTAs)."""
-    shapes = [(9, 132, 30), (5, 256, 50), (3, 128, 97), (6, 260, 48), (11, 520, 7), (21, 128, 4), (2, 4, 24)]
-    flags = [S | F, S | F, S | F, S, S | F | randes.SKIP(2), S | F, S | F]
-    run_full_cycle(make_workload(shapes, flags=flags, n_tasks=n_tasks), out_dtypes=(wl.F32,), extra_task=False)
+    groups of 30, 48 and 50 members (3, 2 and 1 rows per unit with fp32 weights; 2, 1 and 1 with bf16),
+    97 members (too large: per-layer path), a group where only every second member is shuffled, ragged rows
+    and widths (with bf16 weights the widths that are no multiple of 8 take the element-wise path); 2 to 32
+    tasks (32 tasks x 48 members exceed the tables that fit beside two resident CTAs)."""
+    shapes = [(9, 132, 30), (5, 256, 50), (3, 128, 97), (6, 260, 48), (11, 520, 7), (21, 128, 4), (2, 4, 24), (7, 264, 48)]
+    flags = [S | F, S | F, S | F, S, S | F | randes.SKIP(2), S | F, S | F, S | F]
+    run_full_cycle(make_workload(shapes, flags=flags, n_tasks=n_tasks, storage=storage), out_dtypes=(wl.F32,), extra_task=False)
 
 
 def test_random_plans():

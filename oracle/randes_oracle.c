@@ -66,6 +66,8 @@
 #define RO_SHIFT 4u                      /* deterministic rotation instead of a random permutation */
 #define RO_SKIP(flags) (((flags) >> 8) & 0xFFu) /* every k-th member of a group takes part; 0 and 1 = all */
 
+#define RO_GAUSS (1u << 16)              /* Gaussian-like diagonal context (Section 5.5, "RD") instead of the +-1 one */
+#define RO_TAG_GAUS 0x47415553u /* "GAUS" */
 #define RO_TAG_PERM 0x5045524Du /* "PERM" */
 #define RO_TAG_SIGN 0x5349474Eu /* "SIGN" */
 
@@ -147,6 +149,33 @@ void ro_sign_row(uint64_t seed, uint32_t task_id, uint32_t slot, uint32_t cols, 
 }
 
 /* ------------------------------------------------------------------------ */
+/* Section 5.5, the "RD" context matrix: a diagonal with (approximately)     */
+/* standard normal entries instead of +-1; not orthogonal, and its inverse   */
+/* divides.  The paper names no generator.  Here: the sum of twelve uniforms */
+/* minus six (mean 0, variance 1), every step an exactly rounded fp32        */
+/* operation so that any IEEE machine gets the same bits: the twelve words   */
+/* of Philox blocks 3c, 3c+1, 3c+2 of the (slot, task) stream, each reduced  */
+/* to u = (word >> 8) * 2^-24, added left to right.  A zero (which could not */
+/* be inverted) is replaced by one.                                          */
+/* ------------------------------------------------------------------------ */
+float ro_gauss(uint64_t seed, uint32_t task_id, uint32_t slot, uint32_t col)
+{
+    uint32_t key[2], ctr[4], blk[4];
+    float sum = 0.0f;
+    seed_key(seed, key);
+    for (uint32_t b = 0; b < 3; ++b) {
+        ctr[0] = 3u * col + b; ctr[1] = slot; ctr[2] = RO_TAG_GAUS; ctr[3] = task_id;
+        ro_philox4x32_10(ctr, key, blk);
+        for (int w = 0; w < 4; ++w) {
+            float u = (float)(blk[w] >> 8) * (1.0f / 16777216.0f); /* exact: 24 bits times a power of two */
+            sum = sum + u;                                          /* one rounding */
+        }
+    }
+    float g = sum - 6.0f;
+    return g == 0.0f ? 1.0f : g;
+}
+
+/* ------------------------------------------------------------------------ */
 /* Per-task layer tables over the whole model.                               */
 /*   src_of_slot[l] = layer whose delta lands on slot l   (sigma)            */
 /*   slot_of_pos[p] = slot that holds layer p's delta     (sigma^-1)         */
@@ -166,6 +195,12 @@ static int takes_part(uint32_t n_layers, const uint32_t *group, const uint32_t *
 int ro_layer_flips(uint32_t n_layers, const uint32_t *group, const uint32_t *gflags, uint32_t l)
 {
     return (gflags[group[l]] & RO_FLIP) != 0 && takes_part(n_layers, group, gflags, l);
+}
+
+/* 1 if slot l carries the Gaussian-like context instead (restricted by the skip rate likewise). */
+int ro_layer_gauss(uint32_t n_layers, const uint32_t *group, const uint32_t *gflags, uint32_t l)
+{
+    return (gflags[group[l]] & RO_GAUSS) != 0 && takes_part(n_layers, group, gflags, l);
 }
 
 int ro_task_tables(uint32_t n_layers, const uint32_t *group, uint32_t n_groups,
@@ -259,7 +294,8 @@ typedef struct {
 static int spec_check(const ro_spec_t *s)
 {
     for (uint32_t g = 0; g < s->n_groups; ++g)
-        if ((s->gflags[g] & RO_SHUFFLE) && (s->gflags[g] & RO_SHIFT)) return -3;
+        if (((s->gflags[g] & RO_SHUFFLE) && (s->gflags[g] & RO_SHIFT)) ||
+            ((s->gflags[g] & RO_FLIP) && (s->gflags[g] & RO_GAUSS))) return -3;
     /* all members of a group must have one shape (Section 4.3: same type) */
     for (uint32_t a = 0; a < s->n_layers; ++a) {
         if (s->group[a] >= s->n_groups) return -1;
@@ -303,10 +339,13 @@ static int accumulate_one(const ro_spec_t *s, int dtype, int m_dtype, int sign_o
         uint32_t rows = s->rows[l], cols = s->cols[l];
         uint32_t src = src_of_slot[l];
         int flip = ro_layer_flips(L, s->group, s->gflags, l);
+        int gauss = ro_layer_gauss(L, s->group, s->gflags, l);
         int8_t *sg = (int8_t *)malloc(cols ? cols : 1);
-        if (!sg) { free(src_of_slot); free(slot_of_pos); return -1; }
+        float *gs = (float *)malloc(sizeof(float) * (cols ? cols : 1));
+        if (!sg || !gs) { free(sg); free(gs); free(src_of_slot); free(slot_of_pos); return -1; }
         if (flip) ro_sign_row(seed, task_id, l, cols, sg);
         else memset(sg, 1, cols);
+        for (uint32_t c = 0; gauss && c < cols; ++c) gs[c] = ro_gauss(seed, task_id, l, c);
         const void *wt = task[src];
         const void *wb = base ? base[src] : NULL;
         void *m = M[l];
@@ -315,12 +354,14 @@ static int accumulate_one(const ro_spec_t *s, int dtype, int m_dtype, int sign_o
             for (uint32_t c = 0; c < cols; ++c) {
                 size_t idx = (size_t)r * cols + c;
                 float x = transformed_delta(wt, wb, dtype, idx, sg[c]);
+                if (gauss) x = x * gs[c];                    /* Delta D with a Gaussian-like D: one rounding */
                 float old = load_m(m, m_dtype, idx);
                 float sum = sign_op < 0 ? old - x : old + x; /* one fp32 rounding */
                 store_m(m, m_dtype, idx, sum);               /* and one more if M is bf16 */
             }
         }
         free(sg);
+        free(gs);
     }
     free(src_of_slot);
     free(slot_of_pos);
@@ -466,10 +507,13 @@ int ro_retrieve(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
         uint32_t nr = rows[p], nc = cols[p];
         uint32_t l = slot_of_pos[p];
         int flip = ro_layer_flips(L, group, gflags, l);
+        int gauss = ro_layer_gauss(L, group, gflags, l);
         int8_t *sg = (int8_t *)malloc(nc ? nc : 1);
-        if (!sg) { free(src_of_slot); free(slot_of_pos); return -1; }
+        float *gs = (float *)malloc(sizeof(float) * (nc ? nc : 1));
+        if (!sg || !gs) { free(sg); free(gs); free(src_of_slot); free(slot_of_pos); return -1; }
         if (flip) ro_sign_row(seed, task_id, l, nc, sg);
         else memset(sg, 1, nc);
+        for (uint32_t c = 0; gauss && c < nc; ++c) gs[c] = ro_gauss(seed, task_id, l, c);
         const void *m = M[l];
         const void *wb = base[p];
         void *o = out[p];
@@ -479,12 +523,14 @@ int ro_retrieve(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
                 size_t idx = (size_t)r * nc + c;
                 float mv = load_m(m, m_dtype, idx);
                 float signed_m = sg[c] < 0 ? -mv : mv;
+                if (gauss) signed_m = mv / gs[c];            /* D^-1 of a diagonal D divides: one rounding */
                 float y = fmaf(lambda, signed_m, load_elem(wb, dtype, idx));
                 if (out_dtype == RO_BF16) ((uint16_t *)o)[idx] = ro_f32_to_bf16(y);
                 else ((float *)o)[idx] = y;
             }
         }
         free(sg);
+        free(gs);
     }
     free(src_of_slot);
     free(slot_of_pos);
@@ -513,6 +559,8 @@ int ro_linear(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
     if (rc) return rc;
     uint32_t L = n_layers;
     if (p >= L) return -1;
+    for (uint32_t g = 0; g < n_groups; ++g)
+        if (gflags[g] & RO_GAUSS) return -4;   /* defined for the orthogonal contexts only */
     uint32_t *src_of_slot = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
     uint32_t *slot_of_pos = (uint32_t *)malloc(sizeof(uint32_t) * (L + 1));
     if (!src_of_slot || !slot_of_pos) { free(src_of_slot); free(slot_of_pos); return -1; }
@@ -564,6 +612,8 @@ int ro_delta_gram(uint32_t n_layers, const uint32_t *rows, const uint32_t *cols,
                   int dtype, uint32_t n_tasks, const uint32_t *task_ids, const uint64_t *seeds,
                   const void *const *base, const void *const *tasks, double *gram)
 {
+    for (uint32_t g = 0; g < n_groups; ++g)
+        if (gflags[g] & RO_GAUSS) return -4;   /* the interference identity rests on orthogonal transforms */
     ro_spec_t s = make_spec(n_layers, rows, cols, group, n_groups, gflags);
     int rc = spec_check(&s);
     if (rc) return rc;

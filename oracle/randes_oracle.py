@@ -28,6 +28,7 @@ BF16 = 1
 SHUFFLE = 1
 FLIP = 2
 SHIFT = 4
+GAUSS = 1 << 16   # Gaussian-like diagonal context (Section 5.5, "RD") instead of the +-1 one
 
 
 def SKIP(k: int) -> int:
@@ -66,6 +67,8 @@ def _load():
         lib.ro_sign_row.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32,
                                     ctypes.c_uint32, ctypes.c_void_p]
         lib.ro_sign_row.restype = None
+        lib.ro_gauss.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32]
+        lib.ro_gauss.restype = ctypes.c_float
         lib.ro_f32_to_bf16.argtypes = [ctypes.c_float]
         lib.ro_f32_to_bf16.restype = ctypes.c_uint16
         lib.ro_task_tables.restype = ctypes.c_int
@@ -110,6 +113,11 @@ def sign_row(seed: int, task_id: int, slot: int, cols: int) -> np.ndarray:
     out = np.zeros(max(cols, 1), dtype=np.int8)
     _load().ro_sign_row(seed, task_id, slot, cols, out.ctypes.data_as(ctypes.c_void_p))
     return out[:cols]
+
+
+def gauss(seed: int, task_id: int, slot: int, col: int) -> float:
+    """Diagonal entry of the Gaussian-like context (Section 5.5, "RD") for (task, slot, column)."""
+    return float(_load().ro_gauss(seed, task_id, slot, col))
 
 
 def f32_to_bf16(x: float) -> int:

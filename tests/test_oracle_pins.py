@@ -80,6 +80,8 @@ def dense_transform(spec, seed, task_id):
     for l in range(L):
         if (gflags[group[l]] & FLIP) and takes_part[l]:
             diag = ro.sign_row(seed, task_id, l, cols[l]).astype(np.float64)
+        elif (gflags[group[l]] & ro.GAUSS) and takes_part[l]:
+            diag = np.array([ro.gauss(seed, task_id, l, c) for c in range(cols[l])], dtype=np.float64)
         else:
             diag = np.ones(cols[l])
         # vec(X diag(s)) for row-major X [rows, cols] = tile(s, rows) * vec(X)
@@ -727,3 +729,83 @@ def test_linear_on_bf16_inputs_and_superposition_stays_close_to_the_retrieved_we
         want = -2.0 * float(np.float32(lam)) * ro.sign(s, t, l, 17) * np.outer(widen(x)[:, 17].astype(np.float64), widen(M[l])[:, 17].astype(np.float64))
         assert np.allclose(y_wrong - y, want, rtol=0, atol=1e-12)
         assert np.abs(y_wrong - y).max() > 2.0 ** -14 * y_abs.max()
+
+
+# --------------------------------------------------------------------------- Gaussian-like diagonal context ("RD", Section 5.5)
+def test_gauss_entries_replay_the_stated_recipe_and_have_unit_variance():
+    """Entry (task, slot, column) = sum of twelve uniforms minus six, uniforms = top 24 bits of the words of
+    Philox blocks 3c .. 3c+2 of the "GAUS" stream, added left to right in fp32: replayed here from the oracle's
+    Philox (itself pinned to published vectors); mean 0, variance 1, support inside (-6, 6)."""
+    seed, task, slot = 2**40 + 5, 9, 3
+    for c in (0, 1, 130, 4095):
+        acc = np.float32(0.0)
+        for b in range(3):
+            blk = ro.philox4x32_10((3 * c + b, slot, 0x47415553, task), (seed & 0xFFFFFFFF, seed >> 32))
+            for w in blk:
+                acc = np.float32(acc + np.float32(w >> 8) * np.float32(2.0 ** -24))
+        want = np.float32(acc - np.float32(6.0))
+        assert np.float32(ro.gauss(seed, task, slot, c)) == (want if want != 0 else np.float32(1.0))
+    g = np.array([ro.gauss(seed, task, slot, c) for c in range(40000)])
+    assert abs(g.mean()) < 4 / np.sqrt(g.size) and abs(g.var() - 1.0) < 0.03
+    assert np.abs(g).max() < 6.0 and np.all(g != 0.0)
+    # fourth moment of the twelve-uniform sum: 3 - 6/(5*12) = 2.9
+    assert abs(np.mean(g ** 4) - 2.9) < 0.15
+    other = np.array([ro.gauss(seed, task + 1, slot, c) for c in range(4000)])
+    assert abs(np.corrcoef(g[:4000], other)[0, 1]) < 0.06
+
+
+@pytest.mark.parametrize("flags", [ro.GAUSS, ro.GAUSS | SHUFFLE, ro.GAUSS | SHUFFLE | ro.SKIP(2)])
+def test_gauss_context_matches_dense_matrices_and_is_not_orthogonal(flags):
+    """Section 5.5: with a Gaussian-like diagonal D the same formulas hold with D^-1 in place of D^T:
+    M = sum_i D_i P_i delta_i, What_t = W_0 + lambda P_t^T D_t^-1 M; the transform is not orthogonal."""
+    spec = tiny_spec(flags, n_a=4, n_b=3)
+    rng = np.random.default_rng(91)
+    ids, seeds = [2, 7, 5], [3, 2**35, 11]
+    base = rand_model(spec, rng, scale=0.02)
+    tasks = [[b + d for b, d in zip(base, rand_model(spec, rng, scale=1e-3))] for _ in ids]
+    Ts = [dense_transform(spec, s, t)[0] for t, s in zip(ids, seeds)]
+    assert not np.allclose(Ts[0].T @ Ts[0], np.eye(Ts[0].shape[0]))
+    deltas = [flat([np.float32(a - b) for a, b in zip(t, base)]) for t in tasks]
+    M_dense = sum(T @ d for T, d in zip(Ts, deltas))
+    M = ro.compress(spec, ro.F32, ids, seeds, base, tasks)
+    scale = sum(np.abs(T) @ np.abs(d) for T, d in zip(Ts, deltas))
+    assert np.all(np.abs(flat(M) - M_dense) <= 2.0 ** -22 * scale + 1e-30)      # one rounding per product and per sum
+    lam = 0.3
+    for j, (t, s) in enumerate(zip(ids, seeds)):
+        what = ro.retrieve(spec, ro.F32, ro.F32, t, s, lam, base, M)
+        want = flat(base) + float(np.float32(lam)) * (np.linalg.inv(Ts[j]) @ flat(M))
+        tol = 2.0 ** -22 * (np.abs(flat(base)) + lam * np.abs(np.linalg.inv(Ts[j])) @ np.abs(flat(M)))
+        assert np.all(np.abs(flat(what) - want) <= tol + 1e-30)
+
+
+def test_gauss_context_single_model_round_trip_and_larger_interference_than_sign_flips():
+    """K = 1: (delta g) / g returns delta within two roundings.  K > 1: the paper's finding of Section 5.5 -- a
+    diagonal that does not preserve magnitudes leaves more interference than the +-1 one on the same models."""
+    rng = np.random.default_rng(92)
+    spec_g = ([16] * 4, [64] * 4, [0] * 4, [ro.GAUSS])
+    spec_f = ([16] * 4, [64] * 4, [0] * 4, [FLIP])
+    base = rand_model(spec_g, rng, scale=0.02)
+    deltas = [rand_model(spec_g, rng, scale=1e-3) for _ in range(6)]
+    tasks = [[b + d for b, d in zip(base, dl)] for dl in deltas]
+    M1 = ro.compress(spec_g, ro.F32, [4], [17], base, tasks[:1])
+    back = ro.retrieve(spec_g, ro.F32, ro.F32, 4, 17, 1.0, base, M1)
+    d0 = [np.float32(t - b) for t, b in zip(tasks[0], base)]
+    for l in range(4):
+        assert np.all(np.abs(back[l].astype(np.float64) - base[l] - d0[l]) <= 2.0 ** -22 * (np.abs(d0[l]) + np.abs(base[l])))
+    ids, seeds = list(range(6)), [50 + i for i in range(6)]
+    err = {}
+    for name, spec in (("gauss", spec_g), ("flip", spec_f)):
+        M = ro.compress(spec, ro.F32, ids, seeds, base, tasks)
+        out = ro.retrieve(spec, ro.F32, ro.F32, 0, seeds[0], 1.0, base, M)
+        err[name] = np.sqrt(sum(np.sum((o.astype(np.float64) - t) ** 2) for o, t in zip(out, tasks[0])))
+    assert err["gauss"] > 2.0 * err["flip"]
+
+
+def test_gauss_and_flip_exclude_each_other_and_diagnostics_refuse_the_gauss_context():
+    spec = ([2, 2], [8, 8], [0, 0], [ro.GAUSS | FLIP])
+    m = rand_model(spec, np.random.default_rng(1))
+    with pytest.raises(ValueError):
+        ro.compress(spec, ro.F32, [0], [1], None, [m])
+    spec = ([2, 2], [8, 8], [0, 0], [ro.GAUSS])
+    with pytest.raises(ValueError):
+        ro.delta_gram(spec, ro.F32, [0, 1], [1, 2], None, [m, m])

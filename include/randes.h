@@ -72,8 +72,17 @@ typedef enum { RANDES_F32 = 0, RANDES_BF16 = 1 } randes_dtype_t;
  *                   Mutually exclusive with RANDES_SHUFFLE.
  *   RANDES_SKIP(k)  skip rate of the same appendix: only the members with index 0, k,
  *                   2k, ... of the group (in layer order) are shuffled / shifted and
- *                   flipped; k = 0 or 1 means all.  1 <= k <= 255. */
-enum { RANDES_SHUFFLE = 1, RANDES_FLIP = 2, RANDES_SHIFT = 4 };
+ *                   flipped; k = 0 or 1 means all.  1 <= k <= 255.
+ *   RANDES_GAUSS    the "RD" context matrix of the ablation in Section 5.5 instead of the +-1 one:
+ *                   a diagonal of (nearly) standard normal entries, one per (task, slot, column).
+ *                   Not orthogonal: compress multiplies by it, retrieve divides (the paper shows
+ *                   that it interferes more; it is here for that comparison).  Entry = sum of
+ *                   twelve uniforms minus six, drawn from the task's Philox stream in exactly
+ *                   rounded fp32 steps.  Mutually exclusive with RANDES_FLIP; needs an fp32
+ *                   superposition.  A plan with such a group runs compress, add, remove and
+ *                   retrieve through plain (not bandwidth-tuned) kernels, and does not offer
+ *                   randes_retrieve_batch, randes_retrieve_static, randes_delta_gram or randes_linear. */
+enum { RANDES_SHUFFLE = 1, RANDES_FLIP = 2, RANDES_SHIFT = 4, RANDES_GAUSS = 1 << 16 };
 #define RANDES_SKIP(k) (((uint32_t)(k) & 0xFFu) << 8)
 
 typedef struct { uint32_t rows, cols, group; } randes_layer_t;

@@ -15,7 +15,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librandes.so")
-SOURCES = ["randes_api.cu", "randes_kernels.cu", "randes_group.cu", "randes_linear.cu", "randes_batch.cu", "randes_diag.cu"]
+SOURCES = ["randes_api.cu", "randes_kernels.cu", "randes_group.cu", "randes_linear.cu", "randes_context.cu", "randes_batch.cu", "randes_diag.cu"]
 HEADERS = [os.path.join(CSRC, "randes_internal.h"), os.path.join(CSRC, "randes_device.cuh"), os.path.join(os.path.dirname(HERE), "include", "randes.h")]
 
 

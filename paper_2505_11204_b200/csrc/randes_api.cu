@@ -227,6 +227,7 @@ struct randes_plan_s {
     int m_dtype = RANDES_F32;                     // element type of the superposition arena
     std::vector<randes_layer_t> layers;
     std::vector<uint32_t> gflags;
+    bool has_gauss = false;                       // some group carries the Gaussian-like context: every call takes the plain kernels
     std::vector<std::vector<uint32_t>> members;   // per group, in layer order
     std::vector<DevLayer> dev_layers;
     std::vector<DevUnit> units;
@@ -409,6 +410,13 @@ int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_
     a.base = p.dev<const void*>(p.lay.base_ptrs);
     a.task_ptrs = p.dev<const void*>(p.lay.task_ptrs);
     a.M = M;
+    if (p.has_gauss) {
+        if (a.n_units == 0) return RANDES_OK;
+        const int e = launch_context_accumulate(p.storage, a, p.sm_count, s);
+        if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the general-context accumulate kernel");
+        ++g_launches;
+        return RANDES_OK;
+    }
     if (staged) {
         CompressGroupArgs g;
         g.layers = a.layers;
@@ -486,10 +494,14 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
     if (n_tasks && (!task_ids || !seeds)) return fail(RANDES_INVALID_ARGUMENT, "task_ids / seeds is NULL");
     for (uint32_t g = 0; g < n_groups; ++g)
     {
-        if (groups[g].flags & ~static_cast<uint32_t>(RANDES_SHUFFLE | RANDES_FLIP | RANDES_SHIFT | RANDES_SKIP(0xFF)))
+        if (groups[g].flags & ~static_cast<uint32_t>(RANDES_SHUFFLE | RANDES_FLIP | RANDES_SHIFT | RANDES_SKIP(0xFF) | RANDES_GAUSS))
             return fail(RANDES_INVALID_ARGUMENT, "group %u: unknown flag bits 0x%x", g, groups[g].flags);
         if ((groups[g].flags & RANDES_SHUFFLE) && (groups[g].flags & RANDES_SHIFT))
             return fail(RANDES_INVALID_ARGUMENT, "group %u: RANDES_SHUFFLE and RANDES_SHIFT exclude each other", g);
+        if ((groups[g].flags & RANDES_FLIP) && (groups[g].flags & RANDES_GAUSS))
+            return fail(RANDES_INVALID_ARGUMENT, "group %u: RANDES_FLIP and RANDES_GAUSS exclude each other", g);
+        if ((groups[g].flags & RANDES_GAUSS) && m_dtype != RANDES_F32)
+            return fail(RANDES_UNSUPPORTED_DTYPE, "group %u: RANDES_GAUSS needs an fp32 superposition", g);
     }
     for (uint32_t i = 0; i < n_tasks; ++i)
         for (uint32_t j = 0; j < i; ++j)
@@ -505,7 +517,10 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         p->m_dtype = m_dtype;
         p->layers.assign(layers, layers + n_layers);
         p->gflags.resize(n_groups);
-        for (uint32_t g = 0; g < n_groups; ++g) p->gflags[g] = groups[g].flags;
+        for (uint32_t g = 0; g < n_groups; ++g) {
+            p->gflags[g] = groups[g].flags;
+            p->has_gauss = p->has_gauss || (groups[g].flags & RANDES_GAUSS);
+        }
         p->members.assign(n_groups, {});
         for (uint32_t l = 0; l < n_layers; ++l) {
             if (layers[l].group >= n_groups) {
@@ -538,6 +553,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
             const bool takes_part = d.member % skip == 0;
             const size_t n_part = (mem.size() + skip - 1) / skip;
             d.flags = ((p->gflags[g] & RANDES_FLIP) && takes_part ? kFlagFlip : 0u) |
+                      ((p->gflags[g] & RANDES_GAUSS) && takes_part ? kFlagGauss : 0u) |
                       ((p->gflags[g] & (RANDES_SHUFFLE | RANDES_SHIFT)) && takes_part && n_part >= 2 ? kFlagShuffle : 0u);
             d.group_size = static_cast<uint32_t>(mem.size());
             p->dev_layers[l] = d;
@@ -561,7 +577,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
                 any = any || shuffled;
                 if (shuffled) p->max_staged_group = std::max<uint32_t>(p->max_staged_group, static_cast<uint32_t>(mem.size()));
             }
-            if (any) {
+            if (any && !p->has_gauss) {
                 build_units(layers, n_layers, p->storage, p->group_units, &p->group_staged, &member_base, kStagedGroups);
                 build_units(layers, n_layers, p->storage, p->other_units, &p->group_staged, &member_base, kOtherGroups);
             }
@@ -885,6 +901,12 @@ static int randes_retrieve_impl(randes_plan_t* plan, uint32_t task_id, float lam
     a.task.pad = 0;
     a.lambda = lambda;
     if (a.n_units == 0) return RANDES_OK;
+    if (plan->has_gauss) {
+        const int ce = launch_context_retrieve(plan->storage, out_dtype, a, plan->sm_count, s);
+        if (ce) return fail_cuda(static_cast<cudaError_t>(ce), "launch of the general-context retrieve kernel");
+        ++g_launches;
+        return RANDES_OK;
+    }
     const int grid = std::min<int>(plan->grid_ret[out_dtype], static_cast<int>(a.n_units));
     const int e = launch_retrieve(plan->storage, out_dtype, plan->m_dtype, a, grid, s);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the retrieve kernel");
@@ -902,6 +924,7 @@ static int randes_delta_gram_impl(randes_plan_t* plan, const void* const* base, 
                       size_t scratch_bytes, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (plan->has_gauss) return fail(RANDES_INVALID_ARGUMENT, "not offered for plans with a RANDES_GAUSS group");
     if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
     const size_t n = plan->tasks.size();
     if (n == 0) return fail(RANDES_INVALID_ARGUMENT, "no task is registered");
@@ -947,6 +970,7 @@ static int randes_retrieve_batch_impl(randes_plan_t* plan, const uint32_t* task_
                           randes_dtype_t out_dtype, const void* const* base, const void* M, void* const* out, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (plan->has_gauss) return fail(RANDES_INVALID_ARGUMENT, "not offered for plans with a RANDES_GAUSS group");
     if (!plan->ws) return fail(RANDES_INVALID_ARGUMENT, "plan was built without a device workspace");
     if (out_dtype != RANDES_F32 && out_dtype != RANDES_BF16)
         return fail(RANDES_UNSUPPORTED_DTYPE, "output dtype %d is not supported", static_cast<int>(out_dtype));
@@ -1024,6 +1048,7 @@ static int randes_retrieve_static_impl(const randes_plan_t* plan, uint32_t task_
                            const void* const* base, const void* M, void* const* out, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (plan->has_gauss) return fail(RANDES_INVALID_ARGUMENT, "not offered for plans with a RANDES_GAUSS group");
     if (out_dtype != RANDES_F32 && out_dtype != RANDES_BF16)
         return fail(RANDES_UNSUPPORTED_DTYPE, "output dtype %d is not supported", static_cast<int>(out_dtype));
     int rc;
@@ -1093,6 +1118,7 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
                               uint32_t n_tokens, const void* const* base, const void* M, void* y, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    if (plan->has_gauss) return fail(RANDES_INVALID_ARGUMENT, "not offered for plans with a RANDES_GAUSS group");
     if (plan->storage != RANDES_BF16 || plan->m_dtype != RANDES_BF16)
         return fail(RANDES_UNSUPPORTED_DTYPE, "randes_linear needs bf16 weights and a bf16 superposition (tensor-core operands)");
     if (layer >= plan->n_layers) return fail(RANDES_INVALID_ARGUMENT, "layer %u out of range (n_layers = %u)", layer, plan->n_layers);

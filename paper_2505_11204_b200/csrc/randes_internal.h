@@ -9,6 +9,7 @@ namespace randes {
 
 constexpr uint32_t kFlagShuffle = 1u;   // layer may move inside its group for some task
 constexpr uint32_t kFlagFlip = 2u;      // per-column sign flip on this slot
+constexpr uint32_t kFlagGauss = 4u;     // per-column Gaussian-like factor on this slot instead (general diagonal context)
 
 constexpr int kWarpsPerCta = 8;
 constexpr int kThreadsPerCta = kWarpsPerCta * 32;
@@ -16,6 +17,7 @@ constexpr int kRowsPerWarp = 16;        // rows one warp walks per unit (8 to 16
 constexpr int kTaskChunk = 32;          // tasks whose pointers / sign blocks a warp holds at once
 constexpr uint32_t kTagSign = 0x5349474Eu;  // counter word 2 of the sign stream ("SIGN")
 constexpr uint32_t kTagPerm = 0x5045524Du;  // counter word 2 of the permutation stream ("PERM")
+constexpr uint32_t kTagGauss = 0x47415553u; // counter word 2 of the Gaussian-like context stream ("GAUS")
 
 // A lane always moves 16 bytes of a weight tensor: 4 fp32 or 8 bf16 columns.  A
 // warp therefore spans 128 (fp32) or 256 (bf16) columns = 1 or 2 Philox blocks
@@ -152,6 +154,10 @@ struct GramArgs {
 // Launchers (randes_kernels.cu).  Return a cudaError_t as int.
 int launch_retrieve(int storage_dtype, int out_dtype, int m_dtype, const RetrieveArgs& a, int grid, void* stream);
 int launch_accumulate(int storage_dtype, int m_dtype, const AccumulateArgs& a, int grid, void* stream);
+// randes_context.cu: all of a plan's layers under a general diagonal context (plans with a RANDES_GAUSS group);
+// fp32 superposition only.  Return a cudaError_t as int.
+int launch_context_accumulate(int storage_dtype, const AccumulateArgs& a, int sm_count, void* stream);
+int launch_context_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, int sm_count, void* stream);
 // randes_group.cu: compress over group units.  `max_group` = the largest staged group.
 int compress_group_prepare(int storage_dtype, int m_dtype);   // once per device: opts into the shared memory the kernel needs
 bool compress_group_fits(int storage_dtype, uint32_t max_group, uint32_t n_tasks);

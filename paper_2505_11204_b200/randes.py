@@ -22,6 +22,7 @@ BF16 = 1
 SHUFFLE = 1
 FLIP = 2
 SHIFT = 4
+GAUSS = 1 << 16   # RANDES_GAUSS: Gaussian-like diagonal context (the paper's "RD" ablation) instead of the +-1 one
 
 
 def SKIP(k: int) -> int:

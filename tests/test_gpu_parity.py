@@ -419,6 +419,44 @@ def test_large_and_partly_shuffled_groups(n_tasks, storage):
     run_full_cycle(make_workload(shapes, flags=flags, n_tasks=n_tasks, storage=storage), out_dtypes=(wl.F32,), extra_task=False)
 
 
+@pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
+@pytest.mark.parametrize("n_tasks", [3, 10])
+def test_gaussian_diagonal_context(storage, n_tasks):
+    """The "RD" ablation of Section 5.5 (a nearly normal diagonal instead of +-1; compress multiplies, retrieve divides):
+    every step bit for bit against the oracle, alone, under a shuffle, with a skip rate, and beside groups that keep
+    the sign flip or no context (a plan with one such group runs all its layers through the plain kernels);
+    10 tasks = two passes of 8 and 2 through M."""
+    G = randes.GAUSS
+    shapes = [(9, 132, 3), (5, 256, 4), (17, 520, 2), (1, 300, 5), (33, 64, 3), (3, 2100, 2)]
+    flags = [G | S, G, S | F, G | S | randes.SKIP(2), S, G | S]
+    run_full_cycle(make_workload(shapes, flags=flags, storage=storage, n_tasks=n_tasks), extra_task=True)
+
+
+def test_gaussian_diagonal_context_limits():
+    G = randes.GAUSS
+    w = make_workload([(8, 64, 2)], flags=[G | S], n_tasks=2)
+    base, tasks = wl.model_set(w, w.task_ids)
+    d_base = model_to_dev(base)
+    with pytest.raises(randes.RandesError) as e:
+        randes.Plan.from_workload(w, max_tasks=2, m_dtype=wl.BF16)
+    assert e.value.code == randes.UNSUPPORTED_DTYPE
+    with pytest.raises(randes.RandesError) as e:
+        randes.Plan.from_workload(make_workload([(8, 64, 2)], flags=[G | F], n_tasks=2), max_tasks=2)
+    assert e.value.code == randes.INVALID_ARGUMENT
+    plan = randes.Plan.from_workload(w, max_tasks=2)
+    M = plan.compress(d_base, [model_to_dev(t) for t in tasks])
+    before = randes.randes_launch_count()
+    for call in (lambda: plan.retrieve_batch(list(w.task_ids), 0.3, d_base, M),
+                 lambda: plan.delta_gram(d_base, [model_to_dev(t) for t in tasks]),
+                 lambda: randes.randes_retrieve_static(plan.handle, w.task_ids[0], 0.3, wl.F32, randes.ptr_array(d_base), M,
+                                                       randes.ptr_array(plan.new_output(wl.F32)), 0)):
+        with pytest.raises(randes.RandesError) as e:
+            call()
+        assert e.value.code == randes.INVALID_ARGUMENT
+    assert randes.randes_launch_count() == before
+    plan.close()
+
+
 def test_random_plans():
     """Seeded random models: shapes, group sizes, flags (shuffle / shift / flip / skip), task counts, ids,
     seeds and storage types drawn at random; every step of the path against the oracle."""

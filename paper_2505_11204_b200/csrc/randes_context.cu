@@ -8,9 +8,11 @@
 // A plan with such a group runs ALL its layers through these kernels; layers with a +-1 context or
 // none use g = +-1 or 1, for which the arithmetic below gives the bits of the streaming kernels
 // (x * +-1 and x / +-1 are exact).  This is an ablation the paper itself discards (it interferes
-// more), so the kernels are plain: one thread per column walks the rows of a unit, four bytes per
-// access, no staging.  Every operation is an explicitly rounded fp32 intrinsic, in the order of the
-// definition, so results are bit-identical to a scalar evaluation.
+// more), so the kernels are plain: a thread takes four neighbouring columns and walks the rows of a
+// unit, with the loads of all tasks of a row issued before the first use; no staging, no tuning
+// beyond that (a third to under a half of the streaming kernels' speed).  Every operation is an
+// explicitly rounded fp32 intrinsic, in the order of the definition, so results are bit-identical
+// to a scalar evaluation.
 //
 // g: the paper names no generator.  Sum of twelve uniforms minus six: the twelve words of Philox
 // blocks 3c, 3c+1, 3c+2 of the (slot, task) stream tagged "GAUS", each reduced to
@@ -65,11 +67,34 @@ template <> __device__ __forceinline__ float load_elem<bf16>(const void* p, size
     return __uint_as_float(static_cast<uint32_t>(static_cast<const unsigned short*>(p)[i]) << 16);
 }
 
+// four neighbouring elements of a row
+template <typename T> __device__ __forceinline__ void load_quad(const void* p, size_t i, float (&v)[4]);
+template <> __device__ __forceinline__ void load_quad<float>(const void* p, size_t i, float (&v)[4])
+{
+    const float4 x = *reinterpret_cast<const float4*>(static_cast<const float*>(p) + i);
+    v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+}
+template <> __device__ __forceinline__ void load_quad<bf16>(const void* p, size_t i, float (&v)[4])
+{
+    const uint2 x = *reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(p) + i);
+    v[0] = __uint_as_float(x.x << 16); v[1] = __uint_as_float(x.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(x.y << 16); v[3] = __uint_as_float(x.y & 0xFFFF0000u);
+}
+template <typename T> __device__ __forceinline__ bool quad_aligned(const void* p)
+{
+    return (reinterpret_cast<uintptr_t>(p) & (4 * sizeof(T) - 1)) == 0;
+}
+__device__ __forceinline__ void store_quad(float* p, const float (&v)[4]) { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); }
+__device__ __forceinline__ void store_quad(bf16* p, const float (&v)[4])
+{
+    *reinterpret_cast<uint2*>(p) = make_uint2(Out<bf16>::pack(v[0], v[1]), Out<bf16>::pack(v[2], v[3]));
+}
+
 template <typename ST>
 __global__ void __launch_bounds__(kThreadsPerCta) context_accumulate_kernel(const AccumulateArgs a)
 {
     constexpr uint32_t WC = 32 * Store<ST>::CPL;          // columns of one column block of the unit list
-    extern __shared__ float gtab[];                       // [kContextChunk][kContextSpan], column-private entries
+    extern __shared__ __align__(16) float gtab[];         // [kContextChunk][kContextSpan]
     const uint32_t L = a.n_layers;
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
@@ -97,8 +122,44 @@ __global__ void __launch_bounds__(kThreadsPerCta) context_accumulate_kernel(cons
                     }
                 }
             }
-            // each thread reads back only the columns it wrote: no barrier
             const bool from_m = chunk0 > 0 || a.init_from_m;
+            bool vec = cols % 4 == 0;
+#pragma unroll
+            for (int k = 0; k < kContextChunk; ++k)
+                if (static_cast<uint32_t>(k) < nt) vec = vec && quad_aligned<ST>(pw[k]) && (!pb[k] || quad_aligned<ST>(pb[k]));
+            if (vec) {
+                // a thread owns columns 4q .. 4q+3, q = its index + 256 j; the factors of those columns were written
+                // by threads 4q .. 4q+3 of the same pass (column c by thread (c - c_begin) % 256)
+                __syncthreads();
+                for (uint32_t r = un.row0; r < un.row0 + un.nrows; ++r) {
+                    for (uint32_t c = c_begin + 4 * threadIdx.x; c < c_end; c += 4 * kThreadsPerCta) {
+                        const size_t idx = static_cast<size_t>(r) * cols + c;
+                        float w[kContextChunk][4], b[kContextChunk][4], acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                        for (int k = 0; k < kContextChunk; ++k)
+                            if (static_cast<uint32_t>(k) < nt) {
+                                load_quad<ST>(pw[k], idx, w[k]);
+                                if (pb[k]) load_quad<ST>(pb[k], idx, b[k]);
+                            }
+                        if (from_m) load_quad<float>(mp, idx, acc);
+#pragma unroll
+                        for (int k = 0; k < kContextChunk; ++k)
+                            if (static_cast<uint32_t>(k) < nt) {
+                                const float4 g = *reinterpret_cast<const float4*>(&gtab[k * kContextSpan + (c - c_begin)]);
+                                const float gv[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float d = pb[k] ? __fsub_rn(w[k][e], b[k][e]) : w[k][e];
+                                    acc[e] = __fadd_rn(acc[e], __fmul_rn(d, gv[e]));
+                                }
+                            }
+                        store_quad(mp + idx, acc);
+                    }
+                }
+                __syncthreads();   // the table is rewritten by the next pass
+                continue;
+            }
+            // element-wise: each thread reads back only the columns it wrote: no barrier
             for (uint32_t r = un.row0; r < un.row0 + un.nrows; ++r) {
                 for (uint32_t c = c_begin + threadIdx.x; c < c_end; c += kThreadsPerCta) {
                     const size_t idx = static_cast<size_t>(r) * cols + c;
@@ -132,6 +193,32 @@ __global__ void __launch_bounds__(kThreadsPerCta) context_retrieve_kernel(const 
         OT* op = static_cast<OT*>(a.out[p]);
         const uint32_t cols = lp.cols;
         const uint32_t c_begin = un.cb0 * WC, c_end = min(cols, (un.cb0 + un.nbc) * WC);
+        if (cols % 4 == 0 && quad_aligned<ST>(wp) && quad_aligned<OT>(op)) {
+            for (uint32_t c = c_begin + 4 * threadIdx.x; c < c_end; c += 4 * kThreadsPerCta) {
+                float g[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) g[e] = context_entry(lp.flags, a.task, slot, c + e);
+                for (uint32_t r0 = un.row0; r0 < un.row0 + un.nrows; r0 += 4) {
+                    float m[4][4], w[4][4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (r0 + j < un.row0 + un.nrows) {
+                            const size_t idx = static_cast<size_t>(r0 + j) * cols + c;
+                            load_quad<float>(mp, idx, m[j]);
+                            load_quad<ST>(wp, idx, w[j]);
+                        }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (r0 + j < un.row0 + un.nrows) {
+                            float y[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) y[e] = __fmaf_rn(a.lambda, __fdiv_rn(m[j][e], g[e]), w[j][e]);
+                            store_quad(op + static_cast<size_t>(r0 + j) * cols + c, y);
+                        }
+                }
+            }
+            continue;
+        }
         for (uint32_t c = c_begin + threadIdx.x; c < c_end; c += kThreadsPerCta) {
             const float g = context_entry(lp.flags, a.task, slot, c);
             for (uint32_t r = un.row0; r < un.row0 + un.nrows; ++r) {

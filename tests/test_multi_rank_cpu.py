@@ -61,6 +61,21 @@ def test_single_rank_is_identity():
     assert bench.aggregate_value(2e9, 1.0, 1) == pytest.approx(2000.0)
 
 
+def test_row_sliced_job_counts_the_model_once():
+    """--shard rows: the slices of all ranks add up to the model, and the job's value is the model's bytes over the
+    slowest rank's time."""
+    import bench
+    from paper_2505_11204_b200 import workloads as wl
+
+    w = wl.vit_b32()
+    for parts in (2, 3, 8):
+        slices = [wl.row_slice(w, r, parts)[0] for r in range(parts)]
+        assert sum(s.n_params for s in slices) == w.n_params
+        assert sum(bench.step_bytes(s, 5)[1] for s in slices) == bench.step_bytes(w, 5)[1]
+    assert bench.aggregate_value_sliced(3e9, 2.0) == pytest.approx(1500.0)
+    assert bench.parse_args(["--shard", "rows"]).shard == "rows" and bench.parse_args([]).shard == "replicas"
+
+
 def test_step_bytes_match_the_per_parameter_figures():
     import bench
     from paper_2505_11204_b200 import workloads as wl

@@ -256,7 +256,8 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda,
  *   x                     device, [n_tokens, cols] bf16 row-major, 16-byte aligned
  *   base[n_layers]        host array of device pointers (only base[layer] is used, 16-byte aligned)
  *   M                     device, the superposition arena
- *   y                     device, [n_tokens, rows] fp32 row-major; must not alias the inputs
+ *   y, y_dtype            device, [n_tokens, rows] row-major, fp32 or bf16 (the fp32 result rounded to nearest
+ *                         even, once); must not alias the inputs
  * Needs no workspace (the plan may have been built without one).  One kernel launch;
  * asynchronous on `stream`.  The result equals the fp64 definition within
  * 2 * cols * 2^-24 * sum_c |x| (|W_0| + |lambda M|) per output (fp32 accumulation of 2 * cols
@@ -264,7 +265,7 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda,
  * MISALIGNED, CUDA_ERROR.
  */
 int randes_linear(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x,
-                  uint32_t n_tokens, const void* const* base, const void* M, void* y, void* stream);
+                  uint32_t n_tokens, const void* const* base, const void* M, void* y, randes_dtype_t y_dtype, void* stream);
 
 /*
  * Every wait inside the randes_linear kernel is bounded; a thread block whose wait runs out

@@ -1115,12 +1115,14 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_
 }
 
 static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x,
-                              uint32_t n_tokens, const void* const* base, const void* M, void* y, void* stream)
+                              uint32_t n_tokens, const void* const* base, const void* M, void* y, randes_dtype_t y_dtype, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
     if (plan->has_gauss) return fail(RANDES_INVALID_ARGUMENT, "not offered for plans with a RANDES_GAUSS group");
     if (plan->storage != RANDES_BF16 || plan->m_dtype != RANDES_BF16)
         return fail(RANDES_UNSUPPORTED_DTYPE, "randes_linear needs bf16 weights and a bf16 superposition (tensor-core operands)");
+    if (y_dtype != RANDES_F32 && y_dtype != RANDES_BF16)
+        return fail(RANDES_UNSUPPORTED_DTYPE, "output dtype %d is not supported", static_cast<int>(y_dtype));
     if (layer >= plan->n_layers) return fail(RANDES_INVALID_ARGUMENT, "layer %u out of range (n_layers = %u)", layer, plan->n_layers);
     const int row = find_task(*plan, task_id);
     if (row < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_id);
@@ -1133,7 +1135,7 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
     if (cols % 8) return fail(RANDES_INVALID_ARGUMENT, "layer %u: cols = %u is not a multiple of 8 (16-byte rows for the tensor maps)", layer, cols);
     if (reinterpret_cast<uintptr_t>(x) % 16 || reinterpret_cast<uintptr_t>(base[layer]) % 16)
         return fail(RANDES_MISALIGNED, "x and base[%u] must be 16-byte aligned", layer);
-    if (reinterpret_cast<uintptr_t>(y) % 4) return fail(RANDES_MISALIGNED, "y = %p is not aligned to 4 bytes", y);
+    if (reinterpret_cast<uintptr_t>(y) % elem_size(y_dtype)) return fail(RANDES_MISALIGNED, "y = %p is not aligned to its element size", y);
     const TaskEntry& t = plan->tasks[row];
     const uint32_t slot = t.slot_of_pos[layer];                    // sigma_t^-1(p)
     const bool flip = (plan->dev_layers[slot].flags & kFlagFlip) != 0;
@@ -1145,16 +1147,16 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
     int e = linear_prepare();
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "set-up of the linear kernel");
     e = launch_linear(x, n_tokens, base[layer], static_cast<const char*>(M) + plan->m_off_bytes[slot], rows, cols, flip, slot, d, lambda,
-                      static_cast<float*>(y), stream);
+                      y, y_dtype == RANDES_BF16, stream);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the linear kernel");
     ++g_launches;
     return RANDES_OK;
 }
 
 int randes_linear(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x, uint32_t n_tokens,
-                  const void* const* base, const void* M, void* y, void* stream)
+                  const void* const* base, const void* M, void* y, randes_dtype_t y_dtype, void* stream)
 {
-    return guarded([&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, stream); });
+    return guarded([&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, y_dtype, stream); });
 }
 
 int randes_linear_giveups(unsigned int* count)

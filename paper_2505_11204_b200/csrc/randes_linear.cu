@@ -62,7 +62,8 @@ struct LinearArgs {
     uint32_t flip;                 // 0: no sign flip on this slot
     uint32_t slot;                 // l = sigma_t^-1(p): counter word 1 of the sign stream
     DevTask task;
-    float* y;                      // [n_tokens, rows]
+    void* y;                       // [n_tokens, rows], fp32 or bf16
+    uint32_t y_bf16;
 };
 
 // ---- mbarrier, TMA, tcgen05 wrappers --------------------------------------------------------
@@ -291,7 +292,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
             tc_fence_after();
             const int quarter = warp & 3;                     // tensor-memory lanes 32 q .. 32 q + 31
             const uint32_t tlane = static_cast<uint32_t>(quarter * 32) << 16;
-            const bool vec = (a.rows & 3u) == 0 && (reinterpret_cast<uintptr_t>(a.y) & 15u) == 0;
+            const bool vec = (a.rows & 3u) == 0 && (reinterpret_cast<uintptr_t>(a.y) & (a.y_bf16 ? 7u : 15u)) == 0;
 #pragma unroll 1
             for (int h = 0; h < HALVES; ++h) {
                 const uint32_t token = m0 + h * kBM + quarter * 32 + lane;
@@ -302,14 +303,24 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                     tc_load32(tmem + tlane + h * 2 * kBN + kBN + cchunk * 32, v1);
                     tc_wait_ld();
                     if (token < a.n_tokens) {
-                        float* yp = a.y + static_cast<size_t>(token) * a.rows + n0 + cchunk * 32;
+                        const size_t y0 = static_cast<size_t>(token) * a.rows + n0 + cchunk * 32;
+                        float* yp = static_cast<float*>(a.y) + y0;
+                        bf16* yh = static_cast<bf16*>(a.y) + y0;
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             float o[4];
 #pragma unroll
                             for (int e = 0; e < 4; ++e) o[e] = __fmaf_rn(a.lambda, __uint_as_float(v1[j + e]), __uint_as_float(v0[j + e]));
                             const uint32_t f = n0 + cchunk * 32 + j;
-                            if (vec && f + 3 < a.rows) {
+                            if (a.y_bf16) {     // rounded to nearest even, once
+                                if (vec && f + 3 < a.rows) {
+                                    *reinterpret_cast<uint2*>(yh + j) = make_uint2(Out<bf16>::pack(o[0], o[1]), Out<bf16>::pack(o[2], o[3]));
+                                } else {
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e)
+                                        if (f + e < a.rows) yh[j + e] = __float2bfloat16_rn(o[e]);
+                                }
+                            } else if (vec && f + 3 < a.rows) {
                                 *reinterpret_cast<float4*>(yp + j) = make_float4(o[0], o[1], o[2], o[3]);
                             } else {
 #pragma unroll
@@ -375,7 +386,7 @@ int linear_prepare()
 }
 
 int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* m_slot, uint32_t rows, uint32_t cols, bool flip,
-                  uint32_t slot, const DevTask& task, float lambda, float* y, void* stream)
+                  uint32_t slot, const DevTask& task, float lambda, void* y, bool y_bf16, void* stream)
 {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return static_cast<int>(cudaErrorNotSupported);
@@ -398,6 +409,7 @@ int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* 
     a.slot = slot;
     a.task = task;
     a.y = y;
+    a.y_bf16 = y_bf16 ? 1u : 0u;
     const dim3 grid((rows + kBN - 1) / kBN, (n_tokens + halves * kBM - 1) / (halves * kBM));
     if (halves == 1) linear_kernel<1><<<grid, kLinearThreads, LinearGeom<1>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
     else linear_kernel<2><<<grid, kLinearThreads, LinearGeom<2>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);

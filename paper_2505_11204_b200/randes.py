@@ -111,7 +111,7 @@ def lib():
         L.randes_retrieve_batch.restype = ctypes.c_int
         L.randes_retrieve_static.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
         L.randes_retrieve_static.restype = ctypes.c_int
-        L.randes_linear.argtypes = [vp, u32, ctypes.c_float, u32, vp, u32, vp, vp, vp, vp]
+        L.randes_linear.argtypes = [vp, u32, ctypes.c_float, u32, vp, u32, vp, vp, vp, ctypes.c_int, vp]
         L.randes_linear.restype = ctypes.c_int
         L.randes_linear_giveups.argtypes = [ctypes.POINTER(ctypes.c_uint)]
         L.randes_linear_giveups.restype = ctypes.c_int
@@ -249,9 +249,9 @@ def randes_retrieve_static(plan, task_id, lam, out_dtype, base, M, out, stream) 
     _check(lib().randes_retrieve_static(plan, task_id, lam, out_dtype, _addr(base), _addr(M), _addr(out), stream))
 
 
-def randes_linear(plan, task_id, lam, layer, x, n_tokens, base, M, y, stream) -> None:
+def randes_linear(plan, task_id, lam, layer, x, n_tokens, base, M, y, stream, y_dtype: int = F32) -> None:
     """y = x What_t[layer]^T on the tensor cores, the retrieved weight never written to memory."""
-    _check(lib().randes_linear(plan, task_id, lam, layer, _addr(x), n_tokens, _addr(base), _addr(M), _addr(y), stream))
+    _check(lib().randes_linear(plan, task_id, lam, layer, _addr(x), n_tokens, _addr(base), _addr(M), _addr(y), y_dtype, stream))
 
 
 def randes_linear_giveups() -> int:
@@ -448,13 +448,15 @@ class Plan:
         randes_retrieve_batch(self.handle, task_ids, lam, out_dtype, _as_ptrs(base), M, _as_ptrs(out), self._stream())
         return out_lists
 
-    def linear(self, task_id: int, lam: float, layer: int, x, base, M, y=None):
-        """x: [n_tokens, cols] bf16 CUDA tensor; returns y [n_tokens, rows] fp32."""
+    def linear(self, task_id: int, lam: float, layer: int, x, base, M, y=None, y_dtype: int = F32):
+        """x: [n_tokens, cols] bf16 CUDA tensor; returns y [n_tokens, rows], fp32 or bf16."""
         import torch
 
         if y is None:
-            y = torch.empty((x.shape[0], self.rows[layer]), dtype=torch.float32, device=x.device)
-        randes_linear(self.handle, task_id, lam, layer, x, int(x.shape[0]), _as_ptrs(base), M, y, self._stream())
+            y = torch.empty((x.shape[0], self.rows[layer]), dtype=torch.bfloat16 if y_dtype == BF16 else torch.float32, device=x.device)
+        else:
+            y_dtype = BF16 if y.dtype == torch.bfloat16 else F32
+        randes_linear(self.handle, task_id, lam, layer, x, int(x.shape[0]), _as_ptrs(base), M, y, self._stream(), y_dtype)
         return y
 
     def retrieve(self, task_id: int, lam: float, base, M, out=None, out_dtype: int = F32):

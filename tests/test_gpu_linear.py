@@ -72,6 +72,24 @@ def test_linear_small_shapes_ragged_tokens_and_features():
     _run(w, [1, 37, 128, 300])
 
 
+def test_linear_bf16_output_is_the_fp32_result_rounded_once():
+    w = _workload([(200, 192, 2), (7, 72, 2)], [S | F, F], n_tasks=2)
+    ids, seeds = list(w.task_ids), list(w.seeds)
+    base, tasks = wl.model_set(w, ids)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, max_tasks=2, m_dtype=wl.BF16)
+    M_dev = plan.compress(d_base, d_tasks)
+    rng = np.random.default_rng(6)
+    for p in range(w.n_layers):
+        x = to_dev(_bf16_normal(rng, (150, w.cols[p])))
+        y32 = plan.linear(ids[0], w.lam, p, x, d_base, M_dev)
+        y16 = plan.linear(ids[0], w.lam, p, x, d_base, M_dev, y_dtype=wl.BF16)
+        assert y16.dtype == torch.bfloat16
+        assert torch.equal(y16, y32.to(torch.bfloat16))           # same accumulators, one rounding to nearest even
+    assert randes.randes_linear_giveups() == 0
+    plan.close()
+
+
 def test_linear_without_flip_and_without_shuffle():
     w = _workload([(136, 128, 3), (64, 72, 2)], [S, 0])
     _run(w, [5, 130])
@@ -104,7 +122,7 @@ def test_linear_unaligned_output_zero_tokens_and_host_only_plan():
     assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - y_ref) <= (2 * 128 + 2) * 2.0 ** -24 * y_abs + 1e-30)
     assert bool(torch.isnan(buf[0]))                           # nothing before y was written
     empty = torch.zeros((0, 128), dtype=torch.bfloat16, device="cuda")
-    randes.randes_linear(plan.handle, ids[0], 0.3, 0, empty, 0, randes.ptr_array(d_base), M_dev, y, torch.cuda.current_stream().cuda_stream)
+    randes.randes_linear(plan.handle, ids[0], 0.3, 0, empty, 0, randes.ptr_array(d_base), M_dev, y, torch.cuda.current_stream().cuda_stream, wl.F32)
     assert randes.randes_launch_count() == before + 1          # no tokens: no launch
     with pytest.raises(randes.RandesError) as e:
         plan.linear(77, 0.3, 0, to_dev(x), d_base, M_dev)

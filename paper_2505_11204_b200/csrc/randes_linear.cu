@@ -289,47 +289,66 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
         }
         if (ok) ok = mbar_wait(bar_acc, 0, abort_flag);
         if (ok) {
+            // The accumulators hold one token per tensor-memory lane, i.e. per thread; stored like that, a warp's
+            // store would touch 32 rows of y at once.  Each warp therefore turns its [32 tokens x 128 features]
+            // block through shared memory (the operand ring is idle now: every product has completed) and writes
+            // whole 512-byte rows.  Row pitch 528 bytes: the 16-byte writes of a quarter-warp fall into distinct banks.
             tc_fence_after();
             const int quarter = warp & 3;                     // tensor-memory lanes 32 q .. 32 q + 31
             const uint32_t tlane = static_cast<uint32_t>(quarter * 32) << 16;
-            const bool vec = (a.rows & 3u) == 0 && (reinterpret_cast<uintptr_t>(a.y) & (a.y_bf16 ? 7u : 15u)) == 0;
+            constexpr uint32_t kPitch = kBN * 4 + 16;
+            const uint32_t stage = smem_base + quarter * (32 * kPitch);
+            const uint32_t esz = a.y_bf16 ? 2u : 4u;
+            const bool vec = (a.rows & 3u) == 0 && (reinterpret_cast<uintptr_t>(a.y) & (4 * esz - 1)) == 0;
+            const uint32_t f0 = n0 + lane * 4;                // this lane's four features when rows are written
 #pragma unroll 1
             for (int h = 0; h < HALVES; ++h) {
-                const uint32_t token = m0 + h * kBM + quarter * 32 + lane;
 #pragma unroll 1
                 for (int cchunk = 0; cchunk < kBN / 32; ++cchunk) {
                     uint32_t v0[32], v1[32];
                     tc_load32(tmem + tlane + h * 2 * kBN + cchunk * 32, v0);
                     tc_load32(tmem + tlane + h * 2 * kBN + kBN + cchunk * 32, v1);
                     tc_wait_ld();
-                    if (token < a.n_tokens) {
-                        const size_t y0 = static_cast<size_t>(token) * a.rows + n0 + cchunk * 32;
-                        float* yp = static_cast<float*>(a.y) + y0;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        uint4 o;
+                        o.x = __float_as_uint(__fmaf_rn(a.lambda, __uint_as_float(v1[j]), __uint_as_float(v0[j])));
+                        o.y = __float_as_uint(__fmaf_rn(a.lambda, __uint_as_float(v1[j + 1]), __uint_as_float(v0[j + 1])));
+                        o.z = __float_as_uint(__fmaf_rn(a.lambda, __uint_as_float(v1[j + 2]), __uint_as_float(v0[j + 2])));
+                        o.w = __float_as_uint(__fmaf_rn(a.lambda, __uint_as_float(v1[j + 3]), __uint_as_float(v0[j + 3])));
+                        sts128(stage + lane * kPitch + (cchunk * 32 + j) * 4, o);
+                    }
+                }
+                __syncwarp();
+                const uint32_t token0 = m0 + h * kBM + quarter * 32;
+#pragma unroll 4
+                for (int i = 0; i < 32; ++i) {
+                    const uint32_t token = token0 + i;
+                    if (token >= a.n_tokens) break;               // warp-uniform
+                    const uint4 o = lds128(stage + i * kPitch + lane * 16);
+                    const size_t y0 = static_cast<size_t>(token) * a.rows + f0;
+                    const float of[4] = {__uint_as_float(o.x), __uint_as_float(o.y), __uint_as_float(o.z), __uint_as_float(o.w)};
+                    if (a.y_bf16) {     // rounded to nearest even, once
                         bf16* yh = static_cast<bf16*>(a.y) + y0;
+                        if (vec && f0 + 3 < a.rows) {
+                            *reinterpret_cast<uint2*>(yh) = make_uint2(Out<bf16>::pack(of[0], of[1]), Out<bf16>::pack(of[2], of[3]));
+                        } else {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            float o[4];
+                            for (int e = 0; e < 4; ++e)
+                                if (f0 + e < a.rows) yh[e] = __float2bfloat16_rn(of[e]);
+                        }
+                    } else {
+                        float* yp = static_cast<float*>(a.y) + y0;
+                        if (vec && f0 + 3 < a.rows) {
+                            *reinterpret_cast<float4*>(yp) = make_float4(of[0], of[1], of[2], of[3]);
+                        } else {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) o[e] = __fmaf_rn(a.lambda, __uint_as_float(v1[j + e]), __uint_as_float(v0[j + e]));
-                            const uint32_t f = n0 + cchunk * 32 + j;
-                            if (a.y_bf16) {     // rounded to nearest even, once
-                                if (vec && f + 3 < a.rows) {
-                                    *reinterpret_cast<uint2*>(yh + j) = make_uint2(Out<bf16>::pack(o[0], o[1]), Out<bf16>::pack(o[2], o[3]));
-                                } else {
-#pragma unroll
-                                    for (int e = 0; e < 4; ++e)
-                                        if (f + e < a.rows) yh[j + e] = __float2bfloat16_rn(o[e]);
-                                }
-                            } else if (vec && f + 3 < a.rows) {
-                                *reinterpret_cast<float4*>(yp + j) = make_float4(o[0], o[1], o[2], o[3]);
-                            } else {
-#pragma unroll
-                                for (int e = 0; e < 4; ++e)
-                                    if (f + e < a.rows) yp[j + e] = o[e];
-                            }
+                            for (int e = 0; e < 4; ++e)
+                                if (f0 + e < a.rows) yp[e] = of[e];
                         }
                     }
                 }
+                __syncwarp();   // the block is reused for the next 128 tokens
             }
         }
     }

@@ -192,7 +192,9 @@ int randes_task_tables(const randes_plan_t* plan, uint32_t task_id,
  *                              registered task.
  * With a bf16 superposition at most 32 tasks can be summed in one call
  * (CAPACITY otherwise): further models are added with randes_add_model.
- * One kernel launch.  Errors: INVALID_ARGUMENT, MISALIGNED, CAPACITY, CUDA_ERROR.
+ * One kernel launch, or two when some groups are shuffled (those groups go through a kernel that stages
+ * the base tiles of a whole group in shared memory, the remaining tensors through the per-layer kernel).
+ * Errors: INVALID_ARGUMENT, MISALIGNED, CAPACITY, CUDA_ERROR.
  */
 int randes_compress(randes_plan_t* plan, const void* const* base, const void* const* tasks,
                     void* M, void* stream);
@@ -281,7 +283,8 @@ int randes_linear_giveups(unsigned int* count);
  * randes_retrieve, but W_0 is read once instead of n_tasks times.
  *   task_ids[n_tasks]           distinct registered ids, 1 <= n_tasks <= 32 and <= max_tasks
  *   out[n_tasks * n_layers]     out[b*n_layers + l] = layer l of the b-th requested model
- * One kernel launch.  Errors: as randes_retrieve, plus DUPLICATE_TASK, CAPACITY.
+ * One kernel launch, or two when some groups are shuffled (fp32 weights and superposition).
+ * Errors: as randes_retrieve, plus DUPLICATE_TASK, CAPACITY.
  */
 int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_t n_tasks, float lambda,
                           randes_dtype_t out_dtype, const void* const* base, const void* M,

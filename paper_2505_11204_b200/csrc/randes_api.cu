@@ -435,6 +435,20 @@ int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_
         ++g_launches;
     }
     if (a.n_units == 0) return RANDES_OK;
+    // one model, bf16 weights, fp32 superposition: the kernel whose requests are contiguous across a warp,
+    // when every layer's width and every tensor's alignment allow it
+    bool halves = n_rows == 1 && init_from_m && p.storage == RANDES_BF16 && p.m_dtype == RANDES_F32;
+    for (uint32_t l = 0; halves && l < p.n_layers; ++l) {
+        if (p.layers[l].rows == 0 || p.layers[l].cols == 0) continue;
+        halves = p.layers[l].cols % 8 == 0 && reinterpret_cast<uintptr_t>(task_ptrs[l]) % 16 == 0 &&
+                 (!base || reinterpret_cast<uintptr_t>(base[l]) % 16 == 0);
+    }
+    if (halves) {
+        const int he = launch_add_halves(a, p.sm_count, s);
+        if (he) return fail_cuda(static_cast<cudaError_t>(he), "launch of the add / remove kernel");
+        ++g_launches;
+        return RANDES_OK;
+    }
     const int grid = std::min<int>(p.grid_acc[n_rows == 1], static_cast<int>(a.n_units));
     const int e = launch_accumulate(p.storage, p.m_dtype, a, grid, s);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the accumulate kernel");

@@ -154,6 +154,8 @@ struct GramArgs {
 // Launchers (randes_kernels.cu).  Return a cudaError_t as int.
 int launch_retrieve(int storage_dtype, int out_dtype, int m_dtype, const RetrieveArgs& a, int grid, void* stream);
 int launch_accumulate(int storage_dtype, int m_dtype, const AccumulateArgs& a, int grid, void* stream);
+// add / remove of one model, bf16 weights, fp32 superposition, every layer cols % 8 == 0 and 16-byte aligned tensors
+int launch_add_halves(const AccumulateArgs& a, int sm_count, void* stream);
 // randes_context.cu: all of a plan's layers under a general diagonal context (plans with a RANDES_GAUSS group);
 // fp32 superposition only.  Return a cudaError_t as int.
 int launch_context_accumulate(int storage_dtype, const AccumulateArgs& a, int sm_count, void* stream);

@@ -90,6 +90,60 @@ __device__ __noinline__ void retrieve_rows_scalar(WarpTile t, uint32_t cols, con
     }
 }
 
+// bf16 weights with an fp32 superposition.  In the layout above a lane owns 8 neighbouring columns, so its M tile
+// and its fp32 output are 32 bytes: two requests whose lanes sit 32 bytes apart, each using half of every sector it
+// touches.  Here a lane owns 4 + 4 columns instead -- columns 4 lane .. 4 lane + 3 of both 128-column halves of the
+// warp's block -- so that every request of the warp is contiguous (512 bytes of M or fp32 output, 256 bytes of
+// weights), and each half has its own Philox block, read like an fp32 warp would.
+template <typename OT>
+__device__ __forceinline__ void retrieve_rows_halves(const WarpTile& t, uint32_t cols, int lane, const float* __restrict__ mp,
+                                                     const bf16* __restrict__ wp, OT* __restrict__ op, float lambda,
+                                                     uint32_t bits0, uint32_t bits1)
+{
+    constexpr int U = 2;                                  // rows per trip (1 and 4 measured slower)
+    const uint32_t c0 = t.cb * 256u + lane * 4u;          // first half; the second is 128 columns further
+    const bool on[2] = {c0 < cols, c0 + 128u < cols};
+    float lam[2][4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        lam[0][e] = flip(lambda, ((bits0 >> e) & 1u) << 31);
+        lam[1][e] = flip(lambda, ((bits1 >> e) & 1u) << 31);
+    }
+    const uint32_t row_stride = t.rstep * cols;
+    uint32_t off = t.r0 * cols + c0;                      // layers hold < 2^32 elements
+    for (uint32_t r = t.r0; r < t.r_end; r += t.rstep * U, off += row_stride * U) {
+        float4 m[U][2];
+        uint2 w[U][2];
+#pragma unroll
+        for (int j = 0; j < U; ++j)
+            if (r + j * t.rstep < t.r_end) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                    if (on[h]) {
+                        const uint32_t o = off + j * row_stride + h * 128u;
+                        m[j][h] = __ldcs(reinterpret_cast<const float4*>(mp + o));
+                        w[j][h] = __ldcs(reinterpret_cast<const uint2*>(wp + o));
+                    }
+            }
+#pragma unroll
+        for (int j = 0; j < U; ++j)
+            if (r + j * t.rstep < t.r_end) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                    if (on[h]) {
+                        const uint32_t o = off + j * row_stride + h * 128u;
+                        const float wv[4] = {__uint_as_float(w[j][h].x << 16), __uint_as_float(w[j][h].x & 0xFFFF0000u),
+                                             __uint_as_float(w[j][h].y << 16), __uint_as_float(w[j][h].y & 0xFFFF0000u)};
+                        const float mv[4] = {m[j][h].x, m[j][h].y, m[j][h].z, m[j][h].w};
+                        float y[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) y[e] = __fmaf_rn(lam[h][e], mv[e], wv[e]);
+                        Out<OT>::template store<4>(op + o, y);
+                    }
+            }
+    }
+}
+
 template <typename ST, typename OT, typename MT>
 __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_kernel(const RetrieveArgs a)
 {
@@ -102,6 +156,21 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_kernel(const Retri
         const uint32_t slot = (lp.flags & kFlagShuffle) ? a.slot_of_pos[p] : p;   // sigma^-1
         const unsigned long long m_off = slot == p ? lp.m_off : a.layers[slot].m_off;
         const WarpTile t = warp_tile<CPL>(un, warp, lane);
+        if constexpr (CPL == 8 && sizeof(MT) == 4) {
+            // bf16 weights, fp32 M: the lane mapping with contiguous requests, when widths and alignment allow
+            const bf16* wp8 = static_cast<const bf16*>(a.base[p]);
+            OT* op8 = static_cast<OT*>(a.out[p]);
+            if (lp.cols % 8 == 0 && aligned16(wp8) && (reinterpret_cast<uintptr_t>(op8) & 15) == 0) {
+                if (t.r0 >= t.r_end || t.cb * 256u >= lp.cols) continue;   // warp-uniform
+                uint32_t b0 = 0, b1 = 0;
+                if (lp.flags & kFlagFlip) {
+                    b0 = lane_bits<4>(philox4x32_10(t.cb * 2, slot, kTagSign, a.task.id, a.task.key0, a.task.key1), lane);
+                    b1 = lane_bits<4>(philox4x32_10(t.cb * 2 + 1, slot, kTagSign, a.task.id, a.task.key0, a.task.key1), lane);
+                }
+                retrieve_rows_halves<OT>(t, lp.cols, lane, static_cast<const float*>(a.M) + m_off, wp8, op8, a.lambda, b0, b1);
+                continue;
+            }
+        }
         if (t.c >= lp.cols || t.r0 >= t.r_end) continue;
 
         uint32_t bits = 0;
@@ -472,6 +541,80 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const Acc
     }
 }
 
+// add / remove for bf16 weights and an fp32 superposition, with the lane mapping of retrieve_rows_halves: a lane
+// owns columns 4 lane .. 4 lane + 3 of both 128-column halves of the warp's block, so the 32 bytes of M it reads
+// and writes per row are two requests that are contiguous across the warp.  Plain register loads, two rows per
+// trip.  Used when every layer has a width that is a multiple of 8 and 16-byte aligned tensors; the result is
+// the same as accumulate_kernel's: d = W_j - W_0 (one rounding), M +- s d (one rounding).
+template <bool HAS_BASE>
+__global__ void __launch_bounds__(kThreadsPerCta, 3) add_halves_kernel(const AccumulateArgs a)
+{
+    constexpr int U = 2;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const DevTask tk = a.tasks[0];
+    const uint32_t neg = a.negate ? 0xFu : 0u;
+    for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+        const DevUnit un = a.units[u];
+        const uint32_t slot = un.layer;
+        const DevLayer ls = a.layers[slot];
+        const WarpTile t = warp_tile<8>(un, warp, lane);
+        const uint32_t cols = ls.cols;
+        if (t.r0 >= t.r_end || t.cb * 256u >= cols) continue;   // warp-uniform
+        const uint32_t src = (ls.flags & kFlagShuffle) ? a.src_of_slot[slot] : slot;   // sigma_j(l)
+        const bf16* wp = static_cast<const bf16*>(a.task_ptrs[src]);
+        const bf16* bp = HAS_BASE ? static_cast<const bf16*>(a.base[src]) : nullptr;
+        float* mp = static_cast<float*>(a.M) + ls.m_off;
+        uint32_t bits[2] = {neg, neg};
+        if (ls.flags & kFlagFlip) {
+            bits[0] ^= lane_bits<4>(philox4x32_10(t.cb * 2, slot, kTagSign, tk.id, tk.key0, tk.key1), lane);
+            bits[1] ^= lane_bits<4>(philox4x32_10(t.cb * 2 + 1, slot, kTagSign, tk.id, tk.key0, tk.key1), lane);
+        }
+        const uint32_t c0 = t.cb * 256u + lane * 4u;
+        const bool on[2] = {c0 < cols, c0 + 128u < cols};
+        const uint32_t row_stride = t.rstep * cols;
+        uint32_t off = t.r0 * cols + c0;                      // layers hold < 2^32 elements
+        for (uint32_t r = t.r0; r < t.r_end; r += t.rstep * U, off += row_stride * U) {
+            float4 m[U][2];
+            uint2 w[U][2], b[U][2];
+#pragma unroll
+            for (int j = 0; j < U; ++j)
+                if (r + j * t.rstep < t.r_end) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        if (on[h]) {
+                            const uint32_t o = off + j * row_stride + h * 128u;
+                            m[j][h] = *reinterpret_cast<const float4*>(mp + o);
+                            w[j][h] = __ldcs(reinterpret_cast<const uint2*>(wp + o));
+                            if (HAS_BASE) b[j][h] = __ldcs(reinterpret_cast<const uint2*>(bp + o));
+                        }
+                }
+#pragma unroll
+            for (int j = 0; j < U; ++j)
+                if (r + j * t.rstep < t.r_end) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        if (on[h]) {
+                            const uint32_t o = off + j * row_stride + h * 128u;
+                            const float wv[4] = {__uint_as_float(w[j][h].x << 16), __uint_as_float(w[j][h].x & 0xFFFF0000u),
+                                                 __uint_as_float(w[j][h].y << 16), __uint_as_float(w[j][h].y & 0xFFFF0000u)};
+                            const float mv[4] = {m[j][h].x, m[j][h].y, m[j][h].z, m[j][h].w};
+                            float y[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                float d = wv[e];
+                                if (HAS_BASE) {
+                                    const uint32_t bw = e < 2 ? b[j][h].x : b[j][h].y;
+                                    d = __fsub_rn(d, __uint_as_float((e & 1) ? (bw & 0xFFFF0000u) : (bw << 16)));
+                                }
+                                y[e] = __fadd_rn(mv[e], flip(d, ((bits[h] >> e) & 1u) << 31));
+                            }
+                            *reinterpret_cast<float4*>(mp + o) = make_float4(y[0], y[1], y[2], y[3]);
+                        }
+                }
+        }
+    }
+}
+
 template <typename K> int ctas_per_sm(K kernel, size_t smem)
 {
     if (smem > 48 * 1024 &&
@@ -505,6 +648,21 @@ int launch_retrieve(int storage_dtype, int out_dtype, int m_dtype, const Retriev
             });
         });
     });
+}
+
+int launch_add_halves(const AccumulateArgs& a, int sm_count, void* stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int per_sm = 0;
+    cudaError_t e = a.has_base ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, add_halves_kernel<true>, kThreadsPerCta, 0)
+                               : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, add_halves_kernel<false>, kThreadsPerCta, 0);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return static_cast<int>(e); }
+    if (per_sm <= 0) return static_cast<int>(cudaErrorInvalidConfiguration);
+    const unsigned long long want = static_cast<unsigned long long>(sm_count) * per_sm;
+    const int grid = static_cast<int>(want < a.n_units ? want : a.n_units);
+    if (a.has_base) add_halves_kernel<true><<<grid, kThreadsPerCta, 0, s>>>(a);
+    else add_halves_kernel<false><<<grid, kThreadsPerCta, 0, s>>>(a);
+    return static_cast<int>(cudaGetLastError());
 }
 
 int launch_accumulate(int storage_dtype, int m_dtype, const AccumulateArgs& a, int grid, void* stream)

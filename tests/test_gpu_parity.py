@@ -419,6 +419,15 @@ def test_large_and_partly_shuffled_groups(n_tasks, storage):
     run_full_cycle(make_workload(shapes, flags=flags, n_tasks=n_tasks, storage=storage), out_dtypes=(wl.F32,), extra_task=False)
 
 
+def test_bf16_weights_with_widths_that_are_multiples_of_eight():
+    """bf16 weights whose every width is a multiple of 8: add / remove and retrieve then take the kernels in which a lane
+    owns 4 + 4 columns of the two halves of a 256-column block (ragged last blocks: 8, 264, 1032 columns)."""
+    shapes = [(9, 256, 3), (5, 264, 2), (17, 1032, 2), (1, 8, 4), (40, 520, 1), (3, 128, 5)]
+    flags = [S | F, S | F, F, S, F, S | F | randes.SKIP(2)]
+    run_full_cycle(make_workload(shapes, flags=flags, storage=wl.BF16, n_tasks=4))
+    run_full_cycle(make_workload(shapes, flags=flags, storage=wl.BF16, n_tasks=2), m_dtype=wl.BF16, out_dtypes=(wl.BF16,))
+
+
 @pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
 @pytest.mark.parametrize("n_tasks", [3, 10])
 def test_gaussian_diagonal_context(storage, n_tasks):

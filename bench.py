@@ -520,6 +520,42 @@ def run_ours(args):
                                 "GBps": byts / (ms * 1e-3) / 1e9, "frac_of_%s_peak" % peak_kind: byts / (ms * 1e-3) / 1e9 / peak,
                                 "speedup_per_model_vs_add": ops["add"]["ms_per_call"] / (ms / n_swap)}
 
+    # ---- adapter deltas (Section 5.8): the tasks' tensors already hold the deltas (base = NULL), only the layers that carry
+    #      an adapter are in the plan; rank-16 deltas materialised beforehand, here random values of that shape
+    if args.workload == "flan_t5_base":
+        try:
+            wa = wl.subset(w, wl.flan_t5_lora_targets(w), w.name + ":adapter-targets")
+            g_a = torch.Generator(device=dev).manual_seed(4321)
+            a_tasks = [[(torch.randn(r, c, device=dev, generator=g_a) * 1e-4).to(tdt) for r, c in zip(wa.rows, wa.cols)] for _ in range(K + 1)]
+            plan_a = randes.Plan.from_workload(wa, max_tasks=K + 1, device=dev)
+            M_a = plan_a.new_superposition()
+            pa = randes.ptr_array(a_tasks[:K])
+            pa_new = randes.ptr_array(a_tasks[K])
+            t_c, t_a = [], []
+            for rep in range(2 + 5):
+                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                e0.record(stream)
+                randes.randes_compress(plan_a.handle, None, pa, M_a, sh)
+                e1.record(stream)
+                randes.randes_add_model(plan_a.handle, 1000, 77, None, pa_new, M_a, sh)
+                e2.record(stream)
+                randes.randes_remove_model(plan_a.handle, 1000, None, pa_new, M_a, sh)
+                if rep >= 2:
+                    t_c.append((e0, e1)); t_a.append((e1, e2))
+            barrier()
+            ms_c = max_over_ranks([sum(x.elapsed_time(y) for x, y in t_c) / len(t_c)], world, dev)[0]
+            ms_a = max_over_ranks([sum(x.elapsed_time(y) for x, y in t_a) / len(t_a)], world, dev)[0]
+            s_el = 2 if w.storage == wl.BF16 else 4
+            extras["adapter_deltas"] = {"layers": wa.n_layers, "params_M": wa.n_params / 1e6, "tasks": K,
+                                        "compress_ms": ms_c, "compress_GBps": (K * s_el + 4) * wa.n_params / (ms_c * 1e-3) / 1e9,
+                                        "add_ms": ms_a, "add_GBps": (8 + s_el) * wa.n_params / (ms_a * 1e-3) / 1e9,
+                                        "note": "tasks given as deltas (no base): compress moves K*s + 4 bytes per parameter, add 8 + s"}
+            plan_a.close()
+            del a_tasks, M_a
+            torch.cuda.empty_cache()
+        except torch.OutOfMemoryError:
+            extras["adapter_deltas"] = None
+
     # ---- a linear layer on the retrieved weight, the weight never written (tensor cores): the largest
     #      repeated matrix of the set, bf16 weights and a bf16 superposition, 8192 tokens, timed alone
     try:

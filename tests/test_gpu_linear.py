@@ -95,6 +95,23 @@ def test_linear_without_flip_and_without_shuffle():
     _run(w, [5, 130])
 
 
+def test_linear_blocks_of_256_tokens():
+    # enough tiles (16 feature tiles x 10 blocks of 256 tokens >= the SM count) for the 256-token CTA, whose second
+    # block of 128 tokens has accumulators of its own; ragged token count, ragged last k-step, bf16 and fp32 output
+    w = _workload([(2048, 136, 2)], [S | F], n_tasks=2)
+    _run(w, [2500], layers=[0])
+    ids = list(w.task_ids)
+    base, tasks = wl.model_set(w, ids)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, max_tasks=2, m_dtype=wl.BF16)
+    M_dev = plan.compress(d_base, d_tasks)
+    x = to_dev(_bf16_normal(np.random.default_rng(8), (2500, 136)))
+    y32 = plan.linear(ids[1], w.lam, 1, x, d_base, M_dev)
+    y16 = plan.linear(ids[1], w.lam, 1, x, d_base, M_dev, y_dtype=wl.BF16)
+    assert torch.equal(y16, y32.to(torch.bfloat16))
+    plan.close()
+
+
 def test_linear_wide_layer_many_k_steps():
     # 16 k-steps: every stage of the ring is reused several times
     w = _workload([(384, 1024, 2)], [S | F], n_tasks=2)

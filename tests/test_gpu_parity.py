@@ -419,6 +419,15 @@ def test_large_and_partly_shuffled_groups(n_tasks, storage):
     run_full_cycle(make_workload(shapes, flags=flags, n_tasks=n_tasks, storage=storage), out_dtypes=(wl.F32,), extra_task=False)
 
 
+@pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
+@pytest.mark.parametrize("n_tasks", [24, 30])
+def test_group_compress_with_shallower_rings(storage, n_tasks):
+    """Many tasks x many members: the per-(slot, task) records take the room of ring stages (fp32: 24 tasks x 30 members
+    leave 5 stages, 30 x 30 leave 4; bf16: 3) while two CTAs still fit an SM."""
+    shapes = [(8, 128, 24), (6, 256, 30), (4, 64, 1)]
+    run_full_cycle(make_workload(shapes, flags=[S | F, S | F, F], storage=storage, n_tasks=n_tasks), out_dtypes=(wl.F32,), extra_task=False)
+
+
 def test_bf16_weights_with_widths_that_are_multiples_of_eight():
     """bf16 weights whose every width is a multiple of 8: add / remove and retrieve then take the kernels in which a lane
     owns 4 + 4 columns of the two halves of a 256-column block (ragged last blocks: 8, 264, 1032 columns)."""

@@ -428,6 +428,24 @@ def test_group_compress_with_shallower_rings(storage, n_tasks):
     run_full_cycle(make_workload(shapes, flags=[S | F, S | F, F], storage=storage, n_tasks=n_tasks), out_dtypes=(wl.F32,), extra_task=False)
 
 
+def test_batched_retrieve_of_many_tasks_and_members():
+    """32 tasks x 30 members: the records of the grouped batched retrieve no longer fit beside two resident CTAs."""
+    import torch
+
+    w = make_workload([(6, 256, 30), (5, 132, 24), (3, 64, 1)], flags=[S | F, S | F, F], n_tasks=32)
+    base, tasks = wl.model_set(w, w.task_ids)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, max_tasks=32)
+    M = plan.compress(d_base, d_tasks)
+    M_ref = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, base, tasks)
+    check_superposition(plan, M, M_ref, "compress")
+    outs = plan.retrieve_batch(list(w.task_ids), w.lam, d_base, M)
+    for b, (t, s_) in enumerate(zip(w.task_ids, w.seeds)):
+        check_model(outs[b], ro.retrieve(w.spec, w.storage, wl.F32, t, s_, w.lam, base, M_ref), "batch task %d" % t)
+    torch.cuda.synchronize()
+    plan.close()
+
+
 def test_bf16_weights_with_widths_that_are_multiples_of_eight():
     """bf16 weights whose every width is a multiple of 8: add / remove and retrieve then take the kernels in which a lane
     owns 4 + 4 columns of the two halves of a 256-column block (ragged last blocks: 8, 264, 1032 columns)."""

@@ -177,9 +177,12 @@ def test_single_task_round_trip_and_lambda_one():
     plan.close()
 
 
-def test_delta_input_without_base():
-    # adapter deltas given directly (Section 5.8): base = NULL
-    w = make_workload([(16, 768, 3), (768, 16, 2), (1, 100, 2)], n_tasks=3)
+@pytest.mark.parametrize("storage,shapes", [(wl.F32, [(16, 768, 3), (768, 16, 2), (1, 100, 2)]),
+                                            (wl.BF16, [(16, 768, 3), (768, 16, 2), (1, 104, 2)])])
+def test_delta_input_without_base(storage, shapes):
+    # adapter deltas given directly (Section 5.8): base = NULL (bf16: all widths multiples of 8, the add / remove
+    # kernel with 4 + 4 columns per lane)
+    w = make_workload(shapes, n_tasks=3, storage=storage)
     deltas = [[wl.lora_delta_layer(w, l, t) for l in range(w.n_layers)] for t in w.task_ids]
     d_deltas = [model_to_dev(d) for d in deltas]
     plan = randes.Plan.from_workload(w)

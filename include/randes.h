@@ -313,6 +313,34 @@ int randes_delta_gram(randes_plan_t* plan, const void* const* base, const void* 
                       double* gram, void* scratch, size_t scratch_bytes, void* stream);
 
 /*
+ * What the Gram matrix says about one retrieval (Section 3, the equation for the norm of
+ * the interference; Section 4, second display: What_t - W_0 - lambda d_t is exactly the
+ * interference term).  For the task in row/column t of `gram`,
+ *     *norm = lambda * sqrt( sum_{j != t} sum_{l != t} gram[j*n + l] )
+ *           = || lambda * sum_{j != t} T_t^-1 T_j d_j ||_2 ,
+ * the rows added in index order, each row in index order, in fp64; a sum that rounding
+ * pushed below zero counts as zero.
+ *   gram   HOST array of n*n doubles (randes_delta_gram's result copied back), n >= 1
+ * Host-only; nothing is launched.  Errors: INVALID_ARGUMENT (NULL, t >= n).
+ */
+int randes_interference_norm(const double* gram, uint32_t n, uint32_t t, double lambda, double* norm);
+
+/*
+ * Pairwise cosine similarity among the deltas that interfere in a retrieval (the paper's
+ * figures on cosine similarity among interfering deltas, main text and appendix):
+ *     cos(j, l) = gram[j*n + l] / sqrt(gram[j*n + j] * gram[l*n + l])
+ * (the same for T_j d_j, T_l d_l and for T_t^-1 T_j d_j, T_t^-1 T_l d_l: T_t is orthogonal).
+ *   gram      HOST array of n*n doubles
+ *   exclude   index of the retrieved task, left out of the mean; negative = none
+ *   cosines   HOST array of n*n doubles or NULL; receives every cos(j, l) (1 on the
+ *             diagonal; 0 where a delta has zero norm)
+ *   mean      or NULL; receives the mean over the pairs j < l with j, l != exclude,
+ *             summed in index order (0 when there is no such pair)
+ * Host-only; nothing is launched.  Errors: INVALID_ARGUMENT (NULL gram, n == 0, exclude >= n).
+ */
+int randes_pairwise_cosines(const double* gram, uint32_t n, int32_t exclude, double* cosines, double* mean);
+
+/*
  * retrieve for callers that cannot provide a device workspace.  (The paper has
  * no counterpart: this entry point exists for deployment, not for the method.)
  *

@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -1191,6 +1192,47 @@ int randes_delta_gram(randes_plan_t* plan, const void* const* base, const void* 
                       size_t scratch_bytes, void* stream)
 {
     return guarded([&] { return randes_delta_gram_impl(plan, base, tasks, gram, scratch, scratch_bytes, stream); });
+}
+
+// Section 3, norm of the interference: || lambda sum_{j != t} T_t^-1 T_j d_j ||^2 = lambda^2 sum_{j,l != t} <T_j d_j, T_l d_l>,
+// because T_t^-1 is orthogonal.
+int randes_interference_norm(const double* gram, uint32_t n, uint32_t t, double lambda, double* norm)
+{
+    if (!gram || !norm) return fail(RANDES_INVALID_ARGUMENT, "gram or norm is NULL");
+    if (n == 0 || t >= n) return fail(RANDES_INVALID_ARGUMENT, "task index %u out of range (n = %u)", t, n);
+    double total = 0.0;
+    for (uint32_t j = 0; j < n; ++j) {
+        if (j == t) continue;
+        double row = 0.0;
+        for (uint32_t l = 0; l < n; ++l)
+            if (l != t) row += gram[static_cast<size_t>(j) * n + l];
+        total += row;
+    }
+    *norm = lambda * std::sqrt(total > 0.0 ? total : 0.0);
+    return RANDES_OK;
+}
+
+int randes_pairwise_cosines(const double* gram, uint32_t n, int32_t exclude, double* cosines, double* mean)
+{
+    if (!gram) return fail(RANDES_INVALID_ARGUMENT, "gram is NULL");
+    if (n == 0) return fail(RANDES_INVALID_ARGUMENT, "n is 0");
+    if (exclude >= 0 && static_cast<uint32_t>(exclude) >= n)
+        return fail(RANDES_INVALID_ARGUMENT, "exclude = %d out of range (n = %u)", exclude, n);
+    auto cosine = [&](uint32_t j, uint32_t l) {
+        if (j == l) return 1.0;
+        const double d = std::sqrt(gram[static_cast<size_t>(j) * n + j] * gram[static_cast<size_t>(l) * n + l]);
+        return d > 0.0 ? gram[static_cast<size_t>(j) * n + l] / d : 0.0;
+    };
+    double sum = 0.0;
+    uint64_t pairs = 0;
+    for (uint32_t j = 0; j < n; ++j)
+        for (uint32_t l = 0; l < n; ++l) {
+            const double c = cosine(j, l);
+            if (cosines) cosines[static_cast<size_t>(j) * n + l] = c;
+            if (j < l && static_cast<int64_t>(j) != exclude && static_cast<int64_t>(l) != exclude) { sum += c; ++pairs; }
+        }
+    if (mean) *mean = pairs ? sum / static_cast<double>(pairs) : 0.0;
+    return RANDES_OK;
 }
 
 int randes_retrieve_static(const randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,

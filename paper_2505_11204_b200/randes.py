@@ -107,6 +107,10 @@ def lib():
         L.randes_delta_gram_scratch_bytes.restype = sz
         L.randes_delta_gram.argtypes = [vp, vp, vp, vp, vp, sz, vp]
         L.randes_delta_gram.restype = ctypes.c_int
+        L.randes_interference_norm.argtypes = [vp, u32, u32, ctypes.c_double, ctypes.POINTER(ctypes.c_double)]
+        L.randes_interference_norm.restype = ctypes.c_int
+        L.randes_pairwise_cosines.argtypes = [vp, u32, ctypes.c_int32, vp, ctypes.POINTER(ctypes.c_double)]
+        L.randes_pairwise_cosines.restype = ctypes.c_int
         L.randes_retrieve_batch.argtypes = [vp, vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
         L.randes_retrieve_batch.restype = ctypes.c_int
         L.randes_retrieve_static.argtypes = [vp, u32, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
@@ -127,7 +131,7 @@ EXPORTS = [
     "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
     "randes_task_tables", "randes_plan_serialize", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_add_models", "randes_remove_model",
-    "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_retrieve_batch", "randes_retrieve_static", "randes_linear", "randes_linear_giveups", "randes_launch_count", "randes_last_error",
+    "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_interference_norm", "randes_pairwise_cosines", "randes_retrieve_batch", "randes_retrieve_static", "randes_linear", "randes_linear_giveups", "randes_launch_count", "randes_last_error",
 ]
 
 
@@ -285,22 +289,32 @@ def _as_ptrs(x):
     return ptr_array(x)
 
 
-def interference_norm(gram, t: int, lam: float) -> float:
-    """|| lam * sum_{j != t} T_t^-1 T_j d_j || from the Gram matrix (Section 3 of the paper)."""
-    import math
-
+def _host_gram(gram):
+    """An [n, n] Gram matrix (torch tensor, numpy array or nested lists) as a host array of doubles."""
+    if hasattr(gram, "detach"):
+        gram = gram.detach().cpu().tolist()
+    elif hasattr(gram, "tolist"):
+        gram = gram.tolist()
     n = len(gram)
-    return lam * math.sqrt(max(0.0, sum(float(gram[j][l]) for j in range(n) for l in range(n) if j != t and l != t)))
+    return (ctypes.c_double * max(n * n, 1))(*[float(v) for row in gram for v in row]), n
 
 
-def mean_pairwise_cosine(gram, exclude=None) -> float:
-    """Average cosine over all pairs of distinct tasks, leaving `exclude` out (the retrieved task)."""
-    import math
+def randes_interference_norm(gram, t: int, lam: float) -> float:
+    """|| lam * sum_{j != t} T_t^-1 T_j d_j || from the Gram matrix; computed by the library."""
+    g, n = _host_gram(gram)
+    out = ctypes.c_double(0.0)
+    _check(lib().randes_interference_norm(ctypes.addressof(g), n, int(t), float(lam), ctypes.byref(out)))
+    return float(out.value)
 
-    n = len(gram)
-    idx = [i for i in range(n) if i != exclude]
-    pairs = [(i, j) for a, i in enumerate(idx) for j in idx[a + 1:]]
-    return sum(float(gram[i][j]) / math.sqrt(float(gram[i][i]) * float(gram[j][j])) for i, j in pairs) / max(len(pairs), 1)
+
+def randes_pairwise_cosines(gram, exclude: int = -1):
+    """(cosines as n lists of n floats, mean over pairs j < l that leave `exclude` out); computed by the library."""
+    g, n = _host_gram(gram)
+    cos = (ctypes.c_double * max(n * n, 1))()
+    mean = ctypes.c_double(0.0)
+    _check(lib().randes_pairwise_cosines(ctypes.addressof(g), n, -1 if exclude is None else int(exclude), ctypes.addressof(cos),
+                                         ctypes.byref(mean)))
+    return [[float(cos[j * n + l]) for l in range(n)] for j in range(n)], float(mean.value)
 
 
 # ---- convenience object over torch tensors --------------------------------------------------

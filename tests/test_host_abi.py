@@ -177,6 +177,52 @@ def test_plan_argument_validation():
     p.close()
 
 
+def test_interference_norm_and_cosines_against_the_oracle():
+    """randes_interference_norm / randes_pairwise_cosines (host entry points) against what the oracle gives:
+    the norm of the interference is measured on the oracle's own retrieved model (Section 4, second display:
+    What_t - W_0 - lambda d_t is the interference), the cosines on the transformed deltas themselves
+    (a one-task compress is T_i d_i).  Dyadic inputs: the Gram matrix and every sum are exact."""
+    S, F = randes.SHUFFLE, randes.FLIP
+    rows, cols, group = [4, 2, 4, 2, 4, 2], [8, 5, 8, 5, 8, 5], [0, 1, 0, 1, 0, 1]
+    spec = (rows, cols, group, [S | F, S])
+    rng = np.random.default_rng(77)
+    model = lambda: [(rng.integers(-512, 513, size=(r, c)) / 1024.0).astype(np.float32) for r, c in zip(rows, cols)]
+    base = model()
+    ids, seeds = [4, 0, 9, 2], [11, 12, 13, 14]
+    tasks = [model() for _ in ids]
+    G = ro.delta_gram(spec, ro.F32, ids, seeds, base, tasks)
+    flat = lambda m: np.concatenate([np.asarray(a, dtype=np.float64).ravel() for a in m])
+    M = ro.compress(spec, ro.F32, ids, seeds, base, tasks)
+    for lam in (1.0, 0.25):
+        for t in range(len(ids)):
+            what = ro.retrieve(spec, ro.F32, ro.F32, ids[t], seeds[t], lam, base, M)
+            inter = flat(what) - flat(base) - lam * (flat(tasks[t]) - flat(base))
+            want = float(np.sqrt(inter @ inter))
+            got = randes.randes_interference_norm(G, t, lam)
+            assert abs(got - want) <= 4 * np.finfo(np.float64).eps * want, (t, got, want)
+    X = [flat(ro.compress(spec, ro.F32, [i], [s], base, [tk])) for i, s, tk in zip(ids, seeds, tasks)]
+    cos, mean = randes.randes_pairwise_cosines(G)
+    n = len(ids)
+    for j in range(n):
+        for l in range(n):
+            want = 1.0 if j == l else float(X[j] @ X[l]) / float(np.sqrt((X[j] @ X[j]) * (X[l] @ X[l])))
+            assert abs(cos[j][l] - want) <= 1e-15, (j, l)
+    pairs = [(j, l) for j in range(n) for l in range(j + 1, n)]
+    assert abs(mean - sum(cos[j][l] for j, l in pairs) / len(pairs)) <= 1e-15
+    _, mean_wo = randes.randes_pairwise_cosines(G, exclude=1)
+    kept = [(j, l) for j, l in pairs if 1 not in (j, l)]
+    assert abs(mean_wo - sum(cos[j][l] for j, l in kept) / len(kept)) <= 1e-15
+    # degenerate inputs: one task (no pair, nothing interferes), a zero delta, bad arguments
+    assert randes.randes_pairwise_cosines([[2.0]])[1] == 0.0
+    assert randes.randes_interference_norm([[2.0]], 0, 1.0) == 0.0
+    assert randes.randes_pairwise_cosines([[0.0, 0.0], [0.0, 4.0]])[0] == [[1.0, 0.0], [0.0, 1.0]]
+    _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_interference_norm(G, n, 1.0))
+    _expect(randes.INVALID_ARGUMENT, lambda: randes.randes_pairwise_cosines(G, exclude=n))
+    out = ctypes.c_double()
+    assert randes.lib().randes_interference_norm(None, 2, 0, 1.0, ctypes.byref(out)) == randes.INVALID_ARGUMENT
+    assert randes.lib().randes_pairwise_cosines(None, 2, -1, None, None) == randes.INVALID_ARGUMENT
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(randes, "_lib", None)
     monkeypatch.setattr(randes, "LIB_PATH", str(tmp_path / "absent.so"))

@@ -47,7 +47,68 @@ def parse_args(argv=None):
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--check-ranks", action="store_true",
+                    help="only bring up the N ranks (nccl with GPUs, gloo without), count them and print "
+                         '{"n_gpus": N, "ranks_joined": N}: a check of the launch plumbing, no kernel runs')
+    ap.add_argument("--reference-budget-s", type=float, default=240.0,
+                    help="--impl reference: wall-clock budget of the timed steps; fewer steps are timed (and the "
+                         "line says so) when the requested number would not fit")
     return ap.parse_args(argv)
+
+
+# --------------------------------------------------------------------------------- ranks
+def rank_env(args):
+    """(rank, world, local_rank) of this process, after checking them against --gpus.
+
+    Launched by torch.distributed.run the environment carries WORLD_SIZE; it must equal --gpus.
+    Launched plainly with --gpus N > 1, bench.py starts the N ranks itself (launch_ranks)."""
+    world = os.environ.get("WORLD_SIZE")
+    if world is None:
+        if args.gpus != 1:
+            raise SystemExit("bench.py: --gpus %d needs %d ranks; none were started" % (args.gpus, args.gpus))
+        return 0, 1, 0
+    world = int(world)
+    if world != args.gpus:
+        raise SystemExit("bench.py: --gpus %d but WORLD_SIZE=%d: start one rank per GPU (or drop WORLD_SIZE and let "
+                         "bench.py start them)" % (args.gpus, world))
+    return int(os.environ.get("RANK", "0")), world, int(os.environ.get("LOCAL_RANK", "0"))
+
+
+def launch_ranks(args, argv):
+    """`python bench.py --gpus N` without a launcher: run N ranks of this script on this node through
+    torch.distributed.run (rendezvous on 127.0.0.1, a free port) and return its exit code."""
+    import socket
+
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def check_ranks(args):
+    """Bring the ranks up, count them with one all-reduce, print the count: nothing else runs."""
+    import torch
+    import torch.distributed as dist
+
+    rank, world, local = rank_env(args)
+    joined = 1
+    if world > 1:
+        if torch.cuda.is_available():
+            torch.cuda.set_device(local)
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+            t = torch.ones(1, dtype=torch.float64, device="cuda")
+        else:
+            dist.init_process_group("gloo")
+            t = torch.ones(1, dtype=torch.float64)
+        dist.all_reduce(t)
+        joined = int(t.item())
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"n_gpus": world, "ranks_joined": joined, "backend": "nccl" if torch.cuda.is_available() else "gloo",
+                          "check": "ranks only; no kernel was launched"}))
+    return 0 if joined == world else 1
 
 
 def make_workload(args) -> wl.Workload:
@@ -192,18 +253,6 @@ def config_dict(w, args, note=""):
 
 
 # --------------------------------------------------------------------------------- CPU oracle legs
-def oracle_sample(w: wl.Workload):
-    """A bounded sample of the workload for the CPU oracle: the layers of the
-    first two blocks plus the unrepeated tensors, same K, same step structure."""
-    keep, sizes = [], w.group_sizes()
-    seen = [0] * len(sizes)
-    for l, g in enumerate(w.group):
-        if sizes[g] == 1 or seen[g] < 2:
-            keep.append(l)
-            seen[g] += 1
-    return wl.subset(w, keep, w.name + ":first-2-blocks")
-
-
 def run_oracle_step(ro, ws, base, tasks, extra, n_swap):
     K = ws.n_tasks
     M = ro.compress(ws.spec, ws.storage, ws.task_ids, ws.seeds, base, tasks)
@@ -216,25 +265,38 @@ def run_oracle_step(ro, ws, base, tasks, extra, n_swap):
     return M
 
 
-def time_oracle(w: wl.Workload, n_swap: int, steps: int, warmup: int):
+def time_oracle(w: wl.Workload, n_swap: int, steps: int, warmup: int, budget_s: float, models=None):
+    """The CPU oracle, as it stands, on the WHOLE workload: `warmup` untimed steps, then up to `steps` timed ones
+    (fewer when they would not fit `budget_s` of wall clock; the result says how many ran).  `models` =
+    (base, [K + n_swap models]) as host arrays, when the caller already holds them."""
     from oracle import randes_oracle as ro
 
-    ws = oracle_sample(w)
-    K = ws.n_tasks
-    ids = list(ws.task_ids) + [K + j for j in range(n_swap)]
-    base, models = wl.model_set(ws, ids, threads=os.cpu_count() or 1)
-    tasks, extra = models[:K], models[K:]
+    K = w.n_tasks
+    if models is None:
+        ids = list(w.task_ids) + [K + j for j in range(n_swap)]
+        models = wl.model_set(w, ids, threads=os.cpu_count() or 1)
+    base, all_models = models
+    tasks, extra = all_models[:K], all_models[K:]
+    t_first = None
     for _ in range(warmup):
-        run_oracle_step(ro, ws, base, tasks, extra, n_swap)
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        run_oracle_step(ro, ws, base, tasks, extra, n_swap)
-    dt = (time.perf_counter() - t0) / max(steps, 1)
-    _, total = step_bytes(ws, n_swap)
+        t0 = time.perf_counter()
+        run_oracle_step(ro, w, base, tasks, extra, n_swap)
+        t_first = time.perf_counter() - t0
+    ran, t_sum = 0, 0.0
+    while ran < steps:
+        est = t_first if ran == 0 else t_sum / ran
+        if ran >= 1 and est is not None and t_sum + est > budget_s:
+            break
+        t0 = time.perf_counter()
+        run_oracle_step(ro, w, base, tasks, extra, n_swap)
+        t_sum += time.perf_counter() - t0
+        ran += 1
+    dt = t_sum / max(ran, 1)
+    _, total = step_bytes(w, n_swap)
     return {"value": total / dt / 1e9, "unit": "GB/s", "cores": ro.num_threads(), "kind": "oracle",
-            "sample": "%s: %d of %d layers, %.1f M of %.1f M params, K=%d, swap=%d, %.2f s per step"
-                      % (ws.name, ws.n_layers, w.n_layers, ws.n_params / 1e6, w.n_params / 1e6, K, n_swap, dt),
-            "ms_per_step": dt * 1e3}
+            "sample": "the whole workload (%s: all %d layers, %.1f M params, K=%d, swap=%d): %d warm-up + %d timed step(s), %.2f s per step"
+                      % (w.name, w.n_layers, w.n_params / 1e6, K, n_swap, warmup, ran, dt),
+            "ms_per_step": dt * 1e3, "steps_timed": ran, "warmup_run": warmup}
 
 
 def run_reference(args):
@@ -242,20 +304,102 @@ def run_reference(args):
         return 0
     w = make_workload(args)
     steps, warmup = max(1, args.steps), max(0, args.warmup)
-    steps_run, warm_run = min(steps, 30), min(warmup, 3)   # bounded: about a second per step on the sample
-    r = time_oracle(w, args.swap, steps_run, warm_run)
+    r = time_oracle(w, args.swap, steps, warmup, args.reference_budget_s)
+    note = "CPU oracle on the whole workload; %d warm-up step(s), %d of the %d requested steps timed" % (warmup, r["steps_timed"], steps)
+    if r["steps_timed"] < steps:
+        note += " (the rest would have exceeded the %.0f s budget of this arm)" % args.reference_budget_s
     line = {
         "impl": "reference", "metric": "hot_path_algorithmic_bandwidth", "value": r["value"], "unit": "GB/s",
-        "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "ms_per_step": r["ms_per_step"],
+        "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "steps_timed": r["steps_timed"], "ms_per_step": r["ms_per_step"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32" if w.storage == wl.F32 else "bf16 storage, f32 arithmetic", "data": "synthetic",
-        "config": config_dict(w, args, "CPU oracle on a bounded sample; timed %d step(s) after %d warm-up" % (steps_run, warm_run)),
+        "config": config_dict(w, args, note),
         "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
     return 0
+
+
+def check_linear_sample(c):
+    """Compare the kept block of randes_linear's output with the CPU oracle (fp64 from the definition) within the
+    tolerance of the GPU tests, sqrt(2 cols + 2) 2^-24 sum_c |x| (|W_0| + |lambda M|).  Runs in the baseline leg."""
+    import numpy as np
+
+    from oracle import randes_oracle as ro
+
+    wq = c["workload"]
+    t = wq.task_ids[c["task"]]
+    s_ = wq.seeds[c["task"]]
+    y_ref, y_abs = ro.linear(wq.spec, wq.storage, t, s_, c["lam"], c["layer"], c["x"], c["base"], c["M"], m_dtype=wl.BF16)
+    cols = wq.cols[c["layer"]]
+    tol = np.sqrt(2.0 * cols + 2.0) * 2.0 ** -24 * y_abs + 1e-30
+    err = np.abs(c["y"].astype(np.float64) - y_ref)
+    return {"checked": bool((err <= tol).all()), "checked_outputs": int(err.size), "worst_error_over_tolerance": float((err / tol).max()),
+            "check": "%d sampled token rows x all %d features against the CPU oracle" % (len(c["tokens"]), y_ref.shape[1])}
+
+
+def time_bf16_storage(w, n_swap, dev, stream, peak, peak_kind, world, barrier):
+    """compress / retrieve / add / remove of the same workload with bf16 weights (fp32 superposition and output).
+    Values are drawn on the device (seeded; the kernels have no data-dependent branches)."""
+    import torch
+
+    from paper_2505_11204_b200 import randes
+
+    wb = w.with_storage(wl.BF16)
+    K = wb.n_tasks
+    offs, total_el = [], 0
+    for r, c in zip(wb.rows, wb.cols):
+        offs.append(total_el)
+        total_el += (r * c + 63) // 64 * 64
+    views = lambda flat: [flat[o:o + r * c].view(r, c) for o, r, c in zip(offs, wb.rows, wb.cols)]
+    g = torch.Generator(device=dev).manual_seed(977)
+    base32 = torch.randn(total_el, device=dev, generator=g) * 0.02
+    shared = torch.randn(total_el, device=dev, generator=g)
+    flats = [base32.to(torch.bfloat16)]
+    for _ in range(K + 1):
+        d = wb.scale * (0.5 * shared + (0.75 ** 0.5) * torch.randn(total_el, device=dev, generator=g))
+        flats.append((base32 + d).to(torch.bfloat16))
+        del d
+    del base32, shared
+    vs = [views(f) for f in flats]
+    p_base, p_tasks, p_new = randes.ptr_array(vs[0]), randes.ptr_array(vs[1:1 + K]), randes.ptr_array(vs[1 + K])
+    plan = randes.Plan.from_workload(wb, max_tasks=K + 1, device=dev)
+    M = plan.new_superposition()
+    out = plan.new_output(wl.F32)
+    p_out = randes.ptr_array(out)
+    sh = stream.cuda_stream
+    b, _ = step_bytes(wb, n_swap)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    spans = {"compress": [], "retrieve": [], "add": [], "remove": []}
+    for rep in range(3 + 10):
+        e = [ev() for _ in range(5)]
+        e[0].record(stream)
+        randes.randes_compress(plan.handle, p_base, p_tasks, M, sh)
+        e[1].record(stream)
+        for t in wb.task_ids:
+            randes.randes_retrieve(plan.handle, t, wb.lam, wl.F32, p_base, M, p_out, sh)
+        e[2].record(stream)
+        randes.randes_add_model(plan.handle, K, wb.seeds[0] + K, p_base, p_new, M, sh)
+        e[3].record(stream)
+        randes.randes_remove_model(plan.handle, K, p_base, p_new, M, sh)
+        e[4].record(stream)
+        if rep >= 3:
+            for j, n in enumerate(("compress", "retrieve", "add", "remove")):
+                spans[n].append((e[j], e[j + 1]))
+    barrier()
+    res = {"storage": "bf16", "superposition": "f32", "output": "f32", "tasks": K, "params_M": wb.n_params / 1e6,
+           "timed": "10 rounds of compress + K retrieves + add + remove after 3 warm-up rounds"}
+    calls = {"compress": 1, "retrieve": K, "add": 1, "remove": 1}
+    for n, sp in spans.items():
+        ms = max_over_ranks([sum(a.elapsed_time(z) for a, z in sp) / (len(sp) * calls[n])], world, dev)[0]
+        gbs = b[n] / (ms * 1e-3) / 1e9
+        res[n] = {"ms_per_call": ms, "GBps": gbs, "Gparams_per_s": wb.n_params / (ms * 1e-3) / 1e9,
+                  "frac_of_%s_peak" % peak_kind: gbs / peak, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+                  "bytes_per_param": b[n] / wb.n_params}
+    plan.close()
+    return res
 
 
 # --------------------------------------------------------------------------------- GPU legs
@@ -266,9 +410,7 @@ def run_ours(args):
 
     from paper_2505_11204_b200 import build, randes
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = rank_env(args)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local)
@@ -556,6 +698,7 @@ def run_ours(args):
         except torch.OutOfMemoryError:
             extras["adapter_deltas"] = None
 
+    lin_check = None
     # ---- a linear layer on the retrieved weight, the weight never written (tensor cores): the largest
     #      repeated matrix of the set, bf16 weights and a bf16 superposition, 8192 tokens, timed alone
     try:
@@ -580,6 +723,13 @@ def run_ours(args):
         for _ in range(3):
             randes.randes_linear(plan_lin.handle, 0, w.lam, 0, x_lin, n_tok, pb_lin, M_lin, y_lin, sh)
         barrier()
+        # a sampled block of this output (both 128-token halves of the first and the last block of tokens, every
+        # feature) is kept, with the operands, for the comparison with the CPU oracle in the baseline leg
+        tok = sorted(set(t for t in (0, 1, 127, 128, 129, 255, n_tok // 2, n_tok - 256, n_tok - 129, n_tok - 128, n_tok - 1) if 0 <= t < n_tok))
+        u16 = lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16)
+        lin_check = {"workload": wl_lin, "task": 0, "layer": 0, "lam": w.lam, "tokens": tok,
+                     "x": u16(x_lin[tok].contiguous()), "y": y_lin[tok].cpu().numpy(), "base": [u16(b) for b in lin_base],
+                     "M": [u16(plan_lin.slot(M_lin, l)) for l in range(wl_lin.n_layers)]}
         a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         reps = 20
         a.record(stream)
@@ -597,7 +747,7 @@ def run_ours(args):
         extras["linear"] = {"layer_shape": [rows_l, cols_l], "tokens": n_tok, "ms_per_call": ms, "TFLOPs": flops / (ms * 1e-3) / 1e12,
                             "bound": "tensor", "peak_TFLOPs": tc_peak, "peak_source": "%s bf16 GEMM (MEASURED_PEAKS.json)" % tc_kind
                             if tc_kind != "fallback" else "fallback bf16 GEMM",
-                            "frac": flops / (ms * 1e-3) / 1e12 / tc_peak, "giveups": randes.randes_linear_giveups(),
+                            "frac": flops / (ms * 1e-3) / 1e12 / tc_peak, "giveups": randes.randes_linear_giveups(), "checked": None,
                             "note": "y = x W_0^T + lambda (x D) M^T, bf16 operands, fp32 accumulators; flops count both products"}
         plan_lin.close()
         del lin_base, lin_tasks, M_lin, x_lin, y_lin
@@ -675,15 +825,37 @@ def run_ours(args):
                "h2d_bytes_per_step": (1 + K + n_swap) * w.n_params * s_b,
                "d2h_bytes_per_step": (K + 1) * w.n_params * 4, "steps": args.e2e_steps,
                "note": "copies and kernels pipelined over three streams; PCIe-bound"}
-        del h_out, h_M, h_flat, sets, o_flat
+        del h_out, h_M, sets, o_flat
 
     plan.close()
+    del d_models, d_base, M, dset
+    torch.cuda.empty_cache()
+
+    # ---- the same workload with the weights stored as bf16 (fp32 superposition, fp32 output), timed alone
+    if w.storage == wl.F32 and args.workload != "toy":
+        try:
+            extras["bf16_storage"] = time_bf16_storage(w, n_swap, dev, stream, peak, peak_kind, world, barrier)
+        except torch.OutOfMemoryError:
+            extras["bf16_storage"] = None
+        torch.cuda.empty_cache()
+
+    # ---- the CPU oracle beside it: the whole workload, one warm-up step and two timed ones (rank 0, one GPU only);
+    #      the sampled block of the linear layer's output is compared with the oracle here as well
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        del d_models, d_base, M, dset
-        torch.cuda.empty_cache()
-        cpu = time_oracle(w, n_swap, 5, 1)
+        host_models = None
+        if want_e2e:
+            def layers_np(flat):
+                vs = views(flat)
+                return [v.view(torch.int16).numpy().view(np.uint16) if v.dtype == torch.bfloat16 else v.numpy() for v in vs]
+            host_models = (layers_np(h_flat[0]), [layers_np(f) for f in h_flat[1:]])
+        cpu = time_oracle(w, n_swap, 2, 1, 120.0, models=host_models)
         cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        del host_models
+        if lin_check is not None and extras.get("linear"):
+            extras["linear"].update(check_linear_sample(lin_check))
+    if want_e2e:
+        del h_flat
 
     if rank == 0:
         line = {
@@ -706,9 +878,18 @@ def run_ours(args):
     return 0
 
 
-def main():
-    args = parse_args()
-    return run_reference(args) if args.impl == "reference" else run_ours(args)
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else list(argv)
+    args = parse_args(argv)
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be at least 1")
+    if args.impl == "reference":
+        return run_reference(args)       # rank 0 alone works, whatever started it
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return launch_ranks(args, argv)
+    if args.check_ranks:
+        return check_ranks(args)
+    return run_ours(args)
 
 
 if __name__ == "__main__":

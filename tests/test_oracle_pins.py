@@ -731,6 +731,27 @@ def test_linear_on_bf16_inputs_and_superposition_stays_close_to_the_retrieved_we
         assert np.abs(y_wrong - y).max() > 2.0 ** -14 * y_abs.max()
 
 
+@pytest.mark.parametrize("cols", [1024, 4096])
+def test_linear_tolerance_of_the_gpu_test_sees_one_wrong_column_at_wide_layers(cols):
+    """The GPU comparison accepts sqrt(2 cols + 2) 2^-24 y_abs.  With weights and a superposition of the
+    magnitudes of the synthetic sets (W_0 ~ 0.02, M ~ 0.002, lambda = 0.3) one column of M with the wrong sign
+    must move some output beyond that at the widths of the paper-shaped layers; the old worst-case bound
+    (2 cols + 2) 2^-24 y_abs would not have seen it."""
+    rng = np.random.default_rng(cols)
+    spec = ([24], [cols], [0], [FLIP])
+    base = [wl.to_bf16_bits((rng.standard_normal((24, cols)) * 0.02).astype(np.float32))]
+    M = [wl.to_bf16_bits((rng.standard_normal((24, cols)) * 0.002).astype(np.float32))]
+    x = wl.to_bf16_bits(rng.standard_normal((64, cols)).astype(np.float32))
+    lam, t, s = 0.3, 1, 43
+    y, y_abs = ro.linear(spec, ro.BF16, t, s, lam, 0, x, base, M, m_dtype=ro.BF16)
+    Mw = [M[0].copy()]
+    Mw[0][:, cols // 3] ^= 0x8000
+    y_wrong, _ = ro.linear(spec, ro.BF16, t, s, lam, 0, x, base, Mw, m_dtype=ro.BF16)
+    tol = np.sqrt(2.0 * cols + 2.0) * 2.0 ** -24 * y_abs
+    assert (np.abs(y_wrong - y) > tol).mean() > 0.5          # most outputs, not just the tail
+    assert (np.abs(y_wrong - y) > (2 * cols + 2) * 2.0 ** -24 * y_abs).mean() < 0.5   # the worst-case bound misses most
+
+
 # --------------------------------------------------------------------------- Gaussian-like diagonal context ("RD", Section 5.5)
 def test_gauss_entries_replay_the_stated_recipe_and_have_unit_variance():
     """Entry (task, slot, column) = sum of twelve uniforms minus six, uniforms = top 24 bits of the words of

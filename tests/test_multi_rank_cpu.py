@@ -122,3 +122,79 @@ def test_row_slices_of_every_layer_are_independent_problems():
         outs = ro.retrieve(ws.spec, ws.storage, wl.F32, 1, ws.seeds[1], 0.3, cut(base), Ms)
         for l, (lo, hi) in enumerate(bounds):
             assert np.array_equal(Ms[l], M[l][lo:hi]) and np.array_equal(outs[l], out[l][lo:hi])
+
+
+def _bench(*argv, env=None, timeout=240):
+    import subprocess
+
+    e = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    e.update(env or {})
+    return subprocess.run([sys.executable, os.path.join(ROOT, "bench.py")] + list(argv), capture_output=True, text=True,
+                          env=e, timeout=timeout)
+
+
+def test_gpus_flag_starts_its_own_ranks_and_counts_them():
+    """`python bench.py --gpus 2` without a launcher starts two ranks itself; --check-ranks stops after the
+    rendezvous (gloo here, where there is no GPU), so the launcher can be checked without a kernel."""
+    import json
+
+    r = _bench("--gpus", "2", "--check-ranks")
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["ranks_joined"] == 2
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the refusal on a machine without a GPU")
+def test_gpus_flag_never_falls_back_to_one_silent_rank():
+    """On a machine without GPUs the two ranks refuse to run (no CPU fallback) and the launcher passes the failure
+    on: what must not happen is a line that reports n_gpus 1."""
+    r = _bench("--gpus", "2", "--steps", "1", "--no-e2e", "--no-cpu-baseline")
+    assert r.returncode != 0
+    assert "needs a CUDA device" in r.stderr
+    assert '"n_gpus"' not in r.stdout
+
+
+def test_world_size_that_contradicts_gpus_is_an_error():
+    import bench
+
+    args = bench.parse_args(["--gpus", "4"])
+    old = {k: os.environ.get(k) for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    try:
+        os.environ.update(WORLD_SIZE="2", RANK="1", LOCAL_RANK="1")
+        with pytest.raises(SystemExit) as e:
+            bench.rank_env(args)
+        assert "WORLD_SIZE=2" in str(e.value)
+        os.environ["WORLD_SIZE"] = "4"
+        assert bench.rank_env(args) == (1, 4, 1)
+        del os.environ["WORLD_SIZE"]
+        with pytest.raises(SystemExit):
+            bench.rank_env(args)                      # --gpus 4 and nobody started ranks
+        assert bench.rank_env(bench.parse_args([])) == (0, 1, 0)
+    finally:
+        for k, v in old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+
+
+def test_reference_arm_times_the_whole_workload_with_the_requested_steps():
+    """--impl reference: the oracle on every layer of the workload, the warm-up and step counts that were asked
+    for (fewer timed steps only when the budget runs out, and then the line says so)."""
+    import json
+
+    r = _bench("--impl", "reference", "--workload", "toy", "--steps", "3", "--warmup", "2", "--gpus", "2",
+               env={"RANK": "0", "WORLD_SIZE": "2"})
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["steps"] == 3 and line["warmup"] == 2 and line["steps_timed"] == 3
+    assert line["n_gpus"] == 2 and line["cpu_baseline"]["kind"] == "oracle"
+    assert "all 12 layers" in line["cpu_baseline"]["sample"] and "2 warm-up + 3 timed" in line["cpu_baseline"]["sample"]
+    assert line["e2e"]["value"] == line["value"] and line["e2e"]["h2d_bytes_per_step"] == 0
+    # the other ranks of the same launch do no work and print nothing
+    r1 = _bench("--impl", "reference", "--workload", "toy", "--gpus", "2", env={"RANK": "1", "WORLD_SIZE": "2"})
+    assert r1.returncode == 0 and r1.stdout.strip() == ""
+    # a budget too small for the request: one step is still timed, and the note says what happened
+    r2 = _bench("--impl", "reference", "--workload", "toy", "--steps", "50", "--warmup", "1", "--reference-budget-s", "0")
+    line2 = json.loads(r2.stdout.strip().splitlines()[-1])
+    assert line2["steps"] == 50 and 1 <= line2["steps_timed"] < 50 and "budget" in line2["config"]["note"]

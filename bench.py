@@ -46,7 +46,7 @@ def parse_args(argv=None):
                          "one row slice of every layer (strong scaling); neither needs a collective on the data path")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--check-ranks", action="store_true",
                     help="only bring up the N ranks (nccl with GPUs, gloo without), count them and print "
                          '{"n_gpus": N, "ranks_joined": N}: a check of the launch plumbing, no kernel runs')

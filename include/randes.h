@@ -32,8 +32,8 @@
  * - M is one arena of randes_superposition_bytes() bytes, 256-byte aligned;
  *   slot l starts at byte randes_layer_offset(plan, l).  Its element type is
  *   the plan's m_dtype: fp32 by default whatever the storage type of the
- *   weights, or bf16 (half the footprint; the "further compression" the
- *   paper's conclusion leaves open).  Sums always run in fp32: with a bf16 M,
+ *   weights, or bf16 (half the footprint; a smaller superposition is what
+ *   the paper's conclusion leaves to future work).  Sums always run in fp32: with a bf16 M,
  *   compress rounds each element once at the end (nearest even), add / remove
  *   widen the stored element, add in fp32 and round again, retrieve widens.
  * - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
@@ -352,14 +352,14 @@ int randes_pairwise_cosines(const double* gram, uint32_t n, int32_t exclude, dou
  * dev_workspace == NULL (host-only) and calls this instead of randes_retrieve.
  *
  * Same arguments, results and errors as randes_retrieve (bit-identical output);
- * `plan` may be host-only.  The tables the kernel reads are copied, on
- * `stream`, into a fixed array of RANDES_STATIC_SCRATCH_BYTES that lives inside
+ * `plan` may be host-only.  The tables the kernel reads are copied, in
+ * one transfer on `stream`, into a fixed array of RANDES_STATIC_SCRATCH_BYTES that lives inside
  * the library on every GPU that loads it, for the life of the process.  The
  * call allocates no device memory and frees none.
- *   - Limit: 72 bytes per layer plus 16 bytes per tile of 16 rows x 1024 fp32
- *     (2048 bf16) columns, rounded up, must fit the array (models up to roughly
- *     a billion parameters); larger plans fail with RANDES_CAPACITY before
- *     anything is launched.
+ *   - Limit: 52 bytes per layer plus 16 bytes per tile of 16 rows x 1024 fp32
+ *     (2048 bf16) columns, each of the five tables rounded up to 256 bytes,
+ *     must fit the array (models up to roughly a billion parameters); larger
+ *     plans fail with RANDES_CAPACITY before anything is launched.
  *   - The first call on each device looks up the array's device address and
  *     sizes the grid; make that first call outside any stream capture.
  *   - All calls on one device share the array.  Calls on one stream are ordered

@@ -23,8 +23,8 @@
  *     is indexed by the position ("slot") the layer lands on in M.
  *   - Shuffle is the gather the paper prints: slot k receives member sigma(k).
  *   - lambda is applied at retrieval; M is kept in fp32 by default, whatever the
- *     storage type of the weights.  With m_dtype = bf16 (the "further
- *     compression of the superposed delta" the conclusion leaves to future work)
+ *     storage type of the weights.  With m_dtype = bf16 (a smaller superposition,
+ *     which the conclusion names as future work without fixing a format)
  *     compress sums in fp32 and rounds each element once at the end; add and
  *     remove widen the stored element, add in fp32 and round again; retrieve
  *     widens it.
@@ -37,8 +37,8 @@
  *     of the members of a group, in layer order, those with index 0, k, 2k, ...
  *     take part in the shuffle (among themselves) and in the flip; the others
  *     are left as they are.
- *   - Layer shifting (same appendix): "one position deeper with wrap-around"
- *     is read as a rotation of the participating members towards higher block
+ *   - Layer shifting (same appendix: a deterministic move of every layer
+ *     to the next depth, the last wrapping to the first) is read as a rotation of the participating members towards higher block
  *     index; task t rotates by 1 + (t mod (n - 1)) positions (n participants),
  *     so that different tasks are misaligned and no task gets the identity.
  *     Slot k then receives member (k - shift) mod n.

@@ -20,7 +20,9 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "randes_device.cuh"
 #include "randes_internal.h"
@@ -690,7 +692,10 @@ namespace {
 constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 unsigned char* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device
-int g_static_grid[kMaxDevices][2][2] = {};       // persistent grid size [storage][out dtype], per device
+int g_static_grid[kMaxDevices][2][2][2] = {};    // persistent grid size [storage][out dtype][M dtype], per device
+// Host image of the tables of the call being enqueued, one per device, kept for the life of the library:
+// the five tables are laid out here and reach the device array in ONE copy.
+std::vector<unsigned char> g_static_host[kMaxDevices];
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 }  // namespace
 
@@ -704,19 +709,20 @@ int launch_retrieve_static(int storage_dtype, int out_dtype, int m_dtype, const 
                            uint32_t n_units, const uint32_t* slot_of_pos, const void* const* base, void* const* out,
                            const void* M, const DevTask& task, float lambda, void* stream)
 {
-    if (retrieve_static_bytes(n_layers, n_units) > kStaticScratchBytes) return -1;
+    const size_t need = retrieve_static_bytes(n_layers, n_units);
+    if (need > kStaticScratchBytes) return -1;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return static_cast<int>(e);
     if (dev < 0 || dev >= kMaxDevices) return static_cast<int>(cudaErrorInvalidDevice);
-    unsigned char* scratch = nullptr;
+    RetrieveArgs a;
     int grid = 0;
     {
-        // once per device, with that device current: the array's name is only a host-side
-        // handle here; the kernel needs the address the symbol has on this device
         std::lock_guard<std::mutex> lock(g_static_mutex);
         if (!g_static_ptr[dev]) {
+            // once per device, with that device current: the array's name is only a host-side
+            // handle here; the kernel needs the address the symbol has on this device
             void* p = nullptr;
             e = cudaGetSymbolAddress(&p, g_static_scratch);
             if (e != cudaSuccess) return static_cast<int>(e);
@@ -724,30 +730,35 @@ int launch_retrieve_static(int storage_dtype, int out_dtype, int m_dtype, const 
             e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
             if (e != cudaSuccess) return static_cast<int>(e);
             for (int st = 0; st < 2; ++st)
-                for (int od = 0; od < 2; ++od) {
-                    const int occ = retrieve_ctas_per_sm(st, od, 0);
-                    if (occ <= 0) return static_cast<int>(cudaErrorInvalidDeviceFunction);
-                    g_static_grid[dev][st][od] = sms * occ;
-                }
+                for (int od = 0; od < 2; ++od)
+                    for (int md = 0; md < 2; ++md) {
+                        const int occ = retrieve_ctas_per_sm(st, od, md);
+                        if (occ <= 0) return static_cast<int>(cudaErrorInvalidDeviceFunction);
+                        g_static_grid[dev][st][od][md] = sms * occ;
+                    }
+            g_static_host[dev].resize(kStaticScratchBytes);
             g_static_ptr[dev] = static_cast<unsigned char*>(p);
         }
-        scratch = g_static_ptr[dev];
-        grid = g_static_grid[dev][storage_dtype][out_dtype];
+        unsigned char* scratch = g_static_ptr[dev];
+        unsigned char* image = g_static_host[dev].data();
+        grid = g_static_grid[dev][storage_dtype][out_dtype][m_dtype];
+        size_t off = 0;
+        auto put = [&](const void* src, size_t bytes) -> unsigned char* {
+            unsigned char* dst = scratch + off;
+            if (bytes) std::memcpy(image + off, src, bytes);
+            off += align256(bytes);
+            return dst;
+        };
+        a.layers = reinterpret_cast<const DevLayer*>(put(layers, n_layers * sizeof(DevLayer)));
+        a.units = reinterpret_cast<const DevUnit*>(put(units, n_units * sizeof(DevUnit)));
+        a.slot_of_pos = reinterpret_cast<const uint32_t*>(put(slot_of_pos, n_layers * sizeof(uint32_t)));
+        a.base = reinterpret_cast<const void* const*>(put(base, n_layers * sizeof(void*)));
+        a.out = reinterpret_cast<void* const*>(put(out, n_layers * sizeof(void*)));
+        // one copy for all five tables; the image is ordinary host memory, so the call returns once the
+        // driver has taken its contents, and the next call may overwrite it
+        if (off) e = cudaMemcpyAsync(scratch, image, off, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return static_cast<int>(e);
     }
-    size_t off = 0;
-    auto put = [&](const void* src, size_t bytes) -> unsigned char* {
-        unsigned char* dst = scratch + off;
-        off += align256(bytes);
-        if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s);
-        return dst;
-    };
-    RetrieveArgs a;
-    a.layers = reinterpret_cast<const DevLayer*>(put(layers, n_layers * sizeof(DevLayer)));
-    a.units = reinterpret_cast<const DevUnit*>(put(units, n_units * sizeof(DevUnit)));
-    a.slot_of_pos = reinterpret_cast<const uint32_t*>(put(slot_of_pos, n_layers * sizeof(uint32_t)));
-    a.base = reinterpret_cast<const void* const*>(put(base, n_layers * sizeof(void*)));
-    a.out = reinterpret_cast<void* const*>(put(out, n_layers * sizeof(void*)));
-    if (e != cudaSuccess) return static_cast<int>(e);
     a.n_units = n_units;
     a.n_layers = n_layers;
     a.M = M;

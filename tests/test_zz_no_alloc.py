@@ -6,15 +6,21 @@ host framework, or a handler that swaps models in a latency-critical loop where
 cudaMalloc would stall the device.  For them the library keeps the retrieve
 kernel's tables in a fixed device array of its own, so the call needs no
 workspace.  This file checks, through the C ABI, that the variant returns
-exactly what the ordinary entry point returns, on two calls in a row (the
-second call reuses the array the first one filled), and that a model too large
-for the array is refused cleanly.  It is collected last on purpose.
+exactly what the ordinary entry point returns -- and what the CPU oracle
+computes -- on two calls in a row (the second call reuses the array the first
+one filled), that the device's free memory does not shrink across a call, that
+the library's sources name no device allocator at all, and that a model too
+large for the array is refused cleanly.  It is collected last on purpose.
 """
 import ctypes
+import glob
+import os
+import re
 
 import numpy as np
 import pytest
 
+from oracle import randes_oracle as ro
 from paper_2505_11204_b200 import build, randes, workloads as wl
 
 from gpu_util import assert_bits_equal, from_dev, model_to_dev, poison
@@ -51,18 +57,26 @@ def test_static_retrieve_matches_retrieve_on_two_calls_in_a_row(storage):
     plan = randes.Plan.from_workload(w)                      # ordinary plan, with a workspace
     host_plan = randes.Plan.from_workload(w, host_only=True)  # what a caller without an allocator builds
     M = plan.compress(d_base, d_tasks)
+    M_ref = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, base, tasks)
     p_base = randes.ptr_array(d_base)
     stream = torch.cuda.current_stream().cuda_stream
+    calls = 0
     for out_dtype in (wl.F32, wl.BF16):
         for task in (2, 0):                                   # two calls in a row, different permutations and signs
             want = plan.retrieve(task, w.lam, d_base, M, out_dtype=out_dtype)
+            ref = ro.retrieve(w.spec, w.storage, out_dtype, task, w.seeds[task], w.lam, base, M_ref)
             got = [poison(o) for o in plan.new_output(out_dtype)]
-            before = torch.cuda.memory_allocated()
-            randes.randes_retrieve_static(host_plan.handle, task, w.lam, out_dtype, p_base, M, randes.ptr_array(got), stream)
-            assert torch.cuda.memory_allocated() == before
+            p_got = randes.ptr_array(got)
             torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]       # the device's own count, not torch's allocator
+            randes.randes_retrieve_static(host_plan.handle, task, w.lam, out_dtype, p_base, M, p_got, stream)
+            torch.cuda.synchronize()
+            calls += 1
+            if calls > 1:                                     # the first call on a device may load the module with its array
+                assert torch.cuda.mem_get_info()[0] >= free_before
             for l in range(w.n_layers):
                 assert_bits_equal(from_dev(got[l]), from_dev(want[l]), "static retrieve task %d layer %d" % (task, l))
+                assert_bits_equal(from_dev(got[l]), ref[l], "static retrieve against the oracle, task %d layer %d" % (task, l))
     # the ordinary plan's handle works too, and argument checks are the same
     got = plan.new_output(wl.F32)
     randes.randes_retrieve_static(plan.handle, 1, w.lam, wl.F32, p_base, M, randes.ptr_array(got), stream)
@@ -74,6 +88,18 @@ def test_static_retrieve_matches_retrieve_on_two_calls_in_a_row(storage):
     assert e.value.code == randes.UNKNOWN_TASK
     plan.close()
     host_plan.close()
+
+
+def test_library_sources_name_no_device_allocator():
+    """No entry point of the library may allocate or free device memory (callers own every buffer): the CUDA
+    sources must not even name the runtime's or the driver's allocation routines."""
+    here = os.path.dirname(os.path.abspath(build.__file__))
+    banned = re.compile(r"\b(cudaMalloc\w*|cudaFree\w*|cudaHostAlloc|cuMemAlloc\w*|cuMemFree\w*|cuMemCreate|cudaMemPool\w*)\b")
+    sources = sorted(glob.glob(os.path.join(here, "csrc", "*")))
+    assert len(sources) >= 8
+    for path in sources:
+        hits = banned.findall(open(path).read())
+        assert not hits, (os.path.basename(path), hits)
 
 
 def test_static_retrieve_refuses_models_beyond_its_scratch():

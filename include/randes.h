@@ -270,6 +270,23 @@ int randes_linear(const randes_plan_t* plan, uint32_t task_id, float lambda, uin
                   uint32_t n_tokens, const void* const* base, const void* M, void* y, randes_dtype_t y_dtype, void* stream);
 
 /*
+ * randes_linear behind a gate (same computation: Section 4, second display, inside y = x What^T).
+ * Every thread block first waits until the 32-bit word *gate in device memory is non-zero --
+ * written, for instance, by the kernel on another stream that produces x -- and only then reads
+ * its operands.  The wait, like every other wait inside the kernel, ends after wait_ns nanoseconds
+ * of the block's life (0 = the default of one second, at most 60 s): a block whose wait runs out
+ * issues no copy and no product, writes nothing to y, frees what it holds, returns, and is counted
+ * by randes_linear_giveups; the call itself still returns RANDES_OK (it only enqueues), so a caller
+ * that uses a gate reads the counter afterwards.  The context stays usable.
+ *   gate      device, 4-byte aligned, not NULL; whoever writes it must make x visible first
+ *             (a release store or a fence before the store)
+ * Errors: those of randes_linear, plus INVALID_ARGUMENT (gate NULL, wait_ns beyond 60 s).
+ */
+int randes_linear_gated(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x,
+                        uint32_t n_tokens, const void* const* base, const void* M, void* y, randes_dtype_t y_dtype,
+                        const uint32_t* gate, uint64_t wait_ns, void* stream);
+
+/*
  * Every wait inside the randes_linear kernel is bounded; a thread block whose wait runs out
  * skips its tile and counts itself here.  *count = number of such blocks since the library was
  * loaded on the current device (0 in a healthy run).  Synchronises with the device.

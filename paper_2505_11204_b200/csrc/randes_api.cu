@@ -1130,7 +1130,8 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_
 }
 
 static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x,
-                              uint32_t n_tokens, const void* const* base, const void* M, void* y, randes_dtype_t y_dtype, void* stream)
+                              uint32_t n_tokens, const void* const* base, const void* M, void* y, randes_dtype_t y_dtype,
+                              const uint32_t* gate, uint64_t wait_ns, void* stream)
 {
     if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
     if (plan->has_gauss) return fail(RANDES_INVALID_ARGUMENT, "not offered for plans with a RANDES_GAUSS group");
@@ -1151,6 +1152,8 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
     if (reinterpret_cast<uintptr_t>(x) % 16 || reinterpret_cast<uintptr_t>(base[layer]) % 16)
         return fail(RANDES_MISALIGNED, "x and base[%u] must be 16-byte aligned", layer);
     if (reinterpret_cast<uintptr_t>(y) % elem_size(y_dtype)) return fail(RANDES_MISALIGNED, "y = %p is not aligned to its element size", y);
+    if (reinterpret_cast<uintptr_t>(gate) % 4) return fail(RANDES_MISALIGNED, "gate = %p is not 4-byte aligned", (const void*)gate);
+    if (wait_ns > 60ull * 1000000000ull) return fail(RANDES_INVALID_ARGUMENT, "wait_ns = %llu exceeds the supported 60 s", (unsigned long long)wait_ns);
     const TaskEntry& t = plan->tasks[row];
     const uint32_t slot = t.slot_of_pos[layer];                    // sigma_t^-1(p)
     const bool flip = (plan->dev_layers[slot].flags & kFlagFlip) != 0;
@@ -1162,7 +1165,7 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
     int e = linear_prepare();
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "set-up of the linear kernel");
     e = launch_linear(x, n_tokens, base[layer], static_cast<const char*>(M) + plan->m_off_bytes[slot], rows, cols, flip, slot, d, lambda,
-                      y, y_dtype == RANDES_BF16, stream);
+                      y, y_dtype == RANDES_BF16, gate, wait_ns, stream);
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the linear kernel");
     ++g_launches;
     return RANDES_OK;
@@ -1171,7 +1174,15 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
 int randes_linear(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x, uint32_t n_tokens,
                   const void* const* base, const void* M, void* y, randes_dtype_t y_dtype, void* stream)
 {
-    return guarded([&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, y_dtype, stream); });
+    return guarded([&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, y_dtype, nullptr, 0, stream); });
+}
+
+int randes_linear_gated(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x, uint32_t n_tokens,
+                        const void* const* base, const void* M, void* y, randes_dtype_t y_dtype, const uint32_t* gate,
+                        uint64_t wait_ns, void* stream)
+{
+    if (!gate) return fail(RANDES_INVALID_ARGUMENT, "gate is NULL (use randes_linear for a call without a gate)");
+    return guarded([&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, y_dtype, gate, wait_ns, stream); });
 }
 
 int randes_linear_giveups(unsigned int* count)

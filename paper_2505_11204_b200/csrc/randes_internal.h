@@ -185,7 +185,8 @@ int launch_retrieve_batch_groups(int out_dtype, const RetrieveBatchArgs& a, uint
 // All return a cudaError_t as int.
 int linear_prepare();   // opts the kernel into its shared memory on the current device
 int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* m_slot, uint32_t rows, uint32_t cols, bool flip,
-                  uint32_t slot, const DevTask& task, float lambda, void* y, bool y_bf16, void* stream);
+                  uint32_t slot, const DevTask& task, float lambda, void* y, bool y_bf16, const uint32_t* gate,
+                  unsigned long long wait_ns, void* stream);   // gate: NULL or a device word to wait on; wait_ns: 0 = one second
 int linear_giveups(unsigned int* count);   // CTAs that gave up on a bounded wait since the library was loaded (synchronises)
 
 // Retrieve with its tables in a fixed device array inside the library (no workspace).

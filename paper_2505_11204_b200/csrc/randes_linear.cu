@@ -20,8 +20,12 @@
 //   * the epilogue reads the accumulators with tcgen05.ld and stores fma(lambda, acc1, acc0).
 //
 // lambda stays in fp32 and is applied once per output, so the operands keep their stored bits.
-// Every wait on an mbarrier is bounded: a CTA that gives up raises a shared flag, every role
-// leaves its loop, tensor memory is freed, and a device counter records the event.
+// Every wait is bounded in time (the global nanosecond timer; one second unless the caller gives
+// another limit): a CTA whose wait runs out raises a shared flag, every role leaves its loop,
+// copies already issued are waited for, tensor memory is freed, nothing is written to y, and a
+// device counter records the event.  The gated form of the call makes every CTA wait first for a
+// word in device memory to become non-zero; a gate that nothing opens is the one wait of this
+// kernel that can run out in a healthy program.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -45,7 +49,8 @@ constexpr int kBK = 64;           // bf16 columns per stage: one 128-byte swizzl
 constexpr int kTileBytes = kBM * kBK * 2;                    // 16 KiB, also for the kBN x kBK tiles
 constexpr int kLinearThreads = 192;                          // warp 0 TMA, warp 1 MMA, warps 2-5 flip + epilogue
 constexpr int kFlipThreads = 128;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 22;                    // iteration cap of the clean-up waits after a give-up
+constexpr unsigned long long kDefaultWaitNs = 1000000000ull; // one second
 constexpr int kMaxStages = 4;
 
 // HALVES = blocks of 128 tokens per CTA (1 or 2)
@@ -64,6 +69,8 @@ struct LinearArgs {
     DevTask task;
     void* y;                       // [n_tokens, rows], fp32 or bf16
     uint32_t y_bf16;
+    const uint32_t* gate;          // NULL, or a device word the CTA waits on (non-zero = go) before its first copy
+    unsigned long long wait_ns;    // limit of every wait of a CTA, measured from its start
 };
 
 // ---- mbarrier, TMA, tcgen05 wrappers --------------------------------------------------------
@@ -91,14 +98,45 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the CTA has given up (here or in another role).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag)
+__device__ __forceinline__ unsigned long long global_ns()
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u && *abort_flag) return false;
-    }
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// The CTA gives up: the first thread to say so counts it.
+__device__ __forceinline__ void give_up(volatile uint32_t* abort_flag)
+{
     if (atomicExch(const_cast<uint32_t*>(abort_flag), 1u) == 0u) atomicAdd(&g_linear_giveups, 1u);
+}
+// Wait bounded by `deadline` (global timer, ns).  Returns false when the CTA has given up (here or in another role).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, unsigned long long deadline)
+{
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (global_ns() > deadline) break;
+        }
+    }
+    give_up(abort_flag);
+    return false;
+}
+// Wait, bounded likewise, for a word in device memory to become non-zero.
+__device__ __forceinline__ bool gate_wait(const uint32_t* gate, volatile uint32_t* abort_flag, unsigned long long deadline)
+{
+    for (;;) {
+        uint32_t v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(gate) : "memory");
+        if (v) {
+            asm volatile("fence.proxy.async.global;" ::: "memory");   // what the gate's writer stored is read by TMA next
+            return true;
+        }
+        if (*abort_flag) return false;
+        if (global_ns() > deadline) break;
+        __nanosleep(200);
+    }
+    give_up(abort_flag);
     return false;
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1)
@@ -196,15 +234,17 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_ptr;
+    const unsigned long long deadline = global_ns() + a.wait_ns;
 
     if (warp == 0) {
         // ---- TMA producer
         if (lane == 0) {
             uint32_t issued = 0;
-            for (uint32_t kk = 0; kk < n_k; ++kk) {
+            const bool open = a.gate == nullptr || gate_wait(a.gate, abort_flag, deadline);
+            for (uint32_t kk = 0; open && kk < n_k; ++kk) {
                 const int s = kk % kStages;
                 const uint32_t ph = (kk / kStages) & 1u;
-                if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag)) break;
+                if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, deadline)) break;
                 const uint32_t st = smem_base + s * kStageBytes;
                 mbar_expect_tx(bar_full(s), kStageBytes);
                 tma_load_2d(st, &map_x, bar_full(s), kk * kBK, m0);             // HALVES x 128 tokens in one box
@@ -226,11 +266,11 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
             for (uint32_t kk = 0; kk < n_k && ok; ++kk) {
                 const int s = kk % kStages;
                 const uint32_t ph = (kk / kStages) & 1u;
-                ok = mbar_wait(bar_full(s), ph, abort_flag);
+                ok = mbar_wait(bar_full(s), ph, abort_flag, deadline);
                 if (!ok) break;
                 tc_fence_after();
                 if (a.flip) {
-                    ok = mbar_wait(bar_flipped(s), ph, abort_flag);
+                    ok = mbar_wait(bar_flipped(s), ph, abort_flag, deadline);
                     if (!ok) break;
                     tc_fence_after();
                 }
@@ -272,7 +312,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 uint32_t mask[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) mask[j] = (((bits >> (2 * j)) & 1u) << 15) | (((bits >> (2 * j + 1)) & 1u) << 31);
-                ok = mbar_wait(bar_full(s), ph, abort_flag);
+                ok = mbar_wait(bar_full(s), ph, abort_flag, deadline);
                 if (!ok) break;
                 const uint32_t tile = smem_base + s * kStageBytes + kOffM + t * 16;
                 uint4 v[kTileBytes / (16 * kFlipThreads)];
@@ -287,7 +327,8 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
                 mbar_arrive(bar_flipped(s));
             }
         }
-        if (ok) ok = mbar_wait(bar_acc, 0, abort_flag);
+        if (ok) ok = mbar_wait(bar_acc, 0, abort_flag, deadline);
+        if (ok && *abort_flag) ok = false;   // the issuer also arrives on this barrier when it gives up: nothing to store then
         if (ok) {
             // The accumulators hold one token per tensor-memory lane, i.e. per thread; stored like that, a warp's
             // store would touch 32 rows of y at once.  Each warp therefore turns its [32 tokens x 128 features]
@@ -405,7 +446,8 @@ int linear_prepare()
 }
 
 int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* m_slot, uint32_t rows, uint32_t cols, bool flip,
-                  uint32_t slot, const DevTask& task, float lambda, void* y, bool y_bf16, void* stream)
+                  uint32_t slot, const DevTask& task, float lambda, void* y, bool y_bf16, const uint32_t* gate,
+                  unsigned long long wait_ns, void* stream)
 {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return static_cast<int>(cudaErrorNotSupported);
@@ -429,6 +471,8 @@ int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* 
     a.task = task;
     a.y = y;
     a.y_bf16 = y_bf16 ? 1u : 0u;
+    a.gate = gate;
+    a.wait_ns = wait_ns ? wait_ns : kDefaultWaitNs;
     const dim3 grid((rows + kBN - 1) / kBN, (n_tokens + halves * kBM - 1) / (halves * kBM));
     if (halves == 1) linear_kernel<1><<<grid, kLinearThreads, LinearGeom<1>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
     else linear_kernel<2><<<grid, kLinearThreads, LinearGeom<2>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);

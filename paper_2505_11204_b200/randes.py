@@ -117,6 +117,8 @@ def lib():
         L.randes_retrieve_static.restype = ctypes.c_int
         L.randes_linear.argtypes = [vp, u32, ctypes.c_float, u32, vp, u32, vp, vp, vp, ctypes.c_int, vp]
         L.randes_linear.restype = ctypes.c_int
+        L.randes_linear_gated.argtypes = [vp, u32, ctypes.c_float, u32, vp, u32, vp, vp, vp, ctypes.c_int, vp, u64, vp]
+        L.randes_linear_gated.restype = ctypes.c_int
         L.randes_linear_giveups.argtypes = [ctypes.POINTER(ctypes.c_uint)]
         L.randes_linear_giveups.restype = ctypes.c_int
         L.randes_launch_count.argtypes = []
@@ -131,7 +133,7 @@ EXPORTS = [
     "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
     "randes_task_tables", "randes_plan_serialize", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_add_models", "randes_remove_model",
-    "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_interference_norm", "randes_pairwise_cosines", "randes_retrieve_batch", "randes_retrieve_static", "randes_linear", "randes_linear_giveups", "randes_launch_count", "randes_last_error",
+    "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_interference_norm", "randes_pairwise_cosines", "randes_retrieve_batch", "randes_retrieve_static", "randes_linear", "randes_linear_gated", "randes_linear_giveups", "randes_launch_count", "randes_last_error",
 ]
 
 
@@ -256,6 +258,13 @@ def randes_retrieve_static(plan, task_id, lam, out_dtype, base, M, out, stream) 
 def randes_linear(plan, task_id, lam, layer, x, n_tokens, base, M, y, stream, y_dtype: int = F32) -> None:
     """y = x What_t[layer]^T on the tensor cores, the retrieved weight never written to memory."""
     _check(lib().randes_linear(plan, task_id, lam, layer, _addr(x), n_tokens, _addr(base), _addr(M), _addr(y), y_dtype, stream))
+
+
+def randes_linear_gated(plan, task_id, lam, layer, x, n_tokens, base, M, y, gate, wait_ns, stream, y_dtype: int = F32) -> None:
+    """randes_linear whose thread blocks first wait (at most wait_ns nanoseconds; 0 = one second) for the device word
+    ``gate`` to become non-zero; blocks whose wait runs out write nothing and count in randes_linear_giveups()."""
+    _check(lib().randes_linear_gated(plan, task_id, lam, layer, _addr(x), n_tokens, _addr(base), _addr(M), _addr(y), y_dtype,
+                                     _addr(gate), int(wait_ns), stream))
 
 
 def randes_linear_giveups() -> int:

@@ -113,13 +113,14 @@ def test_linear_bf16_output_is_the_fp32_result_rounded_once():
     plan = randes.Plan.from_workload(w, max_tasks=2, m_dtype=wl.BF16)
     M_dev = plan.compress(d_base, d_tasks)
     rng = np.random.default_rng(6)
+    giveups = randes.randes_linear_giveups()
     for p in range(w.n_layers):
         x = to_dev(_bf16_normal(rng, (150, w.cols[p])))
         y32 = plan.linear(ids[0], w.lam, p, x, d_base, M_dev)
         y16 = plan.linear(ids[0], w.lam, p, x, d_base, M_dev, y_dtype=wl.BF16)
         assert y16.dtype == torch.bfloat16
         assert torch.equal(y16, y32.to(torch.bfloat16))           # same accumulators, one rounding to nearest even
-    assert randes.randes_linear_giveups() == 0
+    assert randes.randes_linear_giveups() == giveups
     plan.close()
 
 
@@ -256,6 +257,7 @@ def test_linear_unaligned_output_zero_tokens_and_host_only_plan():
     buf = torch.full((45 * 136 + 1,), float("nan"), dtype=torch.float32, device="cuda")
     y = buf[1:].view(45, 136)                                  # 4 bytes past a 16-byte boundary
     before = randes.randes_launch_count()
+    giveups = randes.randes_linear_giveups()
     host_plan.linear(ids[1], 0.3, 1, to_dev(x), d_base, M_dev, y=y)
     assert randes.randes_launch_count() == before + 1
     y_ref, y_abs = ro.linear(w.spec, w.storage, ids[1], seeds[1], 0.3, 1, x, base, M_ref, m_dtype=wl.BF16)
@@ -267,8 +269,48 @@ def test_linear_unaligned_output_zero_tokens_and_host_only_plan():
     with pytest.raises(randes.RandesError) as e:
         plan.linear(77, 0.3, 0, to_dev(x), d_base, M_dev)
     assert e.value.code == randes.UNKNOWN_TASK
-    assert randes.randes_linear_giveups() == 0
+    assert randes.randes_linear_giveups() == giveups
     plan.close(); host_plan.close()
+
+
+@pytest.mark.parametrize("gflag", [S | F, S])
+def test_linear_behind_a_gate_that_nothing_opens_gives_up_and_leaves_the_context_usable(gflag):
+    """Failure detection of the one kernel that waits.  The gated call makes every thread block wait for a device
+    word; here nothing sets it, so the (3 ms) wait runs out in all 3 x 2 blocks: each must return without a copy,
+    a product or a store (y keeps its poison), count itself in randes_linear_giveups, and leave the context healthy.
+    With the gate open the same call computes the layer, and the ordinary call still works afterwards."""
+    w = _workload([(300, 192, 2)], [gflag], n_tasks=2)
+    ids, seeds = list(w.task_ids), list(w.seeds)
+    base, tasks = wl.model_set(w, ids)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, max_tasks=2, m_dtype=wl.BF16)
+    M_dev = plan.compress(d_base, d_tasks)
+    M_ref = ro.compress(w.spec, w.storage, ids, seeds, base, tasks, m_dtype=wl.BF16)
+    n_tok, p, t, s = 200, 1, ids[1], seeds[1]
+    x = _bf16_normal(np.random.default_rng(12), (n_tok, 192))
+    d_x, p_base = to_dev(x), randes.ptr_array(d_base)
+    stream = torch.cuda.current_stream().cuda_stream
+    gate = torch.zeros(1, dtype=torch.int32, device="cuda")
+    guard = torch.full((n_tok + 2, 300), float("nan"), dtype=torch.float32, device="cuda")
+    y = guard[1:-1]
+    before = randes.randes_linear_giveups()
+    randes.randes_linear_gated(plan.handle, t, w.lam, p, d_x, n_tok, p_base, M_dev, y, gate, 3_000_000, stream)
+    torch.cuda.synchronize()                                   # returns: the kernel ended by itself
+    assert randes.randes_linear_giveups() - before == 3 * 2    # ceil(300 / 128) feature tiles x ceil(200 / 128) token blocks
+    assert bool(torch.isnan(guard).all())                      # nothing was written, inside or around y
+    gate.fill_(1)
+    y_ref, y_abs = ro.linear(w.spec, w.storage, t, s, w.lam, p, x, base, M_ref, m_dtype=wl.BF16)
+    tol = _tolerance(192, y_abs)
+    randes.randes_linear_gated(plan.handle, t, w.lam, p, d_x, n_tok, p_base, M_dev, y, gate, 0, stream)
+    assert np.all(np.abs(y.cpu().numpy().astype(np.float64) - y_ref) <= tol)
+    y2 = plan.linear(t, w.lam, p, d_x, d_base, M_dev)
+    assert torch.equal(y2, y)                                  # the ordinary call, same bits
+    assert bool(torch.isnan(guard[0]).all()) and bool(torch.isnan(guard[-1]).all())
+    assert randes.randes_linear_giveups() - before == 6        # no further give-ups
+    with pytest.raises(randes.RandesError) as e:
+        randes.randes_linear_gated(plan.handle, t, w.lam, p, d_x, n_tok, p_base, M_dev, y, None, 0, stream)
+    assert e.value.code == randes.INVALID_ARGUMENT
+    plan.close()
 
 
 def test_linear_rejects_what_it_cannot_run():

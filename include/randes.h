@@ -320,9 +320,10 @@ int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_
  *   base / tasks     as for randes_compress (base may be NULL: tasks hold deltas)
  *   gram             DEVICE array of n*n doubles, written on `stream`
  *   scratch          device memory of at least randes_delta_gram_scratch_bytes(plan) bytes
- * Products are exact in fp64 and summed in a fixed order: the result is
- * reproducible bit for bit.  At most 32 tasks.  ceil(n/4) passes over the
- * weights, two kernel launches each.
+ * Products are exact in fp64 and summed in a fixed order (fp64 tensor-core
+ * products over blocks of 8 x 8 tasks, upper triangle, mirrored): the result is
+ * symmetric and reproducible bit for bit.  At most 32 tasks.  One pass over the
+ * weights, two kernel launches.
  * Errors: INVALID_ARGUMENT, CAPACITY, MISALIGNED, WORKSPACE_TOO_SMALL, CUDA_ERROR.
  */
 size_t randes_delta_gram_scratch_bytes(const randes_plan_t* plan);

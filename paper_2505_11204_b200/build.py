@@ -1,6 +1,8 @@
 """Compile the CUDA library for sm_100a into the package directory.
 
-    python -m paper_2505_11204_b200.build [--force] [--verbose]
+    python -m paper_2505_11204_b200.build [--force] [--verbose] [--nvtx]
+
+--nvtx brackets every computing entry point with an NVTX range (off by default).
 
 nvcc cross-compiles without a GPU.  The shared object is kept in-tree (it is
 not committed) so that it travels with the source tree to the machine that has
@@ -27,21 +29,31 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
-    if not force and not _stale():
-        return LIB
+def nvcc_command(out: str, extra_flags=(), opt: str = "-O3"):
+    """The one nvcc invocation that builds the library into `out`."""
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + ".%d.tmp" % os.getpid()
-    cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-           "-Xcompiler", "-fPIC", "-shared", "-o", tmp]
-    if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += list(extra_flags)
-    cmd += [os.path.join(CSRC, s) for s in SOURCES]
-    subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    return ([nvcc, opt, "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "--threads", "0",
+             "-Xcompiler", "-fPIC", "-shared", "-o", out] + list(extra_flags) + [os.path.join(CSRC, s) for s in SOURCES])
+
+
+# host code of the library under AddressSanitizer and UndefinedBehaviorSanitizer (device code is unaffected);
+# load the result with the sanitizer run-times preloaded
+SANITIZER_FLAGS = ["-Xcompiler", "-fsanitize=address,-fsanitize=undefined,-fno-sanitize-recover=undefined,-fno-omit-frame-pointer", "-g"]
+# every computing entry point bracketed by an NVTX range named after it
+NVTX_FLAGS = ["-DRANDES_NVTX", "-ldl"]
+
+
+def build_library(force: bool = False, verbose: bool = False, extra_flags=(), out: str = LIB) -> str:
+    """Build the library (into the package directory unless `out` names another file)."""
+    if out == LIB and not force and not _stale():
+        return LIB
+    tmp = out + ".%d.tmp" % os.getpid()
+    flags = list(extra_flags) + (["-Xptxas", "-v"] if verbose else [])
+    subprocess.run(nvcc_command(tmp, flags), check=True)
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    nvtx = "--nvtx" in sys.argv
+    print(build_library(force="--force" in sys.argv or nvtx, verbose="--verbose" in sys.argv, extra_flags=NVTX_FLAGS if nvtx else ()))

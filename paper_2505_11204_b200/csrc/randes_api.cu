@@ -13,6 +13,10 @@
 #include <string>
 #include <vector>
 
+#ifdef RANDES_NVTX
+#include <nvtx3/nvToolsExt.h>
+#endif
+
 #include "../../include/randes.h"
 #include "randes_internal.h"
 
@@ -126,7 +130,7 @@ WorkspaceLayout layout_workspace(size_t n_layers, size_t n_units, size_t n_stage
 enum { kAllGroups = 0, kStagedGroups = 1, kOtherGroups = 2 };
 void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, std::vector<DevUnit>& units,
                  const std::vector<char>* staged = nullptr, const std::vector<uint32_t>* member_base = nullptr,
-                 int which = kAllGroups, std::vector<size_t>* per_group = nullptr)
+                 int which = kAllGroups, std::vector<size_t>* per_group = nullptr, uint32_t rows_per_warp = kRowsPerWarp)
 {
     const uint32_t wcols = cols_per_warp(storage);
     units.clear();
@@ -159,7 +163,7 @@ void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, s
         } else {
             uint32_t nbc = 1;
             while (nbc < static_cast<uint32_t>(kWarpsPerCta) && nb % (nbc * 2) == 0) nbc *= 2;
-            const uint32_t rows_per_unit = kRowsPerWarp * (kWarpsPerCta / nbc);
+            const uint32_t rows_per_unit = rows_per_warp * (kWarpsPerCta / nbc);
             for (uint32_t r0 = 0; r0 < rows; r0 += rows_per_unit)
                 for (uint32_t cb0 = 0; cb0 < nb; cb0 += nbc)
                     for (uint32_t l : members) {
@@ -255,6 +259,8 @@ struct randes_plan_s {
     std::vector<DevTask> h_dev_tasks;
     bool base_valid = false, out_valid = false;
     size_t tasks_valid = 0;
+    const void* checked_m = nullptr;              // M and output element size of the last retrieve whose tensors were found disjoint
+    size_t checked_out_elem = 0;
 
     template <typename T> T* dev(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -457,9 +463,59 @@ int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_
     return RANDES_OK;
 }
 
-// Runs the body of an entry point; nothing may cross the C ABI as an exception.
-template <typename F> int guarded(F&& body)
+// The outputs of a retrieve may overlap neither the base tensors, nor M, nor each other (an output element is
+// written by one thread while others still read their inputs).  Byte ranges, so that partial overlaps are caught
+// too: the ranges of all tensors are sorted by their start and swept once.
+int check_outputs_disjoint(const randes_plan_t& p, const void* const* base, const void* const* out, size_t n_out_models,
+                           size_t out_elem, const void* M)
 {
+    struct Range { uintptr_t lo, hi; uint32_t layer; int kind; };   // kind: 0 base, 1 M, 2 + b output of model b
+    std::vector<Range> r;
+    r.reserve((n_out_models + 1) * p.n_layers + 1);
+    for (uint32_t l = 0; l < p.n_layers; ++l) {
+        const size_t elems = static_cast<size_t>(p.layers[l].rows) * p.layers[l].cols;
+        if (!elems) continue;
+        const uintptr_t b = reinterpret_cast<uintptr_t>(base[l]);
+        r.push_back({b, b + elems * elem_size(p.storage), l, 0});
+        for (size_t m = 0; m < n_out_models; ++m) {
+            const uintptr_t o = reinterpret_cast<uintptr_t>(out[m * p.n_layers + l]);
+            r.push_back({o, o + elems * out_elem, l, static_cast<int>(2 + m)});
+        }
+    }
+    const uintptr_t m0 = reinterpret_cast<uintptr_t>(M);
+    r.push_back({m0, m0 + p.m_bytes, 0, 1});
+    std::sort(r.begin(), r.end(), [](const Range& a, const Range& b) { return a.lo < b.lo; });
+    uintptr_t reach = 0;          // furthest end seen so far, and whose it is
+    const Range* owner = nullptr;
+    for (const Range& x : r) {
+        if (owner && x.lo < reach && (x.kind >= 2 || owner->kind >= 2)) {
+            const Range& o = x.kind >= 2 ? x : *owner;
+            const Range& other = x.kind >= 2 ? *owner : x;
+            return fail(RANDES_INVALID_ARGUMENT, "out[%d][%u] overlaps %s", o.kind - 2, o.layer,
+                        other.kind == 0 ? "a base tensor" : (other.kind == 1 ? "M" : "another output tensor"));
+        }
+        if (x.hi > reach) { reach = x.hi; owner = &x; }
+    }
+    return RANDES_OK;
+}
+
+// Built with -DRANDES_NVTX every computing entry point is bracketed by an NVTX range named after it, so that
+// a timeline shows which call enqueued which kernels.  Off by default: the header is not even included.
+#ifdef RANDES_NVTX
+struct CallRange {
+    explicit CallRange(const char* name) { nvtxRangePushA(name); }
+    ~CallRange() { nvtxRangePop(); }
+};
+#else
+struct CallRange {
+    explicit CallRange(const char*) {}
+};
+#endif
+
+// Runs the body of an entry point; nothing may cross the C ABI as an exception.
+template <typename F> int guarded(const char* name, F&& body)
+{
+    const CallRange range(name);
     try {
         return body();
     } catch (const std::bad_alloc&) {
@@ -576,7 +632,17 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
             off = align_up(off + static_cast<size_t>(layers[l].rows) * layers[l].cols * elem_size(m_dtype), 256);
         }
         p->m_bytes = off;
-        build_units(layers, n_layers, p->storage, p->units);
+        // A general diagonal context costs three Philox blocks per (task, column) and unit: its plans get taller units
+        // (up to eight times), so that the factors are reused over more rows -- as tall as still leaves about two
+        // thousand units for the grid (fewer units than the workspace holds, which is sized for the short ones).
+        uint32_t rows_per_warp = kRowsPerWarp;
+        if (p->has_gauss) {
+            unsigned long long params = 0;
+            for (uint32_t l = 0; l < n_layers; ++l) params += static_cast<unsigned long long>(layers[l].rows) * layers[l].cols;
+            while (rows_per_warp < static_cast<uint32_t>(kContextRowsPerWarp) && params / (2ull * rows_per_warp * 1024ull) >= 2000ull)
+                rows_per_warp *= 2;
+        }
+        build_units(layers, n_layers, p->storage, p->units, nullptr, nullptr, kAllGroups, nullptr, rows_per_warp);
         {
             std::vector<uint32_t> member_base(n_groups, 0);
             p->group_staged.assign(n_groups, 0);
@@ -735,7 +801,7 @@ int randes_plan_deserialize(const void* buffer, size_t buffer_bytes, uint32_t ma
     if (h.n_layers > (1u << 24) || h.n_groups > (1u << 24) || h.n_tasks > (1u << 24) ||
         buffer_bytes < blob_bytes(h.n_layers, h.n_groups, h.n_tasks))
         return fail(RANDES_INVALID_ARGUMENT, "serialized plan is truncated or corrupt");
-    return guarded([&] {
+    return guarded("randes_plan_deserialize", [&] {
         const char* in = static_cast<const char*>(buffer) + sizeof h;
         std::vector<randes_layer_t> layers(h.n_layers);
         std::memcpy(layers.data(), in, h.n_layers * sizeof(randes_layer_t)); in += h.n_layers * sizeof(randes_layer_t);
@@ -890,13 +956,13 @@ static int randes_retrieve_impl(randes_plan_t* plan, uint32_t task_id, float lam
     if (row < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_id);
     if ((rc = check_ptrs(*plan, base, "base", elem_size(plan->storage), false))) return rc;
     if ((rc = check_ptrs(*plan, const_cast<const void* const*>(out), "out", elem_size(out_dtype), false))) return rc;
-    const char* m_lo = static_cast<const char*>(M);
-    const char* m_hi = m_lo + plan->m_bytes;
-    for (uint32_t l = 0; l < plan->n_layers; ++l) {
-        const char* o = static_cast<const char*>(out[l]);
-        if (out[l] && (out[l] == base[l] || (o >= m_lo && o < m_hi)))
-            return fail(RANDES_INVALID_ARGUMENT, "out[%u] aliases base or M", l);
-    }
+    // (skipped when both pointer tables are the ones the last successful call checked)
+    const size_t table_bytes = plan->n_layers * sizeof(void*);
+    const bool seen = plan->base_valid && plan->out_valid && plan->checked_m == M && plan->checked_out_elem == elem_size(out_dtype) &&
+                      std::memcmp(plan->h_base.data(), base, table_bytes) == 0 && std::memcmp(plan->h_out.data(), out, table_bytes) == 0;
+    if (!seen && (rc = check_outputs_disjoint(*plan, base, const_cast<const void* const*>(out), 1, elem_size(out_dtype), M))) return rc;
+    plan->checked_m = M;
+    plan->checked_out_elem = elem_size(out_dtype);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((rc = stage_ptrs(*plan, plan->h_base, plan->base_valid, plan->lay.base_ptrs, base, s))) return rc;
     if ((rc = stage_ptrs(*plan, plan->h_out, plan->out_valid, plan->lay.out_ptrs, const_cast<const void* const*>(out), s)))
@@ -932,7 +998,7 @@ static int randes_retrieve_impl(randes_plan_t* plan, uint32_t task_id, float lam
 size_t randes_delta_gram_scratch_bytes(const randes_plan_t* plan)
 {
     if (!plan || !plan->ws) return 0;
-    return static_cast<size_t>(plan->grid_gram) * kWarpsPerCta * kGramAnchors * kTaskChunk * sizeof(double);
+    return static_cast<size_t>(plan->grid_gram) * kGramPartialDoubles * sizeof(double);
 }
 
 static int randes_delta_gram_impl(randes_plan_t* plan, const void* const* base, const void* const* tasks, double* gram, void* scratch,
@@ -971,13 +1037,9 @@ static int randes_delta_gram_impl(randes_plan_t* plan, const void* const* base, 
     a.task_ptrs = plan->dev<const void*>(plan->lay.task_ptrs);
     a.partial = static_cast<double*>(scratch);
     const int grid = std::max(1, std::min<int>(plan->grid_gram, static_cast<int>(a.n_units)));
-    for (uint32_t a0 = 0; a0 < n; a0 += kGramAnchors) {
-        a.a0 = a0;
-        a.na = std::min<uint32_t>(kGramAnchors, static_cast<uint32_t>(n) - a0);
-        const int e = launch_gram_pass(plan->storage, a, grid, gram, s);
-        if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the Gram kernels");
-        g_launches += 2;
-    }
+    const int e = launch_gram(plan->storage, a, grid, gram, s);
+    if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the Gram kernels");
+    g_launches += 2;
     return RANDES_OK;
 }
 
@@ -998,8 +1060,6 @@ static int randes_retrieve_batch_impl(randes_plan_t* plan, const uint32_t* task_
     if ((rc = check_ptrs(*plan, base, "base", elem_size(plan->storage), false))) return rc;
     if (!out) return fail(RANDES_INVALID_ARGUMENT, "out is NULL");
     RetrieveBatchArgs a;
-    const char* m_lo = static_cast<const char*>(M);
-    const char* m_hi = m_lo + plan->m_bytes;
     for (uint32_t b = 0; b < n_tasks; ++b) {
         const int row = find_task(*plan, task_ids[b]);
         if (row < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_ids[b]);
@@ -1008,12 +1068,8 @@ static int randes_retrieve_batch_impl(randes_plan_t* plan, const uint32_t* task_
         a.task_rows[b] = static_cast<uint32_t>(row);
         void* const* ob = out + static_cast<size_t>(b) * plan->n_layers;
         if ((rc = check_ptrs(*plan, const_cast<const void* const*>(ob), "out", elem_size(out_dtype), false))) return rc;
-        for (uint32_t l = 0; l < plan->n_layers; ++l) {
-            const char* o = static_cast<const char*>(ob[l]);
-            if (ob[l] && (ob[l] == base[l] || (o >= m_lo && o < m_hi)))
-                return fail(RANDES_INVALID_ARGUMENT, "out[%u][%u] aliases base or M", b, l);
-        }
     }
+    if ((rc = check_outputs_disjoint(*plan, base, const_cast<const void* const*>(out), n_tasks, elem_size(out_dtype), M))) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if ((rc = stage_ptrs(*plan, plan->h_base, plan->base_valid, plan->lay.base_ptrs, base, s))) return rc;
     // the batch's output tables share the device area of the task pointer tables
@@ -1072,13 +1128,7 @@ static int randes_retrieve_static_impl(const randes_plan_t* plan, uint32_t task_
     if (row < 0) return fail(RANDES_UNKNOWN_TASK, "task id %u is not registered", task_id);
     if ((rc = check_ptrs(*plan, base, "base", elem_size(plan->storage), false))) return rc;
     if ((rc = check_ptrs(*plan, const_cast<const void* const*>(out), "out", elem_size(out_dtype), false))) return rc;
-    const char* m_lo = static_cast<const char*>(M);
-    const char* m_hi = m_lo + plan->m_bytes;
-    for (uint32_t l = 0; l < plan->n_layers; ++l) {
-        const char* o = static_cast<const char*>(out[l]);
-        if (out[l] && (out[l] == base[l] || (o >= m_lo && o < m_hi)))
-            return fail(RANDES_INVALID_ARGUMENT, "out[%u] aliases base or M", l);
-    }
+    if ((rc = check_outputs_disjoint(*plan, base, const_cast<const void* const*>(out), 1, elem_size(out_dtype), M))) return rc;
     const size_t need = retrieve_static_bytes(plan->n_layers, static_cast<uint32_t>(plan->units.size()));
     if (need > kStaticScratchBytes)
         return fail(RANDES_CAPACITY,
@@ -1102,31 +1152,31 @@ static int randes_retrieve_static_impl(const randes_plan_t* plan, uint32_t task_
 
 int randes_compress(randes_plan_t* plan, const void* const* base, const void* const* tasks, void* M, void* stream)
 {
-    return guarded([&] { return randes_compress_impl(plan, base, tasks, M, stream); });
+    return guarded("randes_compress", [&] { return randes_compress_impl(plan, base, tasks, M, stream); });
 }
 
 int randes_add_model(randes_plan_t* plan, uint32_t task_id, uint64_t seed, const void* const* base,
                      const void* const* task, void* M, void* stream)
 {
-    return guarded([&] { return randes_add_model_impl(plan, task_id, seed, base, task, M, stream); });
+    return guarded("randes_add_model", [&] { return randes_add_model_impl(plan, task_id, seed, base, task, M, stream); });
 }
 
 int randes_add_models(randes_plan_t* plan, const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
                       const void* const* base, const void* const* tasks, void* M, void* stream)
 {
-    return guarded([&] { return randes_add_models_impl(plan, task_ids, seeds, n_tasks, base, tasks, M, stream); });
+    return guarded("randes_add_models", [&] { return randes_add_models_impl(plan, task_ids, seeds, n_tasks, base, tasks, M, stream); });
 }
 
 int randes_remove_model(randes_plan_t* plan, uint32_t task_id, const void* const* base, const void* const* task,
                         void* M, void* stream)
 {
-    return guarded([&] { return randes_remove_model_impl(plan, task_id, base, task, M, stream); });
+    return guarded("randes_remove_model", [&] { return randes_remove_model_impl(plan, task_id, base, task, M, stream); });
 }
 
 int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
                     const void* const* base, const void* M, void* const* out, void* stream)
 {
-    return guarded([&] { return randes_retrieve_impl(plan, task_id, lambda, out_dtype, base, M, out, stream); });
+    return guarded("randes_retrieve", [&] { return randes_retrieve_impl(plan, task_id, lambda, out_dtype, base, M, out, stream); });
 }
 
 static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x,
@@ -1174,7 +1224,7 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
 int randes_linear(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x, uint32_t n_tokens,
                   const void* const* base, const void* M, void* y, randes_dtype_t y_dtype, void* stream)
 {
-    return guarded([&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, y_dtype, nullptr, 0, stream); });
+    return guarded("randes_linear", [&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, y_dtype, nullptr, 0, stream); });
 }
 
 int randes_linear_gated(const randes_plan_t* plan, uint32_t task_id, float lambda, uint32_t layer, const void* x, uint32_t n_tokens,
@@ -1182,7 +1232,7 @@ int randes_linear_gated(const randes_plan_t* plan, uint32_t task_id, float lambd
                         uint64_t wait_ns, void* stream)
 {
     if (!gate) return fail(RANDES_INVALID_ARGUMENT, "gate is NULL (use randes_linear for a call without a gate)");
-    return guarded([&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, y_dtype, gate, wait_ns, stream); });
+    return guarded("randes_linear_gated", [&] { return randes_linear_impl(plan, task_id, lambda, layer, x, n_tokens, base, M, y, y_dtype, gate, wait_ns, stream); });
 }
 
 int randes_linear_giveups(unsigned int* count)
@@ -1196,13 +1246,13 @@ int randes_linear_giveups(unsigned int* count)
 int randes_retrieve_batch(randes_plan_t* plan, const uint32_t* task_ids, uint32_t n_tasks, float lambda,
                           randes_dtype_t out_dtype, const void* const* base, const void* M, void* const* out, void* stream)
 {
-    return guarded([&] { return randes_retrieve_batch_impl(plan, task_ids, n_tasks, lambda, out_dtype, base, M, out, stream); });
+    return guarded("randes_retrieve_batch", [&] { return randes_retrieve_batch_impl(plan, task_ids, n_tasks, lambda, out_dtype, base, M, out, stream); });
 }
 
 int randes_delta_gram(randes_plan_t* plan, const void* const* base, const void* const* tasks, double* gram, void* scratch,
                       size_t scratch_bytes, void* stream)
 {
-    return guarded([&] { return randes_delta_gram_impl(plan, base, tasks, gram, scratch, scratch_bytes, stream); });
+    return guarded("randes_delta_gram", [&] { return randes_delta_gram_impl(plan, base, tasks, gram, scratch, scratch_bytes, stream); });
 }
 
 // Section 3, norm of the interference: || lambda sum_{j != t} T_t^-1 T_j d_j ||^2 = lambda^2 sum_{j,l != t} <T_j d_j, T_l d_l>,
@@ -1249,7 +1299,7 @@ int randes_pairwise_cosines(const double* gram, uint32_t n, int32_t exclude, dou
 int randes_retrieve_static(const randes_plan_t* plan, uint32_t task_id, float lambda, randes_dtype_t out_dtype,
                            const void* const* base, const void* M, void* const* out, void* stream)
 {
-    return guarded([&] { return randes_retrieve_static_impl(plan, task_id, lambda, out_dtype, base, M, out, stream); });
+    return guarded("randes_retrieve_static", [&] { return randes_retrieve_static_impl(plan, task_id, lambda, out_dtype, base, M, out, stream); });
 }
 
 }  // extern "C"

@@ -14,6 +14,7 @@ constexpr uint32_t kFlagGauss = 4u;     // per-column Gaussian-like factor on th
 constexpr int kWarpsPerCta = 8;
 constexpr int kThreadsPerCta = kWarpsPerCta * 32;
 constexpr int kRowsPerWarp = 16;        // rows one warp walks per unit (8 to 16 measured best; 32 and 64 slower)
+constexpr int kContextRowsPerWarp = 128; // upper limit of the same for plans with a general diagonal context (randes_context.cu)
 constexpr int kTaskChunk = 32;          // tasks whose pointers / sign blocks a warp holds at once
 constexpr uint32_t kTagSign = 0x5349474Eu;  // counter word 2 of the sign stream ("SIGN")
 constexpr uint32_t kTagPerm = 0x5045524Du;  // counter word 2 of the permutation stream ("PERM")
@@ -134,7 +135,8 @@ struct RetrieveBatchArgs {
     const uint32_t* members;       // layers of every group, group after group, in member order (group units only)
 };
 
-constexpr int kGramAnchors = 4;   // rows of the Gram matrix produced per pass
+constexpr int kGramBlocks = 10;   // blocks of 8 x 8 in the upper triangle of a kTaskChunk x kTaskChunk Gram matrix
+constexpr int kGramPartialDoubles = kGramBlocks * 64;   // what one CTA hands to the final reduction
 
 struct GramArgs {
     const DevLayer* layers;
@@ -144,11 +146,10 @@ struct GramArgs {
     const uint32_t* src_of_slot;   // sigma rows of all registered tasks
     const DevTask* tasks;
     uint32_t n_tasks;              // <= kTaskChunk
-    uint32_t a0, na;               // this pass produces rows [a0, a0 + na), na <= kGramAnchors
     uint32_t has_base;
     const void* const* base;
     const void* const* task_ptrs;  // [n_tasks][n_layers]
-    double* partial;               // [grid * kWarpsPerCta][kGramAnchors][kTaskChunk]
+    double* partial;               // [grid][kGramPartialDoubles]
 };
 
 // Launchers (randes_kernels.cu).  Return a cudaError_t as int.
@@ -169,8 +170,8 @@ int launch_compress_groups(int storage_dtype, int m_dtype, const CompressGroupAr
 // dynamic shared memory they need: call once per device before launching.
 int retrieve_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype);
 int accumulate_ctas_per_sm(int storage_dtype, int m_dtype, bool single_task);
-// randes_diag.cu: one pass = the Gram kernel plus the fixed-order reduction into gram[a0 .. a0+na)[*]
-int launch_gram_pass(int storage_dtype, const GramArgs& a, int grid, double* gram, void* stream);
+// randes_diag.cu: the Gram kernel (one pass over the weights) plus the fixed-order reduction into gram
+int launch_gram(int storage_dtype, const GramArgs& a, int grid, double* gram, void* stream);
 int gram_ctas_per_sm(int storage_dtype);
 // randes_batch.cu
 int launch_retrieve_batch(int storage_dtype, int out_dtype, int m_dtype, const RetrieveBatchArgs& a, int grid, void* stream);

@@ -102,10 +102,7 @@ __device__ __forceinline__ void retrieve_rows_halves(const WarpTile& t, uint32_t
                                                      const bf16* __restrict__ wp, OT* __restrict__ op, float lambda,
                                                      uint32_t bits0, uint32_t bits1)
 {
-#ifndef RANDES_RET_H_U
-#define RANDES_RET_H_U 2
-#endif
-    constexpr int U = RANDES_RET_H_U;                                  // rows per trip (1 and 4 measured slower)
+    constexpr int U = 2;                                  // rows per trip (1 and 4 measured slower, with two or three CTAs per SM)
     const uint32_t c0 = t.cb * 256u + lane * 4u;          // first half; the second is 128 columns further
     const bool on[2] = {c0 < cols, c0 + 128u < cols};
     float lam[2][4];
@@ -149,11 +146,8 @@ __device__ __forceinline__ void retrieve_rows_halves(const WarpTile& t, uint32_t
     }
 }
 
-#ifndef RANDES_RET_OCC
-#define RANDES_RET_OCC 2
-#endif
 template <typename ST, typename OT, typename MT>
-__global__ void __launch_bounds__(kThreadsPerCta, (sizeof(ST) == 2 && sizeof(MT) == 4) ? RANDES_RET_OCC : 2) retrieve_kernel(const RetrieveArgs a)
+__global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_kernel(const RetrieveArgs a)
 {
     constexpr int CPL = Store<ST>::CPL;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

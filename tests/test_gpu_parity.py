@@ -643,3 +643,29 @@ def test_flan_t5_shaped_full_and_lora_variant():
     ref = ro.retrieve(wlora.spec, wlora.storage, wl.F32, 2, wlora.seeds[2], w.lam, lbase, M_ref)
     check_model(out, ref, "lora retrieve")
     plan.close()
+    # the other form of the same case: the plan of the WHOLE model, every layer without an adapter given as a zero
+    # tensor (one zero tensor per shape, shared by all tasks).  M is zero there, and retrieval returns W_0 itself.
+    is_target = set(targets)
+    zeros_h, zeros_d = {}, {}
+    for l in range(w.n_layers):
+        shape = (w.rows[l], w.cols[l])
+        if l not in is_target and shape not in zeros_h:
+            zeros_h[shape] = np.zeros(shape, dtype=np.float32)
+            zeros_d[shape] = to_dev(zeros_h[shape])
+    pos = {l: k for k, l in enumerate(targets)}
+    full_h = [[deltas[i][pos[l]] if l in is_target else zeros_h[(w.rows[l], w.cols[l])] for l in range(w.n_layers)]
+              for i in range(w.n_tasks)]
+    d_deltas = [model_to_dev(d) for d in deltas]
+    full_d = [[d_deltas[i][pos[l]] if l in is_target else zeros_d[(w.rows[l], w.cols[l])] for l in range(w.n_layers)]
+              for i in range(w.n_tasks)]
+    plan = randes.Plan.from_workload(w)
+    M = plan.compress(None, full_d)
+    M_ref = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, None, full_h)
+    check_superposition(plan, M, M_ref, "lora compress, whole model with zero tensors")
+    out = plan.retrieve(2, w.lam, d_base, M)
+    ref = ro.retrieve(w.spec, w.storage, wl.F32, 2, w.seeds[2], w.lam, base, M_ref)
+    check_model(out, ref, "lora retrieve, whole model")
+    for l in range(w.n_layers):
+        if l not in is_target:
+            assert_bits_equal(from_dev(out[l]), base[l], "layer %d has no adapter: retrieval must return W_0" % l)
+    plan.close()

@@ -223,6 +223,29 @@ def test_interference_norm_and_cosines_against_the_oracle():
     assert randes.lib().randes_pairwise_cosines(None, 2, -1, None, None) == randes.INVALID_ARGUMENT
 
 
+def test_outputs_that_overlap_an_input_or_each_other_are_refused():
+    """out may overlap neither base, nor M, nor another output tensor -- not even part-way.  The check runs on the
+    host before anything is launched (shown here through the entry point that accepts a host-only plan)."""
+    n, rows, cols = 3, 4, 8
+    nbytes = rows * cols * 4
+    plan = randes.Plan([rows] * n, [cols] * n, [0] * n, [randes.SHUFFLE | randes.FLIP], task_ids=[0], seeds=[1], host_only=True)
+    arr = lambda xs: (ctypes.c_void_p * n)(*xs)
+    base = arr([0x10000 + i * 0x1000 for i in range(n)])
+    M = 0x100000
+    call = lambda out: randes.randes_retrieve_static(plan.handle, 0, 1.0, randes.F32, base, M, arr(out), None)
+    good = [0x20000 + i * 0x1000 for i in range(n)]
+    cases = {
+        "a base tensor": [good[0], 0x10000 + 0x1000 + nbytes - 4, good[2]],          # last element of base[1], from another layer
+        "M": [good[0], good[1], M + plan.m_bytes - 4],
+        "another output tensor": [good[0], good[0] + nbytes - 16, good[2]],
+    }
+    for what, out in cases.items():
+        with pytest.raises(randes.RandesError) as e:
+            call(out)
+        assert e.value.code == randes.INVALID_ARGUMENT and what in str(e.value), (what, str(e.value))
+    plan.close()
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(randes, "_lib", None)
     monkeypatch.setattr(randes, "LIB_PATH", str(tmp_path / "absent.so"))

@@ -149,17 +149,22 @@ void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, s
         const size_t before = units.size();
         const uint32_t nb = (cols + wcols - 1) / wcols;
         if (is_staged) {
+            // kUnitChunk consecutive blocks of rows of one column block lie next to each other (a CTA takes them together
+            // and builds its per-(group, column block) tables once); the column blocks of such a band of rows follow, so
+            // that CTAs working side by side read neighbouring pieces of the same rows
             const uint32_t R = group_unit_rows(static_cast<uint32_t>(members.size()), storage);
-            for (uint32_t r0 = 0; r0 < rows; r0 += R)
-                for (uint32_t cb0 = 0; cb0 < nb; ++cb0) {
-                    DevUnit u;
-                    u.layer = (*member_base)[g];
-                    u.row0 = r0;
-                    u.nrows = std::min(R, rows - r0);
-                    u.cb0 = static_cast<uint16_t>(cb0);
-                    u.nbc = 0;
-                    units.push_back(u);
-                }
+            const uint32_t band = R * kUnitChunk;
+            for (uint32_t band0 = 0; band0 < rows; band0 += band)
+                for (uint32_t cb0 = 0; cb0 < nb; ++cb0)
+                    for (uint32_t r0 = band0; r0 < std::min(rows, band0 + band); r0 += R) {
+                        DevUnit u;
+                        u.layer = (*member_base)[g];
+                        u.row0 = r0;
+                        u.nrows = std::min(R, rows - r0);
+                        u.cb0 = static_cast<uint16_t>(cb0);
+                        u.nbc = 0;
+                        units.push_back(u);
+                    }
         } else {
             uint32_t nbc = 1;
             while (nbc < static_cast<uint32_t>(kWarpsPerCta) && nb % (nbc * 2) == 0) nbc *= 2;

@@ -136,6 +136,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
 // of sign bits -- in parallel over its threads.  After that the row loop only reads shared memory
 // and streams 16-byte stores: the call is bound by HBM writes, as it should be.
 constexpr uint32_t kBatchRecBytes = 32;   // {out pointer, slot member, pad, Philox block}
+constexpr uint32_t kBatchMemberBytes = (kStashBytes / kStashTileBytes) * 16;   // per member: {its slot of M, its W_0 tensor}
 
 __device__ __forceinline__ void store_plain(float* p, const float (&y)[4])
 {
@@ -153,47 +154,64 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_group_kernel
     extern __shared__ __align__(16) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_s = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
-    const uint32_t m_stash = smem_s, w_stash = smem_s + kStashBytes, s_rec = smem_s + 2 * kStashBytes;
+    const uint32_t m_stash = smem_s, w_stash = smem_s + kStashBytes, s_mem = smem_s + 2 * kStashBytes, s_rec = s_mem + kBatchMemberBytes;
     const uint32_t L = a.n_layers, n = a.n_tasks;
     const uint32_t sign_word = 16 + (lane >> 3) * 4u, sign_shift = (lane & 7) * 4u;
-    for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+    // The unit list keeps kUnitChunk units of one (group, column block) next to each other and a CTA takes whole
+    // chunks: the records and the member table depend on the group, the column block and the tasks only, so they are
+    // built once per chunk; every further unit of the chunk just refills the two stashes.
+    uint32_t key_group = 0xFFFFFFFFu, key_cb = 0xFFFFFFFFu;
+    uint32_t G = 0, cols = 0, c = 0;
+    bool lane_on = false;
+    const uint32_t n_chunked = (a.n_units + kUnitChunk - 1) / kUnitChunk;
+    for (uint32_t chunk = blockIdx.x; chunk < n_chunked; chunk += gridDim.x)
+    for (uint32_t u = chunk * kUnitChunk; u < min(a.n_units, (chunk + 1) * kUnitChunk); ++u) {
         const DevUnit un = a.units[u];
-        const uint32_t* mem = a.members + un.layer;
-        const DevLayer l0 = a.layers[mem[0]];
-        const uint32_t G = l0.group_size, cols = l0.cols, Rn = un.nrows;
-        const uint32_t c = (un.cb0 * 32u + lane) * CPL;
-        const bool lane_on = c < cols;
+        const uint32_t Rn = un.nrows;
+        if (un.layer != key_group || un.cb0 != key_cb) {
+            const uint32_t* mem = a.members + un.layer;
+            const DevLayer l0 = a.layers[mem[0]];
+            G = l0.group_size;
+            cols = l0.cols;
+            c = (un.cb0 * 32u + lane) * CPL;
+            lane_on = c < cols;
+            const uint32_t npairs = G * n;
+            for (uint32_t p = threadIdx.x; p < npairs; p += kThreadsPerCta) {
+                const uint32_t mp = p / n, b = p - mp * n;
+                const uint32_t pos = mem[mp];
+                const uint32_t fl = a.layers[pos].flags;
+                const uint32_t row = a.task_rows[b];
+                const uint32_t slot = (fl & kFlagShuffle) ? a.slot_of_pos[static_cast<size_t>(row) * L + pos] : pos;   // sigma_b^-1(p)
+                sts_ptrs(s_rec + p * kBatchRecBytes, a.out[static_cast<size_t>(b) * L + pos],
+                         reinterpret_cast<const void*>(static_cast<uintptr_t>(a.layers[slot].member)));
+                uint4 blk = make_uint4(0, 0, 0, 0);
+                if (fl & kFlagFlip) {
+                    const DevTask tk = a.tasks[row];
+                    blk = philox4x32_10(un.cb0, slot, kTagSign, tk.id, tk.key0, tk.key1);
+                }
+                sts128(s_rec + p * kBatchRecBytes + 16, blk);
+            }
+            // per member: where its slot of M and its W_0 tensor start
+            for (uint32_t m = threadIdx.x; m < G; m += kThreadsPerCta)
+                sts_ptrs(s_mem + m * 16, static_cast<const float*>(a.M) + a.layers[mem[m]].m_off, a.base[mem[m]]);
+            key_group = un.layer;
+            key_cb = un.cb0;
+            __syncthreads();   // records and member table are complete and visible to every warp
+        }
         const uint32_t off0 = un.row0 * cols + c;          // layers hold < 2^32 elements
 
         if (lane_on) {
             const uint32_t ntiles = G * Rn;
             for (uint32_t q = warp; q < ntiles; q += kWarpsPerCta) {
                 const uint32_t m = q / Rn, r = q - m * Rn;
-                const uint32_t layer = mem[m];
                 const uint32_t off = off0 + r * cols;
-                cp_async16(m_stash + q * kStashTileBytes + lane * 16, static_cast<const float*>(a.M) + a.layers[layer].m_off + off);
-                cp_async16(w_stash + q * kStashTileBytes + lane * 16, static_cast<const float*>(a.base[layer]) + off);
+                cp_async16(m_stash + q * kStashTileBytes + lane * 16, reinterpret_cast<const float*>(lds_ptr(s_mem + m * 16)) + off);
+                cp_async16(w_stash + q * kStashTileBytes + lane * 16, reinterpret_cast<const float*>(lds_ptr(s_mem + m * 16 + 8)) + off);
             }
         }
         cp_async_commit();
-        const uint32_t npairs = G * n;
-        for (uint32_t p = threadIdx.x; p < npairs; p += kThreadsPerCta) {
-            const uint32_t mp = p / n, b = p - mp * n;
-            const uint32_t pos = mem[mp];
-            const uint32_t fl = a.layers[pos].flags;
-            const uint32_t row = a.task_rows[b];
-            const uint32_t slot = (fl & kFlagShuffle) ? a.slot_of_pos[static_cast<size_t>(row) * L + pos] : pos;   // sigma_b^-1(p)
-            sts_ptrs(s_rec + p * kBatchRecBytes, a.out[static_cast<size_t>(b) * L + pos],
-                     reinterpret_cast<const void*>(static_cast<uintptr_t>(a.layers[slot].member)));
-            uint4 blk = make_uint4(0, 0, 0, 0);
-            if (fl & kFlagFlip) {
-                const DevTask tk = a.tasks[row];
-                blk = philox4x32_10(un.cb0, slot, kTagSign, tk.id, tk.key0, tk.key1);
-            }
-            sts128(s_rec + p * kBatchRecBytes + 16, blk);
-        }
         cp_async_wait<0>();
-        __syncthreads();   // stashes and records are complete and visible to every warp
+        __syncthreads();   // both stashes are complete and visible to every warp
 
         if (lane_on) {
             const uint32_t n_chunks = (Rn + kItemRows - 1) / kItemRows;
@@ -233,7 +251,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_group_kernel
     }
 }
 
-size_t batch_group_smem(uint32_t pairs) { return 2 * static_cast<size_t>(kStashBytes) + static_cast<size_t>(pairs) * kBatchRecBytes; }
+size_t batch_group_smem(uint32_t pairs) { return 2 * static_cast<size_t>(kStashBytes) + kBatchMemberBytes + static_cast<size_t>(pairs) * kBatchRecBytes; }
 
 template <typename K> int occupancy(K kernel)
 {
@@ -289,7 +307,8 @@ int launch_retrieve_batch_groups(int out_dtype, const RetrieveBatchArgs& a, uint
         if (e != cudaSuccess) { (void)cudaGetLastError(); return static_cast<int>(e); }
         if (per_sm <= 0) return static_cast<int>(cudaErrorInvalidConfiguration);
         const uint64_t want = static_cast<uint64_t>(sm_count) * per_sm;
-        const int grid = static_cast<int>(want < a.n_units ? want : a.n_units);
+        const uint64_t chunks = (a.n_units + kUnitChunk - 1) / kUnitChunk;
+        const int grid = static_cast<int>(want < chunks ? want : chunks);
         retrieve_batch_group_kernel<OT><<<grid, kThreadsPerCta, smem, s>>>(a);
         return static_cast<int>(cudaGetLastError());
     });

@@ -32,7 +32,7 @@ namespace {
 using namespace device;
 
 constexpr uint32_t kMaxGroup = kStashBytes / kStashTileBytes;   // members whose tiles fit the largest stash at one row each
-constexpr uint32_t kOffTableBytes = kMaxGroup * 8;
+constexpr uint32_t kOffTableBytes = kMaxGroup * 16;             // per member: first element of its slot in M, its W_0 tensor
 
 // rows per stage (SR), rows per item (IR) and stash size per weight type
 template <typename ST> struct GroupGeom;
@@ -83,7 +83,7 @@ __device__ __forceinline__ void cursor_set(Cursor& c, uint32_t item, uint32_t n_
 {
     c.item = item;
     const uint32_t ms = item / n_chunks;
-    c.m_off = s_rec - kOffTableBytes + ms * 8;
+    c.m_off = s_rec - kOffTableBytes + ms * 16;
     const uint32_t chunk = item - ms * n_chunks;
     c.row = chunk * IR;
     c.rows_left = min(IR, Rn - c.row);
@@ -136,45 +136,62 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
     const uint32_t sign_shift = CPL == 4 ? (lane & 7) * 4u : (lane & 3) * 8u;
     const uint32_t one = 0x3F800000u;
 
-    for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+    // The unit list keeps kUnitChunk units of one (group, column block) next to each other (consecutive blocks of
+    // rows), and a CTA takes whole chunks: the tables below depend on the group, the column block and the tasks only,
+    // so they are built once per chunk and every further unit of the chunk just refills the stash.
+    uint32_t key_group = 0xFFFFFFFFu, key_cb = 0xFFFFFFFFu;
+    uint32_t G = 0, cols = 0, c = 0;
+    bool lane_on = false;
+    const uint32_t n_chunked = (a.n_units + kUnitChunk - 1) / kUnitChunk;
+    for (uint32_t chunk = blockIdx.x; chunk < n_chunked; chunk += gridDim.x)
+    for (uint32_t u = chunk * kUnitChunk; u < min(a.n_units, (chunk + 1) * kUnitChunk); ++u) {
         const DevUnit un = a.units[u];
-        const uint32_t* mem = a.members + un.layer;
-        const DevLayer l0 = a.layers[mem[0]];
-        const uint32_t G = l0.group_size, cols = l0.cols, Rn = un.nrows, row0 = un.row0;
-        const uint32_t c = (un.cb0 * 32u + lane) * CPL;
-        const bool lane_on = c < cols;
+        const uint32_t Rn = un.nrows, row0 = un.row0;
+        if (un.layer != key_group || un.cb0 != key_cb) {
+            // ---- tables, all threads: per (slot, task) pair the source tensor and the sign bits; per member its slot's
+            //      place in M and its W_0 tensor
+            const uint32_t* mem = a.members + un.layer;
+            const DevLayer l0 = a.layers[mem[0]];
+            G = l0.group_size;
+            cols = l0.cols;
+            c = (un.cb0 * 32u + lane) * CPL;
+            lane_on = c < cols;
+            const uint32_t npairs = G * nt;
+            for (uint32_t p = threadIdx.x; p < npairs; p += kThreadsPerCta) {
+                const uint32_t ms = p / nt, i = p - ms * nt;
+                const uint32_t slot = mem[ms];
+                const uint32_t fl = a.layers[slot].flags;
+                const uint32_t src = (fl & kFlagShuffle) ? a.src_of_slot[static_cast<size_t>(i) * L + slot] : slot;   // sigma_i(l)
+                const void* pw = a.task_ptrs[static_cast<size_t>(i) * L + src];
+                sts_ptrs(s_rec + p * REC + Rec::kPtr, pw, reinterpret_cast<const void*>(static_cast<uintptr_t>(a.layers[src].member)));
+                const DevTask tk = a.tasks[i];
+#pragma unroll
+                for (int h = 0; h < HB; ++h) {
+                    uint4 blk = make_uint4(0, 0, 0, 0);
+                    if (fl & kFlagFlip) blk = philox4x32_10(un.cb0 * HB + h, slot, kTagSign, tk.id, tk.key0, tk.key1);
+                    sts128(s_rec + p * REC + Rec::kBlocks + h * 16, blk);
+                }
+            }
+            for (uint32_t ms = threadIdx.x; ms < G; ms += kThreadsPerCta)
+                sts_ptrs(s_off + ms * 16, reinterpret_cast<const void*>(static_cast<uintptr_t>(a.layers[mem[ms]].m_off)), a.base[mem[ms]]);
+            key_group = un.layer;
+            key_cb = un.cb0;
+            __syncthreads();   // the tables are complete and visible to every warp
+        }
         const uint32_t off0 = row0 * cols + c;           // layers hold < 2^32 elements
 
-        // ---- prologue, all threads: W_0 tiles of every member into the stash ...
+        // ---- W_0 tiles of every member into the stash
         if (lane_on) {
             const uint32_t ntiles = G * Rn;
             for (uint32_t q = warp; q < ntiles; q += kWarpsPerCta) {
                 const uint32_t m = q / Rn, r = q - m * Rn;
-                const char* pb = static_cast<const char*>(a.base[mem[m]]);
+                const char* pb = lds_ptr(s_off + m * 16 + 8);
                 cp_async16(stash + q * kStashTileBytes + lane * 16, pb + static_cast<size_t>(off0 + r * cols) * ES);
             }
         }
         cp_async_commit();
-        // ... and, per (slot, task) pair, the source tensor and the sign bits
-        const uint32_t npairs = G * nt;
-        for (uint32_t p = threadIdx.x; p < npairs; p += kThreadsPerCta) {
-            const uint32_t ms = p / nt, i = p - ms * nt;
-            const uint32_t slot = mem[ms];
-            const uint32_t fl = a.layers[slot].flags;
-            const uint32_t src = (fl & kFlagShuffle) ? a.src_of_slot[static_cast<size_t>(i) * L + slot] : slot;   // sigma_i(l)
-            const void* pw = a.task_ptrs[static_cast<size_t>(i) * L + src];
-            sts_ptrs(s_rec + p * REC + Rec::kPtr, pw, reinterpret_cast<const void*>(static_cast<uintptr_t>(a.layers[src].member)));
-            const DevTask tk = a.tasks[i];
-#pragma unroll
-            for (int h = 0; h < HB; ++h) {
-                uint4 blk = make_uint4(0, 0, 0, 0);
-                if (fl & kFlagFlip) blk = philox4x32_10(un.cb0 * HB + h, slot, kTagSign, tk.id, tk.key0, tk.key1);
-                sts128(s_rec + p * REC + Rec::kBlocks + h * 16, blk);
-            }
-        }
-        for (uint32_t ms = threadIdx.x; ms < G; ms += kThreadsPerCta) sts_u64(s_off + ms * 8, a.layers[mem[ms]].m_off);
         cp_async_wait<0>();
-        __syncthreads();   // stash and tables are complete and visible to every warp
+        __syncthreads();   // the stash is complete and visible to every warp
 
         if (lane_on) {
             const uint32_t n_chunks = (Rn + IR - 1) / IR;
@@ -327,7 +344,7 @@ int launch_compress_groups(int storage_dtype, int m_dtype, const CompressGroupAr
                 cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_group_kernel<ST, MT, NS>, kThreadsPerCta, smem);
                 if (e != cudaSuccess) { (void)cudaGetLastError(); return static_cast<int>(e); }
                 if (per_sm <= 0) return static_cast<int>(cudaErrorInvalidConfiguration);
-                const int grid = static_cast<int>(std::min<uint64_t>(static_cast<uint64_t>(sm_count) * per_sm, a.n_units));
+                const int grid = static_cast<int>(std::min<uint64_t>(static_cast<uint64_t>(sm_count) * per_sm, (a.n_units + kUnitChunk - 1) / kUnitChunk));
                 compress_group_kernel<ST, MT, NS><<<grid, kThreadsPerCta, smem, s>>>(a);
                 return static_cast<int>(cudaGetLastError());
             });

@@ -53,6 +53,7 @@ static_assert(sizeof(DevUnit) == 16, "DevUnit layout");
 // shuffled group: the CTA first stashes the W_0 tiles of all members in shared memory, then its
 // warps sum the tasks' deltas slot by slot, subtracting W_0[sigma_i(l)] from the stash.  `layer`
 // is then the index of the group's first entry in the member table.
+constexpr uint32_t kUnitChunk = 8;                    // group units of one (group, column block) kept adjacent in the unit list
 constexpr uint32_t kStashTileBytes = 512;             // 32 lanes x 16 bytes
 constexpr uint32_t kStashBytes = 48 * 1024;           // fp32 weights
 constexpr uint32_t kItemRows = 4;                     // rows of one slot a warp sums in one go, fp32 weights

@@ -457,7 +457,12 @@ int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* 
     if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (ce != cudaSuccess) return static_cast<int>(ce);
     const uint64_t tiles256 = static_cast<uint64_t>((rows + kBN - 1) / kBN) * ((n_tokens + 2 * kBM - 1) / (2 * kBM));
+#ifdef RANDES_LINEAR_FORCE_HALVES
+    const int halves = (n_tokens > static_cast<uint32_t>(kBM)) ? RANDES_LINEAR_FORCE_HALVES : 1;
+    (void)tiles256;
+#else
     const int halves = (n_tokens > static_cast<uint32_t>(kBM) && tiles256 >= static_cast<uint64_t>(sms)) ? 2 : 1;
+#endif
     CUtensorMap mx, mw, mm;
     if (!make_map(enc, &mx, x, cols, n_tokens, halves * kBM) || !make_map(enc, &mw, w0, cols, rows, kBN) || !make_map(enc, &mm, m_slot, cols, rows, kBN))
         return static_cast<int>(cudaErrorInvalidValue);

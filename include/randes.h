@@ -157,6 +157,17 @@ uint32_t randes_num_tasks(const randes_plan_t* plan);
 int randes_task_list(const randes_plan_t* plan, uint32_t* task_ids, uint64_t* seeds);
 
 /*
+ * Self-check of a plan, on the host (a debugging aid: no compute call needs it).  Verifies what the
+ * kernels take for granted: every task's sigma is a bijection that stays inside its group and
+ * sigma^-1 inverts it (Section 4.3: layers are shuffled among layers of the same type only); the slots
+ * of M are aligned, ordered and disjoint; and each of the plan's tile lists covers every
+ * (row, column block) of every layer exactly once and never leaves a layer -- so every element of M or
+ * of a retrieved model is written by exactly one thread block.  Returns RANDES_OK, or
+ * INVALID_ARGUMENT with randes_last_error() naming the first violation.
+ */
+int randes_plan_validate(const randes_plan_t* plan);
+
+/*
  * Persistence.  What RanDeS keeps per model is a seed (Section 4.1), so a plan
  * is fully described by its layer shapes, group flags, element types and the
  * registered (id, seed) pairs in summation order; M itself is the caller's

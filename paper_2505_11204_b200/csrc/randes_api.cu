@@ -1260,6 +1260,89 @@ int randes_delta_gram(randes_plan_t* plan, const void* const* base, const void* 
     return guarded("randes_delta_gram", [&] { return randes_delta_gram_impl(plan, base, tasks, gram, scratch, scratch_bytes, stream); });
 }
 
+// Self-check of a plan (a debugging aid; nothing in the compute calls depends on it having run).
+static int randes_plan_validate_impl(const randes_plan_t* plan)
+{
+    if (!plan) return fail(RANDES_INVALID_ARGUMENT, "plan is NULL");
+    const uint32_t L = plan->n_layers;
+    // (1) slots of M: aligned, in order, not overlapping, inside the arena
+    size_t end = 0;
+    for (uint32_t l = 0; l < L; ++l) {
+        const size_t off = plan->m_off_bytes[l];
+        if (off % 256 || off < end) return fail(RANDES_INVALID_ARGUMENT, "slot %u of M starts at byte %zu (previous slot ends at %zu)", l, off, end);
+        end = off + static_cast<size_t>(plan->layers[l].rows) * plan->layers[l].cols * elem_size(plan->m_dtype);
+        if (plan->dev_layers[l].m_off * elem_size(plan->m_dtype) != off) return fail(RANDES_INVALID_ARGUMENT, "slot %u: element and byte offsets disagree", l);
+    }
+    if (end > plan->m_bytes) return fail(RANDES_INVALID_ARGUMENT, "M holds %zu bytes but the last slot ends at %zu", plan->m_bytes, end);
+    // (2) every task's sigma is a bijection that stays inside groups (Section 4.3), and sigma^-1 inverts it
+    for (const TaskEntry& t : plan->tasks) {
+        std::vector<char> hit(L, 0);
+        for (uint32_t l = 0; l < L; ++l) {
+            const uint32_t src = t.src_of_slot[l];
+            if (src >= L || hit[src]) return fail(RANDES_INVALID_ARGUMENT, "task %u: sigma is not a bijection at slot %u", t.id, l);
+            hit[src] = 1;
+            if (plan->layers[src].group != plan->layers[l].group) return fail(RANDES_INVALID_ARGUMENT, "task %u: slot %u receives layer %u of another group", t.id, l, src);
+            if (t.slot_of_pos[src] != l) return fail(RANDES_INVALID_ARGUMENT, "task %u: sigma^-1(sigma(%u)) = %u", t.id, l, t.slot_of_pos[src]);
+            if (src != l && !(plan->dev_layers[l].flags & kFlagShuffle)) return fail(RANDES_INVALID_ARGUMENT, "task %u: slot %u moved without the shuffle flag", t.id, l);
+        }
+    }
+    // (3) each unit list tiles every layer exactly once: cells = (row, warp-wide column block)
+    const uint32_t span = cols_per_warp(plan->storage);
+    std::vector<size_t> first(L + 1, 0);
+    for (uint32_t l = 0; l < L; ++l)
+        first[l + 1] = first[l] + static_cast<size_t>(plan->layers[l].rows) * ((plan->layers[l].cols + span - 1) / span);
+    auto check_list = [&](const std::vector<DevUnit>& per_layer, const std::vector<DevUnit>& per_group, const char* name) -> int {
+        std::vector<unsigned char> seen(first[L], 0);
+        auto mark = [&](uint32_t layer, uint32_t row0, uint32_t nrows, uint32_t cb0, uint32_t nbc, size_t index) -> int {
+            if (layer >= L) return fail(RANDES_INVALID_ARGUMENT, "%s unit %zu: layer %u out of range", name, index, layer);
+            const uint32_t rows = plan->layers[layer].rows, nb = (plan->layers[layer].cols + span - 1) / span;
+            if (nrows == 0 || row0 + nrows > rows) return fail(RANDES_INVALID_ARGUMENT, "%s unit %zu: rows [%u, %u) leave layer %u (%u rows)", name, index, row0, row0 + nrows, layer, rows);
+            for (uint32_t cb = cb0; cb < cb0 + nbc; ++cb) {
+                if (cb >= nb) continue;   // a unit may be wider than a ragged layer: the kernels skip those column blocks
+                for (uint32_t r = row0; r < row0 + nrows; ++r) {
+                    unsigned char& cell = seen[first[layer] + static_cast<size_t>(r) * nb + cb];
+                    if (cell) return fail(RANDES_INVALID_ARGUMENT, "%s unit %zu: layer %u row %u column block %u is covered twice", name, index, layer, r, cb);
+                    cell = 1;
+                }
+            }
+            return RANDES_OK;
+        };
+        int rc;
+        for (size_t i = 0; i < per_layer.size(); ++i) {
+            const DevUnit& u = per_layer[i];
+            if (u.nbc == 0 || u.nbc > kWarpsPerCta || (u.nbc & (u.nbc - 1))) return fail(RANDES_INVALID_ARGUMENT, "%s unit %zu: %u column blocks", name, i, u.nbc);
+            if ((rc = mark(u.layer, u.row0, u.nrows, u.cb0, u.nbc, i))) return rc;
+        }
+        for (size_t i = 0; i < per_group.size(); ++i) {
+            const DevUnit& u = per_group[i];
+            if (u.nbc != 0 || u.layer >= plan->member_table.size()) return fail(RANDES_INVALID_ARGUMENT, "%s group unit %zu is malformed", name, i);
+            const uint32_t g = plan->layers[plan->member_table[u.layer]].group;
+            const std::vector<uint32_t>& mem = plan->members[g];
+            if (plan->member_table[u.layer] != mem[0]) return fail(RANDES_INVALID_ARGUMENT, "%s group unit %zu does not start at its group's first member", name, i);
+            if (static_cast<size_t>(mem.size()) * u.nrows * kStashTileBytes > stash_bytes(plan->storage))
+                return fail(RANDES_INVALID_ARGUMENT, "%s group unit %zu: %zu members x %u rows exceed the stash", name, i, mem.size(), u.nrows);
+            for (uint32_t l : mem)
+                if ((rc = mark(l, u.row0, u.nrows, u.cb0, 1, i))) return rc;
+        }
+        for (uint32_t l = 0; l < L; ++l)
+            for (size_t c = first[l]; c < first[l + 1]; ++c)
+                if (!seen[c]) {
+                    const uint32_t nb = (plan->layers[l].cols + span - 1) / span;
+                    return fail(RANDES_INVALID_ARGUMENT, "%s: layer %u row %zu column block %zu is covered by no unit", name, l, (c - first[l]) / nb, (c - first[l]) % nb);
+                }
+        return RANDES_OK;
+    };
+    int rc;
+    if ((rc = check_list(plan->units, {}, "the unit list"))) return rc;
+    if (!plan->group_units.empty() && (rc = check_list(plan->other_units, plan->group_units, "the grouped unit list"))) return rc;
+    return RANDES_OK;
+}
+
+int randes_plan_validate(const randes_plan_t* plan)
+{
+    return guarded("randes_plan_validate", [&] { return randes_plan_validate_impl(plan); });
+}
+
 // Section 3, norm of the interference: || lambda sum_{j != t} T_t^-1 T_j d_j ||^2 = lambda^2 sum_{j,l != t} <T_j d_j, T_l d_l>,
 // because T_t^-1 is orthogonal.
 int randes_interference_norm(const double* gram, uint32_t n, uint32_t t, double lambda, double* norm)

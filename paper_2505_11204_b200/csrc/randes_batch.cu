@@ -163,9 +163,15 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_group_kernel
     uint32_t key_group = 0xFFFFFFFFu, key_cb = 0xFFFFFFFFu;
     uint32_t G = 0, cols = 0, c = 0;
     bool lane_on = false;
-    const uint32_t n_chunked = (a.n_units + kUnitChunk - 1) / kUnitChunk;
-    for (uint32_t chunk = blockIdx.x; chunk < n_chunked; chunk += gridDim.x)
-    for (uint32_t u = chunk * kUnitChunk; u < min(a.n_units, (chunk + 1) * kUnitChunk); ++u) {
+    // Whole rounds of chunks first (round r: CTA b takes chunk r * grid + b); what is left -- fewer than grid chunks --
+    // is dealt out unit by unit, so that the last round is as short as one unit instead of one chunk.
+    const uint32_t chunk_rounds = a.n_units / (kUnitChunk * gridDim.x);
+    const uint32_t chunked_units = chunk_rounds * gridDim.x * kUnitChunk;
+    const uint32_t my_chunked = chunk_rounds * kUnitChunk;
+    const uint32_t my_units = my_chunked + (a.n_units - chunked_units > blockIdx.x ? (a.n_units - chunked_units - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u);
+    for (uint32_t t = 0; t < my_units; ++t) {
+        const uint32_t u = t < my_chunked ? ((t / kUnitChunk) * gridDim.x + blockIdx.x) * kUnitChunk + t % kUnitChunk
+                                          : chunked_units + blockIdx.x + (t - my_chunked) * gridDim.x;
         const DevUnit un = a.units[u];
         const uint32_t Rn = un.nrows;
         if (un.layer != key_group || un.cb0 != key_cb) {
@@ -307,8 +313,7 @@ int launch_retrieve_batch_groups(int out_dtype, const RetrieveBatchArgs& a, uint
         if (e != cudaSuccess) { (void)cudaGetLastError(); return static_cast<int>(e); }
         if (per_sm <= 0) return static_cast<int>(cudaErrorInvalidConfiguration);
         const uint64_t want = static_cast<uint64_t>(sm_count) * per_sm;
-        const uint64_t chunks = (a.n_units + kUnitChunk - 1) / kUnitChunk;
-        const int grid = static_cast<int>(want < chunks ? want : chunks);
+        const int grid = static_cast<int>(want < a.n_units ? want : a.n_units);
         retrieve_batch_group_kernel<OT><<<grid, kThreadsPerCta, smem, s>>>(a);
         return static_cast<int>(cudaGetLastError());
     });

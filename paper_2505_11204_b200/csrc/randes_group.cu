@@ -137,14 +137,20 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
     const uint32_t one = 0x3F800000u;
 
     // The unit list keeps kUnitChunk units of one (group, column block) next to each other (consecutive blocks of
-    // rows), and a CTA takes whole chunks: the tables below depend on the group, the column block and the tasks only,
+    // rows), and a CTA takes whole chunks (see the loop): the tables below depend on the group, the column block and the tasks only,
     // so they are built once per chunk and every further unit of the chunk just refills the stash.
     uint32_t key_group = 0xFFFFFFFFu, key_cb = 0xFFFFFFFFu;
     uint32_t G = 0, cols = 0, c = 0;
     bool lane_on = false;
-    const uint32_t n_chunked = (a.n_units + kUnitChunk - 1) / kUnitChunk;
-    for (uint32_t chunk = blockIdx.x; chunk < n_chunked; chunk += gridDim.x)
-    for (uint32_t u = chunk * kUnitChunk; u < min(a.n_units, (chunk + 1) * kUnitChunk); ++u) {
+    // Whole rounds of chunks first (round r: CTA b takes chunk r * grid + b); what is left -- fewer than grid chunks --
+    // is dealt out unit by unit, so that the last round is as short as one unit instead of one chunk.
+    const uint32_t chunk_rounds = a.n_units / (kUnitChunk * gridDim.x);
+    const uint32_t chunked_units = chunk_rounds * gridDim.x * kUnitChunk;
+    const uint32_t my_chunked = chunk_rounds * kUnitChunk;
+    const uint32_t my_units = my_chunked + (a.n_units - chunked_units > blockIdx.x ? (a.n_units - chunked_units - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u);
+    for (uint32_t t = 0; t < my_units; ++t) {
+        const uint32_t u = t < my_chunked ? ((t / kUnitChunk) * gridDim.x + blockIdx.x) * kUnitChunk + t % kUnitChunk
+                                          : chunked_units + blockIdx.x + (t - my_chunked) * gridDim.x;
         const DevUnit un = a.units[u];
         const uint32_t Rn = un.nrows, row0 = un.row0;
         if (un.layer != key_group || un.cb0 != key_cb) {
@@ -344,7 +350,7 @@ int launch_compress_groups(int storage_dtype, int m_dtype, const CompressGroupAr
                 cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_group_kernel<ST, MT, NS>, kThreadsPerCta, smem);
                 if (e != cudaSuccess) { (void)cudaGetLastError(); return static_cast<int>(e); }
                 if (per_sm <= 0) return static_cast<int>(cudaErrorInvalidConfiguration);
-                const int grid = static_cast<int>(std::min<uint64_t>(static_cast<uint64_t>(sm_count) * per_sm, (a.n_units + kUnitChunk - 1) / kUnitChunk));
+                const int grid = static_cast<int>(std::min<uint64_t>(static_cast<uint64_t>(sm_count) * per_sm, a.n_units));
                 compress_group_kernel<ST, MT, NS><<<grid, kThreadsPerCta, smem, s>>>(a);
                 return static_cast<int>(cudaGetLastError());
             });

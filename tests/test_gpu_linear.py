@@ -130,7 +130,7 @@ def test_linear_without_flip_and_without_shuffle():
 
 
 def test_linear_blocks_of_256_tokens():
-    # enough tiles (16 feature tiles x 10 blocks of 256 tokens >= the SM count) for the 256-token CTA, whose second
+    # enough tiles (16 feature tiles x 10 blocks of 256 tokens: two waves, against three of the 128-token shape) for the 256-token CTA, whose second
     # block of 128 tokens has accumulators of its own; ragged token count, ragged last k-step, bf16 and fp32 output
     w = _workload([(2048, 136, 2)], [S | F], n_tasks=2)
     _run(w, [2500], layers=[0])
@@ -158,9 +158,11 @@ def _dyadic_bits(rng, shape, kmax=8):
 
 
 def _uses_256_token_blocks(rows, n_tok):
-    """The library's choice of CTA shape: 256 tokens per CTA once that still gives every SM a tile."""
+    """The library's choice of CTA shape: a 128-token tile costs about 3/4 of a 256-token tile; the shape with the lower
+    (number of waves over the SMs) x (cost of a tile) wins, 256 tokens on a tie."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    return n_tok > 128 and ((rows + 127) // 128) * ((n_tok + 255) // 256) >= sms
+    waves = lambda tokens_per_tile: -(-(((rows + 127) // 128) * ((n_tok + tokens_per_tile - 1) // tokens_per_tile)) // sms)
+    return n_tok > 128 and waves(256) * 4 <= waves(128) * 3
 
 
 def _run_dyadic(shape, gflag, n_tok, sample_tokens, want_256, lam=0.25, members=2):

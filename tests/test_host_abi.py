@@ -246,6 +246,40 @@ def test_outputs_that_overlap_an_input_or_each_other_are_refused():
     plan.close()
 
 
+def test_every_plan_passes_its_self_check():
+    """randes_plan_validate: permutations are bijections inside groups, slots of M are disjoint, and every tile
+    list covers every (row, column block) of every layer exactly once -- on the five paper-shaped sets in both
+    storage types, with the skip / shift / Gaussian-context variants, and on ragged random shapes."""
+    S, F = randes.SHUFFLE, randes.FLIP
+    for make in (wl.toy, wl.vit_b32, wl.gpt2_small, wl.flan_t5_base, wl.vit_l14):
+        for storage in (wl.F32, wl.BF16):
+            for m_dtype in (wl.F32, wl.BF16):
+                w = make().with_storage(storage)
+                p = randes.Plan.from_workload(w, host_only=True, m_dtype=m_dtype)
+                randes.randes_plan_validate(p.handle)
+                p.close()
+    w = wl.vit_b32()
+    for variant in (lambda f: f | randes.SKIP(2), lambda f: (f & ~S) | randes.SHIFT if f & S else f,
+                    lambda f: (f & ~F) | randes.GAUSS if f & F else f):
+        p = randes.Plan(w.rows, w.cols, w.group, [variant(f) for f in w.gflags], task_ids=[0, 5], seeds=[1, 2], host_only=True)
+        randes.randes_plan_validate(p.handle)
+        p.close()
+    rng = np.random.default_rng(3)
+    for _ in range(40):
+        n_groups = int(rng.integers(1, 5))
+        rows, cols, group = [], [], []
+        for g in range(n_groups):
+            r, c, n = int(rng.integers(1, 300)), int(rng.integers(1, 2100)), int(rng.integers(1, 30))
+            rows += [r] * n; cols += [c] * n; group += [g] * n
+        order = rng.permutation(len(rows))
+        rows, cols, group = [rows[i] for i in order], [cols[i] for i in order], [group[i] for i in order]
+        flags = [int(rng.choice([0, S, F, S | F])) for _ in range(n_groups)]
+        p = randes.Plan(rows, cols, group, flags, storage=int(rng.integers(0, 2)), task_ids=[3, 9, 4], seeds=[7, 8, 9], host_only=True)
+        randes.randes_plan_validate(p.handle)
+        p.close()
+    assert randes.lib().randes_plan_validate(None) == randes.INVALID_ARGUMENT
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(randes, "_lib", None)
     monkeypatch.setattr(randes, "LIB_PATH", str(tmp_path / "absent.so"))

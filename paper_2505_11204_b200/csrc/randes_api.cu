@@ -191,7 +191,7 @@ void build_units(const randes_layer_t* layers, uint32_t n_layers, int storage, s
 // Could group g (of `size` members, `cols` wide) be cut into group units at all?
 bool group_fits_stash(size_t size, uint32_t cols, int storage)
 {
-    return size >= 2 && cols % cols_per_lane(storage) == 0 && group_unit_rows(static_cast<uint32_t>(size), storage) >= 1;
+    return size >= 1 && cols % cols_per_lane(storage) == 0 && group_unit_rows(static_cast<uint32_t>(size), storage) >= 1;
 }
 
 // Upper bound of the length of a unit list in which any subset of the groups is staged.
@@ -659,9 +659,13 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
                 if (mem.empty() || !group_fits_stash(mem.size(), layers[mem[0]].cols, p->storage)) continue;
                 bool shuffled = false;
                 for (uint32_t l : mem) shuffled = shuffled || (p->dev_layers[l].flags & kFlagShuffle);
-                p->group_staged[g] = shuffled;
-                any = any || shuffled;
-                if (shuffled) p->max_staged_group = std::max<uint32_t>(p->max_staged_group, static_cast<uint32_t>(mem.size()));
+                // bf16 weights: the group kernel decodes a task's signs once per three rows and is the faster one
+                // even without a shuffle, so the large unrepeated matrices (embeddings) go through it too
+                const bool large_single = p->storage == RANDES_BF16 && mem.size() == 1 && layers[mem[0]].rows >= 256;
+                const bool stage = shuffled || large_single;
+                p->group_staged[g] = stage;
+                any = any || stage;
+                if (stage) p->max_staged_group = std::max<uint32_t>(p->max_staged_group, static_cast<uint32_t>(mem.size()));
             }
             if (any && !p->has_gauss) {
                 build_units(layers, n_layers, p->storage, p->group_units, &p->group_staged, &member_base, kStagedGroups);

@@ -67,7 +67,9 @@ constexpr uint32_t group_unit_rows(uint32_t G, int storage_dtype)
 {
     const uint32_t ir = item_rows(storage_dtype);
     const uint32_t fit = G ? stash_bytes(storage_dtype) / kStashTileBytes / G : 0;
-    return fit >= 4 * ir ? 4 * ir : (fit >= ir ? fit / ir * ir : fit);
+    // four items per member, and at least one item for each of the CTA's warps (a group of one member: eight items)
+    const uint32_t items = G && (static_cast<uint32_t>(kWarpsPerCta) + G - 1) / G > 4u ? (static_cast<uint32_t>(kWarpsPerCta) + G - 1) / G : 4u;
+    return fit >= items * ir ? items * ir : (fit >= ir ? fit / ir * ir : fit);
 }
 
 struct DevTask {

@@ -662,6 +662,34 @@ def run_ours(args):
                                 "GBps": byts / (ms * 1e-3) / 1e9, "frac_of_%s_peak" % peak_kind: byts / (ms * 1e-3) / 1e9 / peak,
                                 "speedup_per_model_vs_add": ops["add"]["ms_per_call"] / (ms / n_swap)}
 
+    # ---- interference diagnostics: the Gram matrix of the K transformed deltas (one pass over all K + 1 models), timed alone
+    if K <= 32:
+        try:
+            gram = torch.empty(K, K, dtype=torch.float64, device=dev)
+            g_bytes = randes.randes_delta_gram_scratch_bytes(plan.handle)
+            g_scratch = torch.empty(g_bytes // 8, dtype=torch.float64, device=dev)
+            spans = []
+            for rep in range(1 + 3):
+                a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                randes.randes_delta_gram(plan.handle, p_base, p_tasks, gram, g_scratch, g_bytes, sh)
+                z.record(stream)
+                if rep >= 1:
+                    spans.append((a, z))
+            barrier()
+            ms = max_over_ranks([sum(a.elapsed_time(z) for a, z in spans) / len(spans)], world, dev)[0]
+            s_el = 2 if w.storage == wl.BF16 else 4
+            byts = (K + 1) * s_el * w.n_params
+            cos, mean_cos = randes.randes_pairwise_cosines(gram)
+            extras["delta_gram"] = {"tasks": K, "ms_per_call": ms, "GBps": byts / (ms * 1e-3) / 1e9,
+                                    "frac_of_%s_peak" % peak_kind: byts / (ms * 1e-3) / 1e9 / peak,
+                                    "mean_pairwise_cosine_after_transform": mean_cos,
+                                    "interference_norm_task0": randes.randes_interference_norm(gram, 0, w.lam),
+                                    "note": "fp64 tensor-core products (mma.m8n8k4), bound by the fp64 pipe; the synthetic deltas have cosine 0.25 before the transforms"}
+            del gram, g_scratch
+        except torch.OutOfMemoryError:
+            extras["delta_gram"] = None
+
     # ---- adapter deltas (Section 5.8): the tasks' tensors already hold the deltas (base = NULL), only the layers that carry
     #      an adapter are in the plan; rank-16 deltas materialised beforehand, here random values of that shape
     if args.workload == "flan_t5_base":

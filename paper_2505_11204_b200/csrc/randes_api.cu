@@ -659,9 +659,11 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
                 if (mem.empty() || !group_fits_stash(mem.size(), layers[mem[0]].cols, p->storage)) continue;
                 bool shuffled = false;
                 for (uint32_t l : mem) shuffled = shuffled || (p->dev_layers[l].flags & kFlagShuffle);
-                // bf16 weights: the group kernel decodes a task's signs once per three rows and is the faster one
-                // even without a shuffle, so the large unrepeated matrices (embeddings) go through it too
-                const bool large_single = p->storage == RANDES_BF16 && mem.size() == 1 && layers[mem[0]].rows >= 256;
+                // bf16 weights and many tasks: the group kernel decodes a task's signs once per three rows and is the faster
+                // one even without a shuffle, so the large unrepeated matrices go through it too.  With few tasks a warp's
+                // pipeline over one member's rows is too short to fill (measured: slower at 7 tasks, faster at 20), so
+                // the choice follows the number of tasks registered when the plan is built.
+                const bool large_single = p->storage == RANDES_BF16 && mem.size() == 1 && layers[mem[0]].rows >= 256 && n_tasks >= 16;
                 const bool stage = shuffled || large_single;
                 p->group_staged[g] = stage;
                 any = any || stage;

@@ -148,10 +148,12 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
     const uint32_t chunked_units = chunk_rounds * gridDim.x * kUnitChunk;
     const uint32_t my_chunked = chunk_rounds * kUnitChunk;
     const uint32_t my_units = my_chunked + (a.n_units - chunked_units > blockIdx.x ? (a.n_units - chunked_units - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u);
+    auto unit_at = [&](uint32_t t) {
+        return t < my_chunked ? ((t / kUnitChunk) * gridDim.x + blockIdx.x) * kUnitChunk + t % kUnitChunk
+                              : chunked_units + blockIdx.x + (t - my_chunked) * gridDim.x;
+    };
     for (uint32_t t = 0; t < my_units; ++t) {
-        const uint32_t u = t < my_chunked ? ((t / kUnitChunk) * gridDim.x + blockIdx.x) * kUnitChunk + t % kUnitChunk
-                                          : chunked_units + blockIdx.x + (t - my_chunked) * gridDim.x;
-        const DevUnit un = a.units[u];
+        const DevUnit un = a.units[unit_at(t)];
         const uint32_t Rn = un.nrows, row0 = un.row0;
         if (un.layer != key_group || un.cb0 != key_cb) {
             // ---- tables, all threads: per (slot, task) pair the source tensor and the sign bits; per member its slot's

@@ -131,19 +131,14 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
 // Batched retrieve of a shuffled group, fp32 weights and superposition.  Task b needs, for layer
 // position p, the slot M[sigma_b^-1(p)]: every slot of the group is wanted by several tasks.  A
 // CTA takes a group unit (a few rows x one warp-wide column block of every member), copies the M
-// tiles of all slots and the W_0 tiles of all positions into shared memory, and resolves one
-// record per (position, task) -- output tensor, which member the wanted slot is, Philox block of
-// sign bits -- in parallel over its threads.  After that the row loop only reads shared memory
+// tiles of all slots and the W_0 tiles of all positions into shared memory once, and resolves
+// one record per (position, task) -- output tensor, which member the wanted slot is, Philox block
+// of sign bits -- in parallel over its threads.  After that the row loop only reads shared memory
 // and streams 16-byte stores: the call is bound by HBM writes, as it should be.
-//
-// The two stashes are double-buffered by halves: a unit is walked in steps of as many rows as fit
-// half a stash, and while the rows of one step are written the tiles of the next step -- of the
-// same unit, or of the CTA's next unit when it belongs to the same group -- are already on their
-// way into the other half.  (With one buffer per stash every unit began with a wait for 96 KiB.)
+// (Measured against this form and slower by 1 - 4 %: tables built once per chunk of units of one column block;
+// the next unit's tiles prefetched into L2 during the row loop; stashes double-buffered by halves with the next
+// step's tiles in flight while a step is written.  What limits the kernel is the stream of stores itself.)
 constexpr uint32_t kBatchRecBytes = 32;   // {out pointer, slot member, pad, Philox block}
-constexpr uint32_t kHalfStash = kStashBytes / 2;
-constexpr uint32_t kBatchMaxGroup = kHalfStash / kStashTileBytes;      // members whose tiles fit half a stash at one row each
-constexpr uint32_t kBatchMemberBytes = kBatchMaxGroup * 16;            // per member: {its slot of M, its W_0 tensor}
 
 __device__ __forceinline__ void store_plain(float* p, const float (&y)[4])
 {
@@ -161,51 +156,29 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_group_kernel
     extern __shared__ __align__(16) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_s = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
-    const uint32_t m_stash = smem_s, w_stash = smem_s + kStashBytes, s_mem = smem_s + 2 * kStashBytes, s_rec = s_mem + kBatchMemberBytes;
+    const uint32_t m_stash = smem_s, w_stash = smem_s + kStashBytes, s_rec = smem_s + 2 * kStashBytes;
     const uint32_t L = a.n_layers, n = a.n_tasks;
     const uint32_t sign_word = 16 + (lane >> 3) * 4u, sign_shift = (lane & 7) * 4u;
-    uint32_t key_group = 0xFFFFFFFFu, G = 0, cols = 0, cap = 1;
-    uint32_t buf = 0;          // the half of the stashes that holds (or is receiving) the step about to be written
-    bool filled = false;       // the first step of the current unit was issued during the previous unit
-
-    // rows [row, row + nr) x column block cb of every member -> half `b` of both stashes (this thread's share)
-    auto fill = [&](uint32_t b, uint32_t row, uint32_t nr, uint32_t cb) {
-        const uint32_t c = (cb * 32u + lane) * CPL;
-        if (c >= cols) return;
-        const uint32_t ntiles = G * nr;
-        for (uint32_t q = warp; q < ntiles; q += kWarpsPerCta) {
-            const uint32_t m = q / nr, r = q - m * nr;
-            const uint32_t off = (row + r) * cols + c;          // layers hold < 2^32 elements
-            cp_async16(m_stash + b * kHalfStash + q * kStashTileBytes + lane * 16, reinterpret_cast<const float*>(lds_ptr(s_mem + m * 16)) + off);
-            cp_async16(w_stash + b * kHalfStash + q * kStashTileBytes + lane * 16, reinterpret_cast<const float*>(lds_ptr(s_mem + m * 16 + 8)) + off);
-        }
-    };
-
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
-        const bool more = u + gridDim.x < a.n_units;
-        DevUnit nx = un;
-        if (more) nx = a.units[u + gridDim.x];
         const uint32_t* mem = a.members + un.layer;
-        if (un.layer != key_group) {
-            // another group: its member table (never with a copy in flight: copies ahead are issued within a group only)
-            const DevLayer l0 = a.layers[mem[0]];
-            G = l0.group_size;
-            cols = l0.cols;
-            cap = kHalfStash / (G * kStashTileBytes);            // rows of a step
-            for (uint32_t m = threadIdx.x; m < G; m += kThreadsPerCta)
-                sts_ptrs(s_mem + m * 16, static_cast<const float*>(a.M) + a.layers[mem[m]].m_off, a.base[mem[m]]);
-            key_group = un.layer;
-            __syncthreads();
-        }
-        const uint32_t Rn = un.nrows;
+        const DevLayer l0 = a.layers[mem[0]];
+        const uint32_t G = l0.group_size, cols = l0.cols, Rn = un.nrows;
         const uint32_t c = (un.cb0 * 32u + lane) * CPL;
         const bool lane_on = c < cols;
-        if (!filled) {
-            fill(buf, un.row0, min(cap, Rn), un.cb0);
-            cp_async_commit();
+        const uint32_t off0 = un.row0 * cols + c;          // layers hold < 2^32 elements
+
+        if (lane_on) {
+            const uint32_t ntiles = G * Rn;
+            for (uint32_t q = warp; q < ntiles; q += kWarpsPerCta) {
+                const uint32_t m = q / Rn, r = q - m * Rn;
+                const uint32_t layer = mem[m];
+                const uint32_t off = off0 + r * cols;
+                cp_async16(m_stash + q * kStashTileBytes + lane * 16, static_cast<const float*>(a.M) + a.layers[layer].m_off + off);
+                cp_async16(w_stash + q * kStashTileBytes + lane * 16, static_cast<const float*>(a.base[layer]) + off);
+            }
         }
-        // one record per (position, task), while the first tiles are on their way
+        cp_async_commit();
         const uint32_t npairs = G * n;
         for (uint32_t p = threadIdx.x; p < npairs; p += kThreadsPerCta) {
             const uint32_t mp = p / n, b = p - mp * n;
@@ -222,63 +195,48 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_group_kernel
             }
             sts128(s_rec + p * kBatchRecBytes + 16, blk);
         }
-        filled = false;
-        for (uint32_t s0 = 0; s0 < Rn; s0 += cap) {
-            const uint32_t nr = min(cap, Rn - s0);
-            // the next step's tiles into the other half: of this unit, or of the CTA's next unit in the same group
-            if (s0 + cap < Rn) {
-                fill(buf ^ 1u, un.row0 + s0 + cap, min(cap, Rn - s0 - cap), un.cb0);
-            } else if (more && nx.layer == key_group) {
-                fill(buf ^ 1u, nx.row0, min(cap, nx.nrows), nx.cb0);
-                filled = true;
-            }
-            cp_async_commit();            // (possibly an empty group: the count below stays the same)
-            cp_async_wait<1>();           // all but the newest group: this step's tiles have landed
-            __syncthreads();              // tiles (and, at the first step, the records) are visible to every warp
+        cp_async_wait<0>();
+        __syncthreads();   // stashes and records are complete and visible to every warp
 
-            if (lane_on) {
-                const uint32_t mb0 = m_stash + buf * kHalfStash + lane * 16, wb0 = w_stash + buf * kHalfStash + lane * 16;
-                const uint32_t n_chunks = (nr + kItemRows - 1) / kItemRows;
-                const uint32_t n_items = G * n_chunks;
-                for (uint32_t item = warp; item < n_items; item += kWarpsPerCta) {
-                    const uint32_t mp = item / n_chunks;
-                    const uint32_t r0 = (item - mp * n_chunks) * kItemRows;
-                    const uint32_t rows_here = min(kItemRows, nr - r0);
-                    float wv[kItemRows][CPL];
+        if (lane_on) {
+            const uint32_t n_chunks = (Rn + kItemRows - 1) / kItemRows;
+            const uint32_t n_items = G * n_chunks;
+            for (uint32_t item = warp; item < n_items; item += kWarpsPerCta) {
+                const uint32_t mp = item / n_chunks;
+                const uint32_t r0 = (item - mp * n_chunks) * kItemRows;
+                const uint32_t nr = min(kItemRows, Rn - r0);
+                float wv[kItemRows][CPL];
 #pragma unroll
-                    for (int r = 0; r < static_cast<int>(kItemRows); ++r)
-                        if (r < static_cast<int>(rows_here)) Store<float>::widen(lds128(wb0 + (mp * nr + r0 + r) * kStashTileBytes), wv[r]);
-                    const uint32_t off = (un.row0 + s0 + r0) * cols + c;
-                    uint32_t rec = s_rec + mp * n * kBatchRecBytes;
-                    for (uint32_t b = 0; b < n; ++b, rec += kBatchRecBytes) {
-                        OT* op = reinterpret_cast<OT*>(const_cast<char*>(lds_ptr(rec))) + off;
-                        const uint32_t member = lds_u32(rec + 8);
-                        const uint32_t bits = lds_u32(rec + sign_word) >> sign_shift;
-                        float lam[CPL];
+                for (int r = 0; r < static_cast<int>(kItemRows); ++r)
+                    if (r < static_cast<int>(nr)) Store<float>::widen(lds128(w_stash + (mp * Rn + r0 + r) * kStashTileBytes + lane * 16), wv[r]);
+                const uint32_t off = off0 + r0 * cols;
+                uint32_t rec = s_rec + mp * n * kBatchRecBytes;
+                for (uint32_t b = 0; b < n; ++b, rec += kBatchRecBytes) {
+                    OT* op = reinterpret_cast<OT*>(const_cast<char*>(lds_ptr(rec))) + off;
+                    const uint32_t member = lds_u32(rec + 8);
+                    const uint32_t bits = lds_u32(rec + sign_word) >> sign_shift;
+                    float lam[CPL];
 #pragma unroll
-                        for (int e = 0; e < CPL; ++e) lam[e] = flip(a.lambda, ((bits >> e) & 1u) << 31);
-                        const uint32_t mb = mb0 + (member * nr + r0) * kStashTileBytes;
+                    for (int e = 0; e < CPL; ++e) lam[e] = flip(a.lambda, ((bits >> e) & 1u) << 31);
+                    const uint32_t mb = m_stash + (member * Rn + r0) * kStashTileBytes + lane * 16;
 #pragma unroll
-                        for (int r = 0; r < static_cast<int>(kItemRows); ++r) {
-                            if (r < static_cast<int>(rows_here)) {
-                                float m[CPL], y[CPL];
-                                Store<float>::widen(lds128(mb + r * kStashTileBytes), m);
+                    for (int r = 0; r < static_cast<int>(kItemRows); ++r) {
+                        if (r < static_cast<int>(nr)) {
+                            float m[CPL], y[CPL];
+                            Store<float>::widen(lds128(mb + r * kStashTileBytes), m);
 #pragma unroll
-                                for (int e = 0; e < CPL; ++e) y[e] = __fmaf_rn(lam[e], m[e], wv[r][e]);
-                                store_plain(op + static_cast<size_t>(r) * cols, y);
-                            }
+                            for (int e = 0; e < CPL; ++e) y[e] = __fmaf_rn(lam[e], m[e], wv[r][e]);
+                            store_plain(op + static_cast<size_t>(r) * cols, y);
                         }
                     }
                 }
             }
-            __syncthreads();   // every warp is done with this half (and, after the last step, with the records)
-            buf ^= 1u;
         }
+        __syncthreads();   // every warp is done with the stashes and records before the next unit overwrites them
     }
-    cp_async_wait<0>();
 }
 
-size_t batch_group_smem(uint32_t pairs) { return 2 * static_cast<size_t>(kStashBytes) + kBatchMemberBytes + static_cast<size_t>(pairs) * kBatchRecBytes; }
+size_t batch_group_smem(uint32_t pairs) { return 2 * static_cast<size_t>(kStashBytes) + static_cast<size_t>(pairs) * kBatchRecBytes; }
 
 template <typename K> int occupancy(K kernel)
 {
@@ -320,7 +278,7 @@ int retrieve_batch_group_prepare()
 
 bool retrieve_batch_group_fits(uint32_t max_group, uint32_t n_tasks)
 {
-    return max_group >= 1 && max_group <= kBatchMaxGroup && batch_group_smem(max_group * n_tasks) <= 227 * 1024;
+    return max_group >= 1 && max_group * kStashTileBytes <= kStashBytes && batch_group_smem(max_group * n_tasks) <= 227 * 1024;
 }
 
 int launch_retrieve_batch_groups(int out_dtype, const RetrieveBatchArgs& a, uint32_t max_group, int sm_count, void* stream)

@@ -16,7 +16,9 @@
 // items: stage = one task x two rows (fp32 weights, items of four rows) or one task x three rows
 // (bf16 weights, items of three rows: the sign decode is shared by more rows).  Sums run in task order, every output
 // element is written by one thread: results are bit-reproducible and equal to the per-layer
-// kernel's.
+// kernel's.  (Measured and not kept: the W_0 tiles of the CTA's next unit prefetched into L2 during the
+// row loop -- slower by 3 - 5 %; the warps' copy pipelines running on across unit boundaries, with
+// the first stages of the next unit in flight during the barrier and the stash refill -- no gain.)
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -108,18 +110,6 @@ __device__ __forceinline__ void cursor_next(Cursor& c, uint32_t n_chunks, uint32
     }
 }
 
-// stages (one task x SR rows) of warp `warp` in a unit of G members x Rn rows: it takes the items warp, warp + 8, ...
-template <uint32_t IR, uint32_t SR>
-__device__ __forceinline__ uint32_t warp_stages(uint32_t warp, uint32_t G, uint32_t n_chunks, uint32_t Rn, uint32_t nt)
-{
-    uint32_t N = 0;
-    for (uint32_t item = warp; item < G * n_chunks; item += kWarpsPerCta) {
-        const uint32_t chunk = item % n_chunks;
-        N += (min(IR, Rn - chunk * IR) + SR - 1) / SR * nt;
-    }
-    return N;
-}
-
 template <typename ST, typename MT, int NSTAGE>
 __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const CompressGroupArgs a)
 {
@@ -154,11 +144,6 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
     uint32_t key_group = 0xFFFFFFFFu, key_cb = 0xFFFFFFFFu;
     uint32_t G = 0, cols = 0, c = 0;
     bool lane_on = false;
-    // this thread's ring of stages: where the next copy goes, where the next stage is read, how many stages of the
-    // coming unit are already in it, and the issue cursor that goes with them
-    uint32_t stage_i = ring, stage_c = ring, pre = 0;
-    Cursor ci;
-    ci.rec = ci.rec_begin = ci.rec_end = ci.off = ci.row = ci.rows_left = ci.item = ci.m_off = 0;
     // Whole rounds of chunks first (round r: CTA b takes chunk r * grid + b); what is left -- fewer than grid chunks --
     // is dealt out unit by unit, so that the last round is as short as one unit instead of one chunk.
     const uint32_t chunk_rounds = a.n_units / (kUnitChunk * gridDim.x);
@@ -220,57 +205,39 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
 
         if (lane_on) {
             const uint32_t n_chunks = (Rn + IR - 1) / IR;
-            const uint32_t N = warp_stages<IR, SR>(warp, G, n_chunks, Rn, nt);   // stages of this warp
-            // The warp's pipeline runs on across the end of a unit: once the last stage of this unit has been issued,
-            // the first stages of the CTA's next unit follow (when it belongs to the same chunk, so that the records
-            // still apply; each lane copies into its own ring slots, which no barrier protects or needs to).  They are
-            // in flight during the barrier and the refill of the stash, so the next unit starts with a full pipeline.
-            uint32_t Rn1 = 0, off1 = 0, n_chunks1 = 1, N1 = 0;
-            if (t + 1 < my_units) {
-                const DevUnit nx = a.units[unit_at(t + 1)];
-                if (nx.layer == key_group && nx.cb0 == key_cb) {
-                    Rn1 = nx.nrows;
-                    off1 = nx.row0 * cols + c;
-                    n_chunks1 = (Rn1 + IR - 1) / IR;
-                    N1 = warp_stages<IR, SR>(warp, G, n_chunks1, Rn1, nt);
-                }
+            const uint32_t n_items = G * n_chunks;
+            uint32_t N = 0;   // stages of this warp
+            for (uint32_t item = warp; item < n_items; item += kWarpsPerCta) {
+                const uint32_t chunk = item % n_chunks;
+                N += (min(IR, Rn - chunk * IR) + SR - 1) / SR * nt;
             }
-            Cursor cc;
-            cursor_set<REC, IR>(cc, warp, n_chunks, Rn, nt, s_rec, off0, cols);
-            if (pre == 0) ci = cc;                      // else: the issue cursor is `pre` stages into this unit already
-            Cursor cn;
-            cursor_set<REC, IR>(cn, warp, n_chunks1, Rn1, nt, s_rec, off1, cols);
-            uint32_t to_issue = N - pre, pre1 = 0;
+            Cursor ci, cc;
+            cursor_set<REC, IR>(ci, warp, n_chunks, Rn, nt, s_rec, off0, cols);
+            cc = ci;
+            uint32_t to_issue = N, stage_i = ring, stage_c = ring;
             const uint32_t stash_lane = stash + lane * 16;
             const uint32_t member_bytes = Rn * kStashTileBytes;
             const size_t row_bytes = static_cast<size_t>(cols) * ES;
 
-            auto copy_stage = [&](Cursor& cur, uint32_t nch, uint32_t rn, uint32_t o0) {
-                const char* src = lds_ptr(cur.rec + Rec::kPtr) + static_cast<size_t>(cur.off) * ES;
+            auto issue = [&]() {
+                const char* src = lds_ptr(ci.rec + Rec::kPtr) + static_cast<size_t>(ci.off) * ES;
 #pragma unroll
                 for (uint32_t r = 0; r < SR; ++r)
-                    if (r == 0 || cur.rows_left > r) cp_async16(stage_i + r * kSlotBytes, src + r * row_bytes);
-                cursor_next<REC, IR, SR>(cur, nch, rn, nt, s_rec, o0, cols);
+                    if (r == 0 || ci.rows_left > r) cp_async16(stage_i + r * kSlotBytes, src + r * row_bytes);
+                cursor_next<REC, IR, SR>(ci, n_chunks, Rn, nt, s_rec, off0, cols);
                 stage_i += kStageBytes;
                 if (stage_i == ring_end) stage_i = ring;
-            };
-            auto issue = [&]() {
-                if (to_issue) {
-                    copy_stage(ci, n_chunks, Rn, off0);
-                    --to_issue;
-                } else if (pre1 < N1) {
-                    copy_stage(cn, n_chunks1, Rn1, off1);
-                    ++pre1;
-                }
+                --to_issue;
             };
 
-            for (uint32_t s = pre; s < static_cast<uint32_t>(NSTAGE - 1); ++s) {
-                issue();
+#pragma unroll
+            for (int s = 0; s < NSTAGE - 1; ++s) {
+                if (to_issue) issue();
                 cp_async_commit();
             }
             f32x2 acc[SR][CPL / 2];
             for (uint32_t it = 0; it < N; ++it) {
-                issue();
+                if (to_issue) issue();
                 cp_async_commit();
                 cp_async_wait<NSTAGE - 1>();   // all but the newest NSTAGE-1 groups have landed: stage_c is ready
                 if (cc.rec == cc.rec_begin) {
@@ -313,13 +280,10 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
                 stage_c += kStageBytes;
                 if (stage_c == ring_end) stage_c = ring;
             }
-            // what was issued beyond this unit belongs to the next one (the wait of its stash fill completes it)
-            pre = pre1;
-            ci = cn;
+            cp_async_wait<0>();
         }
         __syncthreads();   // every warp is done with the stash and the tables before the next unit overwrites them
     }
-    cp_async_wait<0>();
 }
 
 template <typename T> struct Tag { typedef T type; };

@@ -107,10 +107,11 @@ def test_static_retrieve_refuses_models_beyond_its_scratch():
     # The check happens on the host before anything is launched, so this needs no GPU.
     n = 12
     plan = randes.Plan([100_000] * n, [1024] * n, [0] * n, [S | F], task_ids=[0], seeds=[1], host_only=True)
-    fake = (ctypes.c_void_p * n)(*[4096 * (i + 1) for i in range(n)])
-    fake_out = (ctypes.c_void_p * n)(*[4096 * (i + 100) for i in range(n)])
+    # (addresses only, a GiB apart so that the 410 MB tensors do not overlap: nothing is ever dereferenced)
+    fake = (ctypes.c_void_p * n)(*[(i + 1) << 30 for i in range(n)])
+    fake_out = (ctypes.c_void_p * n)(*[(i + 100) << 30 for i in range(n)])
     with pytest.raises(randes.RandesError) as e:
-        randes.randes_retrieve_static(plan.handle, 0, 1.0, randes.F32, fake, 1 << 40, fake_out, None)
+        randes.randes_retrieve_static(plan.handle, 0, 1.0, randes.F32, fake, 1 << 50, fake_out, None)
     assert e.value.code == randes.CAPACITY
     assert "scratch" in str(e.value)
     plan.close()

@@ -605,7 +605,7 @@ def run_ours(args):
                                else "fallback copy bandwidth",
                 "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                 "traffic_source": "ncu dram bytes on the ViT-B/32-shaped case scaled by parameter count (profiles/)"
-                                  if traffic else "none valid for this build",
+                                  if traffic else "none valid for the current kernel sources",
                 "share_of_step": shares[dom] / total_ms,
                 "per_kernel": {k: {"achieved": ops[k]["GBps"], "frac": ops[k]["GBps"] / peak, "bytes_per_launch": b[k]}
                                for k in ops}}

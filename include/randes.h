@@ -168,6 +168,21 @@ int randes_task_list(const randes_plan_t* plan, uint32_t* task_ids, uint64_t* se
 int randes_plan_validate(const randes_plan_t* plan);
 
 /*
+ * Checked build (a debugging aid: the library compiled with -DRANDES_CHECKED, see the build script).  In that
+ * build the streaming kernels (retrieve, compress / add / remove, their group and batched forms) compare, before a
+ * thread block touches a tile, every index the tile's addresses are derived from -- the tile's layer, the layers and
+ * slots it reaches through sigma / sigma^-1 (Section 4.3), its rows -- with the plan's bounds; a tile that fails is
+ * skipped instead of read or written, and the first failure is kept in a device word.  This call synchronises with
+ * the current device and returns that word: 0 = none; else bit 63 set, bits 48-55 the kernel (1 retrieve,
+ * 2 compress / add / remove, 3 add / remove for bf16 weights, 4 group compress, 5 batched retrieve, 6 batched group
+ * retrieve), bits 40-47 what failed (1 the tile's layer, 2 a permuted layer or slot, 3 the rows), bits 0-31 the tile.
+ * *checked_build (may be NULL) tells whether this library is a checked build; the ordinary build always reports 0.
+ * What such a word means in practice: the plan's device workspace was overwritten, or the plan does not belong to
+ * these tensors.  Errors: INVALID_ARGUMENT, CUDA_ERROR.
+ */
+int randes_debug_violation(uint64_t* word, int* checked_build);
+
+/*
  * Persistence.  What RanDeS keeps per model is a seed (Section 4.1), so a plan
  * is fully described by its layer shapes, group flags, element types and the
  * registered (id, seed) pairs in summation order; M itself is the caller's

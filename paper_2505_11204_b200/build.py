@@ -1,8 +1,9 @@
 """Compile the CUDA library for sm_100a into the package directory.
 
-    python -m paper_2505_11204_b200.build [--force] [--verbose] [--nvtx]
+    python -m paper_2505_11204_b200.build [--force] [--verbose] [--nvtx] [--checked]
 
 --nvtx brackets every computing entry point with an NVTX range (off by default).
+--checked builds the kernels with their bounds predicates (slower; see randes_debug_violation).
 
 nvcc cross-compiles without a GPU.  The shared object is kept in-tree (it is
 not committed) so that it travels with the source tree to the machine that has
@@ -41,6 +42,8 @@ def nvcc_command(out: str, extra_flags=(), opt: str = "-O3"):
 SANITIZER_FLAGS = ["-Xcompiler", "-fsanitize=address,-fsanitize=undefined,-fno-sanitize-recover=undefined,-fno-omit-frame-pointer", "-g"]
 # every computing entry point bracketed by an NVTX range named after it
 NVTX_FLAGS = ["-DRANDES_NVTX", "-ldl"]
+# the streaming kernels check the indices of every tile against the plan's bounds (randes_debug_violation)
+CHECKED_FLAGS = ["-DRANDES_CHECKED"]
 
 
 def build_library(force: bool = False, verbose: bool = False, extra_flags=(), out: str = LIB) -> str:
@@ -55,5 +58,5 @@ def build_library(force: bool = False, verbose: bool = False, extra_flags=(), ou
 
 
 if __name__ == "__main__":
-    nvtx = "--nvtx" in sys.argv
-    print(build_library(force="--force" in sys.argv or nvtx, verbose="--verbose" in sys.argv, extra_flags=NVTX_FLAGS if nvtx else ()))
+    flags = (NVTX_FLAGS if "--nvtx" in sys.argv else []) + (CHECKED_FLAGS if "--checked" in sys.argv else [])
+    print(build_library(force="--force" in sys.argv or bool(flags), verbose="--verbose" in sys.argv, extra_flags=flags))

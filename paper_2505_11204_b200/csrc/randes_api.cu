@@ -1349,6 +1349,20 @@ int randes_plan_validate(const randes_plan_t* plan)
     return guarded("randes_plan_validate", [&] { return randes_plan_validate_impl(plan); });
 }
 
+int randes_debug_violation(uint64_t* word, int* checked_build)
+{
+    if (!word) return fail(RANDES_INVALID_ARGUMENT, "word is NULL");
+#ifdef RANDES_CHECKED
+    if (checked_build) *checked_build = 1;
+#else
+    if (checked_build) *checked_build = 0;
+#endif
+    const unsigned long long w[3] = {violation_in_streaming_kernels(), violation_in_group_kernel(), violation_in_batch_kernels()};
+    *word = w[0] ? w[0] : (w[1] ? w[1] : w[2]);
+    if (*word == ~0ull) return fail(RANDES_CUDA_ERROR, "the violation word could not be read");
+    return RANDES_OK;
+}
+
 // Section 3, norm of the interference: || lambda sum_{j != t} T_t^-1 T_j d_j ||^2 = lambda^2 sum_{j,l != t} <T_j d_j, T_l d_l>,
 // because T_t^-1 is orthogonal.
 int randes_interference_norm(const double* gram, uint32_t n, uint32_t t, double lambda, double* norm)

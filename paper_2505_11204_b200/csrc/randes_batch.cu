@@ -40,7 +40,9 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
         const uint32_t p = un.layer;
+        if (!checked(p < a.n_layers, 5, kCheckLayer, u)) continue;
         const DevLayer lp = a.layers[p];
+        if (!checked(un.row0 + un.nrows <= lp.rows, 5, kCheckRows, u)) continue;
         const WarpTile t = warp_tile<CPL>(un, warp, lane);
         if (t.r0 >= t.r_end || t.cb * 32 * CPL >= lp.cols) continue;   // warp-uniform
         const bool flipped = (lp.flags & kFlagFlip) != 0;
@@ -50,7 +52,8 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
         bool ok = aligned16(wp);
         if (lane < n) {
             const uint32_t row = a.task_rows[lane];
-            const uint32_t slot = (lp.flags & kFlagShuffle) ? a.slot_of_pos[static_cast<size_t>(row) * L + p] : p;   // sigma^-1
+            uint32_t slot = (lp.flags & kFlagShuffle) ? a.slot_of_pos[static_cast<size_t>(row) * L + p] : p;   // sigma^-1
+            if (!checked(slot < L, 5, kCheckPermuted, u)) slot = p;   // (checked build: recorded; the tile reads its own slot)
             ws.m[lane] = static_cast<const MT*>(a.M) + a.layers[slot].m_off;
             void* o = a.out[static_cast<size_t>(lane) * L + p];
             ws.out[lane] = o;
@@ -162,6 +165,20 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_group_kernel
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
         const uint32_t* mem = a.members + un.layer;
+#ifdef RANDES_CHECKED
+        {   // every member, every permuted slot and the unit's rows must lie inside the plan; else the unit is skipped
+            bool sound = checked(mem[0] < L, 6, kCheckLayer, u);
+            const uint32_t G_claimed = sound ? a.layers[mem[0]].group_size : 0;
+            for (uint32_t m = 0; sound && m < G_claimed; ++m) {
+                sound = checked(mem[m] < L, 6, kCheckLayer, u);
+                for (uint32_t b = 0; sound && b < n; ++b)
+                    sound = checked(!(a.layers[mem[m]].flags & kFlagShuffle) || a.slot_of_pos[static_cast<size_t>(a.task_rows[b]) * L + mem[m]] < L, 6,
+                                    kCheckPermuted, u);
+            }
+            sound = sound && checked(un.row0 + un.nrows <= a.layers[mem[0]].rows, 6, kCheckRows, u);
+            if (!sound) continue;       // (uniform over the CTA: every thread evaluates the same tables)
+        }
+#endif
         const DevLayer l0 = a.layers[mem[0]];
         const uint32_t G = l0.group_size, cols = l0.cols, Rn = un.nrows;
         const uint32_t c = (un.cb0 * 32u + lane) * CPL;
@@ -252,6 +269,8 @@ template <typename T> struct Tag { typedef T type; };
 template <typename F> int with_type(int dtype, F&& f) { return dtype == 0 ? f(Tag<float>{}) : f(Tag<__nv_bfloat16>{}); }
 
 }  // namespace
+
+RANDES_VIOLATION_READER(violation_in_batch_kernels)
 
 int launch_retrieve_batch(int storage_dtype, int out_dtype, int m_dtype, const RetrieveBatchArgs& a, int grid, void* stream)
 {

@@ -32,6 +32,33 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
+// Checked build (-DRANDES_CHECKED): before a thread block touches a tile, the indices that every later address of the
+// tile is derived from -- the unit's layer, the permuted layer, the unit's rows -- are compared with the plan's
+// bounds; a tile that fails is skipped and the first failure is recorded in a device word (kernel, what, unit) that
+// randes_debug_violation() reads.  In the ordinary build checked() is the constant true and costs nothing.
+enum { kCheckLayer = 1, kCheckPermuted = 2, kCheckRows = 3 };
+#ifdef RANDES_CHECKED
+static __device__ unsigned long long g_violation;     // of the kernels of this translation unit
+__device__ __forceinline__ bool checked(bool ok, uint32_t kernel_id, uint32_t what, uint32_t unit)
+{
+    if (ok) return true;
+    atomicCAS(&g_violation, 0ull, (1ull << 63) | (static_cast<unsigned long long>(kernel_id) << 48) |
+                                      (static_cast<unsigned long long>(what) << 40) | unit);
+    return false;
+}
+#define RANDES_VIOLATION_READER(name)                                                              \
+    unsigned long long name()                                                                      \
+    {                                                                                              \
+        unsigned long long w = 0;                                                                  \
+        if (cudaMemcpyFromSymbol(&w, device::g_violation, sizeof w) != cudaSuccess) w = ~0ull;     \
+        return w;                                                                                  \
+    }
+#else
+__device__ __forceinline__ constexpr bool checked(bool, uint32_t, uint32_t, uint32_t) { return true; }
+#define RANDES_VIOLATION_READER(name) \
+    unsigned long long name() { return 0; }
+#endif
+
 __device__ __forceinline__ float flip(float x, uint32_t mask) { return __uint_as_float(__float_as_uint(x) ^ mask); }
 
 // Two fp32 values in one 64-bit register, for the packed add / sub / fma of sm_100.

@@ -46,10 +46,6 @@ template <> struct GroupGeom<__nv_bfloat16> {
 };
 constexpr uint32_t stage_rows(int storage_dtype) { return storage_dtype == 1 ? 3u : 2u; }
 
-__device__ __forceinline__ void sts_u64(uint32_t saddr, unsigned long long v)
-{
-    asm volatile("st.shared.u64 [%0], %1;" ::"r"(saddr), "l"(v) : "memory");
-}
 __device__ __forceinline__ unsigned long long lds_u64(uint32_t saddr)
 {
     unsigned long long v;
@@ -161,6 +157,24 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
             // ---- tables, all threads: per (slot, task) pair the source tensor and the sign bits; per member its slot's
             //      place in M and its W_0 tensor
             const uint32_t* mem = a.members + un.layer;
+#ifdef RANDES_CHECKED
+            // every member and every permuted source layer of the chunk must be a layer of the plan
+            bool sound = checked(mem[0] < L, 4, kCheckLayer, unit_at(t));
+            const uint32_t G_claimed = sound ? a.layers[mem[0]].group_size : 0;
+            for (uint32_t ms = 0; sound && ms < G_claimed; ++ms) {
+                sound = checked(mem[ms] < L, 4, kCheckLayer, unit_at(t));
+                for (uint32_t i = 0; sound && i < nt; ++i)
+                    sound = checked(!(a.layers[mem[ms]].flags & kFlagShuffle) || a.src_of_slot[static_cast<size_t>(i) * L + mem[ms]] < L, 4,
+                                    kCheckPermuted, unit_at(t));
+            }
+            if (!sound) {       // nothing is copied, summed or stored for this chunk
+                G = cols = 0;
+                lane_on = false;
+                key_group = un.layer;
+                key_cb = un.cb0;
+                continue;
+            }
+#endif
             const DevLayer l0 = a.layers[mem[0]];
             G = l0.group_size;
             cols = l0.cols;
@@ -189,9 +203,15 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
             __syncthreads();   // the tables are complete and visible to every warp
         }
         const uint32_t off0 = row0 * cols + c;           // layers hold < 2^32 elements
+#ifdef RANDES_CHECKED
+        if (G == 0) continue;                            // a chunk that failed its check above
+        const bool rows_ok = checked(row0 + Rn <= a.layers[a.members[un.layer]].rows, 4, kCheckRows, unit_at(t));
+#else
+        constexpr bool rows_ok = true;
+#endif
 
         // ---- W_0 tiles of every member into the stash
-        if (lane_on) {
+        if (lane_on && rows_ok) {
             const uint32_t ntiles = G * Rn;
             for (uint32_t q = warp; q < ntiles; q += kWarpsPerCta) {
                 const uint32_t m = q / Rn, r = q - m * Rn;
@@ -203,7 +223,7 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) compress_group_kernel(const
         cp_async_wait<0>();
         __syncthreads();   // the stash is complete and visible to every warp
 
-        if (lane_on) {
+        if (lane_on && rows_ok) {
             const uint32_t n_chunks = (Rn + IR - 1) / IR;
             const uint32_t n_items = G * n_chunks;
             uint32_t N = 0;   // stages of this warp
@@ -309,6 +329,8 @@ int max_stages(int storage_dtype) { return storage_dtype == 1 ? 4 : 6; }
 int min_stages(int storage_dtype) { return storage_dtype == 1 ? 3 : 4; }
 
 }  // namespace
+
+RANDES_VIOLATION_READER(violation_in_group_kernel)
 
 int compress_group_prepare(int storage_dtype, int m_dtype)
 {

@@ -185,6 +185,12 @@ bool retrieve_batch_group_fits(uint32_t max_group, uint32_t n_tasks);
 int launch_retrieve_batch_groups(int out_dtype, const RetrieveBatchArgs& a, uint32_t max_group, int sm_count, void* stream);
 
 
+// Checked build (-DRANDES_CHECKED): the first bounds violation recorded by the kernels of each file, 0 if none
+// (always 0 in the ordinary build); all-ones if the word could not be read.
+unsigned long long violation_in_streaming_kernels();
+unsigned long long violation_in_group_kernel();
+unsigned long long violation_in_batch_kernels();
+
 // randes_linear.cu: y = x W_0^T + lambda (x D) M_slot^T on the tensor cores (bf16 operands, fp32 accumulators).
 // All return a cudaError_t as int.
 int linear_prepare();   // opts the kernel into its shared memory on the current device

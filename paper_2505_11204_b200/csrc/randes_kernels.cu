@@ -154,8 +154,10 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_kernel(const Retri
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
         const uint32_t p = un.layer;                       // layer position being rebuilt
+        if (!checked(p < a.n_layers, 1, kCheckLayer, u)) continue;
         const DevLayer lp = a.layers[p];
         const uint32_t slot = (lp.flags & kFlagShuffle) ? a.slot_of_pos[p] : p;   // sigma^-1
+        if (!checked(slot < a.n_layers, 1, kCheckPermuted, u) || !checked(un.row0 + un.nrows <= lp.rows, 1, kCheckRows, u)) continue;
         const unsigned long long m_off = slot == p ? lp.m_off : a.layers[slot].m_off;
         const WarpTile t = warp_tile<CPL>(un, warp, lane);
         if constexpr (CPL == 8 && sizeof(MT) == 4) {
@@ -477,7 +479,9 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const Acc
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
         const uint32_t slot = un.layer;
+        if (!checked(slot < a.n_layers, 2, kCheckLayer, u)) continue;
         const DevLayer ls = a.layers[slot];
+        if (!checked(un.row0 + un.nrows <= ls.rows, 2, kCheckRows, u)) continue;
         const WarpTile t = warp_tile<CPL>(un, warp, lane);
         if (t.r0 >= t.r_end || t.cb * 32 * CPL >= ls.cols) continue;   // warp-uniform: nothing for this warp
         const bool lane_on = t.c < ls.cols;
@@ -492,7 +496,8 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) accumulate_kernel(const Acc
             bool ok = true;
             if (lane < nt) {
                 const uint32_t ti = chunk0 + lane;
-                const uint32_t src = shuffled ? a.src_of_slot[static_cast<size_t>(ti) * L + slot] : slot;   // sigma_i(l)
+                uint32_t src = shuffled ? a.src_of_slot[static_cast<size_t>(ti) * L + slot] : slot;   // sigma_i(l)
+                if (!checked(src < L, 2, kCheckPermuted, u)) src = slot;   // (checked build: recorded; the tile reads its own layer)
                 const void* pw = a.task_ptrs[static_cast<size_t>(ti) * L + src];
                 const void* pb = a.has_base ? a.base[src] : nullptr;
                 sts_ptrs(sptr + lane * 16, pw, pb);
@@ -558,11 +563,14 @@ __global__ void __launch_bounds__(kThreadsPerCta, 3) add_halves_kernel(const Acc
     for (uint32_t u = blockIdx.x; u < a.n_units; u += gridDim.x) {
         const DevUnit un = a.units[u];
         const uint32_t slot = un.layer;
+        if (!checked(slot < a.n_layers, 3, kCheckLayer, u)) continue;
         const DevLayer ls = a.layers[slot];
+        if (!checked(un.row0 + un.nrows <= ls.rows, 3, kCheckRows, u)) continue;
         const WarpTile t = warp_tile<8>(un, warp, lane);
         const uint32_t cols = ls.cols;
         if (t.r0 >= t.r_end || t.cb * 256u >= cols) continue;   // warp-uniform
         const uint32_t src = (ls.flags & kFlagShuffle) ? a.src_of_slot[slot] : slot;   // sigma_j(l)
+        if (!checked(src < a.n_layers, 3, kCheckPermuted, u)) continue;
         const bf16* wp = static_cast<const bf16*>(a.task_ptrs[src]);
         const bf16* bp = HAS_BASE ? static_cast<const bf16*>(a.base[src]) : nullptr;
         float* mp = static_cast<float*>(a.M) + ls.m_off;
@@ -767,6 +775,8 @@ int launch_retrieve_static(int storage_dtype, int out_dtype, int m_dtype, const 
     if (n_units == 0) return 0;
     return launch_retrieve(storage_dtype, out_dtype, m_dtype, a, grid < static_cast<int>(n_units) ? grid : static_cast<int>(n_units), stream);
 }
+
+RANDES_VIOLATION_READER(violation_in_streaming_kernels)
 
 int retrieve_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype)
 {

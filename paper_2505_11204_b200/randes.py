@@ -79,6 +79,8 @@ def lib():
         L.randes_plan_destroy.restype = None
         L.randes_plan_validate.argtypes = [vp]
         L.randes_plan_validate.restype = ctypes.c_int
+        L.randes_debug_violation.argtypes = [ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_int)]
+        L.randes_debug_violation.restype = ctypes.c_int
         L.randes_superposition_bytes.argtypes = [vp]
         L.randes_superposition_bytes.restype = sz
         L.randes_layer_offset.argtypes = [vp, u32]
@@ -132,7 +134,7 @@ def lib():
 
 
 EXPORTS = [
-    "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_plan_validate", "randes_superposition_bytes",
+    "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_plan_validate", "randes_debug_violation", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
     "randes_task_tables", "randes_plan_serialize", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_add_models", "randes_remove_model",
     "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_interference_norm", "randes_pairwise_cosines", "randes_retrieve_batch", "randes_retrieve_static", "randes_linear", "randes_linear_gated", "randes_linear_giveups", "randes_launch_count", "randes_last_error",
@@ -200,6 +202,13 @@ def randes_plan_destroy(plan) -> None:
 def randes_plan_validate(plan) -> None:
     """Host-side self-check of a plan's tables; raises RandesError naming the first violation."""
     _check(lib().randes_plan_validate(plan))
+
+
+def randes_debug_violation():
+    """(word, checked_build): the first bounds violation recorded by a checked build's kernels (0 = none)."""
+    word, flag = ctypes.c_uint64(0), ctypes.c_int(0)
+    _check(lib().randes_debug_violation(ctypes.byref(word), ctypes.byref(flag)))
+    return int(word.value), bool(flag.value)
 
 
 def randes_superposition_bytes(plan) -> int:

@@ -162,3 +162,68 @@ def test_vit_l14_shaped_fp32_full_size_sampled():
 
 def test_vit_l14_shaped_bf16_full_size_sampled():
     run_full_size(wl.BF16, n_swap=2)
+
+
+def test_gaussian_context_full_size_sampled():
+    """The Gaussian-diagonal ("RD") context of Section 5.5 on the ViT-L/14-shaped set (fp32, 3 tasks + 1 added and
+    removed): plans with such a group get taller tiles on large models (up to 128 rows per warp), which the small
+    parity cases never reach.  Sampled slots of M and the layers they feed are compared with the oracle bit for bit."""
+    import torch
+
+    w = wl.vit_l14(storage=wl.F32).with_tasks(3)
+    w.gflags = [(f & ~wl.FLIP) | randes.GAUSS if f & wl.FLIP else f for f in w.gflags]
+    L = w.n_layers
+    ids, seeds = list(w.task_ids), list(w.seeds)
+    all_ids, all_seeds = ids + [9], seeds + [1234]
+    src_of = {t: ro.task_tables(w.spec, s, t)[0] for t, s in zip(all_ids, all_seeds)}
+    slots = sampled_slots(w)[::2]
+    need_base, need_task = set(), set()
+    for l in slots:
+        for t in all_ids:
+            src = int(src_of[t][l])
+            need_base.add(src)
+            need_task.add((t, src))
+    base_h, tasks_h = [None] * L, {t: [None] * L for t in all_ids}
+    d_base, d_tasks = [None] * L, {t: [None] * L for t in all_ids}
+    with ThreadPoolExecutor(max_workers=16) as ex:
+        for l, (b, ts) in enumerate(ex.map(lambda l: wl.layer_all_tasks(w, l, all_ids), range(L))):
+            d_base[l] = to_dev(b)
+            if l in need_base:
+                base_h[l] = b
+            for t, a in zip(all_ids, ts):
+                d_tasks[t][l] = to_dev(a)
+                if (t, l) in need_task:
+                    tasks_h[t][l] = a
+    plan = randes.Plan.from_workload(w, max_tasks=4)
+    randes.randes_plan_validate(plan.handle)
+    M = plan.new_superposition().zero_()
+    out = plan.new_output(wl.F32)
+    p_base, p_out = randes.ptr_array(d_base), randes.ptr_array(out)
+    sh = torch.cuda.current_stream().cuda_stream
+
+    def check_m(tag):
+        for l in slots:
+            assert_bits_equal(from_dev(plan.slot(M, l)), M_ref[l], "%s slot %d (%s)" % (tag, l, w.layer_names[l]))
+
+    def check_retrieve(t, s, tag):
+        randes.randes_retrieve(plan.handle, t, w.lam, wl.F32, p_base, M, p_out, sh)
+        pos = sorted(set(int(src_of[t][l]) for l in slots))
+        ref = ro.retrieve(w.spec, wl.F32, wl.F32, t, s, w.lam, base_h, M_ref, positions=pos)
+        for p in pos:
+            assert_bits_equal(from_dev(out[p]), ref[p], "%s retrieve task %d layer %d (%s)" % (tag, t, p, w.layer_names[p]))
+
+    randes.randes_compress(plan.handle, p_base, randes.ptr_array([d_tasks[t] for t in ids]), M, sh)
+    M_ref = ro.compress(w.spec, wl.F32, ids, seeds, base_h, [tasks_h[t] for t in ids], slots=slots)
+    check_m("compress")
+    for t, s in zip(ids, seeds):
+        check_retrieve(t, s, "sweep")
+    randes.randes_add_model(plan.handle, 9, 1234, p_base, randes.ptr_array(d_tasks[9]), M, sh)
+    ro.add_model(w.spec, wl.F32, 9, 1234, base_h, tasks_h[9], M_ref, slots=slots)
+    check_m("add")
+    check_retrieve(9, 1234, "after add")
+    randes.randes_remove_model(plan.handle, 1, p_base, randes.ptr_array(d_tasks[1]), M, sh)
+    ro.remove_model(w.spec, wl.F32, 1, seeds[1], base_h, tasks_h[1], M_ref, slots=slots)
+    check_m("remove")
+    assert bool(torch.isfinite(M).all())
+    torch.cuda.synchronize()
+    plan.close()

@@ -67,6 +67,59 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_kernel(const
         }
         const bool vec = lp.cols % CPL == 0 && __all_sync(0xFFFFFFFFu, ok);
         __syncwarp();
+        if constexpr (CPL == 8 && sizeof(MT) == 4) {
+            // bf16 weights, fp32 M: with 8 neighbouring columns per lane the 32-byte M tiles and fp32 outputs of a warp are
+            // requests whose lanes sit 32 bytes apart.  When widths and alignment allow, a lane takes columns 4 lane ..
+            // 4 lane + 3 of BOTH 128-column halves of the warp's block instead (as retrieve_kernel does): every request is
+            // contiguous across the warp, and each half reads its own Philox block like an fp32 warp.
+            if (vec) {
+                for (uint32_t i = 0; i < n; ++i)
+                    ws.bits[i][lane] = flipped ? static_cast<unsigned short>(lane_bits<4>(ws.block[0][i], lane) | (lane_bits<4>(ws.block[1][i], lane) << 4)) : 0;
+                __syncwarp();
+                const uint32_t c0 = t.cb * 256u + lane * 4u;
+                const bool on[2] = {c0 < lp.cols, c0 + 128u < lp.cols};
+                const uint32_t row_stride = t.rstep * lp.cols;
+                uint32_t off = t.r0 * lp.cols + c0;
+                for (uint32_t r = t.r0; r < t.r_end; r += t.rstep, off += row_stride) {
+                    float wv[2][4];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        if (on[h]) {
+                            const uint2 w = __ldcs(reinterpret_cast<const uint2*>(wp + off + h * 128u));
+                            wv[h][0] = __uint_as_float(w.x << 16); wv[h][1] = __uint_as_float(w.x & 0xFFFF0000u);
+                            wv[h][2] = __uint_as_float(w.y << 16); wv[h][3] = __uint_as_float(w.y & 0xFFFF0000u);
+                        }
+                    for (uint32_t i0 = 0; i0 < n; i0 += TB) {
+                        float4 m[TB][2];
+#pragma unroll
+                        for (int b = 0; b < TB; ++b)
+                            if (i0 + b < n) {
+                                const float* mp = static_cast<const float*>(ws.m[i0 + b]);
+#pragma unroll
+                                for (int h = 0; h < 2; ++h)
+                                    if (on[h]) m[b][h] = __ldg(reinterpret_cast<const float4*>(mp + off + h * 128u));
+                            }
+#pragma unroll
+                        for (int b = 0; b < TB; ++b)
+                            if (i0 + b < n) {
+                                const uint32_t bits = ws.bits[i0 + b][lane];
+                                OT* op = static_cast<OT*>(ws.out[i0 + b]);
+#pragma unroll
+                                for (int h = 0; h < 2; ++h)
+                                    if (on[h]) {
+                                        const float mv[4] = {m[b][h].x, m[b][h].y, m[b][h].z, m[b][h].w};
+                                        float y[4];
+#pragma unroll
+                                        for (int e = 0; e < 4; ++e)
+                                            y[e] = __fmaf_rn(flip(a.lambda, ((bits >> (4 * h + e)) & 1u) << 31), mv[e], wv[h][e]);
+                                        Out<OT>::template store<4>(op + off + h * 128u, y);
+                                    }
+                            }
+                    }
+                }
+                continue;
+            }
+        }
         for (uint32_t i = 0; i < n; ++i)
             ws.bits[i][lane] = flipped ? static_cast<unsigned short>(lane_bits<CPL>(ws.block[CPL == 8 ? (lane >> 4) : 0][i], lane)) : 0;
         __syncwarp();

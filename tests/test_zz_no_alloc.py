@@ -69,7 +69,12 @@ def test_static_retrieve_matches_retrieve_on_two_calls_in_a_row(storage):
             p_got = randes.ptr_array(got)
             torch.cuda.synchronize()
             free_before = torch.cuda.mem_get_info()[0]       # the device's own count, not torch's allocator
-            randes.randes_retrieve_static(host_plan.handle, task, w.lam, out_dtype, p_base, M, p_got, stream)
+            p_base_call = randes.ptr_array(d_base)
+            randes.randes_retrieve_static(host_plan.handle, task, w.lam, out_dtype, p_base_call, M, p_got, stream)
+            # the pointer arrays are the caller's again as soon as the call returns: scribble over them before the
+            # kernel has (necessarily) run -- the library works from its own copy of the tables
+            ctypes.memset(ctypes.addressof(p_base_call), 0xFF, ctypes.sizeof(p_base_call))
+            ctypes.memset(ctypes.addressof(p_got), 0xFF, ctypes.sizeof(p_got))
             torch.cuda.synchronize()
             calls += 1
             if calls > 1:                                     # the first call on a device may load the module with its array

@@ -30,7 +30,8 @@
  *   handed.  Weight tensors must be aligned to their element size; 16-byte
  *   aligned tensors with cols % 4 == 0 take the vectorised path.
  * - M is one arena of randes_superposition_bytes() bytes, 256-byte aligned;
- *   slot l starts at byte randes_layer_offset(plan, l).  Its element type is
+ *   slot l starts at byte randes_layer_offset(plan, l) (the first slot a little
+ *   way in, not at 0: ask, do not assume).  Its element type is
  *   the plan's m_dtype: fp32 by default whatever the storage type of the
  *   weights, or bf16 (half the footprint; a smaller superposition is what
  *   the paper's conclusion leaves to future work).  Sums always run in fp32: with a bf16 M,

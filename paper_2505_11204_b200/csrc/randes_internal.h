@@ -11,6 +11,7 @@ constexpr uint32_t kFlagShuffle = 1u;   // layer may move inside its group for s
 constexpr uint32_t kFlagFlip = 2u;      // per-column sign flip on this slot
 constexpr uint32_t kFlagGauss = 4u;     // per-column Gaussian-like factor on this slot instead (general diagonal context)
 
+constexpr size_t kSuperpositionLeadIn = 1024;   // bytes before the first slot of M (see randes_plan)
 constexpr int kWarpsPerCta = 8;
 constexpr int kThreadsPerCta = kWarpsPerCta * 32;
 constexpr int kRowsPerWarp = 16;        // rows one warp walks per unit (8 to 16 measured best; 32 and 64 slower)

@@ -143,8 +143,8 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers,
 
 void randes_plan_destroy(randes_plan_t* plan); /* NULL is allowed; frees host memory only */
 
-/* Size of the arena M: sum of rows*cols elements of m_dtype, each slot padded to 256 bytes.
- * Independent of the number of tasks (Section 4.1: a seed per added model). */
+/* Size of the arena M: 1 KiB of lead-in, then rows*cols elements of m_dtype per layer, each slot padded to
+ * 256 bytes.  Independent of the number of tasks (Section 4.1: a seed per added model). */
 size_t randes_superposition_bytes(const randes_plan_t* plan);
 
 /* Byte offset of slot `layer` inside M; (size_t)-1 if out of range. */

@@ -242,14 +242,14 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def config_dict(w, args, note=""):
+def config_dict(w, args):
+    """What was run -- the same dict from both arms for the same flags (what differs between them goes into `note`)."""
     return {"workload": "%s-shaped synthetic weights, K=%d tasks, %d layers, %.1f M params; step = compress + %d retrieves + %d adds + %d removes"
                         % (w.name, w.n_tasks, w.n_layers, w.n_params / 1e6, w.n_tasks, args.swap, args.swap),
             "storage": "bf16" if w.storage == wl.BF16 else "f32", "lambda": w.lam,
             "l2": ("inputs exceed L2: every call streams at least %.2f GB" if (4 + 4) * w.n_params > 2 * 126e6 else
                    "working set of %.3f GB fits in L2: latency-bound, not a roofline case")
-                  % ((4 + (2 if w.storage == wl.BF16 else 4)) * w.n_params / 1e9),
-            "note": note}
+                  % ((4 + (2 if w.storage == wl.BF16 else 4)) * w.n_params / 1e9)}
 
 
 # --------------------------------------------------------------------------------- CPU oracle legs
@@ -313,7 +313,7 @@ def run_reference(args):
         "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "steps_timed": r["steps_timed"], "ms_per_step": r["ms_per_step"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32" if w.storage == wl.F32 else "bf16 storage, f32 arithmetic", "data": "synthetic",
-        "config": config_dict(w, args, note),
+        "config": config_dict(w, args), "note": note,
         "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -891,9 +891,10 @@ def run_ours(args):
             "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "strong" if sliced else "weak", "vs_baseline": None,
             "dtype": "f32" if w.storage == wl.F32 else "bf16 storage, f32 arithmetic", "data": "synthetic",
-            "config": config_dict(w_whole, args, ("every rank holds one row slice of every layer (1/%d of the rows); per-call figures under "
-                                                  "'ops' are rank 0's slice; no collective on the data path" % world) if sliced else
-                                  "every rank runs the whole workload on its own GPU; no collective on the data path"),
+            "config": config_dict(w_whole, args),
+            "note": ("every rank holds one row slice of every layer (1/%d of the rows); per-call figures under "
+                     "'ops' are rank 0's slice; no collective on the data path" % world) if sliced else
+                    "every rank runs the whole workload on its own GPU; no collective on the data path",
             "Gparams_per_s": {n: ops[n]["Gparams_per_s"] for n in ops},
             "ops": ops, "extras": extras, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e if e2e is not None else ({"value": None, "note": e2e_skipped} if e2e_skipped else None), "gpu_launches": int(launches),
             "clocks": clocks,

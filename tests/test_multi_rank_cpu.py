@@ -197,4 +197,4 @@ def test_reference_arm_times_the_whole_workload_with_the_requested_steps():
     # a budget too small for the request: one step is still timed, and the note says what happened
     r2 = _bench("--impl", "reference", "--workload", "toy", "--steps", "50", "--warmup", "1", "--reference-budget-s", "0")
     line2 = json.loads(r2.stdout.strip().splitlines()[-1])
-    assert line2["steps"] == 50 and 1 <= line2["steps_timed"] < 50 and "budget" in line2["config"]["note"]
+    assert line2["steps"] == 50 and 1 <= line2["steps_timed"] < 50 and "budget" in line2["note"]

@@ -539,6 +539,55 @@ def test_row_slices_shard_without_exchange():
         plan.close()
 
 
+def test_two_plans_on_two_streams_do_not_disturb_each_other():
+    """Calls on one plan are ordered on the stream they are given; distinct plans share nothing.  Two plans (fp32 and
+    bf16 weights) are driven on two CUDA streams with their calls interleaved on the host -- compress, adds, removes
+    and retrieves of one plan enqueued between those of the other, nothing synchronised in between -- and every result
+    equals the oracle's bit for bit."""
+    import torch
+
+    ws = [wl.toy(n_tasks=3, width=384, n_blocks=5), wl.toy(n_tasks=4, width=256, n_blocks=7).with_storage(wl.BF16)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    st = []
+    for w in ws:
+        ids = list(w.task_ids) + [77]
+        base, models = wl.model_set(w, ids)
+        st.append({"w": w, "base": base, "tasks": models[:w.n_tasks], "extra": models[w.n_tasks],
+                   "d_base": model_to_dev(base), "d_tasks": [model_to_dev(t) for t in models[:w.n_tasks]],
+                   "d_extra": model_to_dev(models[w.n_tasks])})
+    torch.cuda.synchronize()
+    for s_, q in zip(streams, st):
+        with torch.cuda.stream(s_):
+            q["plan"] = randes.Plan.from_workload(q["w"], max_tasks=q["w"].n_tasks + 1)
+            q["M"] = q["plan"].new_superposition()
+            q["outs"] = {}
+    order = ["compress", "retrieve0", "add", "retrieve77", "remove", "retrieve1"]
+    for step in order:
+        for s_, q in zip(streams, st):                       # plan A's call, then plan B's, never a synchronisation
+            w, plan = q["w"], q["plan"]
+            with torch.cuda.stream(s_):
+                if step == "compress":
+                    plan.compress(q["d_base"], q["d_tasks"], q["M"])
+                elif step == "add":
+                    plan.add_model(77, 1234, q["d_base"], q["d_extra"], q["M"])
+                elif step == "remove":
+                    plan.remove_model(w.task_ids[0], q["d_base"], q["d_tasks"][0], q["M"])
+                else:
+                    t = int(step[len("retrieve"):])
+                    q["outs"][step] = plan.retrieve(t, w.lam, q["d_base"], q["M"])
+    torch.cuda.synchronize()
+    for q in st:
+        w = q["w"]
+        M_ref = ro.compress(w.spec, w.storage, w.task_ids, w.seeds, q["base"], q["tasks"])
+        check_model(q["outs"]["retrieve0"], ro.retrieve(w.spec, w.storage, wl.F32, 0, w.seeds[0], w.lam, q["base"], M_ref), "retrieve 0")
+        ro.add_model(w.spec, w.storage, 77, 1234, q["base"], q["extra"], M_ref)
+        check_model(q["outs"]["retrieve77"], ro.retrieve(w.spec, w.storage, wl.F32, 77, 1234, w.lam, q["base"], M_ref), "retrieve 77")
+        ro.remove_model(w.spec, w.storage, w.task_ids[0], w.seeds[0], q["base"], q["tasks"][0], M_ref)
+        check_model(q["outs"]["retrieve1"], ro.retrieve(w.spec, w.storage, wl.F32, 1, w.seeds[1], w.lam, q["base"], M_ref), "retrieve 1")
+        check_superposition(q["plan"], q["M"], M_ref, "final M")
+        q["plan"].close()
+
+
 def test_gpu_argument_validation():
     import torch
 

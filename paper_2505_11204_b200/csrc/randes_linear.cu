@@ -63,6 +63,7 @@ template <int HALVES> struct LinearGeom {
 
 struct LinearArgs {
     uint32_t n_tokens, rows, cols;
+    uint32_t token0;               // first token of this launch (a call may cover its tokens with two launches)
     float lambda;
     uint32_t flip;                 // 0: no sign flip on this slot
     uint32_t slot;                 // l = sigma_t^-1(p): counter word 1 of the sign stream
@@ -213,7 +214,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__
     volatile uint32_t* abort_flag = tmem_ptr + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * kBN, m0 = blockIdx.y * (HALVES * kBM);
+    const int n0 = blockIdx.x * kBN, m0 = a.token0 + blockIdx.y * (HALVES * kBM);
     const uint32_t n_k = (a.cols + kBK - 1) / kBK;
 
     if (threadIdx.x == 0) {
@@ -456,15 +457,25 @@ int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* 
     cudaError_t ce = cudaGetDevice(&dev);
     if (ce == cudaSuccess) ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (ce != cudaSuccess) return static_cast<int>(ce);
-    const uint64_t tiles256 = static_cast<uint64_t>((rows + kBN - 1) / kBN) * ((n_tokens + 2 * kBM - 1) / (2 * kBM));
     // measured: a 128-token tile takes about 3/4 of the time of a 256-token tile (half the products, but each staged
-    // weight tile then feeds one product instead of two); the shape whose number of waves x that cost is lower wins
-    const uint64_t tiles128 = static_cast<uint64_t>((rows + kBN - 1) / kBN) * ((n_tokens + kBM - 1) / kBM);
-    const uint64_t cost128 = (tiles128 + sms - 1) / sms * 3, cost256 = (tiles256 + sms - 1) / sms * 4;
-    const int halves = (n_tokens > static_cast<uint32_t>(kBM) && cost256 <= cost128) ? 2 : 1;
+    // weight tile then feeds one product instead of two). The first `lead` tokens (a multiple of 256) go to a launch of
+    // 256-token tiles, the rest to a launch of 128-token tiles in the same stream; the split whose
+    // (waves over the SMs) x (cost of a tile), summed over the two launches, is lowest wins, ties going to the larger lead.
+    const uint64_t feature_tiles = (rows + kBN - 1) / kBN;
+    const uint32_t blocks256 = (n_tokens + 2 * kBM - 1) / (2 * kBM);
+    uint32_t lead = 0;
+    uint64_t best = ~0ull;
+    for (uint32_t b = 0; b <= blocks256; ++b) {
+        const uint32_t covered = b * 2u * kBM;
+        const uint64_t rest = covered >= n_tokens ? 0 : (n_tokens - covered + kBM - 1) / kBM;
+        const uint64_t cost = (feature_tiles * b + sms - 1) / sms * 4 + (feature_tiles * rest + sms - 1) / sms * 3;
+        if (cost <= best) {
+            best = cost;
+            lead = covered < n_tokens ? covered : n_tokens;
+        }
+    }
     CUtensorMap mx, mw, mm;
-    if (!make_map(enc, &mx, x, cols, n_tokens, halves * kBM) || !make_map(enc, &mw, w0, cols, rows, kBN) || !make_map(enc, &mm, m_slot, cols, rows, kBN))
-        return static_cast<int>(cudaErrorInvalidValue);
+    if (!make_map(enc, &mw, w0, cols, rows, kBN) || !make_map(enc, &mm, m_slot, cols, rows, kBN)) return static_cast<int>(cudaErrorInvalidValue);
     LinearArgs a;
     a.n_tokens = n_tokens;
     a.rows = rows;
@@ -477,9 +488,18 @@ int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* 
     a.y_bf16 = y_bf16 ? 1u : 0u;
     a.gate = gate;
     a.wait_ns = wait_ns ? wait_ns : kDefaultWaitNs;
-    const dim3 grid((rows + kBN - 1) / kBN, (n_tokens + halves * kBM - 1) / (halves * kBM));
-    if (halves == 1) linear_kernel<1><<<grid, kLinearThreads, LinearGeom<1>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
-    else linear_kernel<2><<<grid, kLinearThreads, LinearGeom<2>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
+    if (lead) {
+        if (!make_map(enc, &mx, x, cols, n_tokens, 2 * kBM)) return static_cast<int>(cudaErrorInvalidValue);
+        a.token0 = 0;
+        const dim3 grid(static_cast<unsigned>(feature_tiles), (lead + 2 * kBM - 1) / (2 * kBM));
+        linear_kernel<2><<<grid, kLinearThreads, LinearGeom<2>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
+    }
+    if (lead < n_tokens) {
+        if (!make_map(enc, &mx, x, cols, n_tokens, kBM)) return static_cast<int>(cudaErrorInvalidValue);
+        a.token0 = lead;
+        const dim3 grid(static_cast<unsigned>(feature_tiles), (n_tokens - lead + kBM - 1) / kBM);
+        linear_kernel<1><<<grid, kLinearThreads, LinearGeom<1>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
+    }
     return static_cast<int>(cudaGetLastError());
 }
 

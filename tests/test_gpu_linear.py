@@ -130,8 +130,8 @@ def test_linear_without_flip_and_without_shuffle():
 
 
 def test_linear_blocks_of_256_tokens():
-    # enough tiles (16 feature tiles x 10 blocks of 256 tokens: two waves, against three of the 128-token shape) for the 256-token CTA, whose second
-    # block of 128 tokens has accumulators of its own; ragged token count, ragged last k-step, bf16 and fp32 output
+    # 16 feature tiles x 9 blocks of 256 tokens (one wave of 256-token CTAs, whose second block of 128 tokens has
+    # accumulators of its own) and the ragged rest in 128-token CTAs; ragged last k-step, bf16 and fp32 output
     w = _workload([(2048, 136, 2)], [S | F], n_tasks=2)
     _run(w, [2500], layers=[0])
     ids = list(w.task_ids)
@@ -157,15 +157,22 @@ def _dyadic_bits(rng, shape, kmax=8):
     return wl.to_bf16_bits((rng.integers(-kmax, kmax + 1, size=shape) / 16.0).astype(np.float32))
 
 
-def _uses_256_token_blocks(rows, n_tok):
-    """The library's choice of CTA shape: a 128-token tile costs about 3/4 of a 256-token tile; the shape with the lower
-    (number of waves over the SMs) x (cost of a tile) wins, 256 tokens on a tie."""
+def _lead_tokens(rows, n_tok):
+    """The library's choice of CTA shapes: the first `lead` tokens (a multiple of 256, or all of them) go to 256-token
+    tiles, the rest to 128-token tiles; a 128-token tile costs about 3/4 of a 256-token tile, and the split with the lowest
+    sum of (number of waves over the SMs) x (cost of a tile) wins, the larger lead on a tie."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    waves = lambda tokens_per_tile: -(-(((rows + 127) // 128) * ((n_tok + tokens_per_tile - 1) // tokens_per_tile)) // sms)
-    return n_tok > 128 and waves(256) * 4 <= waves(128) * 3
+    feature_tiles = (rows + 127) // 128
+    best, lead = None, 0
+    for b in range((n_tok + 255) // 256 + 1):
+        rest = max(0, n_tok - 256 * b)
+        cost = -(-feature_tiles * b // sms) * 4 + -(-feature_tiles * ((rest + 127) // 128) // sms) * 3
+        if best is None or cost <= best:
+            best, lead = cost, min(256 * b, n_tok)
+    return lead
 
 
-def _run_dyadic(shape, gflag, n_tok, sample_tokens, want_256, lam=0.25, members=2):
+def _run_dyadic(shape, gflag, n_tok, sample_tokens, want_lead, lam=0.25, members=2):
     """Bit equality with the oracle on dyadic inputs: layer [rows, cols], `members` same-shape layers in one group
     (so that the shuffle picks a slot), x [n_tok, cols].  The oracle runs on `sample_tokens` rows of x; every row
     is also checked against an fp32 library product on the weight formed from the oracle's slot and sign row
@@ -173,9 +180,9 @@ def _run_dyadic(shape, gflag, n_tok, sample_tokens, want_256, lam=0.25, members=
     rows, cols = shape
     w = _workload([(rows, cols, members)], [gflag], n_tasks=2)
     ids, seeds = list(w.task_ids), list(w.seeds)
-    assert _uses_256_token_blocks(rows, n_tok) == want_256
+    assert _lead_tokens(rows, n_tok) == want_lead                          # tokens covered by 256-token tiles
     n_k = (cols + 63) // 64
-    assert n_k >= (2 * 3 + 1 if want_256 else 2 * 4 + 1), "every stage of the operand ring must be reused"
+    assert n_k >= (2 * 3 + 1 if want_lead else 2 * 4 + 1), "every stage of the operand ring must be reused"
     rng = np.random.default_rng(rows * 7 + cols)
     base = [_dyadic_bits(rng, (rows, cols)) for _ in range(w.n_layers)]
     M_ref = [_dyadic_bits(rng, (rows, cols)) for _ in range(w.n_layers)]
@@ -222,20 +229,33 @@ def _block_edges(n_tok):
 
 def test_linear_bit_exact_on_dyadic_inputs_in_the_benchmarked_shape():
     # [1024 x 4096] x 8192 tokens: 256-token CTAs, 64 k-steps through the 3-stage ring (every stage reused 21 times)
-    _run_dyadic((1024, 4096), S | F, 8192, _block_edges(8192), want_256=True, members=2)
+    _run_dyadic((1024, 4096), S | F, 8192, _block_edges(8192), want_lead=8192, members=2)
 
 
 def test_linear_bit_exact_on_dyadic_inputs_256_token_blocks_ragged():
-    # 256-token CTAs with a ragged last k-step (648 = 10 x 64 + 8), ragged token and feature counts; with and without flip
-    _run_dyadic((2000, 648), S | F, 2500, _block_edges(2500), want_256=True)
-    _run_dyadic((2048, 456), S, 2400, _block_edges(2400), want_256=True)
+    # 256-token CTAs alone (16 feature tiles x 9 token blocks: one wave) with a ragged last k-step (648 = 10 x 64 + 8),
+    # ragged token and feature counts
+    _run_dyadic((2000, 648), S | F, 2300, _block_edges(2300), want_lead=2300)
+
+
+def test_linear_bit_exact_on_dyadic_inputs_two_tile_shapes_in_one_call():
+    # the first 2304 tokens in one wave of 256-token CTAs, the ragged rest in 128-token CTAs (a second launch whose
+    # token offset is not zero); with and without flip
+    _run_dyadic((2000, 648), S | F, 2500, _block_edges(2500) + list(range(2296, 2312)), want_lead=2304)
+    _run_dyadic((2048, 456), S, 2400, _block_edges(2400) + list(range(2296, 2312)), want_lead=2304)
+
+
+def test_linear_bit_exact_on_dyadic_inputs_two_tile_shapes_vit_b32_mlp():
+    # [768 x 3072] x 8192 tokens: 6144 tokens in one wave of 144 256-token CTAs, 2048 tokens in 96 128-token CTAs
+    edges = _block_edges(8192) + [6143, 6144, 6145, 6271, 6272, 8063, 8064]
+    _run_dyadic((768, 3072), S | F, 8192, edges, want_lead=6144, members=2)
 
 
 def test_linear_bit_exact_on_dyadic_inputs_128_token_blocks():
     # 128-token CTAs (too few tiles for the wider shape), 17 and 9 k-steps through the 4-stage ring, ragged last k-step
-    _run_dyadic((384, 1032), S | F, 257, range(257), want_256=False)
-    _run_dyadic((200, 576), S, 130, range(130), want_256=False)
-    _run_dyadic((136, 4096), F, 100, range(100), want_256=False, members=1)
+    _run_dyadic((384, 1032), S | F, 257, range(257), want_lead=0)
+    _run_dyadic((200, 576), S, 130, range(130), want_lead=0)
+    _run_dyadic((136, 4096), F, 100, range(100), want_lead=0, members=1)
 
 
 def test_linear_gaussian_inputs_wide_layers_see_one_wrong_column():

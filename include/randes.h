@@ -287,8 +287,10 @@ int randes_retrieve(randes_plan_t* plan, uint32_t task_id, float lambda,
  *   M                     device, the superposition arena
  *   y, y_dtype            device, [n_tokens, rows] row-major, fp32 or bf16 (the fp32 result rounded to nearest
  *                         even, once); must not alias the inputs
- * Needs no workspace (the plan may have been built without one).  One kernel launch;
- * asynchronous on `stream`.  The result equals the fp64 definition within
+ *   n_tokens              at most 8388480 (65535 blocks of 128 tokens)
+ * Needs no workspace (the plan may have been built without one).  One or two kernel launches
+ * (the first tokens in blocks of 256, the rest in blocks of 128, split where that takes the fewest
+ * waves over the SMs); asynchronous on `stream`.  The result equals the fp64 definition within
  * 2 * cols * 2^-24 * sum_c |x| (|W_0| + |lambda M|) per output (fp32 accumulation of 2 * cols
  * exact products in any order).  Errors: UNSUPPORTED_DTYPE, UNKNOWN_TASK, INVALID_ARGUMENT,
  * MISALIGNED, CUDA_ERROR.

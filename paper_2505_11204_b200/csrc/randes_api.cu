@@ -1218,6 +1218,7 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
         return fail(RANDES_MISALIGNED, "x and base[%u] must be 16-byte aligned", layer);
     if (reinterpret_cast<uintptr_t>(y) % elem_size(y_dtype)) return fail(RANDES_MISALIGNED, "y = %p is not aligned to its element size", y);
     if (reinterpret_cast<uintptr_t>(gate) % 4) return fail(RANDES_MISALIGNED, "gate = %p is not 4-byte aligned", (const void*)gate);
+    if (n_tokens > 65535u * 128u) return fail(RANDES_INVALID_ARGUMENT, "n_tokens = %u exceeds the supported %u", n_tokens, 65535u * 128u);
     if (wait_ns > 60ull * 1000000000ull) return fail(RANDES_INVALID_ARGUMENT, "wait_ns = %llu exceeds the supported 60 s", (unsigned long long)wait_ns);
     const TaskEntry& t = plan->tasks[row];
     const uint32_t slot = t.slot_of_pos[layer];                    // sigma_t^-1(p)
@@ -1227,12 +1228,12 @@ static int randes_linear_impl(const randes_plan_t* plan, uint32_t task_id, float
     d.key0 = static_cast<uint32_t>(t.seed);
     d.key1 = static_cast<uint32_t>(t.seed >> 32);
     d.pad = 0;
-    int e = linear_prepare();
+    int e = linear_prepare(), launched = 0;
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "set-up of the linear kernel");
     e = launch_linear(x, n_tokens, base[layer], static_cast<const char*>(M) + plan->m_off_bytes[slot], rows, cols, flip, slot, d, lambda,
-                      y, y_dtype == RANDES_BF16, gate, wait_ns, stream);
+                      y, y_dtype == RANDES_BF16, gate, wait_ns, stream, &launched);
+    g_launches += launched;
     if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the linear kernel");
-    ++g_launches;
     return RANDES_OK;
 }
 

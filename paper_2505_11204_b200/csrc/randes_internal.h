@@ -197,7 +197,7 @@ unsigned long long violation_in_batch_kernels();
 int linear_prepare();   // opts the kernel into its shared memory on the current device
 int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* m_slot, uint32_t rows, uint32_t cols, bool flip,
                   uint32_t slot, const DevTask& task, float lambda, void* y, bool y_bf16, const uint32_t* gate,
-                  unsigned long long wait_ns, void* stream);   // gate: NULL or a device word to wait on; wait_ns: 0 = one second
+                  unsigned long long wait_ns, void* stream, int* n_launched);   // gate: NULL or a device word to wait on; wait_ns: 0 = one second
 int linear_giveups(unsigned int* count);   // CTAs that gave up on a bounded wait since the library was loaded (synchronises)
 
 // Retrieve with its tables in a fixed device array inside the library (no workspace).

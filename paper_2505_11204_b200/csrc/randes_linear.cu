@@ -448,8 +448,9 @@ int linear_prepare()
 
 int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* m_slot, uint32_t rows, uint32_t cols, bool flip,
                   uint32_t slot, const DevTask& task, float lambda, void* y, bool y_bf16, const uint32_t* gate,
-                  unsigned long long wait_ns, void* stream)
+                  unsigned long long wait_ns, void* stream, int* n_launched)
 {
+    *n_launched = 0;
     EncodeTiledFn enc = encode_fn();
     if (!enc) return static_cast<int>(cudaErrorNotSupported);
     // 128 or 256 tokens per CTA (with 256 each staged weight tile feeds two products)
@@ -493,14 +494,20 @@ int launch_linear(const void* x, uint32_t n_tokens, const void* w0, const void* 
         a.token0 = 0;
         const dim3 grid(static_cast<unsigned>(feature_tiles), (lead + 2 * kBM - 1) / (2 * kBM));
         linear_kernel<2><<<grid, kLinearThreads, LinearGeom<2>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
+        const cudaError_t le = cudaGetLastError();
+        if (le != cudaSuccess) return static_cast<int>(le);
+        ++*n_launched;
     }
     if (lead < n_tokens) {
         if (!make_map(enc, &mx, x, cols, n_tokens, kBM)) return static_cast<int>(cudaErrorInvalidValue);
         a.token0 = lead;
         const dim3 grid(static_cast<unsigned>(feature_tiles), (n_tokens - lead + kBM - 1) / kBM);
         linear_kernel<1><<<grid, kLinearThreads, LinearGeom<1>::kSmem, static_cast<cudaStream_t>(stream)>>>(mx, mw, mm, a);
+        const cudaError_t le = cudaGetLastError();
+        if (le != cudaSuccess) return static_cast<int>(le);
+        ++*n_launched;
     }
-    return static_cast<int>(cudaGetLastError());
+    return static_cast<int>(cudaSuccess);
 }
 
 int linear_giveups(unsigned int* count)

@@ -199,7 +199,9 @@ def _run_dyadic(shape, gflag, n_tok, sample_tokens, want_lead, lam=0.25, members
     for p in range(w.n_layers):
         for t, s in zip(ids, seeds):
             y = torch.full((n_tok, rows), float("nan"), dtype=torch.float32, device="cuda")
+            launches = randes.randes_launch_count()
             plan.linear(t, lam, p, d_x, d_base, M_dev, y=y)
+            assert randes.randes_launch_count() - launches == (want_lead > 0) + (want_lead < n_tok)
             got = y.cpu().numpy()
             y_ref, _ = ro.linear(w.spec, w.storage, t, s, lam, p, np.ascontiguousarray(x[sample]), base, M_ref, m_dtype=wl.BF16)
             want = y_ref.astype(np.float32)
@@ -346,6 +348,18 @@ def test_linear_rejects_what_it_cannot_run():
         plan.linear(w.task_ids[0], 0.3, 0, x, d_base, M)
     assert e.value.code == randes.INVALID_ARGUMENT
     plan.close()
+    w8 = _workload([(16, 8, 1)], [F], n_tasks=1)
+    d8 = model_to_dev(wl.model_set(w8, w8.task_ids)[0])
+    plan8 = randes.Plan.from_workload(w8, max_tasks=1, m_dtype=wl.BF16)
+    M8 = plan8.new_superposition()
+    x8 = torch.zeros((4, 8), dtype=torch.bfloat16, device="cuda")
+    y8 = torch.zeros((4, 16), dtype=torch.float32, device="cuda")
+    before = randes.randes_launch_count()
+    with pytest.raises(randes.RandesError) as e:           # more tokens than the grid can hold: refused before any launch
+        randes.randes_linear(plan8.handle, w8.task_ids[0], 0.3, 0, x8, 65535 * 128 + 1, randes.ptr_array(d8), M8, y8,
+                             torch.cuda.current_stream().cuda_stream, wl.F32)
+    assert e.value.code == randes.INVALID_ARGUMENT and randes.randes_launch_count() == before
+    plan8.close()
     w32 = wl.toy()
     plan32 = randes.Plan.from_workload(w32, max_tasks=4)
     b32 = model_to_dev(wl.model_set(w32, [])[0])

@@ -11,6 +11,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
+
 #include "randes_device.cuh"
 #include "randes_internal.h"
 
@@ -308,16 +310,6 @@ __global__ void __launch_bounds__(kThreadsPerCta, 2) retrieve_batch_group_kernel
 
 size_t batch_group_smem(uint32_t pairs) { return 2 * static_cast<size_t>(kStashBytes) + static_cast<size_t>(pairs) * kBatchRecBytes; }
 
-template <typename K> int occupancy(K kernel)
-{
-    int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreadsPerCta, 0) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return 0;
-    }
-    return n;
-}
-
 template <typename T> struct Tag { typedef T type; };
 template <typename F> int with_type(int dtype, F&& f) { return dtype == 0 ? f(Tag<float>{}) : f(Tag<__nv_bfloat16>{}); }
 
@@ -359,25 +351,13 @@ int launch_retrieve_batch_groups(int out_dtype, const RetrieveBatchArgs& a, uint
     const size_t smem = batch_group_smem(max_group * a.n_tasks);
     return with_type(out_dtype, [&](auto ot) {
         typedef typename decltype(ot)::type OT;
-        int per_sm = 0;
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, retrieve_batch_group_kernel<OT>, kThreadsPerCta, smem);
-        if (e != cudaSuccess) { (void)cudaGetLastError(); return static_cast<int>(e); }
-        if (per_sm <= 0) return static_cast<int>(cudaErrorInvalidConfiguration);
-        const uint64_t want = static_cast<uint64_t>(sm_count) * per_sm;
-        const int grid = static_cast<int>(want < a.n_units ? want : a.n_units);
+        // One CTA per unit, not a resident loop: the block scheduler hands the next unit to whichever SM has room.
+        // This kernel is bound by its stores, and SMs do not drain stores at equal rates; with the units dealt out
+        // evenly in advance the slowest SM set the time (measured: 5.1 -> 4.6 ms for 20 ViT-L/14-shaped models).
+        const int grid = static_cast<int>(std::min<uint64_t>(a.n_units, 0x7FFFFFFFull));
+        (void)sm_count;
         retrieve_batch_group_kernel<OT><<<grid, kThreadsPerCta, smem, s>>>(a);
         return static_cast<int>(cudaGetLastError());
-    });
-}
-
-int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype)
-{
-    return with_type(storage_dtype, [&](auto st) {
-        return with_type(out_dtype, [&](auto ot) {
-            return with_type(m_dtype, [&](auto mt) {
-                return occupancy(retrieve_batch_kernel<typename decltype(st)::type, typename decltype(ot)::type, typename decltype(mt)::type>);
-            });
-        });
     });
 }
 

@@ -179,7 +179,6 @@ int launch_gram(int storage_dtype, const GramArgs& a, int grid, double* gram, vo
 int gram_ctas_per_sm(int storage_dtype);
 // randes_batch.cu
 int launch_retrieve_batch(int storage_dtype, int out_dtype, int m_dtype, const RetrieveBatchArgs& a, int grid, void* stream);
-int retrieve_batch_ctas_per_sm(int storage_dtype, int out_dtype, int m_dtype);
 // batched retrieve over group units (fp32 weights and superposition): M and W_0 tiles of a whole group staged in shared memory
 int retrieve_batch_group_prepare();
 bool retrieve_batch_group_fits(uint32_t max_group, uint32_t n_tasks);

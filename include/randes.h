@@ -111,6 +111,17 @@ size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_laye
                                    uint32_t max_tasks);
 
 /*
+ * The same for a plan with these groups.  Equal to randes_plan_workspace_bytes unless a group
+ * carries RANDES_GAUSS (the diagonal context of Section 5.5): such a plan also keeps, in its
+ * workspace, a table of the context's factors -- 4 bytes per registered task and column of every
+ * layer, written when a task is registered -- and randes_plan answers WORKSPACE_TOO_SMALL to less.
+ * Returns 0 on invalid arguments.  Host-only.
+ */
+size_t randes_plan_workspace_bytes_groups(const randes_layer_t* layers, uint32_t n_layers,
+                                          const randes_group_t* groups, uint32_t n_groups,
+                                          uint32_t max_tasks);
+
+/*
  * Build a plan (Sections 4.2-4.4; seeds as in the appendix on the default
  * experimental setup: one seed per model drives both its shuffle and its sign
  * matrices).
@@ -122,7 +133,7 @@ size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_laye
  *                   which compress sums them.  Ids must be distinct.
  *   max_tasks       capacity of the registry (>= n_tasks, >= 1).
  *   dev_workspace   device memory, 256-byte aligned, at least
- *                   randes_plan_workspace_bytes() bytes; used by the plan until
+ *                   randes_plan_workspace_bytes_groups() bytes; used by the plan until
  *                   randes_plan_destroy.  The layer, tile and permutation
  *                   tables are copied into it on `stream`.
  *   out_plan        receives the plan; free with randes_plan_destroy.

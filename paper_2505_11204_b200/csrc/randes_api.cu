@@ -96,7 +96,27 @@ struct TaskEntry {
 
 struct WorkspaceLayout {
     size_t layers, units, tasks, src_of_slot, slot_of_pos, base_ptrs, out_ptrs, task_ptrs, members, staged_units, total;
+    size_t ctx_off = 0, ctx_table = 0;   // plans with a general diagonal context only (appended after `total` is first set)
 };
+
+// floats per task row of the context table: every layer's columns, each span padded to a multiple of four
+size_t context_stride(const randes_layer_t* layers, uint32_t n_layers)
+{
+    size_t n = 0;
+    for (uint32_t l = 0; l < n_layers; ++l) n += align_up(static_cast<size_t>(layers[l].cols), 4);
+    return n;
+}
+
+// append the column offsets and the factor table of a general diagonal context to a layout
+void layout_context(WorkspaceLayout& w, const randes_layer_t* layers, uint32_t n_layers, size_t max_tasks)
+{
+    size_t off = align_up(w.total, 256);
+    w.ctx_off = off;
+    off = align_up(off + n_layers * sizeof(uint32_t), 256);
+    w.ctx_table = off;
+    off = align_up(off + max_tasks * context_stride(layers, n_layers) * sizeof(float), 256);
+    w.total = off;
+}
 
 WorkspaceLayout layout_workspace(size_t n_layers, size_t n_units, size_t n_staged_units, size_t max_tasks)
 {
@@ -238,6 +258,7 @@ struct randes_plan_s {
     std::vector<randes_layer_t> layers;
     std::vector<uint32_t> gflags;
     bool has_gauss = false;                       // some group carries the Gaussian-like context: every call takes the plain kernels
+    uint32_t ctx_stride = 0, max_cols = 0;        // has_gauss: floats per task row of the factor table; widest layer
     std::vector<std::vector<uint32_t>> members;   // per group, in layer order
     std::vector<DevLayer> dev_layers;
     std::vector<DevUnit> units;
@@ -314,6 +335,16 @@ int find_task(const randes_plan_t& p, uint32_t id)
     return -1;
 }
 
+// the factor table of a plan with a general diagonal context, seen from task row `row`
+ContextArgs context_args(const randes_plan_t& p, size_t row)
+{
+    ContextArgs x;
+    x.table = p.dev<float>(p.lay.ctx_table) + row * p.ctx_stride;
+    x.off = p.dev<uint32_t>(p.lay.ctx_off);
+    x.stride = p.ctx_stride;
+    return x;
+}
+
 // copy task rows [first, end) (descriptors + both tables) to the device
 int upload_task_rows(randes_plan_t& p, size_t first, cudaStream_t s)
 {
@@ -338,6 +369,12 @@ int upload_task_rows(randes_plan_t& p, size_t first, cudaStream_t s)
         cudaError_t e = cudaMemcpyAsync(p.dev<DevTask>(p.lay.tasks) + first, p.h_dev_tasks.data() + first,
                                         (p.tasks.size() - first) * sizeof(DevTask), cudaMemcpyHostToDevice, s);
         if (e != cudaSuccess) return fail_cuda(e, "copy of task descriptors");
+        if (p.has_gauss) {   // the factors of these tasks, once, for every later call
+            const int ce = launch_context_fill(context_args(p, 0), p.dev<DevLayer>(p.lay.layers), p.n_layers, p.max_cols, p.dev<DevTask>(p.lay.tasks),
+                                               static_cast<uint32_t>(first), static_cast<uint32_t>(p.tasks.size() - first), s);
+            if (ce) return fail_cuda(static_cast<cudaError_t>(ce), "launch of the context table kernel");
+            ++g_launches;
+        }
     }
     return RANDES_OK;
 }
@@ -423,7 +460,7 @@ int run_accumulate(randes_plan_t& p, size_t first_row, size_t n_rows, bool init_
     a.M = M;
     if (p.has_gauss) {
         if (a.n_units == 0) return RANDES_OK;
-        const int e = launch_context_accumulate(p.storage, a, p.sm_count, s);
+        const int e = launch_context_accumulate(p.storage, a, context_args(p, first_row), s);
         if (e) return fail_cuda(static_cast<cudaError_t>(e), "launch of the general-context accumulate kernel");
         ++g_launches;
         return RANDES_OK;
@@ -550,6 +587,21 @@ size_t randes_plan_workspace_bytes(const randes_layer_t* layers, uint32_t n_laye
     return layout_workspace(n_layers, n_units, n_staged, max_tasks).total;
 }
 
+size_t randes_plan_workspace_bytes_groups(const randes_layer_t* layers, uint32_t n_layers, const randes_group_t* groups, uint32_t n_groups,
+                                          uint32_t max_tasks)
+{
+    const size_t plain = randes_plan_workspace_bytes(layers, n_layers, max_tasks);
+    if (plain == 0 || !groups) return plain;
+    bool gauss = false;
+    for (uint32_t g = 0; g < n_groups; ++g) gauss = gauss || (groups[g].flags & RANDES_GAUSS);
+    if (!gauss) return plain;
+    if (context_stride(layers, n_layers) > 0xFFFFFFFFull) return 0;
+    WorkspaceLayout w{};
+    w.total = plain;
+    layout_context(w, layers, n_layers, max_tasks);
+    return w.total;
+}
+
 int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_group_t* groups, uint32_t n_groups,
                 randes_dtype_t storage_dtype, randes_dtype_t m_dtype, const uint32_t* task_ids, const uint64_t* seeds, uint32_t n_tasks,
                 uint32_t max_tasks, void* dev_workspace, size_t dev_workspace_bytes, void* stream,
@@ -640,17 +692,7 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
             off = align_up(off + static_cast<size_t>(layers[l].rows) * layers[l].cols * elem_size(m_dtype), 256);
         }
         p->m_bytes = off;
-        // A general diagonal context costs three Philox blocks per (task, column) and unit: its plans get taller units
-        // (up to eight times), so that the factors are reused over more rows -- as tall as still leaves about two
-        // thousand units for the grid (fewer units than the workspace holds, which is sized for the short ones).
-        uint32_t rows_per_warp = kRowsPerWarp;
-        if (p->has_gauss) {
-            unsigned long long params = 0;
-            for (uint32_t l = 0; l < n_layers; ++l) params += static_cast<unsigned long long>(layers[l].rows) * layers[l].cols;
-            while (rows_per_warp < static_cast<uint32_t>(kContextRowsPerWarp) && params / (2ull * rows_per_warp * 1024ull) >= 2000ull)
-                rows_per_warp *= 2;
-        }
-        build_units(layers, n_layers, p->storage, p->units, nullptr, nullptr, kAllGroups, nullptr, rows_per_warp);
+        build_units(layers, n_layers, p->storage, p->units);
         {
             std::vector<uint32_t> member_base(n_groups, 0);
             p->group_staged.assign(n_groups, 0);
@@ -684,6 +726,16 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
             make_task_tables(*p, p->tasks[i]);
         }
         p->lay = layout_workspace(n_layers, p->units.size(), p->group_units.size() + p->other_units.size(), max_tasks);
+        if (p->has_gauss) {
+            const size_t stride = context_stride(layers, n_layers);
+            if (stride > 0xFFFFFFFFull) {
+                delete p;
+                return fail(RANDES_INVALID_ARGUMENT, "the layers have %zu columns in all: more than the factor table of a RANDES_GAUSS plan indexes", stride);
+            }
+            p->ctx_stride = static_cast<uint32_t>(stride);
+            for (uint32_t l = 0; l < n_layers; ++l) p->max_cols = std::max(p->max_cols, layers[l].cols);
+            layout_context(p->lay, layers, n_layers, max_tasks);
+        }
     } catch (const std::bad_alloc&) {
         delete p;
         return fail(RANDES_OUT_OF_MEMORY, "host allocation failed");
@@ -698,8 +750,10 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         }
         if (dev_workspace_bytes < p->lay.total) {
             const size_t need = p->lay.total;
+            const bool gauss = p->has_gauss;
             delete p;
-            return fail(RANDES_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, plan needs %zu", dev_workspace_bytes, need);
+            return fail(RANDES_WORKSPACE_TOO_SMALL, "workspace has %zu bytes, plan needs %zu%s", dev_workspace_bytes, need,
+                        gauss ? " (a plan with a RANDES_GAUSS group holds a table of its factors: size it with randes_plan_workspace_bytes_groups)" : "");
         }
         p->ws = static_cast<char*>(dev_workspace);
         cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -738,6 +792,13 @@ int randes_plan(const randes_layer_t* layers, uint32_t n_layers, const randes_gr
         if (e == cudaSuccess && !p->group_units.empty()) {
             const int ge = compress_group_prepare(p->storage, p->m_dtype);
             if (ge) { delete p; return fail_cuda(static_cast<cudaError_t>(ge), "set-up of the group compress kernel"); }
+        }
+        if (e == cudaSuccess && p->has_gauss) {
+            std::vector<uint32_t> ctx_off(n_layers);
+            size_t o = 0;
+            for (uint32_t l = 0; l < n_layers; ++l) { ctx_off[l] = static_cast<uint32_t>(o); o += align_up(static_cast<size_t>(layers[l].cols), 4); }
+            // pageable host memory: the copy has left the vector when the call returns
+            e = cudaMemcpyAsync(p->ws + p->lay.ctx_off, ctx_off.data(), n_layers * sizeof(uint32_t), cudaMemcpyHostToDevice, s);
         }
         if (e != cudaSuccess) { delete p; return fail_cuda(e, "copy of plan tables"); }
         if ((rc = upload_task_rows(*p, 0, s))) { delete p; return rc; }
@@ -995,7 +1056,7 @@ static int randes_retrieve_impl(randes_plan_t* plan, uint32_t task_id, float lam
     a.lambda = lambda;
     if (a.n_units == 0) return RANDES_OK;
     if (plan->has_gauss) {
-        const int ce = launch_context_retrieve(plan->storage, out_dtype, a, plan->sm_count, s);
+        const int ce = launch_context_retrieve(plan->storage, out_dtype, a, context_args(*plan, static_cast<size_t>(row)), s);
         if (ce) return fail_cuda(static_cast<cudaError_t>(ce), "launch of the general-context retrieve kernel");
         ++g_launches;
         return RANDES_OK;

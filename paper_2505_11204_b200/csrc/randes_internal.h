@@ -15,7 +15,6 @@ constexpr size_t kSuperpositionLeadIn = 1024;   // bytes before the first slot o
 constexpr int kWarpsPerCta = 8;
 constexpr int kThreadsPerCta = kWarpsPerCta * 32;
 constexpr int kRowsPerWarp = 16;        // rows one warp walks per unit (8 to 16 measured best; 32 and 64 slower)
-constexpr int kContextRowsPerWarp = 128; // upper limit of the same for plans with a general diagonal context (randes_context.cu)
 constexpr int kTaskChunk = 32;          // tasks whose pointers / sign blocks a warp holds at once
 constexpr uint32_t kTagSign = 0x5349474Eu;  // counter word 2 of the sign stream ("SIGN")
 constexpr uint32_t kTagPerm = 0x5045524Du;  // counter word 2 of the permutation stream ("PERM")
@@ -161,10 +160,20 @@ int launch_retrieve(int storage_dtype, int out_dtype, int m_dtype, const Retriev
 int launch_accumulate(int storage_dtype, int m_dtype, const AccumulateArgs& a, int grid, void* stream);
 // add / remove of one model, bf16 weights, fp32 superposition, every layer cols % 8 == 0 and 16-byte aligned tensors
 int launch_add_halves(const AccumulateArgs& a, int sm_count, void* stream);
-// randes_context.cu: all of a plan's layers under a general diagonal context (plans with a RANDES_GAUSS group);
-// fp32 superposition only.  Return a cudaError_t as int.
-int launch_context_accumulate(int storage_dtype, const AccumulateArgs& a, int sm_count, void* stream);
-int launch_context_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, int sm_count, void* stream);
+// randes_context.cu: all of a plan's layers under a general diagonal context (plans with a RANDES_GAUSS group).
+// The diagonal factors live in a table in the plan's workspace: table[task row][off[slot] + column], `stride` floats per
+// row (every slot's span padded to a multiple of four, so that four neighbouring factors are one aligned 16-byte load).
+// launch_context_fill writes the rows of newly registered tasks; for accumulate `table` points at the first task row
+// to sum, for retrieve at the row of the task to rebuild.
+struct ContextArgs {
+    const float* table;
+    const uint32_t* off;           // device array [n_layers]
+    uint32_t stride;
+};
+int launch_context_fill(const ContextArgs& x, const DevLayer* layers, uint32_t n_layers, uint32_t max_cols, const DevTask* tasks,
+                        uint32_t first_row, uint32_t n_rows, void* stream);
+int launch_context_accumulate(int storage_dtype, const AccumulateArgs& a, const ContextArgs& x, void* stream);
+int launch_context_retrieve(int storage_dtype, int out_dtype, const RetrieveArgs& a, const ContextArgs& x, void* stream);
 // randes_group.cu: compress over group units.  `max_group` = the largest staged group.
 int compress_group_prepare(int storage_dtype, int m_dtype);   // once per device: opts into the shared memory the kernel needs
 bool compress_group_fits(int storage_dtype, uint32_t max_group, uint32_t n_tasks);

@@ -72,6 +72,8 @@ def lib():
         vp, u32, u64, sz = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_size_t
         L.randes_plan_workspace_bytes.argtypes = [vp, u32, u32]
         L.randes_plan_workspace_bytes.restype = sz
+        L.randes_plan_workspace_bytes_groups.argtypes = [vp, u32, vp, u32, u32]
+        L.randes_plan_workspace_bytes_groups.restype = sz
         L.randes_plan.argtypes = [vp, u32, vp, u32, ctypes.c_int, ctypes.c_int, vp, vp, u32, u32, vp, sz, vp,
                                   ctypes.POINTER(vp)]
         L.randes_plan.restype = ctypes.c_int
@@ -134,7 +136,7 @@ def lib():
 
 
 EXPORTS = [
-    "randes_plan_workspace_bytes", "randes_plan", "randes_plan_destroy", "randes_plan_validate", "randes_debug_violation", "randes_superposition_bytes",
+    "randes_plan_workspace_bytes", "randes_plan_workspace_bytes_groups", "randes_plan", "randes_plan_destroy", "randes_plan_validate", "randes_debug_violation", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
     "randes_task_tables", "randes_plan_serialize", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_add_models", "randes_remove_model",
     "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_interference_norm", "randes_pairwise_cosines", "randes_retrieve_batch", "randes_retrieve_static", "randes_linear", "randes_linear_gated", "randes_linear_giveups", "randes_launch_count", "randes_last_error",
@@ -163,6 +165,11 @@ def _addr(x) -> Optional[int]:
 # ---- C-named entry points (raw addresses / ctypes arrays) ----------------------------------
 def randes_plan_workspace_bytes(layers, n_layers: int, max_tasks: int) -> int:
     return int(lib().randes_plan_workspace_bytes(_addr(layers), n_layers, max_tasks))
+
+
+def randes_plan_workspace_bytes_groups(layers, n_layers: int, groups, n_groups: int, max_tasks: int) -> int:
+    """Workspace bytes of a plan with these groups (larger than the plain figure only with a RANDES_GAUSS group)."""
+    return int(lib().randes_plan_workspace_bytes_groups(_addr(layers), n_layers, _addr(groups), n_groups, max_tasks))
 
 
 def randes_plan(layers, n_layers, groups, n_groups, storage_dtype, m_dtype, task_ids, seeds, n_tasks, max_tasks,
@@ -376,7 +383,7 @@ class Plan:
         if not host_only:
             import torch
 
-            ws_bytes = randes_plan_workspace_bytes(self._layers, n_layers, max_tasks)
+            ws_bytes = randes_plan_workspace_bytes_groups(self._layers, n_layers, self._groups, n_groups, max_tasks)
             if ws_bytes == 0:
                 raise RandesError(INVALID_ARGUMENT, randes_last_error())
             self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=device)

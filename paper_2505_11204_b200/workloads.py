@@ -29,6 +29,7 @@ F32 = 0
 BF16 = 1
 SHUFFLE = 1
 FLIP = 2
+GAUSS = 1 << 16   # Gaussian-like diagonal context instead of the +-1 one (RANDES_GAUSS)
 
 
 @dataclass
@@ -72,6 +73,14 @@ class Workload:
         w = Workload(**{**self.__dict__})
         w.storage = storage
         w.name = self.name.split(":")[0] + (":bf16" if storage == BF16 else ":f32")
+        return w
+
+    def with_gaussian_context(self) -> "Workload":
+        """The same set with the +-1 context of every flipped group replaced by the Gaussian-like diagonal of the paper's
+        RD ablation (Section 5.5)."""
+        w = Workload(**{**self.__dict__})
+        w.gflags = [(f & ~FLIP) | GAUSS if f & FLIP else f for f in self.gflags]
+        w.name = self.name + ":rd"
         return w
 
     def with_tasks(self, n_tasks: int, first_seed: Optional[int] = None) -> "Workload":

@@ -5,6 +5,8 @@ fp32 outputs of retrieve are bit-exact (one fused multiply-add on both sides;
 the accepted bound would be 1e-6 * max|W|); bf16 outputs are bit-exact (accepted
 bound: 1 bf16 ulp).  All inputs are seeded and synthetic.
 """
+import ctypes
+
 import numpy as np
 import pytest
 
@@ -483,6 +485,19 @@ def test_gaussian_diagonal_context_limits():
         randes.Plan.from_workload(make_workload([(8, 64, 2)], flags=[G | F], n_tasks=2), max_tasks=2)
     assert e.value.code == randes.INVALID_ARGUMENT
     plan = randes.Plan.from_workload(w, max_tasks=2)
+    import torch
+
+    # the plan keeps a table of its factors in the workspace: the plain workspace figure is refused, with a message that
+    # names the query to use
+    small = randes.randes_plan_workspace_bytes(plan._layers, w.n_layers, 2)
+    assert small < randes.randes_plan_workspace_bytes_groups(plan._layers, w.n_layers, plan._groups, len(w.gflags), 2) == plan.workspace.numel()
+    ids = (ctypes.c_uint32 * 2)(*w.task_ids)
+    sds = (ctypes.c_uint64 * 2)(*w.seeds)
+    ws = torch.empty(small, dtype=torch.uint8, device="cuda")
+    with pytest.raises(randes.RandesError) as e:
+        randes.randes_plan(plan._layers, w.n_layers, plan._groups, len(w.gflags), w.storage, wl.F32, ids, sds, 2, 2, ws.data_ptr(), small,
+                           torch.cuda.current_stream().cuda_stream)
+    assert e.value.code == randes.WORKSPACE_TOO_SMALL and "randes_plan_workspace_bytes_groups" in str(e.value)
     M = plan.compress(d_base, [model_to_dev(t) for t in tasks])
     before = randes.randes_launch_count()
     for call in (lambda: plan.retrieve_batch(list(w.task_ids), 0.3, d_base, M),

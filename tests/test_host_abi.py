@@ -112,6 +112,21 @@ def test_workspace_size_grows_with_capacity_and_rejects_bad_input():
     assert 0 < a < b
     assert randes.randes_plan_workspace_bytes(p._layers, w.n_layers, 0) == 0
     assert randes.randes_plan_workspace_bytes(None, 3, 4) == 0
+    # the group-aware figure: the same without a RANDES_GAUSS group; with one, larger by at least the table of factors
+    # (4 bytes per task and column of every layer)
+    n_groups = len(w.gflags)
+    assert randes.randes_plan_workspace_bytes_groups(p._layers, w.n_layers, p._groups, n_groups, 4) == a
+    assert randes.randes_plan_workspace_bytes_groups(p._layers, w.n_layers, None, 0, 4) == a
+    assert randes.randes_plan_workspace_bytes_groups(p._layers, w.n_layers, p._groups, n_groups, 0) == 0
+    wg = wl.Workload(**{**w.__dict__})
+    wg.gflags = [(f & ~wl.FLIP) | randes.GAUSS if f & wl.FLIP else f for f in w.gflags]
+    assert any(f & randes.GAUSS for f in wg.gflags)
+    pg = randes.Plan.from_workload(wg, host_only=True)
+    for cap in (4, 64):
+        plain = randes.randes_plan_workspace_bytes(pg._layers, wg.n_layers, cap)
+        with_table = randes.randes_plan_workspace_bytes_groups(pg._layers, wg.n_layers, pg._groups, n_groups, cap)
+        assert with_table >= plain + 4 * cap * sum(wg.cols)
+        assert with_table <= plain + 4 * cap * sum(c + 3 for c in wg.cols) + 4 * wg.n_layers + 1024
 
 
 def test_plan_round_trips_through_its_serialized_form():

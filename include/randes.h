@@ -81,7 +81,9 @@ typedef enum { RANDES_F32 = 0, RANDES_BF16 = 1 } randes_dtype_t;
  *                   twelve uniforms minus six, drawn from the task's Philox stream in exactly
  *                   rounded fp32 steps.  Mutually exclusive with RANDES_FLIP; needs an fp32
  *                   superposition.  A plan with such a group runs compress, add, remove and
- *                   retrieve through plain (not bandwidth-tuned) kernels, and does not offer
+ *                   retrieve through kernels of their own, which read the entries from a table
+ *                   kept in the plan's workspace (size it with randes_plan_workspace_bytes_groups;
+ *                   one extra kernel launch whenever tasks are registered or removed), and does not offer
  *                   randes_retrieve_batch, randes_retrieve_static, randes_delta_gram or randes_linear. */
 enum { RANDES_SHUFFLE = 1, RANDES_FLIP = 2, RANDES_SHIFT = 4, RANDES_GAUSS = 1 << 16 };
 #define RANDES_SKIP(k) (((uint32_t)(k) & 0xFFu) << 8)

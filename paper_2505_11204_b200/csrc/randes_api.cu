@@ -1406,6 +1406,14 @@ static int randes_plan_validate_impl(const randes_plan_t* plan)
     int rc;
     if ((rc = check_list(plan->units, {}, "the unit list"))) return rc;
     if (!plan->group_units.empty() && (rc = check_list(plan->other_units, plan->group_units, "the grouped unit list"))) return rc;
+    // a general diagonal context: the factor table holds every column of every layer for max_tasks rows, inside the workspace
+    if (plan->has_gauss) {
+        if (plan->ctx_stride != context_stride(plan->layers.data(), L))
+            return fail(RANDES_INVALID_ARGUMENT, "the factor table has %u floats per task, the layers need %zu", plan->ctx_stride, context_stride(plan->layers.data(), L));
+        if (plan->ws && (plan->lay.ctx_off + L * sizeof(uint32_t) > plan->lay.ctx_table ||
+                         plan->lay.ctx_table + static_cast<size_t>(plan->max_tasks) * plan->ctx_stride * sizeof(float) > plan->lay.total))
+            return fail(RANDES_INVALID_ARGUMENT, "the factor table does not fit the workspace layout");
+    }
     return RANDES_OK;
 }
 

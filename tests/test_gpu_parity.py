@@ -468,9 +468,46 @@ def test_gaussian_diagonal_context(storage, n_tasks):
     the sign flip or no context (a plan with one such group runs all its layers through the plain kernels);
     10 tasks = two passes of 8 and 2 through M."""
     G = randes.GAUSS
-    shapes = [(9, 132, 3), (5, 256, 4), (17, 520, 2), (1, 300, 5), (33, 64, 3), (3, 2100, 2)]
-    flags = [G | S, G, S | F, G | S | randes.SKIP(2), S, G | S]
+    shapes = [(9, 132, 3), (5, 256, 4), (17, 520, 2), (1, 300, 5), (33, 64, 3), (3, 2100, 2), (7, 131, 2), (4, 6, 3), (21, 1030, 2)]
+    flags = [G | S, G, S | F, G | S | randes.SKIP(2), S, G | S, G | S, G, S | F]     # (widths 131, 6, 1030: the element-wise path)
     run_full_cycle(make_workload(shapes, flags=flags, storage=storage, n_tasks=n_tasks), extra_task=True)
+
+
+@pytest.mark.parametrize("storage", [wl.F32, wl.BF16])
+def test_gaussian_diagonal_context_registry_changes(storage):
+    """The factors of the RD context are kept per registered task in a table in the plan's workspace.  A remove shifts the
+    later tasks up one row, a batched add appends rows: after each change every remaining task must still be retrieved
+    with ITS factors, and the sums must equal the oracle's replay of the same calls (six tasks = two passes of four and
+    two; the batched add continues from M)."""
+    G = randes.GAUSS
+    w = make_workload([(9, 132, 3), (6, 257, 2), (17, 520, 2), (1, 300, 4)], flags=[G | S, G | S, S | F, G], storage=storage, n_tasks=6)
+    ids, seeds = list(w.task_ids), list(w.seeds)
+    new_ids, new_seeds = [40, 41, 42], [900, 901, 902]
+    base, tasks = wl.model_set(w, ids + new_ids)
+    d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+    plan = randes.Plan.from_workload(w, max_tasks=9)
+    M_dev = poison(plan.new_superposition())
+    plan.compress(d_base, d_tasks[:6], M_dev)
+    M_ref = ro.compress(w.spec, storage, ids, seeds, base, tasks[:6])
+    check_superposition(plan, M_dev, M_ref, "compress")
+    # remove the second task: rows 2 .. 5 of the table move up
+    plan.remove_model(ids[1], d_base, d_tasks[1], M_dev)
+    ro.remove_model(w.spec, storage, ids[1], seeds[1], base, tasks[1], M_ref)
+    check_superposition(plan, M_dev, M_ref, "remove of a middle task")
+    for t in (0, 2, 5):
+        check_model(plan.retrieve(ids[t], 0.3, d_base, M_dev), ro.retrieve(w.spec, storage, wl.F32, ids[t], seeds[t], 0.3, base, M_ref),
+                    "retrieve of task %d after the shift" % ids[t])
+    # three more in one pass, then one of the old ones leaves
+    plan.add_models(new_ids, new_seeds, d_base, d_tasks[6:], M_dev)
+    ro.add_models(w.spec, storage, new_ids, new_seeds, base, tasks[6:], M_ref)
+    check_superposition(plan, M_dev, M_ref, "add_models")
+    plan.remove_model(ids[4], d_base, d_tasks[4], M_dev)
+    ro.remove_model(w.spec, storage, ids[4], seeds[4], base, tasks[4], M_ref)
+    check_superposition(plan, M_dev, M_ref, "second remove")
+    for t, sd in ((ids[5], seeds[5]), (new_ids[0], new_seeds[0]), (new_ids[2], new_seeds[2])):
+        check_model(plan.retrieve(t, 0.3, d_base, M_dev, out_dtype=wl.BF16), ro.retrieve(w.spec, storage, wl.BF16, t, sd, 0.3, base, M_ref),
+                    "retrieve of task %d after the second shift" % t)
+    plan.close()
 
 
 def test_gaussian_diagonal_context_limits():

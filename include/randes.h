@@ -208,6 +208,13 @@ int randes_debug_violation(uint64_t* word, int* checked_build);
  * Errors: INVALID_ARGUMENT (not a blob, truncated), plus those of randes_plan.
  */
 size_t randes_plan_serialize(const randes_plan_t* plan, void* buffer, size_t buffer_bytes);
+/*
+ * Bytes of device workspace a plan equal to this one needs (same layers, groups, element types and
+ * max_tasks): the figure randes_plan checks, at most randes_plan_workspace_bytes_groups().  Also
+ * answered by a host-only plan -- to size the workspace of a plan kept as a blob, deserialize it
+ * without a workspace, ask, and deserialize again with the memory.  0 for a NULL plan.
+ */
+size_t randes_plan_workspace_needed(const randes_plan_t* plan);
 int randes_plan_deserialize(const void* buffer, size_t buffer_bytes, uint32_t max_tasks,
                             void* dev_workspace, size_t dev_workspace_bytes, void* stream,
                             randes_plan_t** out_plan);

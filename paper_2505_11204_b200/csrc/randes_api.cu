@@ -861,6 +861,8 @@ size_t randes_plan_serialize(const randes_plan_t* plan, void* buffer, size_t buf
     return need;
 }
 
+size_t randes_plan_workspace_needed(const randes_plan_t* plan) { return plan ? plan->lay.total : 0; }
+
 int randes_plan_deserialize(const void* buffer, size_t buffer_bytes, uint32_t max_tasks, void* dev_workspace,
                             size_t dev_workspace_bytes, void* stream, randes_plan_t** out_plan)
 {

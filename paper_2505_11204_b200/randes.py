@@ -109,6 +109,8 @@ def lib():
         L.randes_plan_serialize.restype = sz
         L.randes_plan_deserialize.argtypes = [vp, sz, u32, vp, sz, vp, ctypes.POINTER(vp)]
         L.randes_plan_deserialize.restype = ctypes.c_int
+        L.randes_plan_workspace_needed.argtypes = [vp]
+        L.randes_plan_workspace_needed.restype = sz
         L.randes_delta_gram_scratch_bytes.argtypes = [vp]
         L.randes_delta_gram_scratch_bytes.restype = sz
         L.randes_delta_gram.argtypes = [vp, vp, vp, vp, vp, sz, vp]
@@ -138,7 +140,7 @@ def lib():
 EXPORTS = [
     "randes_plan_workspace_bytes", "randes_plan_workspace_bytes_groups", "randes_plan", "randes_plan_destroy", "randes_plan_validate", "randes_debug_violation", "randes_superposition_bytes",
     "randes_layer_offset", "randes_num_layers", "randes_num_tasks", "randes_task_list",
-    "randes_task_tables", "randes_plan_serialize", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_add_models", "randes_remove_model",
+    "randes_task_tables", "randes_plan_serialize", "randes_plan_workspace_needed", "randes_plan_deserialize", "randes_compress", "randes_add_model", "randes_add_models", "randes_remove_model",
     "randes_retrieve", "randes_delta_gram_scratch_bytes", "randes_delta_gram", "randes_interference_norm", "randes_pairwise_cosines", "randes_retrieve_batch", "randes_retrieve_static", "randes_linear", "randes_linear_gated", "randes_linear_giveups", "randes_launch_count", "randes_last_error",
 ]
 
@@ -191,6 +193,11 @@ def randes_plan_serialize(plan) -> bytes:
     if int(lib().randes_plan_serialize(plan, ctypes.addressof(buf), n)) != n:
         raise RandesError(INVALID_ARGUMENT, randes_last_error())
     return buf.raw
+
+
+def randes_plan_workspace_needed(plan) -> int:
+    """Workspace bytes a plan equal to this one needs (also answered by a host-only plan)."""
+    return int(lib().randes_plan_workspace_needed(plan))
 
 
 def randes_plan_deserialize(blob: bytes, max_tasks: int = 0, dev_workspace=None, dev_workspace_bytes: int = 0, stream=None) -> int:

@@ -510,6 +510,44 @@ def test_gaussian_diagonal_context_registry_changes(storage):
     plan.close()
 
 
+def test_plan_rebuilt_from_its_blob_on_the_device():
+    """A plan kept as a blob comes back in two steps: deserialized host-only it tells the workspace it needs, deserialized
+    again with that memory it computes the same bits as the original -- also for a plan whose workspace holds the factor
+    table of the Gaussian-like context."""
+    import torch
+
+    G = randes.GAUSS
+    for flags in ([S | F, S, F], [G | S, G, S | F]):
+        w = make_workload([(9, 132, 3), (5, 256, 2), (17, 520, 2)], flags=flags, n_tasks=3)
+        base, tasks = wl.model_set(w, w.task_ids)
+        d_base, d_tasks = model_to_dev(base), [model_to_dev(t) for t in tasks]
+        plan = randes.Plan.from_workload(w, max_tasks=4)
+        M_a = plan.compress(d_base, d_tasks)
+        blob = randes.randes_plan_serialize(plan.handle)
+        host = randes.randes_plan_deserialize(blob, max_tasks=4)
+        need = randes.randes_plan_workspace_needed(host)
+        randes.randes_plan_destroy(host)
+        assert 0 < need <= plan.workspace.numel()
+        stream = torch.cuda.current_stream().cuda_stream
+        ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        with pytest.raises(randes.RandesError) as e:
+            randes.randes_plan_deserialize(blob, 4, ws.data_ptr(), need - 256, stream)
+        assert e.value.code == randes.WORKSPACE_TOO_SMALL
+        twin = randes.randes_plan_deserialize(blob, 4, ws.data_ptr(), need, stream)
+        try:
+            M_b = poison(plan.new_superposition())
+            randes.randes_compress(twin, randes.ptr_array(d_base), randes.ptr_array(d_tasks), M_b, stream)
+            for l in range(w.n_layers):          # slot by slot: the lead-in and the padding between slots are never written
+                assert torch.equal(plan.slot(M_a, l).view(torch.int32), plan.slot(M_b, l).view(torch.int32)), "slot %d" % l
+            out_a = plan.retrieve(w.task_ids[1], 0.3, d_base, M_a)
+            out_b = plan.new_output(wl.F32)
+            randes.randes_retrieve(twin, w.task_ids[1], 0.3, wl.F32, randes.ptr_array(d_base), M_b, randes.ptr_array(out_b), stream)
+            assert all(torch.equal(a.view(torch.int32), b.view(torch.int32)) for a, b in zip(out_a, out_b))
+        finally:
+            randes.randes_plan_destroy(twin)
+        plan.close()
+
+
 def test_gaussian_diagonal_context_limits():
     G = randes.GAUSS
     w = make_workload([(8, 64, 2)], flags=[G | S], n_tasks=2)

@@ -146,6 +146,11 @@ def test_plan_round_trips_through_its_serialized_form():
             assert randes.lib().randes_task_tables(q, t, ctypes.addressof(a), ctypes.addressof(b)) == 0
             assert (list(a), list(b)) == p.task_tables(t)
         assert randes.randes_plan_serialize(q) == blob
+        # a host-only plan already tells what workspace its device twin needs: no more than the a-priori figure
+        need = randes.randes_plan_workspace_needed(q)
+        assert 0 < need <= randes.randes_plan_workspace_needed(p.handle)       # (q holds room for its 3 tasks only)
+        assert need <= randes.randes_plan_workspace_bytes_groups(p._layers, L, p._groups, len(gflags), 3)
+        assert randes.randes_plan_workspace_needed(None) == 0
     finally:
         randes.randes_plan_destroy(q)
     for bad in (blob[:20], b"\0" * len(blob), blob[:-8]):

@@ -175,17 +175,10 @@ template <int CH> struct ContextRing {
 };
 // copies with an L2 eviction priority: the task weights stream through once (evict first), the W_0 tiles are read again by
 // the other slots of the group under a shuffle (evict last)
-__device__ __forceinline__ uint64_t l2_policy(bool keep)
-{
-    uint64_t pol;
-    if (keep) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-    else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
 template <typename T> __device__ __forceinline__ void copy_quad(uint32_t dst, const void* p, size_t i, uint64_t pol);
 template <> __device__ __forceinline__ void copy_quad<float>(uint32_t dst, const void* p, size_t i, uint64_t pol)
 {
-    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(static_cast<const float*>(p) + i), "l"(pol) : "memory");
+    cp_async16_hint(dst, static_cast<const float*>(p) + i, pol);
 }
 template <> __device__ __forceinline__ void copy_quad<bf16>(uint32_t dst, const void* p, size_t i, uint64_t pol)
 {
@@ -210,7 +203,7 @@ __device__ __forceinline__ void accumulate_quads_ring(const AccumulateArgs& a, c
                                                       const void* const (&pb)[CH], bool from_m, uint32_t ring)
 {
     typedef ContextRing<CH> R;
-    const uint64_t pol_stream = l2_policy(false), pol_keep = l2_policy(true);
+    const uint64_t pol_stream = l2_evict_first_policy(), pol_keep = l2_evict_last_policy();
     for (uint32_t c = c_begin + 4 * threadIdx.x; c < c_end; c += 4 * kThreadsPerCta) {
         float g[CH][4];
 #pragma unroll

@@ -304,6 +304,14 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
     uint32_t stage_c = ring, stage_i = ring;
     const uint32_t ring_end = ring + NSTAGE * G::kStageBytes;
 
+    // Under a shuffle without staging (more than 32 tasks, several models added at once) every W_0 tile is read by
+    // several slots of its group and the repeats are meant to hit in L2: the W_0 copies ask L2 to keep their lines, the
+    // task weights, which pass through once, to drop theirs first (2 - 3 % on those paths).
+    uint64_t pol_stream = 0, pol_keep = 0;
+    if (BASE == kPerTaskBase) {
+        pol_stream = l2_evict_first_policy();
+        pol_keep = l2_evict_last_policy();
+    }
     auto issue = [&]() {
 #pragma unroll
         for (int k = 0; k < NB; ++k) {
@@ -315,8 +323,12 @@ __device__ __forceinline__ void accumulate_rows_async(const WarpTile& t, uint32_
                 for (int u = 0; u < U; ++u) {
                     if (u == 0 || left_i > u) {
                         const size_t byte_off = static_cast<size_t>(off_i + u * row_stride) * ES;
-                        cp_async16(stage_i + (G::kW + u * NB + k) * kSlotBytes, pw + byte_off);
-                        if (BASE == kPerTaskBase) cp_async16(stage_i + (G::kB + u * NB + k) * kSlotBytes, pb + byte_off);
+                        if (BASE == kPerTaskBase) {
+                            cp_async16_hint(stage_i + (G::kW + u * NB + k) * kSlotBytes, pw + byte_off, pol_stream);
+                            cp_async16_hint(stage_i + (G::kB + u * NB + k) * kSlotBytes, pb + byte_off, pol_keep);
+                        } else {
+                            cp_async16(stage_i + (G::kW + u * NB + k) * kSlotBytes, pw + byte_off);
+                        }
                     }
                 }
             }

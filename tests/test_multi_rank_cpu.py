@@ -102,6 +102,23 @@ def test_workload_parameter_counts():
     assert len(wl.flan_t5_lora_targets(wl.flan_t5_base())) == 72
 
 
+def test_context_switch_of_the_benchmark_swaps_the_flip_for_the_gaussian_diagonal():
+    """--context gauss: every group that flips signs carries the Gaussian-like context instead, nothing else changes,
+    and the line's config says so (the same dict from both arms)."""
+    import bench
+    from paper_2505_11204_b200 import workloads as wl
+
+    plain = bench.make_workload(bench.parse_args(["--workload", "vit_b32"]))
+    args = bench.parse_args(["--workload", "vit_b32", "--context", "gauss"])
+    rd = bench.make_workload(args)
+    assert rd.name.endswith(":rd") and (rd.rows, rd.cols, rd.group) == (plain.rows, plain.cols, plain.group)
+    assert any(f & wl.FLIP for f in plain.gflags)
+    for f0, f1 in zip(plain.gflags, rd.gflags):
+        assert f1 == ((f0 & ~wl.FLIP) | wl.GAUSS if f0 & wl.FLIP else f0)
+    assert "context" in bench.config_dict(rd, args) and "context" not in bench.config_dict(plain, bench.parse_args(["--workload", "vit_b32"]))
+    assert bench.step_bytes(rd, 5) == bench.step_bytes(plain, 5)
+
+
 def test_row_slices_of_every_layer_are_independent_problems():
     """Sharding by row slices needs no collective: the oracle on each slice equals the slice of the oracle."""
     import numpy as np

@@ -608,6 +608,32 @@ def test_random_plans():
         run_full_cycle(w, out_dtypes=(int(rng.integers(0, 2)),), lam=float(rng.choice([0.1, 0.3, 1.0, 2.0])))
 
 
+def test_random_plans_with_a_gaussian_context():
+    """The same draw with the Gaussian-like diagonal in some groups (such a plan runs all its layers, flipped or not,
+    through the kernels of the general context; up to twelve tasks = three passes of four): every step against the oracle."""
+    rng = np.random.default_rng(4711)
+    SH, SK, G = randes.SHIFT, randes.SKIP, randes.GAUSS
+    for case in range(10):
+        n_groups = int(rng.integers(1, 5))
+        shapes, flags = [], []
+        for g in range(n_groups):
+            rows = int(rng.choice([1, 2, 5, 16, 17, 33, 70]))
+            cols = int(rng.choice([4, 6, 12, 64, 130, 136, 256, 264, 520, 1024, 1032, 2056]))
+            shapes.append((rows, cols, int(rng.choice([1, 2, 3, 5, 12]))))
+            f = int(rng.choice([0, S, S, SH]))
+            if g == 0 or rng.random() < 0.6:
+                f |= G
+            elif rng.random() < 0.7:
+                f |= F
+            if rng.random() < 0.25:
+                f |= SK(int(rng.integers(2, 4)))
+            flags.append(f)
+        w = make_workload(shapes, flags=flags, storage=int(rng.integers(0, 2)), n_tasks=int(rng.choice([1, 2, 4, 5, 9, 12])),
+                          seed0=int(rng.integers(0, 2**62)), data_seed=300 + case, interleave=bool(rng.integers(0, 2)))
+        w.task_ids = [int(x) for x in rng.choice(1000, size=w.n_tasks, replace=False)]
+        run_full_cycle(w, out_dtypes=(int(rng.integers(0, 2)),), lam=float(rng.choice([0.1, 0.3, 1.0])))
+
+
 def test_row_slices_shard_without_exchange():
     # what each of several GPUs would hold under row-slice sharding, run here one slice after the other
     w = make_workload([(37, 256, 3), (1, 256, 3), (50, 132, 2)], n_tasks=3)
